@@ -1,0 +1,133 @@
+"""CPU oracle of the streaming-scan hot path. TEST INFRASTRUCTURE ONLY.
+
+Only tests/, the smoke check and the benchmark's CPU-baseline leg may import this package; the
+product package never does. The arithmetic lives in s3_oracle.cpp (plain C++, fp64); this file only
+marshals numpy arrays into it.
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+
+from .build import build as _build
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(_build())
+        _lib.s3o_idf.restype = C.c_double
+        _lib.s3o_idf.argtypes = [C.c_double]
+        _lib.s3o_num_threads.restype = C.c_int
+    return _lib
+
+
+def _p(a, t):
+    return None if a is None else a.ctypes.data_as(C.POINTER(t))
+
+
+def _f32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def num_threads() -> int:
+    return int(lib().s3o_num_threads())
+
+
+def preact(x, W, b_enc, b_dec) -> np.ndarray:
+    """Eq. 1 before the ReLU, fp64 [T, d_sae]."""
+    x, W, b_enc, b_dec = _f32(x), _f32(W), _f32(b_enc), _f32(b_dec)
+    T, d_in = x.shape
+    d_sae = W.shape[1]
+    assert W.shape[0] == d_in and b_enc.shape == (d_sae,) and b_dec.shape == (d_in,)
+    pre = np.empty((T, d_sae), dtype=np.float64)
+    lib().s3o_preact(_p(x, C.c_float), _p(W, C.c_float), _p(b_enc, C.c_float), _p(b_dec, C.c_float),
+                     C.c_int64(T), C.c_int(d_in), C.c_int(d_sae), _p(pre, C.c_double))
+    return pre
+
+
+def topk(pre, k: int):
+    """ReLU + Top-k (Eq. 1-3): ids int32 [T,k] (pad -1), vals fp32 [T,k] (pad 0)."""
+    pre = np.ascontiguousarray(pre, dtype=np.float64)
+    T, d_sae = pre.shape
+    ids = np.empty((T, k), dtype=np.int32)
+    vals = np.empty((T, k), dtype=np.float32)
+    lib().s3o_topk(_p(pre, C.c_double), C.c_int64(T), C.c_int(d_sae), C.c_int(k), _p(ids, C.c_int32), _p(vals, C.c_float))
+    return ids, vals
+
+
+def encode_topk(x, W, b_enc, b_dec, k: int):
+    return topk(preact(x, W, b_enc, b_dec), k)
+
+
+def postings(ids, d_sae: int, pos_base: int = 0, vals=None):
+    """Eq. 4 for one chunk: (row_ptr uint32 [d_sae+1], pos int32 [nnz], pval fp32 [nnz] or None)."""
+    ids = _i32(ids)
+    T, k = ids.shape
+    v = None if vals is None else _f32(vals)
+    row_ptr = np.empty(d_sae + 1, dtype=np.uint32)
+    pos = np.empty(max(T * k, 1), dtype=np.int32)
+    pval = None if v is None else np.empty(max(T * k, 1), dtype=np.float32)
+    lib().s3o_postings(_p(ids, C.c_int32), _p(v, C.c_float), C.c_int64(T), C.c_int(k), C.c_int(d_sae),
+                       C.c_int64(pos_base), _p(row_ptr, C.c_uint32), _p(pos, C.c_int32), _p(pval, C.c_float))
+    nnz = int(row_ptr[-1])
+    return row_ptr, pos[:nnz].copy(), (None if pval is None else pval[:nnz].copy())
+
+
+def index_merge(chunks, d_sae: int):
+    """Concatenate per-chunk CSRs [(row_ptr, pos), ...] (arrival order) into one CSR per layer."""
+    n = len(chunks)
+    rps = [np.ascontiguousarray(c[0], dtype=np.uint32) for c in chunks]
+    pss = [np.ascontiguousarray(c[1], dtype=np.int32) for c in chunks]
+    total = int(sum(int(r[-1]) for r in rps))
+    row_ptr = np.empty(d_sae + 1, dtype=np.uint64)
+    pos = np.empty(max(total, 1), dtype=np.int32)
+    RP = (C.POINTER(C.c_uint32) * n)(*[_p(r, C.c_uint32) for r in rps])
+    PP = (C.POINTER(C.c_int32) * n)(*[_p(p if p.size else np.zeros(1, np.int32), C.c_int32) for p in pss])
+    lib().s3o_index_merge(C.c_int(n), RP, PP, C.c_int(d_sae), _p(row_ptr, C.c_uint64), _p(pos, C.c_int32))
+    return row_ptr, pos[:total].copy()
+
+
+def idf(freq: float) -> float:
+    return float(lib().s3o_idf(C.c_double(freq)))
+
+
+def score_spans(ctx_ids, q_ids, q_vals, d_sae: int, width: int, stride: int, mode: int = 0, stop_freq: int = 0):
+    """ctx_ids [n_layers, L, k]; q_ids/q_vals [n_layers, Q, nq, kq]. Returns int64 coact [Q,n_spans]
+    (mode 0) or fp64 weighted scores (mode 1)."""
+    ctx_ids, q_ids, q_vals = _i32(ctx_ids), _i32(q_ids), _f32(q_vals)
+    n_layers, L, k = ctx_ids.shape
+    _, Q, nq, kq = q_ids.shape
+    assert q_ids.shape[0] == n_layers and q_vals.shape == q_ids.shape
+    ns = (L - width) // stride + 1 if L >= width else 0
+    co = np.zeros((Q, ns), dtype=np.int64) if mode == 0 else None
+    ws = np.zeros((Q, ns), dtype=np.float64) if mode == 1 else None
+    lib().s3o_score_spans(_p(ctx_ids, C.c_int32), C.c_int64(L), C.c_int(k), C.c_int(d_sae), C.c_int(n_layers),
+                          _p(q_ids, C.c_int32), _p(q_vals, C.c_float), C.c_int(Q), C.c_int(nq), C.c_int(kq),
+                          C.c_int(width), C.c_int(stride), C.c_int(mode), C.c_int64(stop_freq),
+                          _p(co, C.c_int64), _p(ws, C.c_double))
+    return co if mode == 0 else ws
+
+
+def fuse_select(base, bm25, alpha: float, beta: float, s: int):
+    """base: int64 coact or fp64 weighted scores [Q, n_spans]; bm25 fp32 [Q, n_spans] or None.
+    Returns (top_idx int32 [Q,s], top_score fp32 [Q,s], all_scores fp32 [Q,n_spans])."""
+    base = np.ascontiguousarray(base)
+    Q, ns = base.shape
+    co = base if base.dtype == np.int64 else None
+    ws = base.astype(np.float64) if co is None else None
+    b = None if bm25 is None else _f32(bm25)
+    top_idx = np.empty((Q, s), dtype=np.int32)
+    top_score = np.empty((Q, s), dtype=np.float32)
+    allsc = np.empty((Q, max(ns, 1)), dtype=np.float32)
+    lib().s3o_fuse_select(_p(co, C.c_int64), _p(ws, C.c_double), _p(b, C.c_float), C.c_float(alpha), C.c_float(beta),
+                          C.c_int(Q), C.c_int64(ns), C.c_int(s), _p(top_idx, C.c_int32), _p(top_score, C.c_float),
+                          _p(allsc, C.c_float))
+    return top_idx, top_score, allsc[:, :ns]
