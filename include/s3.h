@@ -1,0 +1,219 @@
+/*
+ * s3scan -- C ABI of the B200 (sm_100a) streaming-scan hot path of S^3-Attention.
+ *
+ *   scan      : SAE encode + ReLU + Top-k  ->  per-chunk CSR postings  ->  async append to a host index
+ *   retrieval : query feature aggregation  ->  span co-activation scores  ->  score fusion + top-s spans
+ *
+ * Conventions
+ *   - Every function returns s3_status (0 = S3_OK, negative = error). No exception crosses the ABI.
+ *     s3_last_error() gives a thread-local message for the last failing call on this thread.
+ *   - Pointer names say where the memory lives: d_* = device, h_* = host. The CALLER owns every
+ *     device buffer; the library never allocates or frees device memory. Sizes of caller-provided
+ *     scratch come from the *_bytes() queries.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). All device work
+ *     is enqueued on it and returns asynchronously; only s3_index_sync, s3_index_export_csr,
+ *     s3_index_stats and s3_workspace_status wait for the device.
+ *   - A workspace (`d_ws`) starts with a 64-byte status block. Zero it once before first use.
+ *     A kernel whose bounded wait runs out writes a non-zero code there (sticky) and returns early;
+ *     s3_workspace_status reads it. Calls that share one workspace must not overlap on the device.
+ *   - Device pointers must be 16-byte aligned unless stated otherwise.
+ *   - sm_100a only. There is no CPU path: without a CUDA device the compute entry points fail with
+ *     S3_ERR_CUDA.
+ */
+#ifndef S3_H_
+#define S3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t s3_status;
+enum {
+    S3_OK = 0,
+    S3_ERR_INVALID_ARG = -1,  /* null / misaligned pointer, size out of range                      */
+    S3_ERR_UNSUPPORTED = -2,  /* valid request outside the implemented limits (stated per call)    */
+    S3_ERR_CUDA = -3,         /* a CUDA runtime/driver call failed (message has the CUDA error)    */
+    S3_ERR_NOMEM = -4,        /* host (pinned) allocation failed                                   */
+    S3_ERR_CAPACITY = -5,     /* a caller-provided buffer or an int32 position range is too small  */
+    S3_ERR_TIMEOUT = -6,      /* a bounded device-side wait ran out (see s3_workspace_status)      */
+    S3_ERR_STATE = -7         /* call not allowed in the object's current state                    */
+};
+
+typedef enum { S3_BF16 = 0, S3_F32 = 1 } s3_dtype;
+
+#define S3_MAX_K 64            /* largest Top-k per token                                           */
+#define S3_MAX_POSTINGS_ITEMS 32
+#define S3_MAX_SCORE_LAYERS 16
+#define S3_WS_HEADER_BYTES 64
+
+const char* s3_last_error(void);
+int s3_version(void);
+
+/* Reads the status block of a workspace after waiting for `stream`.
+ * Returns S3_OK, or S3_ERR_TIMEOUT if a kernel gave up on a bounded wait; *code_out (nullable, host)
+ * receives the raw code (which wait ran out). */
+s3_status s3_workspace_status(const void* d_ws, void* stream, uint32_t* code_out);
+
+/* ------------------------------------------------------------------------------------------------
+ * SAE encode + ReLU + Top-k            (paper Sec. 3.3 Eq. 1-2; Sec. 3.4 Eq. 3; Sec. 3.5 Eq. 5)
+ *
+ *   pre[t,f] = sum_i W_enc[i,f] * (x[t,i] - b_dec[i]) + b_enc[f]
+ *   per token: the min(k, #{f : pre[t,f] > 0}) largest strictly positive pre[t,.]; ids and values,
+ *   ordered by (value descending, id ascending); the row is padded with id -1 / value 0.
+ *   The [T, d_sae] pre-activation is never written to device memory.
+ *
+ * W_enc is [d_in, d_sae] row-major (feature f = column f), dtype bf16 or fp32; b_enc [d_sae] and
+ * b_dec [d_in] are fp32. x is [T, d_in] row-major with row pitch ldx (elements), same dtype as W_enc.
+ *
+ * S3_BF16: products of bf16 inputs accumulated in fp32 on the tensor cores; b_dec is folded into an
+ *          effective bias b_eff[f] = b_enc[f] - sum_i W_enc[i,f] b_dec[i] (fp64 sum, stored fp32).
+ *          Requires d_in % 8 == 0, ldx % 8 == 0, d_sae % 8 == 0.
+ * S3_F32 : fp32 FMA accumulation of W_enc[i,f] * (x[t,i] - b_dec[i]) in index order, no folding.
+ * Limits : 1 <= k <= min(S3_MAX_K, d_sae); d_sae <= 65536 * 4; anything else -> S3_ERR_UNSUPPORTED /
+ *          S3_ERR_INVALID_ARG. T == 0 is a no-op.
+ *
+ * s3_sae_create runs a one-time preparation on `stream` (bf16: a K-major copy of W_enc and b_eff)
+ * into the caller's `d_prepared` buffer of s3_sae_prepared_bytes() bytes, which must stay alive and
+ * untouched, like W_enc/b_enc/b_dec themselves, for the life of the handle. The handle is host
+ * memory only.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct s3_sae s3_sae;
+
+size_t s3_sae_prepared_bytes(int d_in, int d_sae, s3_dtype dtype);
+s3_status s3_sae_create(s3_sae** out, const void* d_W_enc, const float* d_b_enc, const float* d_b_dec,
+                        int d_in, int d_sae, s3_dtype dtype, void* d_prepared, size_t prepared_bytes,
+                        void* stream);
+s3_status s3_sae_destroy(s3_sae* sae);
+/* Scratch for partial Top-k lists of up to T_max tokens (includes the status block). */
+size_t s3_sae_encode_workspace_bytes(const s3_sae* sae, int T_max, int k);
+s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, int T, int k,
+                             int32_t* d_ids /*[T,k]*/, float* d_vals /*[T,k]*/,
+                             void* d_ws, size_t ws_bytes, void* stream);
+/* Tuning knob: number of column slices each row block of the encode is split into (0 = automatic)
+ * and the largest number of thread blocks a launch may use (0 = all SMs). Results do not depend on
+ * either. */
+s3_status s3_sae_set_schedule(s3_sae* sae, int n_slices, int max_ctas);
+
+/* ------------------------------------------------------------------------------------------------
+ * Postings build                                             (paper Sec. 3.4 Eq. 4: I[f] <- I[f] U {t})
+ *
+ * Groups the (feature, position) pairs of one chunk of one layer into a CSR:
+ *   row_ptr[f] = number of pairs with id < f  (row_ptr has d_sae + 1 entries, uint32)
+ *   pos[row_ptr[f] .. row_ptr[f+1]) = ascending absolute positions pos_base + t with f in F_t
+ * ids [T,k] int32; entries < 0 are padding and are skipped; ids within a token must be distinct.
+ * d_vals / d_pval (both null or both non-null) carry each pair's activation next to its position.
+ * d_pos (and d_pval) must hold T*k entries. The result is bit-exact and run-to-run identical.
+ * Limits: d_sae <= 49152 (per-feature cursors live in shared memory), T < 2^24,
+ *         pos_base + T <= 2^31 - 1 (S3_ERR_CAPACITY: positions are int32). T == 0 writes zeros to row_ptr.
+ * The batched form processes up to S3_MAX_POSTINGS_ITEMS independent chunk-layers in one launch;
+ * `items` is a HOST array.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    const int32_t* d_ids;
+    const float* d_vals; /* nullable */
+    int32_t T, k, d_sae, reserved;
+    int64_t pos_base;
+    uint32_t* d_row_ptr; /* [d_sae+1] */
+    int32_t* d_pos;      /* [T*k]     */
+    float* d_pval;       /* nullable  */
+} s3_postings_item;
+
+size_t s3_postings_workspace_bytes(int T_max, int k, int d_sae);
+s3_status s3_postings_build(const int32_t* d_ids, const float* d_vals, int T, int k, int d_sae,
+                            int64_t pos_base, uint32_t* d_row_ptr, int32_t* d_pos, float* d_pval,
+                            void* d_ws, size_t ws_bytes, void* stream);
+s3_status s3_postings_build_batched(const s3_postings_item* h_items, int n_items,
+                                    void* d_ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Host-resident inverted index                         (paper Sec. 3.4: the index lives on the CPU and
+ *                                                        device memory is bounded by the chunk size)
+ *
+ * s3_index_append enqueues, without blocking the host: an event on `producer_stream`, then on the
+ * index's own copy stream device->pinned-host copies of row_ptr (d_sae+1 words) and of T*k
+ * positions (and values if d_pval != NULL). Chunks of one layer must arrive in ascending,
+ * non-overlapping position order (else S3_ERR_STATE). The device buffers may be overwritten once
+ * the copy is done: pass the stream that will overwrite them to s3_index_stream_wait (device-side
+ * wait, host does not block), or use *reuse_event_out (a cudaEvent_t owned by the index, valid
+ * until the next append of the same layer).
+ * Pinned memory grows in slabs of `pinned_slab_bytes`; growing calls the pinned allocator, which
+ * may synchronise the device, so reserve up front (s3_index_reserve) for an uninterrupted scan.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct s3_index s3_index;
+typedef struct {
+    int64_t n_chunks;        /* appended chunk-layers                       */
+    int64_t n_postings;      /* sum of row_ptr[d_sae] over synced segments  */
+    int64_t host_bytes;      /* pinned bytes in use                         */
+    int64_t host_bytes_reserved;
+    int64_t max_list_len;    /* longest merged posting list over all layers */
+    int64_t n_positions;     /* largest position + 1 seen                   */
+} s3_index_stats_t;
+
+s3_status s3_index_create(s3_index** out, int n_layers, int d_sae, size_t pinned_slab_bytes);
+s3_status s3_index_reserve(s3_index* index, size_t bytes);
+s3_status s3_index_append(s3_index* index, int layer, const uint32_t* d_row_ptr, const int32_t* d_pos,
+                          const float* d_pval, int T, int k, int64_t pos_base, void* producer_stream,
+                          void** reuse_event_out /*nullable*/);
+s3_status s3_index_stream_wait(s3_index* index, void* stream);
+/* Waits for every copy; checks that each segment's row_ptr is monotone and ends at <= T*k. */
+s3_status s3_index_sync(s3_index* index);
+s3_status s3_index_stats(s3_index* index, s3_index_stats_t* out);
+s3_status s3_index_layer_postings(s3_index* index, int layer, uint64_t* n_out);
+/* Merges the layer's chunk segments into one CSR on the host: per feature the chunk lists
+ * concatenated in arrival order (ascending positions). h_row_ptr [d_sae+1] uint64; h_pos (and
+ * h_pval, nullable) must hold s3_index_layer_postings() entries. */
+s3_status s3_index_export_csr(s3_index* index, int layer, uint64_t* h_row_ptr, int32_t* h_pos, float* h_pval);
+s3_status s3_index_destroy(s3_index* index);
+
+/* ------------------------------------------------------------------------------------------------
+ * Co-activation span scoring + fusion + top-s
+ *            (paper Sec. 3.5 Eq. 5-6 and the appendix IDF definition; fixed-width spans, min-count
+ *             score and score fusion follow the benchmark definition, see below)
+ *
+ * Spans: span j covers positions [j*stride, j*stride + width); n_spans = (L - width)/stride + 1
+ * (0 if L < width); positions after the last full span are ignored.
+ * Per query q and layer l, from the query tokens' Top-k (q_ids/q_vals [n_layers, Q, nq, k], ids < 0
+ * skipped):  cQ(f) = number of query tokens whose set contains f,  aQ(f) = sum of their activations
+ * (fp32, token order).
+ *   mode S3_SCORE_MINCOUNT : base[q,j] = sum_l sum_f min(cQ_l(f), cS_l(f,j))          (integer, exact)
+ *   mode S3_SCORE_WEIGHTED : base[q,j] = sum_l sum_f aQ_l(f) * IDF_l(f) * cS_l(f,j)   (Eq. 6 summed over
+ *        the span; IDF(f) = 1/(ln(1+freq(f))+1), freq = the feature's posting-list length in layer l;
+ *        features with freq > stop_freq are skipped when stop_freq > 0; accumulated in fp64)
+ * with cS_l(f,j) = number of postings of f inside span j.
+ * Fusion: score = fl32(fl32(alpha*base) + fl32(beta*bm25[q,j])) (bm25 nullable: score = fl32(alpha*base)).
+ * Output: the s best spans per query by (score descending, span index ascending); padded with
+ * index -1 / score 0 when n_spans < s. d_all_scores (nullable) receives every fused score.
+ *
+ * `h_layers` is a HOST array of n_layers views whose pointers are DEVICE pointers to one merged CSR
+ * per layer (row_ptr uint64 [d_sae+1], pos int32 ascending per feature).
+ * Limits: n_layers <= S3_MAX_SCORE_LAYERS; nq*k <= 4096; n_spans <= 16384; s <= 64;
+ *         width, stride >= 1.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    const uint64_t* d_row_ptr;
+    const int32_t* d_pos;
+} s3_csr_view;
+
+enum { S3_SCORE_MINCOUNT = 0, S3_SCORE_WEIGHTED = 1 };
+
+typedef struct {
+    int32_t width, stride, mode, s;
+    float alpha, beta;
+    int64_t stop_freq; /* 0 = off */
+} s3_score_params;
+
+size_t s3_score_workspace_bytes(int Q, int nq, int k, int n_layers, int n_spans, int s);
+s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L,
+                                         const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
+                                         const s3_score_params* params, const float* d_bm25, int64_t ld_bm25,
+                                         int32_t* d_top_idx /*[Q,s]*/, float* d_top_score /*[Q,s]*/,
+                                         float* d_all_scores /*[Q,n_spans] nullable*/,
+                                         void* d_ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* S3_H_ */

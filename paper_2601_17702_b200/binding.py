@@ -1,0 +1,287 @@
+"""ctypes binding of libs3scan.so: the same entry points as include/s3.h, taking torch tensors for
+device memory and the current torch stream. Argument marshalling only: every step of the path runs
+in the library's kernels. There is no fallback: a missing library or a failing call raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libs3scan.so")
+
+S3_OK = 0
+S3_ERR_INVALID_ARG, S3_ERR_UNSUPPORTED, S3_ERR_CUDA, S3_ERR_NOMEM = -1, -2, -3, -4
+S3_ERR_CAPACITY, S3_ERR_TIMEOUT, S3_ERR_STATE = -5, -6, -7
+S3_BF16, S3_F32 = 0, 1
+S3_SCORE_MINCOUNT, S3_SCORE_WEIGHTED = 0, 1
+S3_WS_HEADER_BYTES = 64
+
+EXPORTS = [
+    "s3_last_error", "s3_version", "s3_workspace_status",
+    "s3_sae_prepared_bytes", "s3_sae_create", "s3_sae_destroy", "s3_sae_encode_workspace_bytes",
+    "s3_sae_encode_topk", "s3_sae_set_schedule",
+    "s3_postings_workspace_bytes", "s3_postings_build", "s3_postings_build_batched",
+    "s3_index_create", "s3_index_reserve", "s3_index_append", "s3_index_stream_wait", "s3_index_sync",
+    "s3_index_stats", "s3_index_layer_postings", "s3_index_export_csr", "s3_index_destroy",
+    "s3_score_workspace_bytes", "s3_coactivation_score_topspans",
+]
+
+
+class S3Error(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"s3 error {code}: {msg}")
+        self.code = code
+
+
+class PostingsItem(C.Structure):
+    _fields_ = [("d_ids", C.c_void_p), ("d_vals", C.c_void_p), ("T", C.c_int32), ("k", C.c_int32),
+                ("d_sae", C.c_int32), ("reserved", C.c_int32), ("pos_base", C.c_int64),
+                ("d_row_ptr", C.c_void_p), ("d_pos", C.c_void_p), ("d_pval", C.c_void_p)]
+
+
+class CsrView(C.Structure):
+    _fields_ = [("d_row_ptr", C.c_void_p), ("d_pos", C.c_void_p)]
+
+
+class ScoreParams(C.Structure):
+    _fields_ = [("width", C.c_int32), ("stride", C.c_int32), ("mode", C.c_int32), ("s", C.c_int32),
+                ("alpha", C.c_float), ("beta", C.c_float), ("stop_freq", C.c_int64)]
+
+
+class IndexStats(C.Structure):
+    _fields_ = [("n_chunks", C.c_int64), ("n_postings", C.c_int64), ("host_bytes", C.c_int64),
+                ("host_bytes_reserved", C.c_int64), ("max_list_len", C.c_int64), ("n_positions", C.c_int64)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads the CUDA library; raises if it has not been built (there is no other implementation)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2601_17702_b200.build` "
+                              "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.s3_last_error.restype = C.c_char_p
+        for name in ("s3_sae_prepared_bytes", "s3_sae_encode_workspace_bytes", "s3_postings_workspace_bytes",
+                     "s3_score_workspace_bytes"):
+            getattr(L, name).restype = C.c_size_t
+        L.s3_sae_prepared_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
+        L.s3_sae_create.argtypes = [C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                    C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_sae_destroy.argtypes = [C.c_void_p]
+        L.s3_sae_set_schedule.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        L.s3_sae_encode_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        L.s3_sae_encode_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_workspace_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
+        L.s3_postings_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
+        L.s3_postings_build.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_void_p,
+                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_postings_build_batched.argtypes = [C.POINTER(PostingsItem), C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_index_create.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int, C.c_size_t]
+        L.s3_index_reserve.argtypes = [C.c_void_p, C.c_size_t]
+        L.s3_index_append.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                      C.c_int64, C.c_void_p, C.POINTER(C.c_void_p)]
+        L.s3_index_stream_wait.argtypes = [C.c_void_p, C.c_void_p]
+        L.s3_index_sync.argtypes = [C.c_void_p]
+        L.s3_index_stats.argtypes = [C.c_void_p, C.POINTER(IndexStats)]
+        L.s3_index_layer_postings.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_uint64)]
+        L.s3_index_export_csr.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.s3_index_destroy.argtypes = [C.c_void_p]
+        L.s3_score_workspace_bytes.argtypes = [C.c_int] * 6
+        L.s3_coactivation_score_topspans.argtypes = [C.POINTER(CsrView), C.c_int, C.c_int, C.c_int64, C.c_void_p,
+                                                     C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(ScoreParams),
+                                                     C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                     C.c_void_p, C.c_size_t, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _check(code: int):
+    if code != S3_OK:
+        raise S3Error(code, lib().s3_last_error().decode())
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def s3_last_error() -> str:
+    return lib().s3_last_error().decode()
+
+
+def s3_version() -> int:
+    return int(lib().s3_version())
+
+
+def new_workspace(n_bytes: int, device="cuda") -> torch.Tensor:
+    """A zeroed device workspace (the status block at its start must start at zero)."""
+    return torch.zeros(max(int(n_bytes), S3_WS_HEADER_BYTES), dtype=torch.uint8, device=device)
+
+
+def s3_workspace_status(ws: torch.Tensor, stream=None) -> int:
+    code = C.c_uint32(0)
+    _check(lib().s3_workspace_status(_ptr(ws), _stream(stream), C.byref(code)))
+    return int(code.value)
+
+
+class Sae:
+    """Handle of one SAE encoder (s3_sae_create / s3_sae_destroy). Keeps the tensors it points to alive."""
+
+    def __init__(self, W_enc: torch.Tensor, b_enc: torch.Tensor, b_dec: torch.Tensor, stream=None):
+        assert W_enc.is_cuda and W_enc.is_contiguous() and W_enc.dim() == 2
+        self.dtype = {torch.bfloat16: S3_BF16, torch.float32: S3_F32}[W_enc.dtype]
+        self.d_in, self.d_sae = W_enc.shape
+        self.W_enc, self.b_enc, self.b_dec = W_enc, b_enc.contiguous(), b_dec.contiguous()
+        assert self.b_enc.dtype == torch.float32 and self.b_dec.dtype == torch.float32
+        n = lib().s3_sae_prepared_bytes(self.d_in, self.d_sae, self.dtype)
+        self.prepared = torch.empty(n, dtype=torch.uint8, device=W_enc.device)
+        h = C.c_void_p()
+        _check(lib().s3_sae_create(C.byref(h), _ptr(W_enc), _ptr(self.b_enc), _ptr(self.b_dec), self.d_in, self.d_sae,
+                                   self.dtype, _ptr(self.prepared), n, _stream(stream)))
+        self.handle = h
+
+    def set_schedule(self, n_slices: int = 0, max_ctas: int = 0):
+        _check(lib().s3_sae_set_schedule(self.handle, n_slices, max_ctas))
+
+    def encode_workspace_bytes(self, T_max: int, k: int) -> int:
+        return int(lib().s3_sae_encode_workspace_bytes(self.handle, T_max, k))
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().s3_sae_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def s3_sae_encode_topk(sae: Sae, x: torch.Tensor, k: int, ids: torch.Tensor, vals: torch.Tensor, ws: torch.Tensor,
+                       stream=None):
+    """ids int32 [T,k], vals fp32 [T,k] are written on the stream; x is [T, d_in] with stride(1) == 1."""
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1 and x.shape[1] == sae.d_in
+    T = x.shape[0]
+    assert ids.dtype == torch.int32 and vals.dtype == torch.float32 and ids.is_contiguous() and vals.is_contiguous()
+    assert tuple(ids.shape) == (T, k) and tuple(vals.shape) == (T, k)
+    _check(lib().s3_sae_encode_topk(sae.handle, _ptr(x), x.stride(0) if T > 1 else max(x.stride(0), sae.d_in), T, k,
+                                    _ptr(ids), _ptr(vals), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def s3_postings_workspace_bytes(T_max: int, k: int, d_sae: int) -> int:
+    return int(lib().s3_postings_workspace_bytes(T_max, k, d_sae))
+
+
+def s3_postings_build(ids: torch.Tensor, d_sae: int, pos_base: int, row_ptr: torch.Tensor, pos: torch.Tensor,
+                      ws: torch.Tensor, vals: torch.Tensor | None = None, pval: torch.Tensor | None = None, stream=None):
+    T, k = ids.shape
+    assert ids.dtype == torch.int32 and ids.is_contiguous() and row_ptr.dtype in (torch.uint32, torch.int32)
+    assert row_ptr.numel() == d_sae + 1 and pos.dtype == torch.int32 and pos.numel() >= T * k
+    _check(lib().s3_postings_build(_ptr(ids), _ptr(vals), T, k, d_sae, pos_base, _ptr(row_ptr), _ptr(pos), _ptr(pval),
+                                   _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def make_postings_item(ids, d_sae, pos_base, row_ptr, pos, vals=None, pval=None) -> PostingsItem:
+    T, k = ids.shape
+    p = lambda t: None if t is None else t.data_ptr()
+    return PostingsItem(p(ids), p(vals), T, k, d_sae, 0, pos_base, p(row_ptr), p(pos), p(pval))
+
+
+def s3_postings_build_batched(items: list[PostingsItem], ws: torch.Tensor, stream=None):
+    arr = (PostingsItem * max(len(items), 1))(*items)
+    _check(lib().s3_postings_build_batched(arr, len(items), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+class Index:
+    """Host-resident inverted index (s3_index_*)."""
+
+    def __init__(self, n_layers: int, d_sae: int, pinned_slab_bytes: int = 64 << 20):
+        h = C.c_void_p()
+        _check(lib().s3_index_create(C.byref(h), n_layers, d_sae, pinned_slab_bytes))
+        self.handle, self.n_layers, self.d_sae = h, n_layers, d_sae
+
+    def reserve(self, n_bytes: int):
+        _check(lib().s3_index_reserve(self.handle, n_bytes))
+
+    def append(self, layer: int, row_ptr: torch.Tensor, pos: torch.Tensor, T: int, k: int, pos_base: int,
+               pval: torch.Tensor | None = None, stream=None):
+        _check(lib().s3_index_append(self.handle, layer, _ptr(row_ptr), _ptr(pos), _ptr(pval), T, k, pos_base,
+                                     _stream(stream), None))
+
+    def stream_wait(self, stream=None):
+        _check(lib().s3_index_stream_wait(self.handle, _stream(stream)))
+
+    def sync(self):
+        _check(lib().s3_index_sync(self.handle))
+
+    def stats(self) -> dict:
+        st = IndexStats()
+        _check(lib().s3_index_stats(self.handle, C.byref(st)))
+        return {f: int(getattr(st, f)) for f, _ in IndexStats._fields_}
+
+    def layer_postings(self, layer: int) -> int:
+        n = C.c_uint64(0)
+        _check(lib().s3_index_layer_postings(self.handle, layer, C.byref(n)))
+        return int(n.value)
+
+    def export_csr(self, layer: int, with_values: bool = False):
+        """(row_ptr int64-viewed uint64 [d_sae+1], pos int32 [P], pval fp32 [P] or None) as host tensors."""
+        n = self.layer_postings(layer)
+        row_ptr = torch.empty(self.d_sae + 1, dtype=torch.int64)
+        pos = torch.empty(max(n, 1), dtype=torch.int32)
+        pval = torch.empty(max(n, 1), dtype=torch.float32) if with_values else None
+        _check(lib().s3_index_export_csr(self.handle, layer, _ptr(row_ptr), _ptr(pos), _ptr(pval)))
+        return row_ptr, pos[:n], (None if pval is None else pval[:n])
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().s3_index_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def s3_score_workspace_bytes(Q, nq, k, n_layers, n_spans, s) -> int:
+    return int(lib().s3_score_workspace_bytes(Q, nq, k, n_layers, n_spans, s))
+
+
+def s3_coactivation_score_topspans(layers, d_sae: int, L: int, q_ids: torch.Tensor, q_vals: torch.Tensor,
+                                   width: int, stride: int, s: int, alpha: float, beta: float, ws: torch.Tensor,
+                                   bm25: torch.Tensor | None = None, mode: int = S3_SCORE_MINCOUNT, stop_freq: int = 0,
+                                   top_idx: torch.Tensor | None = None, top_score: torch.Tensor | None = None,
+                                   all_scores: torch.Tensor | None = None, stream=None):
+    """layers: list of (row_ptr int64 [d_sae+1], pos int32) device tensors, one merged CSR per layer.
+    q_ids/q_vals: [n_layers, Q, nq, k]. Returns (top_idx [Q,s] int32, top_score [Q,s] fp32)."""
+    n_layers, Q, nq, k = q_ids.shape
+    assert len(layers) == n_layers and q_ids.dtype == torch.int32 and q_vals.dtype == torch.float32
+    assert q_ids.is_contiguous() and q_vals.is_contiguous()
+    views = (CsrView * n_layers)(*[CsrView(rp.data_ptr(), ps.data_ptr()) for rp, ps in layers])
+    for rp, ps in layers:
+        assert rp.dtype == torch.int64 and ps.dtype == torch.int32 and rp.numel() == d_sae + 1
+    dev = q_ids.device
+    if top_idx is None:
+        top_idx = torch.empty((Q, s), dtype=torch.int32, device=dev)
+    if top_score is None:
+        top_score = torch.empty((Q, s), dtype=torch.float32, device=dev)
+    params = ScoreParams(width, stride, mode, s, alpha, beta, stop_freq)
+    ld = 0 if bm25 is None else bm25.stride(0)
+    _check(lib().s3_coactivation_score_topspans(views, n_layers, d_sae, L, _ptr(q_ids), _ptr(q_vals), Q, nq, k,
+                                                C.byref(params), _ptr(bm25), ld, _ptr(top_idx), _ptr(top_score),
+                                                _ptr(all_scores), _ptr(ws), ws.numel(), _stream(stream)))
+    return top_idx, top_score

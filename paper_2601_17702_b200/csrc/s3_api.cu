@@ -1,0 +1,300 @@
+// C ABI of the s3scan library: argument checks, handles and dispatch. All compute is in the kernels.
+#include <stdarg.h>
+#include <string.h>
+
+#include <new>
+
+#include "s3_encode_tc.cuh"
+#include "s3_topk.cuh"
+
+namespace s3 {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+s3_status fail(s3_status code, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int device_sm_count()
+{
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+    if (dev < 64 && cached[dev]) return cached[dev];
+    int n = 1;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 1;
+    if (dev < 64) cached[dev] = n;
+    return n;
+}
+
+int device_cc_major()
+{
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return 0;
+    return major;
+}
+
+}  // namespace s3
+
+using namespace s3;
+
+struct s3_sae {
+    const void* d_W;
+    const float* d_b_enc;
+    const float* d_b_dec;
+    int d_in, d_sae;
+    s3_dtype dtype;
+    int n_slices_override, max_ctas;
+    EncodeTcState tc;
+};
+
+namespace {
+
+constexpr int kMaxSlices = 16;
+
+int col_tiles(const s3_sae* sae) { return sae->dtype == S3_BF16 ? encode_tc_col_tiles(sae->d_sae) : encode_simt_col_tiles(sae->d_sae); }
+int row_tiles(const s3_sae* sae, int T) { return sae->dtype == S3_BF16 ? encode_tc_row_tiles(T) : encode_simt_row_tiles(T); }
+
+// Number of column slices per row block. The kernel runs `units = row_tiles * slices` work units on
+// at most n_sm thread blocks; the modelled time is waves * tiles-per-slice plus a small charge per
+// slice for restarting the Top-k filter and for the merge.
+int pick_slices(const s3_sae* sae, int T)
+{
+    const int nct = col_tiles(sae);
+    int cap = nct < kMaxSlices ? nct : kMaxSlices;
+    if (sae->n_slices_override > 0) return sae->n_slices_override < cap ? sae->n_slices_override : cap;
+    const int nrt = row_tiles(sae, T);
+    int n_sm = device_sm_count();
+    if (sae->max_ctas > 0 && sae->max_ctas < n_sm) n_sm = sae->max_ctas;
+    if (sae->dtype == S3_F32) {   // non-persistent kernel: enough blocks to cover the SMs
+        int s = (n_sm + nrt - 1) / nrt;
+        return s < 1 ? 1 : (s > cap ? cap : s);
+    }
+    int best = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= cap; ++s) {
+        const int units = nrt * s;
+        const int waves = (units + n_sm - 1) / n_sm;
+        const int len = (nct + s - 1) / s;
+        const double cost = (double)waves * len + 0.25 * s * waves;
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+    }
+    return best;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* s3_last_error(void) { return g_err; }
+int s3_version(void) { return 100; }
+
+s3_status s3_workspace_status(const void* d_ws, void* stream, uint32_t* code_out)
+{
+    S3_REQUIRE(d_ws != nullptr, S3_ERR_INVALID_ARG, "d_ws is null");
+    uint32_t code = 0;
+    S3_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    S3_CUDA_TRY(cudaMemcpy(&code, d_ws, sizeof(code), cudaMemcpyDeviceToHost));
+    if (code_out) *code_out = code;
+    if (code == DEV_OK) return S3_OK;
+    if (code == DEV_BAD_FEATURE_ID) return fail(S3_ERR_INVALID_ARG, "a feature id >= d_sae was met on the device (code %u)", code);
+    return fail(S3_ERR_TIMEOUT, "a bounded device-side wait ran out (code %u)", code);
+}
+
+// ---------------------------------------------------------------------------------------------- SAE
+size_t s3_sae_prepared_bytes(int d_in, int d_sae, s3_dtype dtype)
+{
+    if (d_in < 1 || d_sae < 1) return 0;
+    return dtype == S3_BF16 ? encode_tc_prepared_bytes(d_in, d_sae) : 256;
+}
+
+s3_status s3_sae_create(s3_sae** out, const void* d_W_enc, const float* d_b_enc, const float* d_b_dec, int d_in,
+                        int d_sae, s3_dtype dtype, void* d_prepared, size_t prepared_bytes, void* stream)
+{
+    S3_REQUIRE(out != nullptr, S3_ERR_INVALID_ARG, "out is null");
+    *out = nullptr;
+    S3_REQUIRE(d_W_enc && d_b_enc && d_b_dec, S3_ERR_INVALID_ARG, "null weight pointer");
+    S3_REQUIRE(aligned16(d_W_enc) && aligned16(d_b_enc) && aligned16(d_b_dec), S3_ERR_INVALID_ARG,
+               "weight pointers must be 16-byte aligned");
+    S3_REQUIRE(dtype == S3_BF16 || dtype == S3_F32, S3_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
+    S3_REQUIRE(d_in >= 1 && d_sae >= 1, S3_ERR_INVALID_ARG, "d_in = %d, d_sae = %d out of range", d_in, d_sae);
+    S3_REQUIRE(d_sae <= 262144, S3_ERR_UNSUPPORTED, "d_sae = %d exceeds 262144", d_sae);
+    if (dtype == S3_BF16) {
+        S3_REQUIRE(d_in % 8 == 0 && d_sae % 8 == 0, S3_ERR_UNSUPPORTED,
+                   "bf16 encode needs d_in and d_sae to be multiples of 8 (got %d, %d)", d_in, d_sae);
+        S3_REQUIRE(d_prepared != nullptr && aligned16(d_prepared), S3_ERR_INVALID_ARG, "d_prepared is null or misaligned");
+        S3_REQUIRE(prepared_bytes >= encode_tc_prepared_bytes(d_in, d_sae), S3_ERR_CAPACITY,
+                   "d_prepared holds %zu bytes, %zu needed", prepared_bytes, encode_tc_prepared_bytes(d_in, d_sae));
+    }
+    int n_dev = 0;
+    S3_CUDA_TRY(cudaGetDeviceCount(&n_dev));
+    S3_REQUIRE(device_cc_major() == 10, S3_ERR_UNSUPPORTED, "this library runs on sm_100 devices only (found compute capability %d.x)",
+               device_cc_major());
+    s3_sae* sae = new (std::nothrow) s3_sae();
+    S3_REQUIRE(sae != nullptr, S3_ERR_NOMEM, "out of host memory");
+    sae->d_W = d_W_enc; sae->d_b_enc = d_b_enc; sae->d_b_dec = d_b_dec;
+    sae->d_in = d_in; sae->d_sae = d_sae; sae->dtype = dtype;
+    sae->n_slices_override = 0; sae->max_ctas = 0;
+    if (dtype == S3_BF16) {
+        const s3_status st = encode_tc_prepare(&sae->tc, d_W_enc, d_b_enc, d_b_dec, d_in, d_sae, d_prepared,
+                                               static_cast<cudaStream_t>(stream));
+        if (st != S3_OK) { delete sae; return st; }
+    }
+    *out = sae;
+    return S3_OK;
+}
+
+s3_status s3_sae_destroy(s3_sae* sae)
+{
+    delete sae;
+    return S3_OK;
+}
+
+s3_status s3_sae_set_schedule(s3_sae* sae, int n_slices, int max_ctas)
+{
+    S3_REQUIRE(sae != nullptr, S3_ERR_INVALID_ARG, "sae is null");
+    S3_REQUIRE(n_slices >= 0 && n_slices <= kMaxSlices && max_ctas >= 0, S3_ERR_INVALID_ARG,
+               "n_slices must be in [0, %d] and max_ctas >= 0", kMaxSlices);
+    sae->n_slices_override = n_slices;
+    sae->max_ctas = max_ctas;
+    return S3_OK;
+}
+
+size_t s3_sae_encode_workspace_bytes(const s3_sae* sae, int T_max, int k)
+{
+    if (!sae || T_max < 0 || k < 1 || k > S3_MAX_K) return 0;
+    const int nct = col_tiles(sae);
+    const int smax = nct < kMaxSlices ? nct : kMaxSlices;
+    return S3_WS_HEADER_BYTES + (size_t)T_max * smax * k * sizeof(uint64_t);
+}
+
+s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, int T, int k, int32_t* d_ids, float* d_vals,
+                             void* d_ws, size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(sae != nullptr, S3_ERR_INVALID_ARG, "sae is null");
+    S3_REQUIRE(T >= 0, S3_ERR_INVALID_ARG, "T = %d is negative", T);
+    S3_REQUIRE(k >= 1 && k <= sae->d_sae, S3_ERR_INVALID_ARG, "k = %d out of range [1, d_sae = %d]", k, sae->d_sae);
+    S3_REQUIRE(k <= S3_MAX_K, S3_ERR_UNSUPPORTED, "k = %d exceeds the supported maximum %d", k, S3_MAX_K);
+    if (T == 0) return S3_OK;
+    S3_REQUIRE(d_x && d_ids && d_vals && d_ws, S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE(aligned16(d_x) && aligned16(d_ws) && (reinterpret_cast<uintptr_t>(d_ids) & 3) == 0 &&
+                   (reinterpret_cast<uintptr_t>(d_vals) & 3) == 0,
+               S3_ERR_INVALID_ARG, "misaligned device pointer");
+    S3_REQUIRE(ldx >= sae->d_in, S3_ERR_INVALID_ARG, "ldx = %lld is smaller than d_in = %d", (long long)ldx, sae->d_in);
+    if (sae->dtype == S3_BF16) S3_REQUIRE(ldx % 8 == 0, S3_ERR_INVALID_ARG, "ldx = %lld must be a multiple of 8 for bf16", (long long)ldx);
+    const int n_slices = pick_slices(sae, T);
+    const size_t need = S3_WS_HEADER_BYTES + (size_t)T * n_slices * k * sizeof(uint64_t);
+    S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t* status = static_cast<uint32_t*>(d_ws);
+    uint64_t* part = reinterpret_cast<uint64_t*>(static_cast<unsigned char*>(d_ws) + S3_WS_HEADER_BYTES);
+    s3_status rc;
+    if (sae->dtype == S3_BF16)
+        rc = launch_encode_tc(&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, k, n_slices, sae->max_ctas, part, status, st);
+    else
+        rc = launch_encode_simt(static_cast<const float*>(d_x), ldx, static_cast<const float*>(sae->d_W), sae->d_b_enc,
+                                sae->d_b_dec, T, sae->d_in, sae->d_sae, k, n_slices, part, st);
+    if (rc != S3_OK) return rc;
+    launch_topk_merge(part, T, n_slices, k, d_ids, d_vals, st);
+    S3_CUDA_TRY(cudaGetLastError());
+    return S3_OK;
+}
+
+// ---------------------------------------------------------------------------------------------- postings
+size_t s3_postings_workspace_bytes(int T_max, int k, int d_sae)
+{
+    (void)T_max; (void)k; (void)d_sae;
+    return S3_WS_HEADER_BYTES;
+}
+
+static s3_status check_item(const s3_postings_item& it, int idx)
+{
+    S3_REQUIRE(it.T >= 0 && it.k >= 1 && it.d_sae >= 1, S3_ERR_INVALID_ARG, "item %d: T = %d, k = %d, d_sae = %d out of range", idx, it.T,
+               it.k, it.d_sae);
+    S3_REQUIRE(it.d_sae <= 49152, S3_ERR_UNSUPPORTED, "item %d: d_sae = %d exceeds 49152", idx, it.d_sae);
+    S3_REQUIRE((int64_t)it.T * it.k < (1ll << 24), S3_ERR_UNSUPPORTED, "item %d: T*k = %lld must be below 2^24", idx,
+               (long long)it.T * it.k);
+    S3_REQUIRE(it.d_row_ptr != nullptr, S3_ERR_INVALID_ARG, "item %d: d_row_ptr is null", idx);
+    S3_REQUIRE(it.T == 0 || (it.d_ids && it.d_pos), S3_ERR_INVALID_ARG, "item %d: null device pointer", idx);
+    S3_REQUIRE((it.d_vals == nullptr) == (it.d_pval == nullptr), S3_ERR_INVALID_ARG,
+               "item %d: d_vals and d_pval must be both null or both non-null", idx);
+    S3_REQUIRE(it.pos_base >= 0, S3_ERR_INVALID_ARG, "item %d: pos_base is negative", idx);
+    S3_REQUIRE(it.pos_base + it.T <= INT32_MAX, S3_ERR_CAPACITY, "item %d: positions beyond int32 (pos_base %lld + T %d)", idx,
+               (long long)it.pos_base, it.T);
+    return S3_OK;
+}
+
+s3_status s3_postings_build_batched(const s3_postings_item* h_items, int n_items, void* d_ws, size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(n_items >= 0, S3_ERR_INVALID_ARG, "n_items is negative");
+    if (n_items == 0) return S3_OK;
+    S3_REQUIRE(h_items != nullptr, S3_ERR_INVALID_ARG, "h_items is null");
+    S3_REQUIRE(n_items <= S3_MAX_POSTINGS_ITEMS, S3_ERR_UNSUPPORTED, "n_items = %d exceeds %d", n_items, S3_MAX_POSTINGS_ITEMS);
+    S3_REQUIRE(d_ws != nullptr && ws_bytes >= S3_WS_HEADER_BYTES, S3_ERR_CAPACITY, "workspace missing or smaller than %d bytes",
+               S3_WS_HEADER_BYTES);
+    for (int i = 0; i < n_items; ++i) {
+        const s3_status st = check_item(h_items[i], i);
+        if (st != S3_OK) return st;
+    }
+    return launch_postings(h_items, n_items, static_cast<uint32_t*>(d_ws), static_cast<cudaStream_t>(stream));
+}
+
+s3_status s3_postings_build(const int32_t* d_ids, const float* d_vals, int T, int k, int d_sae, int64_t pos_base,
+                            uint32_t* d_row_ptr, int32_t* d_pos, float* d_pval, void* d_ws, size_t ws_bytes, void* stream)
+{
+    s3_postings_item it;
+    it.d_ids = d_ids; it.d_vals = d_vals; it.T = T; it.k = k; it.d_sae = d_sae; it.reserved = 0;
+    it.pos_base = pos_base; it.d_row_ptr = d_row_ptr; it.d_pos = d_pos; it.d_pval = d_pval;
+    return s3_postings_build_batched(&it, 1, d_ws, ws_bytes, stream);
+}
+
+// ---------------------------------------------------------------------------------------------- scoring
+size_t s3_score_workspace_bytes(int Q, int nq, int k, int n_layers, int n_spans, int s)
+{
+    (void)Q; (void)nq; (void)k; (void)n_layers; (void)n_spans; (void)s;
+    return S3_WS_HEADER_BYTES;
+}
+
+s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L,
+                                         const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
+                                         const s3_score_params* p, const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx,
+                                         float* d_top_score, float* d_all_scores, void* d_ws, size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(h_layers && p, S3_ERR_INVALID_ARG, "null argument");
+    S3_REQUIRE(n_layers >= 1 && n_layers <= S3_MAX_SCORE_LAYERS, S3_ERR_UNSUPPORTED, "n_layers = %d out of [1, %d]", n_layers,
+               S3_MAX_SCORE_LAYERS);
+    S3_REQUIRE(d_sae >= 1 && d_sae <= (1 << 20), S3_ERR_INVALID_ARG, "d_sae = %d out of range", d_sae);
+    S3_REQUIRE(L >= 0 && L <= INT32_MAX, S3_ERR_INVALID_ARG, "L out of range");
+    S3_REQUIRE(Q >= 0 && nq >= 1 && k >= 1, S3_ERR_INVALID_ARG, "Q = %d, nq = %d, k = %d out of range", Q, nq, k);
+    S3_REQUIRE((int64_t)nq * k <= 4096, S3_ERR_UNSUPPORTED, "nq*k = %lld exceeds 4096", (long long)nq * k);
+    S3_REQUIRE(p->width >= 1 && p->stride >= 1, S3_ERR_INVALID_ARG, "width = %d, stride = %d must be >= 1", p->width, p->stride);
+    S3_REQUIRE(p->mode == S3_SCORE_MINCOUNT || p->mode == S3_SCORE_WEIGHTED, S3_ERR_INVALID_ARG, "unknown mode %d", p->mode);
+    S3_REQUIRE(p->s >= 1 && p->s <= 64, S3_ERR_UNSUPPORTED, "s = %d out of [1, 64]", p->s);
+    const int64_t n_spans = (L >= p->width) ? (L - p->width) / p->stride + 1 : 0;
+    S3_REQUIRE(n_spans <= 16384, S3_ERR_UNSUPPORTED, "n_spans = %lld exceeds 16384", (long long)n_spans);
+    if (Q == 0) return S3_OK;
+    S3_REQUIRE(d_q_ids && d_q_vals && d_top_idx && d_top_score, S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE(d_ws != nullptr && ws_bytes >= S3_WS_HEADER_BYTES, S3_ERR_CAPACITY, "workspace missing or smaller than %d bytes",
+               S3_WS_HEADER_BYTES);
+    S3_REQUIRE(d_bm25 == nullptr || ld_bm25 >= n_spans, S3_ERR_INVALID_ARG, "ld_bm25 smaller than n_spans");
+    for (int l = 0; l < n_layers; ++l)
+        S3_REQUIRE(h_layers[l].d_row_ptr && (h_layers[l].d_pos || n_spans == 0), S3_ERR_INVALID_ARG, "layer %d: null CSR pointer", l);
+    return launch_score(h_layers, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, (int)n_spans, p, d_bm25, ld_bm25, d_top_idx,
+                        d_top_score, d_all_scores, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,512 @@
+// bf16 SAE encode + ReLU + running Top-k (Sec. 3.3, Eq. 1-2) on the sm_100a tensor cores.
+//
+//   pre[t,f] = sum_i x[t,i] * W_enc[i,f] + b_eff[f],   b_eff = b_enc - W_enc^T b_dec   (folded once)
+//
+// Persistent, warp-specialised kernel, one CTA per SM:
+//   warp 0      TMA producer: streams 128x64 tiles of x and 256x64 tiles of W_enc^T (K-major, 128-byte
+//               swizzle) into a ring of shared-memory stages, completion on mbarriers;
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 x bf16 -> fp32) into
+//               one of two 128x256 accumulators in tensor memory, tcgen05.commit frees the stage /
+//               publishes the accumulator;
+//   warps 2-5   epilogue: thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
+//               biased, filtered against the row's current k-th best value, survivors are parked in a
+//               per-thread shared-memory strip and then folded into the row's heap in lock-step, so a
+//               warp pays for the busiest lane of a batch, not for every lane's hit separately.
+// A work unit is (128-token block, slice of 256-column tiles); the accumulator ring keeps the tensor
+// pipe busy with tile n+1 while the epilogue filters tile n. Only the k survivors per (token, slice)
+// leave the SM (as 64-bit keys); the pre-activation matrix is never written to memory.
+//
+// Every mbarrier wait is bounded; a wait that runs out records which one in the workspace status
+// word, raises a CTA-wide abort flag, and the CTA drains its own TMA copies, frees its tensor memory
+// and exits.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "s3_encode_tc.cuh"
+#include "s3_topk.cuh"
+
+namespace s3 {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
+constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
+constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KB
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int NUM_THREADS = 192;
+constexpr int EPI_THREADS = 128;
+constexpr int TMEM_COLS = 512;
+constexpr int BATCH = 32;                    // columns per tcgen05.ld
+constexpr int HALF = 16;                     // columns filtered between two heap drains (strip depth)
+constexpr uint32_t WAIT_LIMIT = 1u << 26;    // try_wait polls before a wait is declared dead (~1 s)
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait. Returns false if the wait ran out or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag)
+{
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 1023u) == 1023u && *abort_flag) return false;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+// Named barrier 1 over the 128 epilogue threads with an AND-reduction of `pred`.
+__device__ __forceinline__ bool epi_all(bool pred)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(static_cast<uint32_t>(pred)), "n"(128)
+        : "memory");
+    return out != 0;
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte rows, 128-byte swizzle, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr >> 4) & 0x3FFFu);        // start address
+    d |= static_cast<uint64_t>(1) << 16;                        // leading byte offset (unused for swizzled K-major)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= static_cast<uint64_t>(1) << 46;                        // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;                        // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128.
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
+                                (static_cast<uint32_t>(BM >> 4) << 24);
+
+struct EncodeTcParams {
+    int T, d_in, d_sae, k;
+    int n_mtiles, n_col_tiles, n_slices, n_units, n_stages;
+    const float* b_eff;
+    uint64_t* part;
+    uint32_t* status;
+};
+
+// Shared-memory carve-up (all offsets from a 1024-byte aligned base).
+struct SmemLayout {
+    uint32_t a_off, b_off, heap_off, strip_off, bias_off, bar_off, total;
+};
+__host__ __device__ inline SmemLayout smem_layout(int n_stages, int k)
+{
+    SmemLayout L;
+    L.a_off = 0;
+    L.b_off = L.a_off + n_stages * A_STAGE_BYTES;
+    L.heap_off = L.b_off + n_stages * B_STAGE_BYTES;
+    L.strip_off = L.heap_off + k * EPI_THREADS * 8;
+    L.bias_off = L.strip_off + HALF * EPI_THREADS * 4;
+    L.bar_off = L.bias_off + 2 * BN * 4;
+    L.total = L.bar_off + (2 * n_stages + 4) * 8 + 16;
+    return L;
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                 const EncodeTcParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const SmemLayout L = smem_layout(p.n_stages, p.k);
+    unsigned char* smem_a = smem + L.a_off;
+    unsigned char* smem_b = smem + L.b_off;
+    uint64_t* heap = reinterpret_cast<uint64_t*>(smem + L.heap_off);
+    float* strip = reinterpret_cast<float*>(smem + L.strip_off);
+    float* bias_s = reinterpret_cast<float*>(smem + L.bias_off);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L.bar_off);
+    uint64_t* empty_bar = full_bar + p.n_stages;
+    uint64_t* acc_full = empty_bar + p.n_stages;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kblocks = (p.d_in + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.n_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_THREADS); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
+            uint32_t stage = 0, phase = 0;
+            uint64_t issued = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+                const int slice = u / p.n_mtiles, mt = u - slice * p.n_mtiles;
+                const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
+                const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
+                for (int nt = tile_lo; nt < tile_hi && ok; ++nt) {
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag)) {
+                            dev_set_error(p.status, DEV_TIMEOUT_SMEM_EMPTY);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
+                        tma_load_2d(smem_a + stage * A_STAGE_BYTES, &map_x, kb * BK, mt * BM, &full_bar[stage]);
+                        tma_load_2d(smem_b + stage * B_STAGE_BYTES, &map_w, kb * BK, nt * BN, &full_bar[stage]);
+                        ++issued;
+                        if (++stage == static_cast<uint32_t>(p.n_stages)) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            // Own copies still in flight: wait (bounded) until the last n_stages loads have landed.
+            const uint64_t back = issued < static_cast<uint64_t>(p.n_stages) ? issued : static_cast<uint64_t>(p.n_stages);
+            uint32_t s = stage, ph = phase;
+            for (uint64_t i = 0; i < back; ++i) {
+                if (s == 0) { s = p.n_stages - 1; ph ^= 1u; } else { --s; }
+                for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
+                    if (mbar_try_wait(&full_bar[s], ph)) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t tile_count = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+                const int slice = u / p.n_mtiles;
+                const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
+                const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
+                for (int nt = tile_lo; nt < tile_hi && ok; ++nt, ++tile_count) {
+                    const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+                    if (!mbar_wait(&acc_empty[ab], acc_phase ^ 1u, abort_flag)) {
+                        dev_set_error(p.status, DEV_TIMEOUT_ACC_EMPTY);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + ab * BN;
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (!mbar_wait(&full_bar[stage], phase, abort_flag)) {
+                            dev_set_error(p.status, DEV_TIMEOUT_TMA_FULL);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint64_t da = make_smem_desc(smem_u32(smem_a + stage * A_STAGE_BYTES));
+                        const uint64_t db = make_smem_desc(smem_u32(smem_b + stage * B_STAGE_BYTES));
+#pragma unroll
+                        for (int kk = 0; kk < BK / UMMA_K; ++kk)
+                            tc_mma_bf16(d_tmem, da + static_cast<uint64_t>(kk * 2), db + static_cast<uint64_t>(kk * 2), kInstrDesc,
+                                        (kb | kk) != 0 ? 1u : 0u);
+                        tc_commit(&empty_bar[stage]);
+                        if (++stage == static_cast<uint32_t>(p.n_stages)) { stage = 0; phase ^= 1u; }
+                    }
+                    if (ok) tc_commit(&acc_full[ab]);
+                }
+            }
+        }
+    } else {
+        // ---------------- epilogue: bias + ReLU + running Top-k ----------------
+        const int quarter = warp & 3;               // TMEM lanes this warp may read
+        const int e = quarter * 32 + lane;          // row inside the 128-token block
+        const int et = threadIdx.x - 64;            // 0..127, used only to spread the bias loads
+        uint32_t tile_count = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+            const int slice = u / p.n_mtiles, mt = u - slice * p.n_mtiles;
+            const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
+            const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
+            heap_init<EPI_THREADS>(heap, e, p.k);
+            float tau = 0.0f;
+            for (int nt = tile_lo; nt < tile_hi && ok; ++nt, ++tile_count) {
+                const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+                float* bias = bias_s + ab * BN;
+                for (int c = et; c < BN; c += EPI_THREADS) {
+                    const int col = nt * BN + c;
+                    bias[c] = (col < p.d_sae) ? p.b_eff[col] : -INFINITY;
+                }
+                const bool arrived = mbar_wait(&acc_full[ab], acc_phase, abort_flag);
+                if (!arrived) {
+                    dev_set_error(p.status, DEV_TIMEOUT_ACC_FULL);
+                    *abort_flag = 1;
+                }
+                // One barrier both publishes the bias tile and makes the go/no-go decision uniform
+                // across the four epilogue warps, so none of them can be left behind at it.
+                if (!epi_all(arrived)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ab * BN + (static_cast<uint32_t>(quarter * 32) << 16);
+#pragma unroll 1
+                for (int cb = 0; cb < BN / BATCH; ++cb) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + cb * BATCH, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int h = 0; h < BATCH / HALF; ++h) {
+                        uint32_t mask = 0;
+                        int cnt = 0;
+#pragma unroll
+                        for (int j = 0; j < HALF; ++j) {
+                            const float v = __uint_as_float(r[h * HALF + j]) + bias[cb * BATCH + h * HALF + j];
+                            if (v > tau) {
+                                strip[cnt * EPI_THREADS + e] = v;
+                                ++cnt;
+                                mask |= 1u << j;
+                            }
+                        }
+                        const int nmax = __reduce_max_sync(0xffffffffu, cnt);
+                        const int col0 = nt * BN + cb * BATCH + h * HALF;
+                        for (int i = 0; i < nmax; ++i) {
+                            if (i < cnt) {
+                                const float v = strip[i * EPI_THREADS + e];
+                                const int j = __ffs(mask) - 1;
+                                mask &= mask - 1;
+                                if (v > tau) {
+                                    const uint64_t root = heap_replace_root<EPI_THREADS>(
+                                        heap, e, p.k, make_key(__float_as_uint(v), static_cast<uint32_t>(col0 + j)));
+                                    tau = __uint_as_float(static_cast<uint32_t>(root >> 32));
+                                }
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(&acc_empty[ab]);
+            }
+            if (ok) {
+                const int t = mt * BM + e;
+                if (t < p.T) {
+                    uint64_t* dst = p.part + (static_cast<size_t>(t) * p.n_slices + slice) * p.k;
+                    for (int j = 0; j < p.k; ++j) dst[j] = heap[j * EPI_THREADS + e];
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- one-time preparation ---------------------------------------------------------------------------
+// W_enc [d_in, d_sae] (feature = column) -> W_t [d_sae, d_in] so that both GEMM operands are K-major.
+__global__ void transpose_bf16_kernel(const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ Wt, int d_in, int d_sae)
+{
+    __shared__ __nv_bfloat16 tile[32][33];
+    const int f0 = blockIdx.x * 32, i0 = blockIdx.y * 32;
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int i = i0 + r, f = f0 + threadIdx.x;
+        tile[r][threadIdx.x] = (i < d_in && f < d_sae) ? W[static_cast<size_t>(i) * d_sae + f] : __float2bfloat16(0.0f);
+    }
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int f = f0 + r, i = i0 + threadIdx.x;
+        if (f < d_sae && i < d_in) Wt[static_cast<size_t>(f) * d_in + i] = tile[threadIdx.x][r];
+    }
+}
+
+// b_eff[f] = b_enc[f] - sum_i W_enc[i,f] * b_dec[i], summed in fp64 in index order, stored as fp32.
+__global__ void folded_bias_kernel(const __nv_bfloat16* __restrict__ W, const float* __restrict__ b_enc,
+                                   const float* __restrict__ b_dec, int d_in, int d_sae, float* __restrict__ b_eff)
+{
+    const int f = blockIdx.x * blockDim.x + threadIdx.x;
+    if (f >= d_sae) return;
+    double s = 0.0;
+    for (int i = 0; i < d_in; ++i)
+        s += static_cast<double>(__bfloat162float(W[static_cast<size_t>(i) * d_sae + f])) * static_cast<double>(b_dec[i]);
+    b_eff[f] = static_cast<float>(static_cast<double>(b_enc[f]) - s);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+s3_status get_encode_fn(EncodeTiledFn* out)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        S3_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres));
+        S3_REQUIRE(sym != nullptr && qres == cudaDriverEntryPointSuccess, S3_ERR_CUDA,
+                   "the driver does not provide cuTensorMapEncodeTiled");
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    *out = fn;
+    return S3_OK;
+}
+
+// 2-D bf16 tensor [rows, cols] with row pitch ld (elements); box = box_rows x 64 columns, 128-byte swizzle.
+s3_status make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows)
+{
+    EncodeTiledFn fn;
+    const s3_status st = get_encode_fn(&fn);
+    if (st != S3_OK) return st;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {ld * 2};
+    const cuuint32_t box[2] = {BK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    S3_REQUIRE(r == CUDA_SUCCESS, S3_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d (rows %llu cols %llu ld %llu)",
+               static_cast<int>(r), static_cast<unsigned long long>(rows), static_cast<unsigned long long>(cols),
+               static_cast<unsigned long long>(ld));
+    return S3_OK;
+}
+
+}  // namespace
+
+size_t encode_tc_prepared_bytes(int d_in, int d_sae)
+{
+    return round_up(static_cast<size_t>(d_sae) * d_in * 2, 256) + round_up(static_cast<size_t>(d_sae) * 4, 256);
+}
+
+s3_status encode_tc_prepare(EncodeTcState* st, const void* d_W, const float* d_b_enc, const float* d_b_dec, int d_in,
+                            int d_sae, void* d_prepared, cudaStream_t stream)
+{
+    st->d_wt = d_prepared;
+    st->d_b_eff = reinterpret_cast<float*>(static_cast<unsigned char*>(d_prepared) +
+                                           round_up(static_cast<size_t>(d_sae) * d_in * 2, 256));
+    const dim3 tb(32, 8), tg((d_sae + 31) / 32, (d_in + 31) / 32);
+    transpose_bf16_kernel<<<tg, tb, 0, stream>>>(static_cast<const __nv_bfloat16*>(d_W),
+                                                 static_cast<__nv_bfloat16*>(st->d_wt), d_in, d_sae);
+    S3_CUDA_TRY(cudaGetLastError());
+    folded_bias_kernel<<<(d_sae + 127) / 128, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(d_W), d_b_enc, d_b_dec, d_in,
+                                                                d_sae, st->d_b_eff);
+    S3_CUDA_TRY(cudaGetLastError());
+    static_assert(sizeof(CUtensorMap) <= sizeof(st->map_w), "tensor map storage too small");
+    return make_map(reinterpret_cast<CUtensorMap*>(st->map_w), st->d_wt, d_sae, d_in, d_in, BN);
+}
+
+int encode_tc_col_tiles(int d_sae) { return (d_sae + BN - 1) / BN; }
+int encode_tc_row_tiles(int T) { return (T + BM - 1) / BM; }
+
+s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
+                           int n_slices, int max_ctas, uint64_t* d_part, uint32_t* d_status, cudaStream_t stream)
+{
+    alignas(64) CUtensorMap map_x;
+    s3_status rc = make_map(&map_x, d_x, static_cast<uint64_t>(T), static_cast<uint64_t>(d_in), static_cast<uint64_t>(ldx), BM);
+    if (rc != S3_OK) return rc;
+
+    EncodeTcParams p;
+    p.T = T; p.d_in = d_in; p.d_sae = d_sae; p.k = k;
+    p.n_mtiles = encode_tc_row_tiles(T);
+    p.n_col_tiles = encode_tc_col_tiles(d_sae);
+    p.n_slices = n_slices;
+    p.n_units = p.n_mtiles * n_slices;
+    p.b_eff = st->d_b_eff;
+    p.part = d_part;
+    p.status = d_status;
+
+    int dev = 0;
+    S3_CUDA_TRY(cudaGetDevice(&dev));
+    int max_smem = 0;
+    S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    int n_stages = 6;
+    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, k).total) + 1024 > max_smem) --n_stages;
+    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, k).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
+               "shared memory too small for the encode pipeline (k = %d)", k);
+    p.n_stages = n_stages;
+    const size_t smem = smem_layout(n_stages, k).total + 1024;
+    static bool attr_set[64] = {};
+    if (dev < 64 && !attr_set[dev]) {
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        attr_set[dev] = true;
+    }
+    int grid = device_sm_count();
+    if (max_ctas > 0 && max_ctas < grid) grid = max_ctas;
+    if (p.n_units < grid) grid = p.n_units;
+    encode_tc_kernel<<<grid, NUM_THREADS, smem, stream>>>(map_x, *reinterpret_cast<const CUtensorMap*>(st->map_w), p);
+    S3_CUDA_TRY(cudaGetLastError());
+    return S3_OK;
+}
+
+}  // namespace s3

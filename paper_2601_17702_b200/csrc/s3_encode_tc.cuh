@@ -1,0 +1,36 @@
+// Host-side interface of the tensor-core (bf16) and FP32-pipe encode kernels.
+#pragma once
+
+#include "s3_common.cuh"
+
+namespace s3 {
+
+struct EncodeTcState {
+    void* d_wt = nullptr;        // W_enc^T [d_sae, d_in] bf16 inside the caller's prepared buffer
+    float* d_b_eff = nullptr;    // folded bias [d_sae]
+    alignas(64) unsigned char map_w[128];   // TMA descriptor of W_enc^T
+};
+
+size_t encode_tc_prepared_bytes(int d_in, int d_sae);
+s3_status encode_tc_prepare(EncodeTcState* st, const void* d_W, const float* d_b_enc, const float* d_b_dec, int d_in,
+                            int d_sae, void* d_prepared, cudaStream_t stream);
+int encode_tc_col_tiles(int d_sae);
+int encode_tc_row_tiles(int T);
+s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
+                           int n_slices, int max_ctas, uint64_t* d_part, uint32_t* d_status, cudaStream_t stream);
+
+size_t encode_simt_smem_bytes(int k);
+int encode_simt_col_tiles(int d_sae);
+int encode_simt_row_tiles(int T);
+s3_status launch_encode_simt(const float* d_x, int64_t ldx, const float* d_W, const float* d_b_enc,
+                             const float* d_b_dec, int T, int d_in, int d_sae, int k, int n_slices,
+                             uint64_t* d_part, cudaStream_t stream);
+
+s3_status launch_postings(const s3_postings_item* h_items, int n_items, uint32_t* d_status, cudaStream_t stream);
+
+s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
+                       const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
+                       const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
+                       float* d_all_scores, cudaStream_t stream);
+
+}  // namespace s3
