@@ -1,0 +1,85 @@
+"""Host driver loop of the streaming scan (Algorithm 1, Phase 1): per context chunk and target layer,
+encode the transient key (and optionally query) projections, build the chunk's CSR postings and hand
+them to the host-resident index. It only sequences calls of the C ABI on torch-owned buffers; device
+memory is allocated once, for one chunk, and reused for every chunk of the context."""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class SaeSlot:
+    """One SAE stream of the scan (e.g. 'key' or 'query'): per-layer encoders plus the chunk-sized
+    device buffers its outputs go through."""
+
+    def __init__(self, name: str, saes: list[B.Sae], k: int, chunk: int, with_values: bool = False):
+        self.name, self.saes, self.k, self.chunk = name, saes, k, chunk
+        dev = saes[0].W_enc.device
+        self.d_sae = saes[0].d_sae
+        n_layers = len(saes)
+        self.ids = [torch.empty((chunk, k), dtype=torch.int32, device=dev) for _ in range(n_layers)]
+        self.vals = [torch.empty((chunk, k), dtype=torch.float32, device=dev) for _ in range(n_layers)]
+        self.row_ptr = [torch.zeros(self.d_sae + 1, dtype=torch.int32, device=dev) for _ in range(n_layers)]
+        self.pos = [torch.zeros(chunk * k, dtype=torch.int32, device=dev) for _ in range(n_layers)]
+        self.pval = [torch.zeros(chunk * k, dtype=torch.float32, device=dev) for _ in range(n_layers)] if with_values else None
+        self.ws = B.new_workspace(max(s.encode_workspace_bytes(chunk, k) for s in saes), dev)
+        self.index = B.Index(n_layers, self.d_sae)
+
+
+class ScanPipeline:
+    def __init__(self, slots: list[SaeSlot]):
+        self.slots = slots
+        self.n_layers = len(slots[0].saes)
+        self.ws_post = B.new_workspace(B.S3_WS_HEADER_BYTES, slots[0].ids[0].device)
+        self.launches = 0          # kernels of this library enqueued so far
+
+    def reserve_index(self, n_tokens: int):
+        for s in self.slots:
+            per_layer = n_tokens * s.k * (8 if s.pval else 4) + (n_tokens // s.chunk + 2) * (s.d_sae + 1 + 64) * 4
+            s.index.reserve(per_layer * self.n_layers + (1 << 20))
+
+    def scan_chunk(self, pos_base: int, x_by_slot: dict[str, list[torch.Tensor]]):
+        """x_by_slot[name][layer] is the [T, d_in] projection of this chunk for that SAE stream."""
+        items = []
+        T = None
+        for s in self.slots:
+            xs = x_by_slot[s.name]
+            for l in range(self.n_layers):
+                x = xs[l]
+                T = x.shape[0]
+                B.s3_sae_encode_topk(s.saes[l], x, s.k, s.ids[l][:T], s.vals[l][:T], s.ws)
+                self.launches += 2
+                items.append(B.make_postings_item(s.ids[l][:T], s.d_sae, pos_base, s.row_ptr[l], s.pos[l],
+                                                  s.vals[l][:T] if s.pval else None, s.pval[l] if s.pval else None))
+        # the previous chunk's device->host copies read row_ptr/pos: order the overwrite after them
+        for s in self.slots:
+            s.index.stream_wait()
+        for i in range(0, len(items), 32):
+            B.s3_postings_build_batched(items[i:i + 32], self.ws_post)
+            self.launches += 1
+        for s in self.slots:
+            for l in range(self.n_layers):
+                s.index.append(l, s.row_ptr[l], s.pos[l], T, s.k, pos_base, s.pval[l] if s.pval else None)
+
+    def finish(self):
+        for s in self.slots:
+            s.index.sync()
+            code = B.s3_workspace_status(s.ws)
+            assert code == 0
+        assert B.s3_workspace_status(self.ws_post) == 0
+
+    def close(self):
+        for s in self.slots:
+            s.index.close()
+
+
+def stage_index_on_device(index: B.Index, device) -> list[tuple[torch.Tensor, torch.Tensor]]:
+    """Merged per-layer CSRs of a host index, uploaded for retrieval."""
+    out = []
+    for l in range(index.n_layers):
+        rp, ps, _ = index.export_csr(l)
+        if ps.numel() == 0:
+            ps = torch.zeros(1, dtype=torch.int32)
+        out.append((rp.to(device), ps.to(device)))
+    return out
