@@ -47,7 +47,7 @@ def load_peaks():
 
 class ClockSampler:
     """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
@@ -58,7 +58,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -66,9 +66,9 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -78,8 +78,10 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            f = [v.strip() for v in ln.split(",")]
+        for ts, ln in self.lines:
+            if t_begin is not None and not (t_begin <= ts <= t_end + 0.06):
+                continue
+            f = [v.strip() for v in ln.split(",")][1:]
             if len(f) < 7:
                 continue
             try:
@@ -176,17 +178,18 @@ def run_ours(args, rank, world, local_rank):
             torch.distributed.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    if rank == 0:
+        sampler.start()
     # ---- device-resident timing (inputs already in HBM)
     for i in range(args.warmup):
         step(i, xk[i % n_distinct], xq[i % n_distinct])
     barrier()
     torch.cuda.reset_peak_memory_stats()
     mem_after_warm = torch.cuda.memory_allocated()
-    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
-                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
-    if rank == 0:
-        sampler.start()
     l0 = pipe.launches + launches[0]
+    wall0 = time.time()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for j in range(args.steps):
@@ -195,7 +198,7 @@ def run_ours(args, rank, world, local_rank):
     t1.record()
     barrier()
     ms = t0.elapsed_time(t1)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(wall0, time.time()) if rank == 0 else None
     gpu_launches = pipe.launches + launches[0] - l0
     peak_mem = torch.cuda.max_memory_allocated()
     enc_ms = [a.elapsed_time(b) for a, b in enc_events]
@@ -327,10 +330,73 @@ def run_reference(args, cpu_only_sample=None):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
+# ------------------------------------------------------------------------------------------ single-kernel cases
+
+def run_case(args):
+    """Runs ONE kernel of the path a few times on a small, L2-exceeding case and prints its event-timed
+    duration: the command line that the ncu captures under profiles/ were taken with."""
+    import paper_2601_17702_b200 as S
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = C.CFG3
+    inp = C.ScanInputs(cfg, device=dev)
+    reps = args.steps
+    out = {"case": args.case, "reps": reps}
+    if args.case in ("encode_key", "encode_query", "encode_retrieval"):
+        which = "query" if args.case == "encode_query" else "key"
+        shp = cfg.query if which == "query" else cfg.key
+        k = C.CFG4.kq if args.case == "encode_retrieval" else shp.k
+        T = args.tokens or (C.CFG4.Q * C.CFG4.nq if args.case == "encode_retrieval" else cfg.chunk)
+        sae = S.Sae(*inp.sae(which, 0))
+        sae.set_schedule(args.slices, args.max_ctas)
+        xs = [inp.x(which, 0, c * T, T) for c in range(2)]
+        ids = torch.empty((T, k), dtype=torch.int32, device=dev)
+        vals = torch.empty((T, k), dtype=torch.float32, device=dev)
+        ws = S.new_workspace(sae.encode_workspace_bytes(T, k), dev)
+        run = lambda i: S.s3_sae_encode_topk(sae, xs[i % 2], k, ids, vals, ws)
+        out.update(T=T, d_in=shp.d_in, d_sae=shp.d_sae, k=k, flop=2.0 * T * shp.d_in * shp.d_sae)
+    elif args.case == "postings":
+        n_items, T, k, D = args.items, cfg.chunk, cfg.query.k, cfg.query.d_sae
+        g = torch.Generator(device=dev).manual_seed(1)
+        idss = [torch.rand((T, D), device=dev, generator=g).topk(k, dim=1).indices.to(torch.int32) for _ in range(n_items)]
+        rps = [torch.zeros(D + 1, dtype=torch.int32, device=dev) for _ in range(n_items)]
+        pss = [torch.zeros(T * k, dtype=torch.int32, device=dev) for _ in range(n_items)]
+        items = [S.make_postings_item(idss[i], D, 0, rps[i], pss[i]) for i in range(n_items)]
+        ws = S.new_workspace(64, dev)
+
+        def run(i):
+            for j in range(0, n_items, 32):
+                S.s3_postings_build_batched(items[j:j + 32], ws)
+        out.update(items=n_items, T=T, k=k, d_sae=D, bytes=n_items * (T * k * 8 + (D + 1) * 4))
+    else:
+        raise SystemExit(f"unknown case {args.case}")
+    for i in range(2):
+        run(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        run(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    out["ms"] = ms
+    if "flop" in out:
+        out["tflops"] = out["flop"] / ms / 1e9
+    if "bytes" in out:
+        out["gbs"] = out["bytes"] / ms / 1e6
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings")
+    ap.add_argument("--tokens", type=int, default=0)
+    ap.add_argument("--slices", type=int, default=0)
+    ap.add_argument("--max-ctas", type=int, default=0)
+    ap.add_argument("--items", type=int, default=8)
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--steps", type=int, default=48)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -339,6 +405,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
+    if args.case:
+        if rank == 0:
+            run_case(args)
+        return
     if args.impl == "reference":
         if rank == 0:
             print(json.dumps(run_reference(args)), flush=True)

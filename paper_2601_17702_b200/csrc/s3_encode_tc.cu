@@ -9,9 +9,11 @@
 //               one of two 128x256 accumulators in tensor memory, tcgen05.commit frees the stage /
 //               publishes the accumulator;
 //   warps 2-5   epilogue: thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
-//               biased, filtered against the row's current k-th best value, survivors are parked in a
-//               per-thread shared-memory strip and then folded into the row's heap in lock-step, so a
-//               warp pays for the busiest lane of a batch, not for every lane's hit separately.
+//               biased and filtered against a lower bound of the row's k-th best value. Survivors are
+//               only appended to a small per-thread pending list in shared memory (a predicated store);
+//               when some lane's list fills up, all lanes fold their lists into their heaps in
+//               lock-step, which raises the bounds. Appends are cheap and the expensive heap updates
+//               run with most lanes busy instead of once per stray hit.
 // A work unit is (128-token block, slice of 256-column tiles); the accumulator ring keeps the tensor
 // pipe busy with tile n+1 while the epilogue filters tile n. Only the k survivors per (token, slice)
 // leave the SM (as 64-bit keys); the pre-activation matrix is never written to memory.
@@ -37,7 +39,7 @@ constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr int TMEM_COLS = 512;
 constexpr int BATCH = 32;                    // columns per tcgen05.ld
-constexpr int HALF = 16;                     // columns filtered between two heap drains (strip depth)
+constexpr int HALF = 16;                     // columns filtered between two checks of the pending lists
 constexpr uint32_t WAIT_LIMIT = 1u << 26;    // try_wait polls before a wait is declared dead (~1 s)
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -151,7 +153,7 @@ constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cas
 
 struct EncodeTcParams {
     int T, d_in, d_sae, k;
-    int n_mtiles, n_col_tiles, n_slices, n_units, n_stages;
+    int n_mtiles, n_col_tiles, n_slices, n_units, n_stages, pend_cap;
     const float* b_eff;
     uint64_t* part;
     uint32_t* status;
@@ -159,33 +161,57 @@ struct EncodeTcParams {
 
 // Shared-memory carve-up (all offsets from a 1024-byte aligned base).
 struct SmemLayout {
-    uint32_t a_off, b_off, heap_off, strip_off, bias_off, bar_off, total;
+    uint32_t a_off, b_off, heap_off, pend_off, bar_off, total;
 };
-__host__ __device__ inline SmemLayout smem_layout(int n_stages, int k)
+// kp = heap slots per row (k rounded up to 8/16/32/64), pend_cap = pending-list slots per row.
+__host__ __device__ inline SmemLayout smem_layout(int n_stages, int kp, int pend_cap)
 {
     SmemLayout L;
     L.a_off = 0;
     L.b_off = L.a_off + n_stages * A_STAGE_BYTES;
     L.heap_off = L.b_off + n_stages * B_STAGE_BYTES;
-    L.strip_off = L.heap_off + k * EPI_THREADS * 8;
-    L.bias_off = L.strip_off + HALF * EPI_THREADS * 4;
-    L.bar_off = L.bias_off + 2 * BN * 4;
+    L.pend_off = L.heap_off + kp * EPI_THREADS * 8;
+    L.bar_off = L.pend_off + pend_cap * EPI_THREADS * 8;
     L.total = L.bar_off + (2 * n_stages + 4) * 8 + 16;
     return L;
 }
 
+// Row-private min-heap with a compile-time number of slots KP (stride EPI_THREADS between slots).
+// Slots k..KP-1 hold the all-ones sentinel, which never leaves the bottom of the heap.
+template <int KP>
+__device__ __forceinline__ uint64_t heap_replace_root_fixed(uint64_t* h, uint64_t key)
+{
+    int i = 0;
+#pragma unroll
+    for (int lvl = 0; lvl < 7; ++lvl) {
+        const int c = 2 * i + 1;
+        if (c >= KP) break;
+        uint64_t kc = h[c * EPI_THREADS];
+        int cc = c;
+        if (c + 1 < KP) {
+            const uint64_t k2 = h[(c + 1) * EPI_THREADS];
+            if (k2 < kc) { kc = k2; cc = c + 1; }
+        }
+        if (kc >= key) break;
+        h[i * EPI_THREADS] = kc;
+        i = cc;
+    }
+    h[i * EPI_THREADS] = key;
+    return h[0];
+}
+
+template <int KP>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const EncodeTcParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const SmemLayout L = smem_layout(p.n_stages, p.k);
+    const SmemLayout L = smem_layout(p.n_stages, KP, p.pend_cap);
     unsigned char* smem_a = smem + L.a_off;
     unsigned char* smem_b = smem + L.b_off;
     uint64_t* heap = reinterpret_cast<uint64_t*>(smem + L.heap_off);
-    float* strip = reinterpret_cast<float*>(smem + L.strip_off);
-    float* bias_s = reinterpret_cast<float*>(smem + L.bias_off);
+    uint64_t* pend = reinterpret_cast<uint64_t*>(smem + L.pend_off);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L.bar_off);
     uint64_t* empty_bar = full_bar + p.n_stages;
     uint64_t* acc_full = empty_bar + p.n_stages;
@@ -294,63 +320,65 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         // ---------------- epilogue: bias + ReLU + running Top-k ----------------
         const int quarter = warp & 3;               // TMEM lanes this warp may read
         const int e = quarter * 32 + lane;          // row inside the 128-token block
-        const int et = threadIdx.x - 64;            // 0..127, used only to spread the bias loads
+        uint64_t* my_heap = heap + e;
+        uint64_t* my_pend = pend + e;
+        const int flush_at = p.pend_cap - HALF;     // fold the lists once a lane holds more than this
         uint32_t tile_count = 0;
         bool ok = true;
         for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
             const int slice = u / p.n_mtiles, mt = u - slice * p.n_mtiles;
             const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
             const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
-            heap_init<EPI_THREADS>(heap, e, p.k);
-            float tau = 0.0f;
+#pragma unroll
+            for (int sl = 0; sl < KP; ++sl) my_heap[sl * EPI_THREADS] = (sl < p.k) ? 0ull : ~0ull;
+            uint64_t root = 0ull;
+            float tau = 0.0f;                       // value of the heap root: a lower bound of the k-th best
+            int cnt = 0;                            // entries in this row's pending list
             for (int nt = tile_lo; nt < tile_hi && ok; ++nt, ++tile_count) {
                 const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
-                float* bias = bias_s + ab * BN;
-                for (int c = et; c < BN; c += EPI_THREADS) {
-                    const int col = nt * BN + c;
-                    bias[c] = (col < p.d_sae) ? p.b_eff[col] : -INFINITY;
-                }
                 const bool arrived = mbar_wait(&acc_full[ab], acc_phase, abort_flag);
                 if (!arrived) {
                     dev_set_error(p.status, DEV_TIMEOUT_ACC_FULL);
                     *abort_flag = 1;
                 }
-                // One barrier both publishes the bias tile and makes the go/no-go decision uniform
-                // across the four epilogue warps, so none of them can be left behind at it.
+                // Make the go/no-go decision uniform across the four epilogue warps.
                 if (!epi_all(arrived)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ab * BN + (static_cast<uint32_t>(quarter * 32) << 16);
+                const float4* bias4 = reinterpret_cast<const float4*>(p.b_eff + static_cast<size_t>(nt) * BN);
 #pragma unroll 1
                 for (int cb = 0; cb < BN / BATCH; ++cb) {
                     uint32_t r[32];
                     tc_ld32(taddr + cb * BATCH, r);
+                    float bias[BATCH];
+#pragma unroll
+                    for (int j4 = 0; j4 < BATCH / 4; ++j4) {
+                        const float4 b4 = __ldg(bias4 + cb * (BATCH / 4) + j4);
+                        bias[4 * j4 + 0] = b4.x; bias[4 * j4 + 1] = b4.y; bias[4 * j4 + 2] = b4.z; bias[4 * j4 + 3] = b4.w;
+                    }
                     tc_wait_ld();
+                    const uint32_t ncol0 = ~static_cast<uint32_t>(nt * BN + cb * BATCH);   // ~(col0 + j) = ncol0 - j
 #pragma unroll
                     for (int h = 0; h < BATCH / HALF; ++h) {
-                        uint32_t mask = 0;
-                        int cnt = 0;
 #pragma unroll
                         for (int j = 0; j < HALF; ++j) {
-                            const float v = __uint_as_float(r[h * HALF + j]) + bias[cb * BATCH + h * HALF + j];
-                            if (v > tau) {
-                                strip[cnt * EPI_THREADS + e] = v;
-                                ++cnt;
-                                mask |= 1u << j;
-                            }
+                            // Branch-free append: the slot after the list is always written and only
+                            // kept (by advancing cnt) when the value beats the bound.
+                            const float v = __uint_as_float(r[h * HALF + j]) + bias[h * HALF + j];
+                            my_pend[cnt * EPI_THREADS] =
+                                (static_cast<uint64_t>(__float_as_uint(v)) << 32) | (ncol0 - static_cast<uint32_t>(h * HALF + j));
+                            cnt += (v > tau) ? 1 : 0;
                         }
-                        const int nmax = __reduce_max_sync(0xffffffffu, cnt);
-                        const int col0 = nt * BN + cb * BATCH + h * HALF;
-                        for (int i = 0; i < nmax; ++i) {
-                            if (i < cnt) {
-                                const float v = strip[i * EPI_THREADS + e];
-                                const int j = __ffs(mask) - 1;
-                                mask &= mask - 1;
-                                if (v > tau) {
-                                    const uint64_t root = heap_replace_root<EPI_THREADS>(
-                                        heap, e, p.k, make_key(__float_as_uint(v), static_cast<uint32_t>(col0 + j)));
-                                    tau = __uint_as_float(static_cast<uint32_t>(root >> 32));
+                        if (__any_sync(0xffffffffu, cnt > flush_at)) {
+                            const int nmax = __reduce_max_sync(0xffffffffu, cnt);
+                            for (int i = 0; i < nmax; ++i) {
+                                if (i < cnt) {
+                                    const uint64_t key = my_pend[i * EPI_THREADS];
+                                    if (key > root) root = heap_replace_root_fixed<KP>(my_heap, key);
                                 }
                             }
+                            cnt = 0;
+                            tau = __uint_as_float(static_cast<uint32_t>(root >> 32));
                         }
                     }
                 }
@@ -358,10 +386,19 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 mbar_arrive(&acc_empty[ab]);
             }
             if (ok) {
+                for (int i = 0; i < cnt; ++i) {     // fold what is still pending (lane-private, no lock-step needed)
+                    const uint64_t key = my_pend[i * EPI_THREADS];
+                    if (key > root) root = heap_replace_root_fixed<KP>(my_heap, key);
+                }
                 const int t = mt * BM + e;
                 if (t < p.T) {
                     uint64_t* dst = p.part + (static_cast<size_t>(t) * p.n_slices + slice) * p.k;
-                    for (int j = 0; j < p.k; ++j) dst[j] = heap[j * EPI_THREADS + e];
+                    int w = 0;
+#pragma unroll 4
+                    for (int sl = 0; sl < KP; ++sl) {
+                        const uint64_t key = my_heap[sl * EPI_THREADS];
+                        if (key != ~0ull && w < p.k) dst[w++] = key;
+                    }
                 }
             }
         }
@@ -393,11 +430,14 @@ __global__ void transpose_bf16_kernel(const __nv_bfloat16* __restrict__ W, __nv_
 }
 
 // b_eff[f] = b_enc[f] - sum_i W_enc[i,f] * b_dec[i], summed in fp64 in index order, stored as fp32.
+// The array is padded to whole 256-column tiles with -inf, which no candidate filter lets through.
 __global__ void folded_bias_kernel(const __nv_bfloat16* __restrict__ W, const float* __restrict__ b_enc,
-                                   const float* __restrict__ b_dec, int d_in, int d_sae, float* __restrict__ b_eff)
+                                   const float* __restrict__ b_dec, int d_in, int d_sae, int d_sae_pad,
+                                   float* __restrict__ b_eff)
 {
     const int f = blockIdx.x * blockDim.x + threadIdx.x;
-    if (f >= d_sae) return;
+    if (f >= d_sae_pad) return;
+    if (f >= d_sae) { b_eff[f] = -INFINITY; return; }
     double s = 0.0;
     for (int i = 0; i < d_in; ++i)
         s += static_cast<double>(__bfloat162float(W[static_cast<size_t>(i) * d_sae + f])) * static_cast<double>(b_dec[i]);
@@ -446,7 +486,8 @@ s3_status make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t c
 
 size_t encode_tc_prepared_bytes(int d_in, int d_sae)
 {
-    return round_up(static_cast<size_t>(d_sae) * d_in * 2, 256) + round_up(static_cast<size_t>(d_sae) * 4, 256);
+    const size_t d_sae_pad = static_cast<size_t>((d_sae + BN - 1) / BN) * BN;
+    return round_up(static_cast<size_t>(d_sae) * d_in * 2, 256) + round_up(d_sae_pad * 4, 256);
 }
 
 s3_status encode_tc_prepare(EncodeTcState* st, const void* d_W, const float* d_b_enc, const float* d_b_dec, int d_in,
@@ -459,8 +500,9 @@ s3_status encode_tc_prepare(EncodeTcState* st, const void* d_W, const float* d_b
     transpose_bf16_kernel<<<tg, tb, 0, stream>>>(static_cast<const __nv_bfloat16*>(d_W),
                                                  static_cast<__nv_bfloat16*>(st->d_wt), d_in, d_sae);
     S3_CUDA_TRY(cudaGetLastError());
-    folded_bias_kernel<<<(d_sae + 127) / 128, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(d_W), d_b_enc, d_b_dec, d_in,
-                                                                d_sae, st->d_b_eff);
+    const int d_sae_pad = (d_sae + BN - 1) / BN * BN;
+    folded_bias_kernel<<<(d_sae_pad + 127) / 128, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(d_W), d_b_enc, d_b_dec, d_in,
+                                                                    d_sae, d_sae_pad, st->d_b_eff);
     S3_CUDA_TRY(cudaGetLastError());
     static_assert(sizeof(CUtensorMap) <= sizeof(st->map_w), "tensor map storage too small");
     return make_map(reinterpret_cast<CUtensorMap*>(st->map_w), st->d_wt, d_sae, d_in, d_in, BN);
@@ -490,21 +532,38 @@ s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx
     S3_CUDA_TRY(cudaGetDevice(&dev));
     int max_smem = 0;
     S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    int n_stages = 6;
-    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, k).total) + 1024 > max_smem) --n_stages;
-    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, k).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
+    const int kp = k <= 8 ? 8 : (k <= 16 ? 16 : (k <= 32 ? 32 : 64));
+    // Prefer three or more pipeline stages; give what is left to the pending lists (16..32 slots).
+    int n_stages = 6, pend_cap = HALF;
+    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, kp, HALF).total) + 1024 > max_smem) --n_stages;
+    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, kp, HALF).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
                "shared memory too small for the encode pipeline (k = %d)", k);
+    if (n_stages > 4) n_stages = 4;
+    for (int cap = 2 * HALF; cap > HALF; cap -= 2)
+        if (static_cast<int>(smem_layout(n_stages, kp, cap).total) + 1024 <= max_smem) { pend_cap = cap; break; }
     p.n_stages = n_stages;
-    const size_t smem = smem_layout(n_stages, k).total + 1024;
-    static bool attr_set[64] = {};
-    if (dev < 64 && !attr_set[dev]) {
-        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
-        attr_set[dev] = true;
-    }
+    p.pend_cap = pend_cap;
+    const size_t smem = smem_layout(n_stages, kp, pend_cap).total + 1024;
     int grid = device_sm_count();
     if (max_ctas > 0 && max_ctas < grid) grid = max_ctas;
     if (p.n_units < grid) grid = p.n_units;
-    encode_tc_kernel<<<grid, NUM_THREADS, smem, stream>>>(map_x, *reinterpret_cast<const CUtensorMap*>(st->map_w), p);
+    const CUtensorMap& map_w = *reinterpret_cast<const CUtensorMap*>(st->map_w);
+    static bool attr_set[64][4] = {};
+#define S3_LAUNCH_ENCODE(KP, SLOT)                                                                                      \
+    do {                                                                                                                \
+        if (dev < 64 && !attr_set[dev][SLOT]) {                                                                         \
+            S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)); \
+            attr_set[dev][SLOT] = true;                                                                                 \
+        }                                                                                                               \
+        encode_tc_kernel<KP><<<grid, NUM_THREADS, smem, stream>>>(map_x, map_w, p);                                     \
+    } while (0)
+    switch (kp) {
+        case 8: S3_LAUNCH_ENCODE(8, 0); break;
+        case 16: S3_LAUNCH_ENCODE(16, 1); break;
+        case 32: S3_LAUNCH_ENCODE(32, 2); break;
+        default: S3_LAUNCH_ENCODE(64, 3); break;
+    }
+#undef S3_LAUNCH_ENCODE
     S3_CUDA_TRY(cudaGetLastError());
     return S3_OK;
 }
