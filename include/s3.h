@@ -98,7 +98,39 @@ s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, in
 s3_status s3_sae_set_schedule(s3_sae* sae, int n_slices, int max_ctas);
 
 /* ------------------------------------------------------------------------------------------------
- * Postings build                                             (paper Sec. 3.4 Eq. 4: I[f] <- I[f] U {t})
+ * SAE encode + ReLU + Top-k without any caller-provided scratch
+ *
+ * (The paper has no counterpart of this call: it exists for the way some programs have to use this
+ *  library, not for the method.)
+ *
+ * Same result as s3_sae_encode_topk, for callers that cannot allocate device memory: a serving
+ * process whose memory pool is sized once and then frozen, a plugin that only ever sees the input
+ * and output buffers its host framework passes in, code that runs while something else owns the
+ * allocator. The partial Top-k lists that s3_sae_encode_topk keeps in the caller's `d_ws` live
+ * here in an array of S3_STATIC_SCRATCH_BYTES bytes built into the library image. Each GPU that
+ * loads the library carries that array until the process exits. The call itself allocates and
+ * frees nothing, on the host side of CUDA or through any library.
+ *
+ *   - Size limit: the call is refused with S3_ERR_CAPACITY when
+ *     s3_sae_encode_workspace_bytes(sae, T, k) > S3_STATIC_SCRATCH_BYTES (for the 16-slice maximum
+ *     that is T*k <= 131071 pairs, e.g. 4095 tokens at k = 32). Split longer inputs by token range.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and remembers it. Make that first call before starting any stream capture.
+ *   - One array per device, shared by every call and keeping the previous call's contents. The
+ *     call clears the 64-byte status block at its start and rewrites the lists it uses, so stale
+ *     contents never reach a result. Two calls whose device work overlaps (different streams or
+ *     threads, same device) race on the array: order them on one stream or with events.
+ *   - d_status_out (device, 4 bytes, nullable) receives the status word of this call on `stream`
+ *     after the kernels: 0, or the code of a bounded wait that ran out (as s3_workspace_status).
+ * Inputs, outputs, alignment rules, dtype rules and asynchrony are those of s3_sae_encode_topk.
+ * ---------------------------------------------------------------------------------------------- */
+#define S3_STATIC_SCRATCH_BYTES (16u << 20)
+s3_status s3_sae_encode_topk_static(const s3_sae* sae, const void* d_x, int64_t ldx, int T, int k,
+                                    int32_t* d_ids /*[T,k]*/, float* d_vals /*[T,k]*/,
+                                    uint32_t* d_status_out /*nullable*/, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Postings build                                       (paper Sec. 3.4 Eq. 4: I[f] <- I[f] U {t})
  *
  * Groups the (feature, position) pairs of one chunk of one layer into a CSR:
  *   row_ptr[f] = number of pairs with id < f  (row_ptr has d_sae + 1 entries, uint32)

@@ -17,11 +17,12 @@ S3_ERR_CAPACITY, S3_ERR_TIMEOUT, S3_ERR_STATE = -5, -6, -7
 S3_BF16, S3_F32 = 0, 1
 S3_SCORE_MINCOUNT, S3_SCORE_WEIGHTED = 0, 1
 S3_WS_HEADER_BYTES = 64
+S3_STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = [
     "s3_last_error", "s3_version", "s3_workspace_status",
     "s3_sae_prepared_bytes", "s3_sae_create", "s3_sae_destroy", "s3_sae_encode_workspace_bytes",
-    "s3_sae_encode_topk", "s3_sae_set_schedule",
+    "s3_sae_encode_topk", "s3_sae_set_schedule", "s3_sae_encode_topk_static",
     "s3_postings_workspace_bytes", "s3_postings_build", "s3_postings_build_batched",
     "s3_index_create", "s3_index_reserve", "s3_index_append", "s3_index_stream_wait", "s3_index_sync",
     "s3_index_stats", "s3_index_layer_postings", "s3_index_export_csr", "s3_index_destroy",
@@ -78,6 +79,8 @@ def lib():
         L.s3_sae_encode_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int]
         L.s3_sae_encode_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_sae_encode_topk_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_void_p,
+                                                C.c_void_p, C.c_void_p, C.c_void_p]
         L.s3_workspace_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
         L.s3_postings_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_postings_build.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_void_p,
@@ -178,6 +181,21 @@ def s3_sae_encode_topk(sae: Sae, x: torch.Tensor, k: int, ids: torch.Tensor, val
     assert tuple(ids.shape) == (T, k) and tuple(vals.shape) == (T, k)
     _check(lib().s3_sae_encode_topk(sae.handle, _ptr(x), x.stride(0) if T > 1 else max(x.stride(0), sae.d_in), T, k,
                                     _ptr(ids), _ptr(vals), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def s3_sae_encode_topk_static(sae: Sae, x: torch.Tensor, k: int, ids: torch.Tensor, vals: torch.Tensor,
+                              status_out: torch.Tensor | None = None, stream=None):
+    """The encode for callers that cannot allocate: same outputs as s3_sae_encode_topk, but the scratch
+    is the fixed array inside the library (S3_STATIC_SCRATCH_BYTES, one per device, shared by all calls),
+    so no workspace is passed. status_out: optional int32/uint32 device tensor (1 element) that receives
+    the call's device status word. Raises S3Error(S3_ERR_CAPACITY) when T*k is too large for the array."""
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1 and x.shape[1] == sae.d_in
+    T = x.shape[0]
+    assert ids.dtype == torch.int32 and vals.dtype == torch.float32 and ids.is_contiguous() and vals.is_contiguous()
+    assert tuple(ids.shape) == (T, k) and tuple(vals.shape) == (T, k)
+    assert status_out is None or (status_out.is_cuda and status_out.element_size() == 4 and status_out.numel() >= 1)
+    _check(lib().s3_sae_encode_topk_static(sae.handle, _ptr(x), x.stride(0) if T > 1 else max(x.stride(0), sae.d_in),
+                                           T, k, _ptr(ids), _ptr(vals), _ptr(status_out), _stream(stream)))
 
 
 def s3_postings_workspace_bytes(T_max: int, k: int, d_sae: int) -> int:
