@@ -362,12 +362,49 @@ def run_case(args):
         rps = [torch.zeros(D + 1, dtype=torch.int32, device=dev) for _ in range(n_items)]
         pss = [torch.zeros(T * k, dtype=torch.int32, device=dev) for _ in range(n_items)]
         items = [S.make_postings_item(idss[i], D, 0, rps[i], pss[i]) for i in range(n_items)]
-        ws = S.new_workspace(64, dev)
+        ws = S.new_workspace(min(n_items, 32) * S.s3_postings_workspace_bytes(T, k, D), dev)
 
         def run(i):
             for j in range(0, n_items, 32):
                 S.s3_postings_build_batched(items[j:j + 32], ws)
         out.update(items=n_items, T=T, k=k, d_sae=D, bytes=n_items * (T * k * 8 + (D + 1) * 4))
+    elif args.case == "score":
+        # retrieval scoring alone: a random index of L tokens (k ids per token out of D features) as one
+        # merged CSR, Q queries of nq tokens with kq ids each; bytes = gathered postings + lexical scores + outputs
+        r = C.CFG4
+        L = args.tokens or r.scan.L
+        k, D = (r.scan.key.k, r.scan.key.d_sae) if not args.tokens else (16, 8192)
+        stride = r.stride if not args.tokens else 64
+        g = torch.Generator(device=dev).manual_seed(1)
+        ids = torch.cat([torch.rand((min(65536, L - t0), D), device=dev, generator=g).topk(k, dim=1).indices.to(torch.int32)
+                         for t0 in range(0, L, 65536)])
+        rp32 = torch.zeros(D + 1, dtype=torch.int32, device=dev)
+        pos = torch.zeros(L * k, dtype=torch.int32, device=dev)
+        step_t = 131072
+        ws = S.new_workspace(S.s3_postings_workspace_bytes(step_t, k, D), dev)
+        ix = S.Index(1, D, 64 << 20)
+        for t0 in range(0, L, step_t):
+            n = min(step_t, L - t0)
+            ix.stream_wait()
+            S.s3_postings_build(ids[t0:t0 + n], D, t0, rp32, pos, ws)
+            ix.append(0, rp32, pos, n, k, t0)
+        rp, ps, _ = ix.export_csr(0)
+        csr = [(rp.to(dev), ps.to(dev))]
+        ix.close()
+        q_ids = torch.rand((r.Q * r.nq, D), device=dev, generator=g).topk(r.kq, dim=1).indices.to(torch.int32).view(1, r.Q, r.nq, r.kq)
+        q_vals = torch.ones(q_ids.shape, dtype=torch.float32, device=dev)
+        ns = C.n_spans(L, r.width, stride)
+        bm25 = G.gamma21(r.bm25_seed, r.Q, ns).to(dev)
+        top_idx = torch.empty((r.Q, r.s), dtype=torch.int32, device=dev)
+        top_score = torch.empty((r.Q, r.s), dtype=torch.float32, device=dev)
+        lens = (csr[0][0][1:] - csr[0][0][:-1])
+        gathered = 0
+        for q in range(r.Q):
+            gathered += int(lens[torch.unique(q_ids[0, q].flatten().long())].sum().item())
+        run = lambda i: S.s3_coactivation_score_topspans(csr, D, L, q_ids, q_vals, r.width, stride, r.s, r.alpha, r.beta, ws,
+                                                         bm25, top_idx=top_idx, top_score=top_score)
+        out.update(L=L, d_sae=D, k=k, Q=r.Q, nq=r.nq, kq=r.kq, spans=ns, stride=stride, gathered_postings=gathered,
+                   index_bytes=int(ps.numel()) * 4, bytes=gathered * 4 + r.Q * ns * 4 + r.Q * r.s * 8)
     else:
         raise SystemExit(f"unknown case {args.case}")
     for i in range(2):
@@ -390,7 +427,7 @@ def run_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings")
+    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)

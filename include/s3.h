@@ -138,10 +138,12 @@ s3_status s3_sae_encode_topk_static(const s3_sae* sae, const void* d_x, int64_t 
  * ids [T,k] int32; entries < 0 are padding and are skipped; ids within a token must be distinct.
  * d_vals / d_pval (both null or both non-null) carry each pair's activation next to its position.
  * d_pos (and d_pval) must hold T*k entries. The result is bit-exact and run-to-run identical.
- * Limits: d_sae <= 49152 (per-feature cursors live in shared memory), T < 2^24,
- *         pos_base + T <= 2^31 - 1 (S3_ERR_CAPACITY: positions are int32). T == 0 writes zeros to row_ptr.
- * The batched form processes up to S3_MAX_POSTINGS_ITEMS independent chunk-layers in one launch;
- * `items` is a HOST array.
+ * Limits: d_sae <= 2^20, k <= 4096, T*k < 2^31, pos_base + T <= 2^31 - 1 (S3_ERR_CAPACITY: positions are
+ *         int32). T == 0 writes zeros to row_ptr.
+ * Workspace: the status block plus a table of per-token-run feature counts;
+ * s3_postings_workspace_bytes(T, k, d_sae) bounds it for one item, and a batch needs the sum of its
+ * items' values. The batched form processes up to S3_MAX_POSTINGS_ITEMS independent chunk-layers in one
+ * sequence of launches; `items` is a HOST array.
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
     const int32_t* d_ids;
@@ -222,7 +224,9 @@ s3_status s3_index_destroy(s3_index* index);
  * `h_layers` is a HOST array of n_layers views whose pointers are DEVICE pointers to one merged CSR
  * per layer (row_ptr uint64 [d_sae+1], pos int32 ascending per feature).
  * Limits: n_layers <= S3_MAX_SCORE_LAYERS; nq*k <= 4096; n_spans <= 16384; s <= 64;
- *         width, stride >= 1.
+ *         width, stride >= 1. Per query the kernel keeps 4 (min-count) or 8 (weighted) bytes per span and
+ *         about 28 bytes per query entry in shared memory; a combination beyond the SM's capacity
+ *         (only weighted mode near both maxima) returns S3_ERR_UNSUPPORTED.
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
     const uint64_t* d_row_ptr;

@@ -217,16 +217,16 @@ s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, in
 // ---------------------------------------------------------------------------------------------- postings
 size_t s3_postings_workspace_bytes(int T_max, int k, int d_sae)
 {
-    (void)T_max; (void)k; (void)d_sae;
-    return S3_WS_HEADER_BYTES;
+    return 256 + postings_workspace_bytes(T_max, k, d_sae);
 }
 
 static s3_status check_item(const s3_postings_item& it, int idx)
 {
     S3_REQUIRE(it.T >= 0 && it.k >= 1 && it.d_sae >= 1, S3_ERR_INVALID_ARG, "item %d: T = %d, k = %d, d_sae = %d out of range", idx, it.T,
                it.k, it.d_sae);
-    S3_REQUIRE(it.d_sae <= 49152, S3_ERR_UNSUPPORTED, "item %d: d_sae = %d exceeds 49152", idx, it.d_sae);
-    S3_REQUIRE((int64_t)it.T * it.k < (1ll << 24), S3_ERR_UNSUPPORTED, "item %d: T*k = %lld must be below 2^24", idx,
+    S3_REQUIRE(it.d_sae <= (1 << 20), S3_ERR_UNSUPPORTED, "item %d: d_sae = %d exceeds 2^20", idx, it.d_sae);
+    S3_REQUIRE(it.k <= 4096, S3_ERR_UNSUPPORTED, "item %d: k = %d exceeds 4096", idx, it.k);
+    S3_REQUIRE((int64_t)it.T * it.k <= INT32_MAX, S3_ERR_UNSUPPORTED, "item %d: T*k = %lld must be below 2^31", idx,
                (long long)it.T * it.k);
     S3_REQUIRE(it.d_row_ptr != nullptr, S3_ERR_INVALID_ARG, "item %d: d_row_ptr is null", idx);
     S3_REQUIRE(it.T == 0 || (it.d_ids && it.d_pos), S3_ERR_INVALID_ARG, "item %d: null device pointer", idx);
@@ -250,7 +250,7 @@ s3_status s3_postings_build_batched(const s3_postings_item* h_items, int n_items
         const s3_status st = check_item(h_items[i], i);
         if (st != S3_OK) return st;
     }
-    return launch_postings(h_items, n_items, static_cast<uint32_t*>(d_ws), static_cast<cudaStream_t>(stream));
+    return launch_postings(h_items, n_items, d_ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 s3_status s3_postings_build(const int32_t* d_ids, const float* d_vals, int T, int k, int d_sae, int64_t pos_base,

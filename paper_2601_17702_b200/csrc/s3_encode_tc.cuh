@@ -26,7 +26,8 @@ s3_status launch_encode_simt(const float* d_x, int64_t ldx, const float* d_W, co
                              const float* d_b_dec, int T, int d_in, int d_sae, int k, int n_slices,
                              uint64_t* d_part, cudaStream_t stream);
 
-s3_status launch_postings(const s3_postings_item* h_items, int n_items, uint32_t* d_status, cudaStream_t stream);
+size_t postings_workspace_bytes(int T, int k, int d_sae);   // table bytes of one item (multiple of 256)
+s3_status launch_postings(const s3_postings_item* h_items, int n_items, void* d_ws, size_t ws_bytes, cudaStream_t stream);
 
 s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
                        const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,

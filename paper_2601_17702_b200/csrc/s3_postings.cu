@@ -1,188 +1,355 @@
 // Per-chunk CSR posting lists (Sec. 3.4, Eq. 4: I[f] <- I[f] U {t} for every f in F_t).
 //
-// One thread block builds one chunk-layer in a single launch, with the per-feature counters /
-// write cursors held in shared memory (4 bytes per feature):
-//   1. histogram of the ids (shared-memory atomics)           -> list lengths
-//   2. exclusive block scan                                   -> row_ptr (global) and cursors (shared)
-//   3. ordered scatter, sub-tile by sub-tile in token order   -> pos (and pval)
-// Step 3 keeps every list in ascending position: a sub-tile is a run of consecutive tokens; inside
-// it each pair takes a ticket from its feature's cursor (the top 8 bits of the cursor word count the
-// sub-tile's tickets, the low 24 bits keep the run start), and pairs that share a feature within
-// the sub-tile then re-rank themselves by position before the final write. Features are distinct
-// within a token, so a feature gets at most one ticket per token and at most 255 per sub-tile.
+// A chunk-layer ("item") is cut into runs of consecutive tokens, one thread block per run, so that a
+// launch over a handful of items still fills the GPU. Four small kernels, all integer, no inter-block
+// waiting:
+//   1. count    block (item, run): histogram of the run's ids in shared memory -> table[run][f]
+//   2. colscan  thread per feature: exclusive prefix of table[.][f] down the runs (in place) and the
+//               feature's total -> row_ptr[f+1]
+//   3. rowscan  block per item: in-place inclusive scan of row_ptr[1..d_sae]
+//   4. scatter  block (item, run): cursor[f] = row_ptr[f] + table[run][f] in shared memory, then the
+//               run's tokens in order, 64 at a time: every pair takes a ticket from its feature's
+//               counter; a feature hit once in the 64 tokens writes straight to cursor[f]; a feature
+//               hit several times records the hitting tokens in a 64-bit mask (small hash table), and
+//               each of its pairs ranks itself by counting the mask bits below its own token.
+// Every list therefore comes out in ascending position whatever the block scheduling, and the result
+// is bit-identical from run to run. Features are handled in ranges of 32768 per pass (one pass for
+// the usual dictionary sizes).
 #include "s3_common.cuh"
+#include "s3_encode_tc.cuh"
 
 namespace s3 {
 
 namespace {
 
-constexpr int PT = 1024;   // threads per block
-constexpr int PER = 4;     // pairs per thread per sub-tile
-constexpr uint32_t LOW24 = 0x00FFFFFFu;
+constexpr int PT = 1024;            // threads per block
+constexpr int PER = 4;              // pairs per thread per sub-tile
+constexpr int SUB_PAIRS = PT * PER; // pairs per sub-tile
+constexpr int SUB_TOK = 64;         // tokens per sub-tile at most (one mask bit each)
+constexpr int RANGE = 32768;        // features per pass
+constexpr int HASH = 4096;          // mask slots (at most SUB_PAIRS/2 features can be hit twice)
+constexpr int MAX_BLOCKS_TOTAL = 1024;
 
-struct PostingsBatch {
+struct PostingsPlan {
     s3_postings_item items[S3_MAX_POSTINGS_ITEMS];
+    unsigned long long table_off[S3_MAX_POSTINGS_ITEMS];   // byte offset of the item's table in the workspace
+    int blk_start[S3_MAX_POSTINGS_ITEMS + 1];              // first block of each item in the flattened grid
+    int tok_per_blk[S3_MAX_POSTINGS_ITEMS];
+    int wide[S3_MAX_POSTINGS_ITEMS];                       // table entries are 32-bit (else 16-bit)
+    int n_items;
+    unsigned char* ws;
+    uint32_t* status;
 };
 
-__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* warp_sums, uint32_t& total)
+__device__ __forceinline__ int find_item(const PostingsPlan& pl, int blk)
 {
+    int it = 0;
+    while (it + 1 < pl.n_items && blk >= pl.blk_start[it + 1]) ++it;
+    return it;
+}
+
+__device__ __forceinline__ uint32_t table_get(const unsigned char* tab, bool wide, size_t idx)
+{
+    return wide ? reinterpret_cast<const uint32_t*>(tab)[idx] : reinterpret_cast<const uint16_t*>(tab)[idx];
+}
+__device__ __forceinline__ void table_put(unsigned char* tab, bool wide, size_t idx, uint32_t v)
+{
+    if (wide) reinterpret_cast<uint32_t*>(tab)[idx] = v;
+    else reinterpret_cast<uint16_t*>(tab)[idx] = static_cast<uint16_t>(v);
+}
+
+// ---- 1. per-run histograms -------------------------------------------------------------------------
+__global__ void __launch_bounds__(PT)
+postings_count_kernel(const __grid_constant__ PostingsPlan pl)
+{
+    extern __shared__ uint32_t hist[];       // [min(d_sae, RANGE)]
+    const int item = find_item(pl, blockIdx.x);
+    const s3_postings_item& it = pl.items[item];
+    const int run = blockIdx.x - pl.blk_start[item];
+    const int tid = threadIdx.x;
+    const int d_sae = it.d_sae, k = it.k;
+    const int t_lo = run * pl.tok_per_blk[item];
+    const int t_hi = min(it.T, t_lo + pl.tok_per_blk[item]);
+    const int64_t p_lo = (int64_t)t_lo * k, p_hi = (int64_t)t_hi * k;
+    const int32_t* __restrict__ ids = it.d_ids;
+    unsigned char* tab = pl.ws + pl.table_off[item];
+    const bool wide = pl.wide[item] != 0;
+
+    for (int f0 = 0; f0 < d_sae; f0 += RANGE) {
+        const int nf = min(RANGE, d_sae - f0);
+        for (int f = tid; f < nf; f += PT) hist[f] = 0;
+        __syncthreads();
+        for (int64_t p = p_lo + tid; p < p_hi; p += PT) {
+            const int32_t f = __ldg(ids + p);
+            if (f >= 0) {
+                if (f >= d_sae) { if (f0 == 0) dev_set_error(pl.status, DEV_BAD_FEATURE_ID); }
+                else if (f >= f0 && f < f0 + nf) atomicAdd(&hist[f - f0], 1u);
+            }
+        }
+        __syncthreads();
+        for (int f = tid; f < nf; f += PT) table_put(tab, wide, (size_t)run * d_sae + f0 + f, hist[f]);
+        __syncthreads();
+    }
+}
+
+// ---- 2. per-feature prefix over the runs ---------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+postings_colscan_kernel(const __grid_constant__ PostingsPlan pl, int max_tiles)
+{
+    const int item = blockIdx.y;
+    const s3_postings_item& it = pl.items[item];
+    const int f = blockIdx.x * 256 + threadIdx.x;
+    if (blockIdx.x >= max_tiles || f >= it.d_sae) return;
+    const int n_runs = pl.blk_start[item + 1] - pl.blk_start[item];
+    unsigned char* tab = pl.ws + pl.table_off[item];
+    const bool wide = pl.wide[item] != 0;
+    uint32_t run_sum = 0;
+    for (int r = 0; r < n_runs; ++r) {
+        const size_t idx = (size_t)r * it.d_sae + f;
+        const uint32_t c = table_get(tab, wide, idx);
+        table_put(tab, wide, idx, run_sum);
+        run_sum += c;
+    }
+    it.d_row_ptr[f + 1] = run_sum;
+    if (f == 0) it.d_row_ptr[0] = 0;
+}
+
+// ---- 3. row_ptr = inclusive scan of the totals ------------------------------------------------------------
+__global__ void __launch_bounds__(PT)
+postings_rowscan_kernel(const __grid_constant__ PostingsPlan pl)
+{
+    __shared__ uint32_t warp_sums[33];
+    const s3_postings_item& it = pl.items[blockIdx.x];
+    uint32_t* rp = it.d_row_ptr + 1;
+    const int n = it.d_sae;
+    const int per = (n + PT - 1) / PT;                 // consecutive entries per thread
+    const int lo = threadIdx.x * per, hi = min(n, lo + per);
+    uint32_t sum = 0;
+    for (int i = lo; i < hi; ++i) sum += rp[i];
+    // block exclusive scan of the per-thread sums
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t inc = v;
+    uint32_t inc = sum;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t n = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += n;
+        const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += v;
     }
     if (lane == 31) warp_sums[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-        uint32_t w = warp_sums[lane];
+        const uint32_t w = warp_sums[lane];
         uint32_t winc = w;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t n = __shfl_up_sync(0xffffffffu, winc, o);
-            if (lane >= o) winc += n;
+            const uint32_t v = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += v;
         }
-        warp_sums[lane] = winc - w;          // exclusive prefix of the warp sums
-        if (lane == 31) warp_sums[32] = winc;  // block total
+        warp_sums[lane] = winc - w;
     }
     __syncthreads();
-    const uint32_t res = warp_sums[warp] + inc - v;
-    total = warp_sums[32];
-    __syncthreads();
-    return res;
+    uint32_t run = warp_sums[warp] + inc - sum;
+    for (int i = lo; i < hi; ++i) { run += rp[i]; rp[i] = run; }
 }
 
-__global__ void __launch_bounds__(PT)
-postings_kernel(const __grid_constant__ PostingsBatch batch, uint32_t* __restrict__ status)
-{
-    extern __shared__ uint32_t cursor[];     // [d_sae]
-    __shared__ uint32_t warp_sums[33];
+// ---- 4. ordered scatter ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t hash_feature(uint32_t f) { return (f * 2654435761u) >> 20; }   // 12 bits
 
-    const s3_postings_item it = batch.items[blockIdx.x];
+__global__ void __launch_bounds__(PT)
+postings_scatter_kernel(const __grid_constant__ PostingsPlan pl)
+{
+    extern __shared__ uint32_t smem_u32[];
+    // cursor[nf] | tick[nf/4 + 1] (one byte per feature) | hkey[HASH] | hbits[2*HASH]
+    const int item = find_item(pl, blockIdx.x);
+    const s3_postings_item& it = pl.items[item];
+    const int run = blockIdx.x - pl.blk_start[item];
     const int tid = threadIdx.x;
     const int d_sae = it.d_sae, k = it.k;
-    const int64_t n_pairs = (int64_t)it.T * k;
+    const int nf_max = min(RANGE, d_sae);
+    uint32_t* cursor = smem_u32;
+    uint32_t* tick = cursor + nf_max;
+    uint32_t* hkey = tick + (nf_max + 3) / 4 + 1;
+    uint32_t* hbits = hkey + HASH;
+
+    const int t_lo = run * pl.tok_per_blk[item];
+    const int t_hi = min(it.T, t_lo + pl.tok_per_blk[item]);
     const int32_t* __restrict__ ids = it.d_ids;
-
-    for (int f = tid; f < d_sae; f += PT) cursor[f] = 0;
-    __syncthreads();
-
-    // 1. histogram
-    for (int64_t p = tid; p < n_pairs; p += PT) {
-        const int32_t f = ids[p];
-        if (f >= 0) {
-            if (f < d_sae) atomicAdd(&cursor[f], 1u);
-            else dev_set_error(status, DEV_BAD_FEATURE_ID);
-        }
-    }
-    __syncthreads();
-
-    // 2. exclusive scan -> row_ptr, cursors
-    uint32_t carry = 0;
-    for (int f0 = 0; f0 < d_sae; f0 += PT) {
-        const int f = f0 + tid;
-        const uint32_t v = (f < d_sae) ? cursor[f] : 0u;
-        uint32_t total;
-        const uint32_t ex = block_exclusive_scan(v, warp_sums, total) + carry;
-        if (f < d_sae) { cursor[f] = ex; it.d_row_ptr[f] = ex; }
-        carry += total;
-    }
-    if (tid == 0) it.d_row_ptr[d_sae] = carry;
-    __syncthreads();
-
-    // 3. ordered scatter
-    int ts = (PT * PER) / k;
-    ts = ts < 1 ? 1 : (ts > 255 ? 255 : ts);
-    const int64_t sub_pairs = (int64_t)ts * k;
-    const int64_t cap = n_pairs;
+    const unsigned char* tab = pl.ws + pl.table_off[item];
+    const bool wide = pl.wide[item] != 0;
     const bool has_val = it.d_vals != nullptr && it.d_pval != nullptr;
-    for (int64_t base = 0; base < n_pairs; base += sub_pairs) {
-        const int64_t lim = (n_pairs - base < sub_pairs) ? (n_pairs - base) : sub_pairs;
-        int32_t f[PER];
-        uint32_t a[PER], cm[PER];
-        int32_t mypos[PER];
-        float myval[PER];
-        bool any_multi = false;
-#pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            const int64_t q = tid + (int64_t)j * PT;
-            f[j] = -1;
-            if (q < lim) {
-                const int64_t p = base + q;
-                const int32_t fj = ids[p];
-                if (fj >= 0 && fj < d_sae) {
-                    f[j] = fj;
-                    mypos[j] = (int32_t)(it.pos_base + p / k);
-                    if (has_val) myval[j] = it.d_vals[p];
-                    a[j] = atomicAdd(&cursor[fj], 1u << 24) >> 24;
-                }
-            }
-        }
+    int sub_tok = SUB_PAIRS / k;
+    sub_tok = sub_tok < 1 ? 1 : (sub_tok > SUB_TOK ? SUB_TOK : sub_tok);
+
+    for (int i = tid; i < HASH; i += PT) { hkey[i] = 0; hbits[2 * i] = 0; hbits[2 * i + 1] = 0; }
+
+    for (int f0 = 0; f0 < d_sae; f0 += RANGE) {
+        const int nf = min(RANGE, d_sae - f0);
+        for (int f = tid; f < nf; f += PT)
+            cursor[f] = it.d_row_ptr[f0 + f] + table_get(tab, wide, (size_t)run * d_sae + f0 + f);
+        for (int f = tid; f < (nf + 3) / 4 + 1; f += PT) tick[f] = 0;
         __syncthreads();
-#pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            if (f[j] >= 0) {
-                cm[j] = cursor[f[j]];
-                const uint32_t m = cm[j] >> 24, c = cm[j] & LOW24;
-                if (m == 1) {
-                    if (c < cap) { it.d_pos[c] = mypos[j]; if (has_val) it.d_pval[c] = myval[j]; }
-                } else {
-                    any_multi = true;
-                    if ((int64_t)c + a[j] < cap) it.d_pos[c + a[j]] = mypos[j];   // provisional slot
-                }
-            }
-        }
-        const int multi = __syncthreads_or(any_multi ? 1 : 0);
-        if (multi) {
-            uint32_t rank[PER];
+
+        for (int ts = t_lo; ts < t_hi; ts += sub_tok) {
+            const int n_tok = min(sub_tok, t_hi - ts);
+            const int n_pairs = n_tok * k;
+            const int64_t p0 = (int64_t)ts * k;
+            int lf[PER];          // feature relative to f0, -1 = nothing to do
+            uint32_t tk[PER];     // ticket within the sub-tile
+            int tau[PER];         // token offset within the sub-tile
+            // tickets
 #pragma unroll
             for (int j = 0; j < PER; ++j) {
-                rank[j] = 0;
-                if (f[j] >= 0 && (cm[j] >> 24) > 1) {
-                    const uint32_t m = cm[j] >> 24, c = cm[j] & LOW24;
-                    for (uint32_t e = 0; e < m; ++e)
-                        if ((int64_t)c + e < cap && __ldcg(&it.d_pos[c + e]) < mypos[j]) ++rank[j];
-                }
-            }
-            __syncthreads();
-#pragma unroll
-            for (int j = 0; j < PER; ++j) {
-                if (f[j] >= 0 && (cm[j] >> 24) > 1) {
-                    const uint32_t c = cm[j] & LOW24;
-                    if ((int64_t)c + rank[j] < cap) {
-                        it.d_pos[c + rank[j]] = mypos[j];
-                        if (has_val) it.d_pval[c + rank[j]] = myval[j];
+                const int q = tid + j * PT;
+                lf[j] = -1;
+                if (q < n_pairs) {
+                    const int32_t f = __ldg(ids + p0 + q);
+                    if (f >= f0 && f < f0 + nf) {
+                        lf[j] = f - f0;
+                        tau[j] = q / k;
+                        const int sh = 8 * (lf[j] & 3);
+                        tk[j] = (atomicAdd(&tick[lf[j] >> 2], 1u << sh) >> sh) & 0xFFu;
                     }
                 }
             }
-        }
+            __syncthreads();
+            // single hits write now; multiple hits publish their token in the feature's mask
+            uint32_t m[PER], slot[PER];
+            bool any_multi = false;
 #pragma unroll
-        for (int j = 0; j < PER; ++j)
-            if (f[j] >= 0 && a[j] == 0) cursor[f[j]] = (cm[j] & LOW24) + (cm[j] >> 24);
-        __syncthreads();
+            for (int j = 0; j < PER; ++j) {
+                if (lf[j] < 0) continue;
+                m[j] = (tick[lf[j] >> 2] >> (8 * (lf[j] & 3))) & 0xFFu;
+                if (m[j] == 1) {
+                    const uint32_t c = cursor[lf[j]];
+                    it.d_pos[c] = (int32_t)(it.pos_base + ts + tau[j]);
+                    if (has_val) it.d_pval[c] = it.d_vals[p0 + tid + j * PT];
+                } else {
+                    any_multi = true;
+                    uint32_t h = hash_feature((uint32_t)lf[j]);
+                    const uint32_t want = (uint32_t)lf[j] + 1u;
+                    for (int probe = 0; probe < HASH; ++probe) {      // the table cannot fill up: <= HASH/2 keys
+                        const uint32_t old = atomicCAS(&hkey[h], 0u, want);
+                        if (old == 0u || old == want) break;
+                        h = (h + 1) & (HASH - 1);
+                    }
+                    slot[j] = h;
+                    atomicOr(&hbits[2 * h + (tau[j] >> 5)], 1u << (tau[j] & 31));
+                }
+            }
+            const int multi = __syncthreads_or(any_multi ? 1 : 0);
+            if (multi) {
+#pragma unroll
+                for (int j = 0; j < PER; ++j) {
+                    if (lf[j] < 0 || m[j] == 1) continue;
+                    const uint32_t b0 = hbits[2 * slot[j]], b1 = hbits[2 * slot[j] + 1];
+                    const uint32_t rank = tau[j] < 32 ? __popc(b0 & ((1u << tau[j]) - 1u))
+                                                      : __popc(b0) + __popc(b1 & ((1u << (tau[j] - 32)) - 1u));
+                    const uint32_t c = cursor[lf[j]] + rank;
+                    it.d_pos[c] = (int32_t)(it.pos_base + ts + tau[j]);
+                    if (has_val) it.d_pval[c] = it.d_vals[p0 + tid + j * PT];
+                }
+                __syncthreads();
+            }
+            // the first ticket holder of each feature advances the cursor and clears the counters
+#pragma unroll
+            for (int j = 0; j < PER; ++j) {
+                if (lf[j] < 0) continue;
+                if (tk[j] == 0) {
+                    cursor[lf[j]] += m[j];
+                    atomicSub(&tick[lf[j] >> 2], m[j] << (8 * (lf[j] & 3)));
+                }
+                if (m[j] != 1) { hkey[slot[j]] = 0; hbits[2 * slot[j]] = 0; hbits[2 * slot[j] + 1] = 0; }
+            }
+            __syncthreads();
+        }
     }
 }
 
+size_t table_bytes(int T, int d_sae, int n_runs)
+{
+    const size_t entry = T > 65535 ? 4 : 2;
+    return round_up((size_t)n_runs * d_sae * entry, 256);
+}
+
+int runs_for(int T, int tok_per_blk) { return T > 0 ? (T + tok_per_blk - 1) / tok_per_blk : 0; }
+
 }  // namespace
 
-s3_status launch_postings(const s3_postings_item* h_items, int n_items, uint32_t* d_status, cudaStream_t stream)
+// Tokens per block such that the launch has about two blocks per SM over all items, at least one
+// 64-token sub-tile each, and no more than MAX_BLOCKS_TOTAL blocks in all.
+static int plan_tokens_per_block(const s3_postings_item* items, int n_items, int target_blocks)
+{
+    int64_t total = 0;
+    for (int i = 0; i < n_items; ++i) total += items[i].T;
+    int64_t tpb = (total + target_blocks - 1) / (target_blocks > 0 ? target_blocks : 1);
+    if (tpb < SUB_TOK) tpb = SUB_TOK;
+    tpb = (tpb + SUB_TOK - 1) / SUB_TOK * SUB_TOK;
+    while (true) {
+        int64_t blocks = 0;
+        for (int i = 0; i < n_items; ++i) blocks += runs_for(items[i].T, (int)tpb);
+        if (blocks <= MAX_BLOCKS_TOTAL) break;
+        tpb *= 2;
+    }
+    return (int)tpb;
+}
+
+size_t postings_workspace_bytes(int T, int k, int d_sae)
+{
+    (void)k;
+    if (T <= 0 || d_sae <= 0) return 0;
+    // the plan of a batch never uses fewer than SUB_TOK tokens per block, nor more than MAX_BLOCKS_TOTAL blocks
+    int runs = runs_for(T, SUB_TOK);
+    if (runs > MAX_BLOCKS_TOTAL) runs = MAX_BLOCKS_TOTAL;
+    return table_bytes(T, d_sae, runs);
+}
+
+s3_status launch_postings(const s3_postings_item* h_items, int n_items, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
     static bool attr_set[64] = {};
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 64 && !attr_set[dev]) {
-        S3_CUDA_TRY(cudaFuncSetAttribute(postings_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 49152 * 4));
+        S3_CUDA_TRY(cudaFuncSetAttribute(postings_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, RANGE * 4));
+        S3_CUDA_TRY(cudaFuncSetAttribute(postings_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         RANGE * 4 + RANGE + 16 + HASH * 12));
         attr_set[dev] = true;
     }
-    PostingsBatch batch;
-    int max_d = 0;
+    PostingsPlan pl;
+    pl.n_items = n_items;
+    pl.ws = static_cast<unsigned char*>(d_ws);
+    pl.status = static_cast<uint32_t*>(d_ws);
+    const int tpb = plan_tokens_per_block(h_items, n_items, 2 * device_sm_count());
+    size_t off = S3_WS_HEADER_BYTES;
+    int blocks = 0, max_d = 0, max_tiles = 0;
     for (int i = 0; i < n_items; ++i) {
-        batch.items[i] = h_items[i];
+        pl.items[i] = h_items[i];
+        pl.tok_per_blk[i] = tpb;
+        pl.blk_start[i] = blocks;
+        const int runs = runs_for(h_items[i].T, tpb);
+        blocks += runs;
+        pl.wide[i] = h_items[i].T > 65535 ? 1 : 0;
+        off = round_up(off, 256);
+        pl.table_off[i] = off;
+        off += table_bytes(h_items[i].T, h_items[i].d_sae, runs);
         if (h_items[i].d_sae > max_d) max_d = h_items[i].d_sae;
+        const int tiles = (h_items[i].d_sae + 255) / 256;
+        if (tiles > max_tiles) max_tiles = tiles;
     }
-    postings_kernel<<<n_items, PT, (size_t)max_d * sizeof(uint32_t), stream>>>(batch, d_status);
+    pl.blk_start[n_items] = blocks;
+    S3_REQUIRE(off <= ws_bytes, S3_ERR_CAPACITY, "postings workspace holds %zu bytes, %zu needed", ws_bytes, off);
+    const int nf = max_d < RANGE ? max_d : RANGE;
+    if (blocks > 0) {
+        postings_count_kernel<<<blocks, PT, (size_t)nf * 4, stream>>>(pl);
+        S3_CUDA_TRY(cudaGetLastError());
+    }
+    postings_colscan_kernel<<<dim3(max_tiles, n_items), 256, 0, stream>>>(pl, max_tiles);
     S3_CUDA_TRY(cudaGetLastError());
+    postings_rowscan_kernel<<<n_items, PT, 0, stream>>>(pl);
+    S3_CUDA_TRY(cudaGetLastError());
+    if (blocks > 0) {
+        const size_t smem = (size_t)nf * 4 + ((size_t)(nf + 3) / 4 + 1) * 4 + (size_t)HASH * 12;
+        postings_scatter_kernel<<<blocks, PT, smem, stream>>>(pl);
+        S3_CUDA_TRY(cudaGetLastError());
+    }
     return S3_OK;
 }
 

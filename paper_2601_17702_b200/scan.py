@@ -31,7 +31,8 @@ class ScanPipeline:
     def __init__(self, slots: list[SaeSlot]):
         self.slots = slots
         self.n_layers = len(slots[0].saes)
-        self.ws_post = B.new_workspace(B.S3_WS_HEADER_BYTES, slots[0].ids[0].device)
+        n_post = sum(B.s3_postings_workspace_bytes(s.chunk, s.k, s.d_sae) for s in slots) * self.n_layers
+        self.ws_post = B.new_workspace(n_post, slots[0].ids[0].device)
         self.launches = 0          # kernels of this library enqueued so far
 
     def reserve_index(self, n_tokens: int):

@@ -52,7 +52,7 @@ def test_host_side_argument_checks():
     ws = C.create_string_buffer(64)
     assert lib.s3_postings_build_batched(arr, 1, ws, 64, None) in (B.S3_ERR_INVALID_ARG, B.S3_ERR_UNSUPPORTED)
     assert lib.s3_postings_build_batched(arr, 33, ws, 64, None) == B.S3_ERR_UNSUPPORTED
-    item = B.PostingsItem(1, None, 4, 2, 60000, 0, 0, 1, 1, None)
+    item = B.PostingsItem(1, None, 4, 2, (1 << 20) + 8, 0, 0, 1, 1, None)
     arr = (B.PostingsItem * 1)(item)
     assert lib.s3_postings_build_batched(arr, 1, ws, 64, None) == B.S3_ERR_UNSUPPORTED       # d_sae limit
     item = B.PostingsItem(1, None, 4, 2, 64, 0, 2**31 - 2, 1, 1, None)

@@ -254,7 +254,8 @@ def test_postings_empty_inputs():
 def test_postings_batched_and_deterministic():
     d = dev()
     items, outs, refs = [], [], []
-    for i, (T, k, d_sae) in enumerate([(512, 32, 16384), (300, 64, 32768), (0, 8, 128), (2000, 16, 8192)]):
+    shapes = [(512, 32, 16384), (300, 64, 32768), (0, 8, 128), (2000, 16, 8192), (700, 8, 40000)]
+    for i, (T, k, d_sae) in enumerate(shapes):
         ids = _rand_ids(T, k, d_sae, 100 + i) if T else np.zeros((0, k), np.int32)
         ids_d = torch.as_tensor(ids).to(d)
         rp = torch.zeros(d_sae + 1, dtype=torch.int32, device=d)
@@ -262,7 +263,7 @@ def test_postings_batched_and_deterministic():
         items.append(S.make_postings_item(ids_d, d_sae, 1000 * i, rp, ps))
         outs.append((ids_d, rp, ps))
         refs.append(O.postings(ids, d_sae, 1000 * i))
-    ws = S.new_workspace(64)
+    ws = S.new_workspace(sum(S.s3_postings_workspace_bytes(T, k, D) for T, k, D in shapes))
     S.s3_postings_build_batched(items, ws)
     first = [(rp.cpu().numpy().copy(), ps.cpu().numpy().copy()) for _, rp, ps in outs]
     for (rp, ps), (orp, opos, _) in zip(first, refs):
@@ -279,7 +280,7 @@ def test_postings_bad_feature_id_is_reported_not_written():
     ids = torch.tensor([[1, 2], [3, 99]], dtype=torch.int32, device=d)
     rp = torch.zeros(9, dtype=torch.int32, device=d)
     ps = torch.zeros(4, dtype=torch.int32, device=d)
-    ws = S.new_workspace(64)
+    ws = S.new_workspace(S.s3_postings_workspace_bytes(2, 2, 8))
     S.s3_postings_build(ids, 8, 0, rp, ps, ws)
     with pytest.raises(S.binding.S3Error) as e:
         S.s3_workspace_status(ws)
@@ -294,7 +295,7 @@ def test_index_append_export_matches_oracle_merge():
     d_sae, k, n_layers = 2048, 8, 2
     chunks = [(0, 700), (700, 300), (1000, 1024), (2024, 1)]
     ix = S.Index(n_layers, d_sae, pinned_slab_bytes=1 << 20)
-    ws = S.new_workspace(64)
+    ws = S.new_workspace(S.s3_postings_workspace_bytes(1024, k, d_sae))
     ref = {l: [] for l in range(n_layers)}
     row_ptr = torch.zeros(d_sae + 1, dtype=torch.int32, device=d)
     pos = torch.zeros(1024 * k, dtype=torch.int32, device=d)
@@ -348,6 +349,9 @@ def gpu_score(ctx_ids, q_ids, q_vals, d_sae, width, stride, s, alpha, beta, bm25
     (777, 4, 64, 2, 3, 5, 4, 48, 20, 8),       # width not a multiple of stride
     (500, 4, 64, 1, 2, 3, 4, 10, 25, 64),      # gaps between spans; s larger than n_spans
     (30, 4, 64, 1, 2, 3, 4, 64, 16, 4),        # no full span at all
+    (12000, 4, 32, 1, 2, 5, 4, 64, 16, 8),     # hot features with lists longer than one warp's share
+    (9000, 4, 16, 2, 2, 3, 4, 50, 30, 8),      # long lists, stride not a power of two, width not a multiple
+    (5000, 8, 16, 1, 2, 40, 8, 64, 8, 8),      # features shared by many query tokens (large cQ), 8 spans per position
 ])
 def test_score_mincount_exact(L, k, d_sae, n_layers, Q, nq, kq, width, stride, s):
     ctx = np.stack([_rand_ids(L, k, d_sae, 50 + l, hot=3) for l in range(n_layers)])
@@ -412,7 +416,7 @@ def test_cfg1_scan_and_retrieval_end_to_end():
     S.s3_sae_encode_topk(sae, x.to(d), k, ids, vals, ws)
     row_ptr = torch.zeros(D + 1, dtype=torch.int32, device=d)
     pos = torch.zeros(cfg.L * k, dtype=torch.int32, device=d)
-    S.s3_postings_build(ids, D, 0, row_ptr, pos, ws)
+    S.s3_postings_build(ids, D, 0, row_ptr, pos, S.new_workspace(S.s3_postings_workspace_bytes(cfg.L, k, D)))
     ix = S.Index(1, D, 1 << 20)
     ix.append(0, row_ptr, pos, cfg.L, k, 0)
     rp, ps, _ = ix.export_csr(0)
