@@ -5,8 +5,8 @@
 // waiting:
 //   1. count    block (item, run): histogram of the run's ids in shared memory -> table[run][f]
 //   2. colscan  thread per feature: exclusive prefix of table[.][f] down the runs (in place) and the
-//               feature's total -> row_ptr[f+1]
-//   3. rowscan  block per item: in-place inclusive scan of row_ptr[1..d_sae]
+//               feature's total (its list length) -> row_ptr[f]
+//   3. rowscan  block per item: in-place exclusive scan of row_ptr[0..d_sae), total -> row_ptr[d_sae]
 //   4. scatter  block (item, run): cursor[f] = row_ptr[f] + table[run][f] in shared memory, then the
 //               run's tokens in order, 64 at a time: every pair takes a ticket from its feature's
 //               counter; a feature hit once in the 64 tokens writes straight to cursor[f]; a feature
@@ -79,11 +79,15 @@ postings_count_kernel(const __grid_constant__ PostingsPlan pl)
         const int nf = min(RANGE, d_sae - f0);
         for (int f = tid; f < nf; f += PT) hist[f] = 0;
         __syncthreads();
-        for (int64_t p = p_lo + tid; p < p_hi; p += PT) {
-            const int32_t f = __ldg(ids + p);
-            if (f >= 0) {
-                if (f >= d_sae) { if (f0 == 0) dev_set_error(pl.status, DEV_BAD_FEATURE_ID); }
-                else if (f >= f0 && f < f0 + nf) atomicAdd(&hist[f - f0], 1u);
+        for (int64_t p = p_lo + tid; p < p_hi; p += 4 * PT) {
+            int32_t f[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) f[j] = (p + (int64_t)j * PT < p_hi) ? __ldg(ids + p + (int64_t)j * PT) : -1;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (f[j] < 0) continue;
+                if (f[j] >= d_sae) { if (f0 == 0) dev_set_error(pl.status, DEV_BAD_FEATURE_ID); }
+                else if (f[j] >= f0 && f[j] < f0 + nf) atomicAdd(&hist[f[j] - f0], 1u);
             }
         }
         __syncthreads();
@@ -93,40 +97,54 @@ postings_count_kernel(const __grid_constant__ PostingsPlan pl)
 }
 
 // ---- 2. per-feature prefix over the runs ---------------------------------------------------------------
+// Thread per feature. The runs are taken eight at a time: eight independent loads, a prefix in
+// registers, eight stores, so that the memory round trips of a column overlap.
+template <typename E>
+__device__ __forceinline__ uint32_t colscan_column(E* col, size_t pitch, int n_runs)
+{
+    uint32_t run_sum = 0;
+    for (int r0 = 0; r0 < n_runs; r0 += 8) {
+        uint32_t c[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c[j] = (r0 + j < n_runs) ? static_cast<uint32_t>(col[(size_t)(r0 + j) * pitch]) : 0u;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (r0 + j < n_runs) col[(size_t)(r0 + j) * pitch] = static_cast<E>(run_sum);
+            run_sum += c[j];
+        }
+    }
+    return run_sum;
+}
+
 __global__ void __launch_bounds__(256)
-postings_colscan_kernel(const __grid_constant__ PostingsPlan pl, int max_tiles)
+postings_colscan_kernel(const __grid_constant__ PostingsPlan pl)
 {
     const int item = blockIdx.y;
     const s3_postings_item& it = pl.items[item];
     const int f = blockIdx.x * 256 + threadIdx.x;
-    if (blockIdx.x >= max_tiles || f >= it.d_sae) return;
+    if (f >= it.d_sae) return;
     const int n_runs = pl.blk_start[item + 1] - pl.blk_start[item];
     unsigned char* tab = pl.ws + pl.table_off[item];
-    const bool wide = pl.wide[item] != 0;
-    uint32_t run_sum = 0;
-    for (int r = 0; r < n_runs; ++r) {
-        const size_t idx = (size_t)r * it.d_sae + f;
-        const uint32_t c = table_get(tab, wide, idx);
-        table_put(tab, wide, idx, run_sum);
-        run_sum += c;
-    }
-    it.d_row_ptr[f + 1] = run_sum;
-    if (f == 0) it.d_row_ptr[0] = 0;
+    const uint32_t total = pl.wide[item] ? colscan_column(reinterpret_cast<uint32_t*>(tab) + f, it.d_sae, n_runs)
+                                         : colscan_column(reinterpret_cast<uint16_t*>(tab) + f, it.d_sae, n_runs);
+    it.d_row_ptr[f] = total;             // list length for now; the row scan turns it into the offset
 }
 
-// ---- 3. row_ptr = inclusive scan of the totals ------------------------------------------------------------
+// ---- 3. row_ptr = exclusive scan of the list lengths, in place ------------------------------------------------
+// Thread t owns entries [t*per, (t+1)*per): a first sweep sums them (independent loads), a block scan
+// of the 1024 sums gives each thread its starting offset, a second sweep writes the offsets.
 __global__ void __launch_bounds__(PT)
 postings_rowscan_kernel(const __grid_constant__ PostingsPlan pl)
 {
     __shared__ uint32_t warp_sums[33];
     const s3_postings_item& it = pl.items[blockIdx.x];
-    uint32_t* rp = it.d_row_ptr + 1;
+    uint32_t* rp = it.d_row_ptr;
     const int n = it.d_sae;
-    const int per = (n + PT - 1) / PT;                 // consecutive entries per thread
-    const int lo = threadIdx.x * per, hi = min(n, lo + per);
+    const int per = (n + PT - 1) / PT;
+    const int lo = min(n, (int)threadIdx.x * per), hi = min(n, lo + per);
     uint32_t sum = 0;
+#pragma unroll 8
     for (int i = lo; i < hi; ++i) sum += rp[i];
-    // block exclusive scan of the per-thread sums
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t inc = sum;
 #pragma unroll
@@ -145,10 +163,21 @@ postings_rowscan_kernel(const __grid_constant__ PostingsPlan pl)
             if (lane >= o) winc += v;
         }
         warp_sums[lane] = winc - w;
+        if (lane == 31) warp_sums[32] = winc;
     }
     __syncthreads();
     uint32_t run = warp_sums[warp] + inc - sum;
-    for (int i = lo; i < hi; ++i) { run += rp[i]; rp[i] = run; }
+    for (int i0 = lo; i0 < hi; i0 += 8) {
+        uint32_t c[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c[j] = (i0 + j < hi) ? rp[i0 + j] : 0u;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (i0 + j < hi) rp[i0 + j] = run;
+            run += c[j];
+        }
+    }
+    if (threadIdx.x == 0) rp[n] = warp_sums[32];
 }
 
 // ---- 4. ordered scatter ---------------------------------------------------------------------------------
@@ -341,7 +370,7 @@ s3_status launch_postings(const s3_postings_item* h_items, int n_items, void* d_
         postings_count_kernel<<<blocks, PT, (size_t)nf * 4, stream>>>(pl);
         S3_CUDA_TRY(cudaGetLastError());
     }
-    postings_colscan_kernel<<<dim3(max_tiles, n_items), 256, 0, stream>>>(pl, max_tiles);
+    postings_colscan_kernel<<<dim3(max_tiles, n_items), 256, 0, stream>>>(pl);
     S3_CUDA_TRY(cudaGetLastError());
     postings_rowscan_kernel<<<n_items, PT, 0, stream>>>(pl);
     S3_CUDA_TRY(cudaGetLastError());
