@@ -87,7 +87,7 @@ s3_status s3_sae_create(s3_sae** out, const void* d_W_enc, const float* d_b_enc,
                         int d_in, int d_sae, s3_dtype dtype, void* d_prepared, size_t prepared_bytes,
                         void* stream);
 s3_status s3_sae_destroy(s3_sae* sae);
-/* Scratch for partial Top-k lists of up to T_max tokens (includes the status block). */
+/* Scratch for the per-slice Top-k candidate lists of up to T_max tokens (includes the status block). */
 size_t s3_sae_encode_workspace_bytes(const s3_sae* sae, int T_max, int k);
 s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, int T, int k,
                              int32_t* d_ids /*[T,k]*/, float* d_vals /*[T,k]*/,
@@ -112,8 +112,9 @@ s3_status s3_sae_set_schedule(s3_sae* sae, int n_slices, int max_ctas);
  * frees nothing, on the host side of CUDA or through any library.
  *
  *   - Size limit: the call is refused with S3_ERR_CAPACITY when
- *     s3_sae_encode_workspace_bytes(sae, T, k) > S3_STATIC_SCRATCH_BYTES (for the 16-slice maximum
- *     that is T*k <= 131071 pairs, e.g. 4095 tokens at k = 32). Split longer inputs by token range.
+ *     s3_sae_encode_workspace_bytes(sae, T, k) > S3_STATIC_SCRATCH_BYTES (for bf16 encoders with 16 or
+ *     more column tiles that is about T*k <= 8100, e.g. 250 tokens at k = 32). Split longer inputs by
+ *     token range.
  *   - The first call on each device looks up the array's device address (with that device
  *     current) and remembers it. Make that first call before starting any stream capture.
  *   - One array per device, shared by every call and keeping the previous call's contents. The

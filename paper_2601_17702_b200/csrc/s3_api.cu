@@ -76,7 +76,11 @@ int pick_slices(const s3_sae* sae, int T)
 {
     const int nct = col_tiles(sae);
     int cap = nct < kMaxSlices ? nct : kMaxSlices;
-    if (sae->n_slices_override > 0) return sae->n_slices_override < cap ? sae->n_slices_override : cap;
+    const int lo = sae->dtype == S3_BF16 ? encode_tc_min_slices(sae->d_sae) : 1;
+    if (sae->n_slices_override > 0) {
+        const int s = sae->n_slices_override < cap ? sae->n_slices_override : cap;
+        return s < lo ? lo : s;
+    }
     const int nrt = row_tiles(sae, T);
     int n_sm = device_sm_count();
     if (sae->max_ctas > 0 && sae->max_ctas < n_sm) n_sm = sae->max_ctas;
@@ -86,7 +90,7 @@ int pick_slices(const s3_sae* sae, int T)
     }
     int best = 1;
     double best_cost = 1e30;
-    for (int s = 1; s <= cap; ++s) {
+    for (int s = lo; s <= cap; ++s) {
         const int units = nrt * s;
         const int waves = (units + n_sm - 1) / n_sm;
         const int len = (nct + s - 1) / s;
@@ -179,6 +183,7 @@ size_t s3_sae_encode_workspace_bytes(const s3_sae* sae, int T_max, int k)
     if (!sae || T_max < 0 || k < 1 || k > S3_MAX_K) return 0;
     const int nct = col_tiles(sae);
     const int smax = nct < kMaxSlices ? nct : kMaxSlices;
+    if (sae->dtype == S3_BF16) return S3_WS_HEADER_BYTES + 192 + encode_tc_workspace_bytes(T_max, smax, k);
     return S3_WS_HEADER_BYTES + (size_t)T_max * smax * k * sizeof(uint64_t);
 }
 
@@ -197,17 +202,19 @@ s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, in
     S3_REQUIRE(ldx >= sae->d_in, S3_ERR_INVALID_ARG, "ldx = %lld is smaller than d_in = %d", (long long)ldx, sae->d_in);
     if (sae->dtype == S3_BF16) S3_REQUIRE(ldx % 8 == 0, S3_ERR_INVALID_ARG, "ldx = %lld must be a multiple of 8 for bf16", (long long)ldx);
     const int n_slices = pick_slices(sae, T);
-    const size_t need = S3_WS_HEADER_BYTES + (size_t)T * n_slices * k * sizeof(uint64_t);
-    S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint32_t* status = static_cast<uint32_t*>(d_ws);
+    if (sae->dtype == S3_BF16) {
+        const size_t need = S3_WS_HEADER_BYTES + 192 + encode_tc_workspace_bytes(T, n_slices, k);
+        S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
+        return launch_encode_tc(&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, k, n_slices, sae->max_ctas,
+                                static_cast<unsigned char*>(d_ws) + 256, status, d_ids, d_vals, st);
+    }
+    const size_t need = S3_WS_HEADER_BYTES + (size_t)T * n_slices * k * sizeof(uint64_t);
+    S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
     uint64_t* part = reinterpret_cast<uint64_t*>(static_cast<unsigned char*>(d_ws) + S3_WS_HEADER_BYTES);
-    s3_status rc;
-    if (sae->dtype == S3_BF16)
-        rc = launch_encode_tc(&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, k, n_slices, sae->max_ctas, part, status, st);
-    else
-        rc = launch_encode_simt(static_cast<const float*>(d_x), ldx, static_cast<const float*>(sae->d_W), sae->d_b_enc,
-                                sae->d_b_dec, T, sae->d_in, sae->d_sae, k, n_slices, part, st);
+    const s3_status rc = launch_encode_simt(static_cast<const float*>(d_x), ldx, static_cast<const float*>(sae->d_W), sae->d_b_enc,
+                                            sae->d_b_dec, T, sae->d_in, sae->d_sae, k, n_slices, part, st);
     if (rc != S3_OK) return rc;
     launch_topk_merge(part, T, n_slices, k, d_ids, d_vals, st);
     S3_CUDA_TRY(cudaGetLastError());

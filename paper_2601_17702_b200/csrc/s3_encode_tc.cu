@@ -1,4 +1,4 @@
-// bf16 SAE encode + ReLU + running Top-k (Sec. 3.3, Eq. 1-2) on the sm_100a tensor cores.
+// bf16 SAE encode + ReLU + Top-k candidate selection (Sec. 3.3, Eq. 1-2) on the sm_100a tensor cores.
 //
 //   pre[t,f] = sum_i x[t,i] * W_enc[i,f] + b_eff[f],   b_eff = b_enc - W_enc^T b_dec   (folded once)
 //
@@ -9,14 +9,23 @@
 //               one of two 128x256 accumulators in tensor memory, tcgen05.commit frees the stage /
 //               publishes the accumulator;
 //   warps 2-5   epilogue: thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
-//               biased and filtered against a lower bound of the row's k-th best value. Survivors are
-//               only appended to a small per-thread pending list in shared memory (a predicated store);
-//               when some lane's list fills up, all lanes fold their lists into their heaps in
-//               lock-step, which raises the bounds. Appends are cheap and the expensive heap updates
-//               run with most lanes busy instead of once per stray hit.
-// A work unit is (128-token block, slice of 256-column tiles); the accumulator ring keeps the tensor
-// pipe busy with tile n+1 while the epilogue filters tile n. Only the k survivors per (token, slice)
-// leave the SM (as 64-bit keys); the pre-activation matrix is never written to memory.
+//               biased and compared with the row's bound tau, a value that at least k pre-activations
+//               of the row are known to exceed. Survivors go, branch-free, to a short pending list in
+//               shared memory. When some lane's list is nearly full the warp folds its lists: each
+//               survivor is appended to the row's candidate list in global memory and counted in a
+//               small per-row histogram over the float's exponent and top mantissa bits; as soon as k
+//               survivors lie in buckets above the bound's bucket, tau moves up to the next bucket edge.
+//               tau therefore tracks the row's running k-th largest value to within one bucket (about
+//               4 %) at a few instructions per survivor, and no ordered structure is kept on the SM.
+// A work unit is (128-token block, slice of 256-column tiles). A finished unit publishes its final
+// bound per row; units of the same rows that start later begin with it (any published bound is valid:
+// k values above it exist). The candidate lists of all slices, a few hundred keys per row, are
+// reduced to the exact Top-k by the merge kernel (s3_topk_merge.cu), which first drops everything not
+// above the best published bound. Only candidates leave the SM (as 64-bit keys); the pre-activation
+// matrix is never written to memory.
+//
+// A candidate list that would overflow is first compacted against the current bound and, if that
+// does not free enough room (many nearly equal values), cut down to its exact k largest keys.
 //
 // Every mbarrier wait is bounded; a wait that runs out records which one in the workspace status
 // word, raises a CTA-wide abort flag, and the CTA drains its own TMA copies, frees its tensor memory
@@ -39,7 +48,10 @@ constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr int TMEM_COLS = 512;
 constexpr int BATCH = 32;                    // columns per tcgen05.ld
-constexpr int HALF = 16;                     // columns filtered between two checks of the pending lists
+constexpr int STEP = 8;                      // columns filtered between two checks of the pending lists
+constexpr int PEND_CAP = 2 * STEP;           // pending-list slots per row
+constexpr int NB = 64;                       // histogram buckets per row
+constexpr int HSHIFT = 19;                   // bucket = float bits >> 19: 16 buckets per octave
 constexpr uint32_t WAIT_LIMIT = 1u << 26;    // try_wait polls before a wait is declared dead (~1 s)
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -153,65 +165,145 @@ constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cas
 
 struct EncodeTcParams {
     int T, d_in, d_sae, k;
-    int n_mtiles, n_col_tiles, n_slices, n_units, n_stages, pend_cap;
+    int n_mtiles, n_col_tiles, n_slices, n_units, n_stages;
+    uint32_t cap;              // candidate-list slots per (token, slice)
     const float* b_eff;
-    uint64_t* part;
+    uint64_t* cand;            // [T][n_slices][cap]
+    uint32_t* counts;          // [T][n_slices]
+    uint32_t* hint;            // [T] float bits of the best published bound
     uint32_t* status;
 };
 
 // Shared-memory carve-up (all offsets from a 1024-byte aligned base).
 struct SmemLayout {
-    uint32_t a_off, b_off, heap_off, pend_off, bar_off, total;
+    uint32_t a_off, b_off, pend_off, hist_off, bar_off, total;
 };
-// kp = heap slots per row (k rounded up to 8/16/32/64), pend_cap = pending-list slots per row.
-__host__ __device__ inline SmemLayout smem_layout(int n_stages, int kp, int pend_cap)
+__host__ __device__ inline SmemLayout smem_layout(int n_stages)
 {
     SmemLayout L;
     L.a_off = 0;
     L.b_off = L.a_off + n_stages * A_STAGE_BYTES;
-    L.heap_off = L.b_off + n_stages * B_STAGE_BYTES;
-    L.pend_off = L.heap_off + kp * EPI_THREADS * 8;
-    L.bar_off = L.pend_off + pend_cap * EPI_THREADS * 8;
+    L.pend_off = L.b_off + n_stages * B_STAGE_BYTES;
+    L.hist_off = L.pend_off + PEND_CAP * EPI_THREADS * 8;
+    L.bar_off = L.hist_off + NB * EPI_THREADS * 2;
     L.total = L.bar_off + (2 * n_stages + 4) * 8 + 16;
     return L;
 }
 
-// Row-private min-heap with a compile-time number of slots KP (stride EPI_THREADS between slots).
-// Slots k..KP-1 hold the all-ones sentinel, which never leaves the bottom of the heap.
-template <int KP>
-__device__ __forceinline__ uint64_t heap_replace_root_fixed(uint64_t* h, uint64_t key)
+// Per-row selection state of an epilogue thread.
+struct RowSel {
+    float tau;          // candidates are values > tau
+    float tau_floor;    // bound while the histogram has not moved yet (0, a published bound, or an exact k-th value)
+    int hbase;          // bucket id of histogram slot 0 (-1: not chosen yet)
+    int istar;          // histogram slot of the current bound
+    uint32_t above;     // survivors counted in slots >= istar
+    uint32_t gcnt;      // entries in the row's candidate list
+    bool floor_exact;   // tau_floor is the value of the list's exact k-th key
+};
+
+// Rare path: the candidate list cannot take the pending entries. Drops what is not above the bound;
+// if the list stays nearly full it keeps only its k largest keys and restarts the histogram from there.
+// New entries always come from later columns than the list's, so after the exact cut a value equal to
+// the k-th key's can no longer win (ties go to the lower id) and the strict comparison stays exact.
+__device__ __noinline__ void prune_list(uint64_t* glist, uint16_t* my_hist, RowSel& r, int k, uint32_t cap)
 {
-    int i = 0;
-#pragma unroll
-    for (int lvl = 0; lvl < 7; ++lvl) {
-        const int c = 2 * i + 1;
-        if (c >= KP) break;
-        uint64_t kc = h[c * EPI_THREADS];
-        int cc = c;
-        if (c + 1 < KP) {
-            const uint64_t k2 = h[(c + 1) * EPI_THREADS];
-            if (k2 < kc) { kc = k2; cc = c + 1; }
-        }
-        if (kc >= key) break;
-        h[i * EPI_THREADS] = kc;
-        i = cc;
+    uint32_t w = 0;
+    for (uint32_t i = 0; i < r.gcnt; ++i) {
+        const uint64_t key = glist[i];
+        if (__uint_as_float(static_cast<uint32_t>(key >> 32)) > r.tau) glist[w++] = key;
     }
-    h[i * EPI_THREADS] = key;
-    return h[0];
+    r.gcnt = w;
+    if (r.gcnt + PEND_CAP <= cap) return;
+    for (int a = 0; a < k; ++a) {
+        uint32_t best = a;
+        uint64_t kb = glist[a];
+        for (uint32_t b = a + 1; b < r.gcnt; ++b) {
+            const uint64_t kk = glist[b];
+            if (kk > kb) { kb = kk; best = b; }
+        }
+        const uint64_t tmp = glist[a];
+        glist[a] = kb;
+        glist[best] = tmp;
+    }
+    r.gcnt = k;
+    const uint32_t vb = static_cast<uint32_t>(glist[k - 1] >> 32);
+    r.tau_floor = r.tau = __uint_as_float(vb);
+    r.floor_exact = true;
+#pragma unroll 1
+    for (int s = 0; s < NB; ++s) my_hist[s * EPI_THREADS] = 0;
+    my_hist[0] = static_cast<uint16_t>(k);
+    r.hbase = static_cast<int>(vb >> HSHIFT);
+    r.istar = 0;
+    r.above = k;
 }
 
-template <int KP>
+// Folds the warp's pending lists (cnt entries per lane) into candidate lists and histograms, then
+// raises each row's bound as far as the histogram allows. Called by all 32 lanes.
+__device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_hist, uint64_t* glist, RowSel& r, int& cnt,
+                                             int k, uint32_t cap)
+{
+    if (__any_sync(0xffffffffu, r.gcnt + cnt > cap)) {
+        if (r.gcnt + cnt > cap) prune_list(glist, my_hist, r, k, cap);
+    }
+    if (r.hbase < 0 && cnt > 0) {
+        uint32_t ref = __float_as_uint(r.tau);
+        if (ref == 0) {      // no bound yet: centre the window on the largest value seen so far
+            for (int i = 0; i < cnt; ++i) {
+                const uint32_t vb = static_cast<uint32_t>(my_pend[i * EPI_THREADS] >> 32);
+                ref = vb > ref ? vb : ref;
+            }
+            const int b = static_cast<int>(ref >> HSHIFT) - NB / 2;
+            r.hbase = b > 0 ? b : 0;
+        } else {
+            r.hbase = static_cast<int>(ref >> HSHIFT);
+        }
+    }
+    const int nmax = __reduce_max_sync(0xffffffffu, cnt);
+    for (int i = 0; i < nmax; ++i) {
+        if (i < cnt) {
+            const uint64_t key = my_pend[i * EPI_THREADS];
+            const uint32_t vb = static_cast<uint32_t>(key >> 32);
+            if (__uint_as_float(vb) > r.tau) {
+                int idx = static_cast<int>(vb >> HSHIFT) - r.hbase;
+                idx = idx < 0 ? 0 : (idx > NB - 1 ? NB - 1 : idx);
+                my_hist[idx * EPI_THREADS] += 1;
+                r.above += 1;
+                glist[r.gcnt++] = key;
+            }
+        }
+    }
+    cnt = 0;
+    while (r.istar < NB - 1) {
+        const uint32_t c = my_hist[r.istar * EPI_THREADS];
+        if (r.above - c < static_cast<uint32_t>(k)) break;
+        r.above -= c;
+        ++r.istar;
+    }
+    if (r.istar == NB - 1) {
+        // k survivors lie at or above the last slot's edge: restart the window there
+        r.hbase += NB - 1;
+#pragma unroll 1
+        for (int s = 0; s < NB; ++s) my_hist[s * EPI_THREADS] = 0;
+        my_hist[0] = static_cast<uint16_t>(r.above);
+        r.istar = 0;
+        r.tau_floor = __uint_as_float((static_cast<uint32_t>(r.hbase) << HSHIFT) - 1u);
+        r.floor_exact = false;
+    }
+    // "value >= edge" is "value > the float just below the edge"
+    r.tau = r.istar > 0 ? __uint_as_float((static_cast<uint32_t>(r.hbase + r.istar) << HSHIFT) - 1u) : r.tau_floor;
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const EncodeTcParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const SmemLayout L = smem_layout(p.n_stages, KP, p.pend_cap);
+    const SmemLayout L = smem_layout(p.n_stages);
     unsigned char* smem_a = smem + L.a_off;
     unsigned char* smem_b = smem + L.b_off;
-    uint64_t* heap = reinterpret_cast<uint64_t*>(smem + L.heap_off);
     uint64_t* pend = reinterpret_cast<uint64_t*>(smem + L.pend_off);
+    uint16_t* hist = reinterpret_cast<uint16_t*>(smem + L.hist_off);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L.bar_off);
     uint64_t* empty_bar = full_bar + p.n_stages;
     uint64_t* acc_full = empty_bar + p.n_stages;
@@ -317,22 +409,28 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             }
         }
     } else {
-        // ---------------- epilogue: bias + ReLU + running Top-k ----------------
+        // ---------------- epilogue: bias + ReLU + candidate selection ----------------
         const int quarter = warp & 3;               // TMEM lanes this warp may read
         const int e = quarter * 32 + lane;          // row inside the 128-token block
-        uint64_t* my_heap = heap + e;
         uint64_t* my_pend = pend + e;
-        const int flush_at = p.pend_cap - HALF;     // fold the lists once a lane holds more than this
+        uint16_t* my_hist = hist + e;
         uint32_t tile_count = 0;
         bool ok = true;
         for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
             const int slice = u / p.n_mtiles, mt = u - slice * p.n_mtiles;
             const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
             const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
-#pragma unroll
-            for (int sl = 0; sl < KP; ++sl) my_heap[sl * EPI_THREADS] = (sl < p.k) ? 0ull : ~0ull;
-            uint64_t root = 0ull;
-            float tau = 0.0f;                       // value of the heap root: a lower bound of the k-th best
+            const int t = mt * BM + e;
+            const bool live = t < p.T;
+            uint64_t* glist = p.cand + (static_cast<size_t>(live ? t : 0) * p.n_slices + slice) * p.cap;
+#pragma unroll 1
+            for (int sl = 0; sl < NB; ++sl) my_hist[sl * EPI_THREADS] = 0;
+            // start from the best bound another slice of these rows has published so far, if any
+            const uint32_t hint_in = live ? *reinterpret_cast<volatile const uint32_t*>(p.hint + t) : 0u;
+            RowSel r;
+            r.tau_floor = live ? __uint_as_float(hint_in) : INFINITY;    // rows past T select nothing
+            r.tau = r.tau_floor;
+            r.hbase = -1; r.istar = 0; r.above = 0; r.gcnt = 0; r.floor_exact = false;
             int cnt = 0;                            // entries in this row's pending list
             for (int nt = tile_lo; nt < tile_hi && ok; ++nt, ++tile_count) {
                 const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
@@ -348,8 +446,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const float4* bias4 = reinterpret_cast<const float4*>(p.b_eff + static_cast<size_t>(nt) * BN);
 #pragma unroll 1
                 for (int cb = 0; cb < BN / BATCH; ++cb) {
-                    uint32_t r[32];
-                    tc_ld32(taddr + cb * BATCH, r);
+                    uint32_t acc[32];
+                    tc_ld32(taddr + cb * BATCH, acc);
                     float bias[BATCH];
 #pragma unroll
                     for (int j4 = 0; j4 < BATCH / 4; ++j4) {
@@ -359,46 +457,31 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     tc_wait_ld();
                     const uint32_t ncol0 = ~static_cast<uint32_t>(nt * BN + cb * BATCH);   // ~(col0 + j) = ncol0 - j
 #pragma unroll
-                    for (int h = 0; h < BATCH / HALF; ++h) {
+                    for (int h = 0; h < BATCH / STEP; ++h) {
 #pragma unroll
-                        for (int j = 0; j < HALF; ++j) {
+                        for (int j = 0; j < STEP; ++j) {
                             // Branch-free append: the slot after the list is always written and only
                             // kept (by advancing cnt) when the value beats the bound.
-                            const float v = __uint_as_float(r[h * HALF + j]) + bias[h * HALF + j];
+                            const float v = __uint_as_float(acc[h * STEP + j]) + bias[h * STEP + j];
                             my_pend[cnt * EPI_THREADS] =
-                                (static_cast<uint64_t>(__float_as_uint(v)) << 32) | (ncol0 - static_cast<uint32_t>(h * HALF + j));
-                            cnt += (v > tau) ? 1 : 0;
+                                (static_cast<uint64_t>(__float_as_uint(v)) << 32) | (ncol0 - static_cast<uint32_t>(h * STEP + j));
+                            cnt += (v > r.tau) ? 1 : 0;
                         }
-                        if (__any_sync(0xffffffffu, cnt > flush_at)) {
-                            const int nmax = __reduce_max_sync(0xffffffffu, cnt);
-                            for (int i = 0; i < nmax; ++i) {
-                                if (i < cnt) {
-                                    const uint64_t key = my_pend[i * EPI_THREADS];
-                                    if (key > root) root = heap_replace_root_fixed<KP>(my_heap, key);
-                                }
-                            }
-                            cnt = 0;
-                            tau = __uint_as_float(static_cast<uint32_t>(root >> 32));
-                        }
+                        if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) fold_pending(my_pend, my_hist, glist, r, cnt, p.k, p.cap);
                     }
                 }
                 tc_fence_before();
                 mbar_arrive(&acc_empty[ab]);
             }
             if (ok) {
-                for (int i = 0; i < cnt; ++i) {     // fold what is still pending (lane-private, no lock-step needed)
-                    const uint64_t key = my_pend[i * EPI_THREADS];
-                    if (key > root) root = heap_replace_root_fixed<KP>(my_heap, key);
-                }
-                const int t = mt * BM + e;
-                if (t < p.T) {
-                    uint64_t* dst = p.part + (static_cast<size_t>(t) * p.n_slices + slice) * p.k;
-                    int w = 0;
-#pragma unroll 4
-                    for (int sl = 0; sl < KP; ++sl) {
-                        const uint64_t key = my_heap[sl * EPI_THREADS];
-                        if (key != ~0ull && w < p.k) dst[w++] = key;
-                    }
+                if (__any_sync(0xffffffffu, cnt > 0)) fold_pending(my_pend, my_hist, glist, r, cnt, p.k, p.cap);
+                if (live) {
+                    p.counts[static_cast<size_t>(t) * p.n_slices + slice] = r.gcnt;
+                    // Publish the bound: at least k values of this slice exceed it. An exact k-th value
+                    // only bounds from below after stepping to the next float down.
+                    uint32_t out = __float_as_uint(r.tau);
+                    if (r.istar == 0 && r.floor_exact && out > 0u) out -= 1u;
+                    if (out > hint_in) atomicMax(p.hint + t, out);
                 }
             }
         }
@@ -511,8 +594,20 @@ s3_status encode_tc_prepare(EncodeTcState* st, const void* d_W, const float* d_b
 int encode_tc_col_tiles(int d_sae) { return (d_sae + BN - 1) / BN; }
 int encode_tc_row_tiles(int T) { return (T + BM - 1) / BM; }
 
+uint32_t encode_tc_list_cap(int k) { return static_cast<uint32_t>(k < 4 ? 64 : 16 * k); }
+
+// Column tiles per slice may not exceed 255: a row's histogram counters are 16 bits wide.
+int encode_tc_min_slices(int d_sae) { return (encode_tc_col_tiles(d_sae) + 254) / 255; }
+
+size_t encode_tc_workspace_bytes(int T, int n_slices, int k)
+{
+    const size_t t = static_cast<size_t>(T), s = static_cast<size_t>(n_slices);
+    return round_up(t * 4, 256) + round_up(t * s * 4, 256) + t * s * encode_tc_list_cap(k) * sizeof(uint64_t);
+}
+
 s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
-                           int n_slices, int max_ctas, uint64_t* d_part, uint32_t* d_status, cudaStream_t stream)
+                           int n_slices, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals,
+                           cudaStream_t stream)
 {
     alignas(64) CUtensorMap map_x;
     s3_status rc = make_map(&map_x, d_x, static_cast<uint64_t>(T), static_cast<uint64_t>(d_in), static_cast<uint64_t>(ldx), BM);
@@ -522,48 +617,43 @@ s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx
     p.T = T; p.d_in = d_in; p.d_sae = d_sae; p.k = k;
     p.n_mtiles = encode_tc_row_tiles(T);
     p.n_col_tiles = encode_tc_col_tiles(d_sae);
+    S3_REQUIRE(n_slices >= encode_tc_min_slices(d_sae), S3_ERR_INVALID_ARG, "d_sae = %d needs at least %d column slices", d_sae,
+               encode_tc_min_slices(d_sae));
     p.n_slices = n_slices;
     p.n_units = p.n_mtiles * n_slices;
+    p.cap = encode_tc_list_cap(k);
     p.b_eff = st->d_b_eff;
-    p.part = d_part;
+    unsigned char* base = static_cast<unsigned char*>(d_scratch);
+    p.hint = reinterpret_cast<uint32_t*>(base);
+    p.counts = reinterpret_cast<uint32_t*>(base + round_up(static_cast<size_t>(T) * 4, 256));
+    p.cand = reinterpret_cast<uint64_t*>(base + round_up(static_cast<size_t>(T) * 4, 256) +
+                                         round_up(static_cast<size_t>(T) * n_slices * 4, 256));
     p.status = d_status;
+    // no bound is known for any row yet
+    S3_CUDA_TRY(cudaMemsetAsync(p.hint, 0, static_cast<size_t>(T) * 4, stream));
 
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
     int max_smem = 0;
     S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    const int kp = k <= 8 ? 8 : (k <= 16 ? 16 : (k <= 32 ? 32 : 64));
-    // Prefer three or more pipeline stages; give what is left to the pending lists (16..32 slots).
-    int n_stages = 6, pend_cap = HALF;
-    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, kp, HALF).total) + 1024 > max_smem) --n_stages;
-    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, kp, HALF).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
-               "shared memory too small for the encode pipeline (k = %d)", k);
-    if (n_stages > 4) n_stages = 4;
-    for (int cap = 2 * HALF; cap > HALF; cap -= 2)
-        if (static_cast<int>(smem_layout(n_stages, kp, cap).total) + 1024 <= max_smem) { pend_cap = cap; break; }
+    int n_stages = 4;
+    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages).total) + 1024 > max_smem) --n_stages;
+    S3_REQUIRE(static_cast<int>(smem_layout(n_stages).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
+               "shared memory too small for the encode pipeline");
     p.n_stages = n_stages;
-    p.pend_cap = pend_cap;
-    const size_t smem = smem_layout(n_stages, kp, pend_cap).total + 1024;
+    const size_t smem = smem_layout(n_stages).total + 1024;
     int grid = device_sm_count();
     if (max_ctas > 0 && max_ctas < grid) grid = max_ctas;
     if (p.n_units < grid) grid = p.n_units;
     const CUtensorMap& map_w = *reinterpret_cast<const CUtensorMap*>(st->map_w);
-    static bool attr_set[64][4] = {};
-#define S3_LAUNCH_ENCODE(KP, SLOT)                                                                                      \
-    do {                                                                                                                \
-        if (dev < 64 && !attr_set[dev][SLOT]) {                                                                         \
-            S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)); \
-            attr_set[dev][SLOT] = true;                                                                                 \
-        }                                                                                                               \
-        encode_tc_kernel<KP><<<grid, NUM_THREADS, smem, stream>>>(map_x, map_w, p);                                     \
-    } while (0)
-    switch (kp) {
-        case 8: S3_LAUNCH_ENCODE(8, 0); break;
-        case 16: S3_LAUNCH_ENCODE(16, 1); break;
-        case 32: S3_LAUNCH_ENCODE(32, 2); break;
-        default: S3_LAUNCH_ENCODE(64, 3); break;
+    static bool attr_set[64] = {};
+    if (dev < 64 && !attr_set[dev]) {
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        attr_set[dev] = true;
     }
-#undef S3_LAUNCH_ENCODE
+    encode_tc_kernel<<<grid, NUM_THREADS, smem, stream>>>(map_x, map_w, p);
+    S3_CUDA_TRY(cudaGetLastError());
+    launch_candidate_merge(p.cand, p.counts, p.hint, T, n_slices, p.cap, k, d_ids, d_vals, stream);
     S3_CUDA_TRY(cudaGetLastError());
     return S3_OK;
 }

@@ -16,8 +16,12 @@ s3_status encode_tc_prepare(EncodeTcState* st, const void* d_W, const float* d_b
                             int d_sae, void* d_prepared, cudaStream_t stream);
 int encode_tc_col_tiles(int d_sae);
 int encode_tc_row_tiles(int T);
+int encode_tc_min_slices(int d_sae);
+size_t encode_tc_workspace_bytes(int T, int n_slices, int k);     // scratch after the status block
+// Encode kernel + candidate merge: writes ids / vals [T,k].
 s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
-                           int n_slices, int max_ctas, uint64_t* d_part, uint32_t* d_status, cudaStream_t stream);
+                           int n_slices, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals,
+                           cudaStream_t stream);
 
 size_t encode_simt_smem_bytes(int k);
 int encode_simt_col_tiles(int d_sae);

@@ -43,4 +43,9 @@ __device__ __forceinline__ uint64_t heap_replace_root(uint64_t* heap, int row, i
 void launch_topk_merge(const uint64_t* d_part, int T, int n_slices, int k, int32_t* d_ids, float* d_vals,
                        cudaStream_t stream);
 
+// Candidate lists of the tensor-core encode: cand[(t * n_slices + slice) * cap + i], i < counts[t * n_slices + slice],
+// unordered keys; hint[t] = float bits of a bound that at least k values of row t exceed.
+void launch_candidate_merge(const uint64_t* d_cand, const uint32_t* d_counts, const uint32_t* d_hint, int T, int n_slices,
+                            uint32_t cap, int k, int32_t* d_ids, float* d_vals, cudaStream_t stream);
+
 }  // namespace s3

@@ -41,6 +41,89 @@ topk_merge_kernel(const uint64_t* __restrict__ part, int T, int n, int npad, int
     }
 }
 
+// Exact Top-k of one row from the candidate lists of its slices. One warp per row:
+//   1. survivors = candidates above the best bound published for the row (at least k values exceed it,
+//      so nothing at or below it can be among the k best), gathered into the warp's shared-memory buffer;
+//   2. bitonic sort of the survivors (a couple of hundred keys at most in the usual case);
+//   3. rows whose survivors do not fit the buffer (long runs of nearly equal values) fall back to k
+//      rounds of "largest key below the previous one" over the lists in global memory.
+constexpr int kCandBuf = 1024;   // survivor slots per warp
+
+__global__ void __launch_bounds__(kMergeWarps * 32)
+candidate_merge_kernel(const uint64_t* __restrict__ cand, const uint32_t* __restrict__ counts,
+                       const uint32_t* __restrict__ hint, int T, int n_slices, uint32_t cap, int k,
+                       int32_t* __restrict__ ids, float* __restrict__ vals)
+{
+    __shared__ uint64_t cand_buf[kMergeWarps][kCandBuf];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * kMergeWarps + warp;
+    if (t >= T) return;
+    uint64_t* buf = cand_buf[warp];
+    const float tau = __uint_as_float(hint[t]);
+    uint32_t n = 0;            // survivors so far (warp-uniform)
+    bool overflow = false;
+    for (int s = 0; s < n_slices && !overflow; ++s) {
+        const uint32_t cnt = counts[(size_t)t * n_slices + s];
+        const uint64_t* list = cand + ((size_t)t * n_slices + s) * cap;
+        for (uint32_t i0 = 0; i0 < cnt; i0 += 32) {
+            const uint32_t i = i0 + lane;
+            const uint64_t key = i < cnt ? list[i] : 0ull;
+            const bool keep = i < cnt && __uint_as_float(static_cast<uint32_t>(key >> 32)) > tau;
+            const uint32_t m = __ballot_sync(0xffffffffu, keep);
+            const uint32_t at = n + __popc(m & ((1u << lane) - 1u));
+            if (n + __popc(m) > kCandBuf) { overflow = true; break; }
+            if (keep) buf[at] = key;
+            n += __popc(m);
+        }
+    }
+    if (!overflow) {
+        uint32_t npad = 32;
+        while (npad < n) npad <<= 1;
+        for (uint32_t i = n + lane; i < npad; i += 32) buf[i] = 0ull;
+        __syncwarp();
+        for (uint32_t size = 2; size <= npad; size <<= 1) {
+            for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+                for (uint32_t i = lane; i < (npad >> 1); i += 32) {
+                    const uint32_t pos = 2 * i - (i & (stride - 1));
+                    const bool desc = (pos & size) == 0;
+                    const uint64_t a = buf[pos], b = buf[pos + stride];
+                    if ((a < b) == desc) { buf[pos] = b; buf[pos + stride] = a; }
+                }
+                __syncwarp();
+            }
+        }
+        for (int j = lane; j < k; j += 32) {
+            const uint64_t key = static_cast<uint32_t>(j) < n ? buf[j] : 0ull;
+            ids[(size_t)t * k + j] = key ? static_cast<int32_t>(~static_cast<uint32_t>(key)) : -1;
+            vals[(size_t)t * k + j] = key ? __uint_as_float(static_cast<uint32_t>(key >> 32)) : 0.0f;
+        }
+        return;
+    }
+    // fallback: selection by repeated maximum (keys are distinct, so "below the previous" removes exactly one)
+    uint64_t prev = ~0ull;
+    for (int j = 0; j < k; ++j) {
+        uint64_t best = 0ull;
+        for (int s = 0; s < n_slices; ++s) {
+            const uint32_t cnt = counts[(size_t)t * n_slices + s];
+            const uint64_t* list = cand + ((size_t)t * n_slices + s) * cap;
+            for (uint32_t i = lane; i < cnt; i += 32) {
+                const uint64_t key = list[i];
+                if (key < prev && key > best) best = key;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const uint64_t other = __shfl_xor_sync(0xffffffffu, best, o);
+            best = other > best ? other : best;
+        }
+        if (lane == 0) {
+            ids[(size_t)t * k + j] = best ? static_cast<int32_t>(~static_cast<uint32_t>(best)) : -1;
+            vals[(size_t)t * k + j] = best ? __uint_as_float(static_cast<uint32_t>(best >> 32)) : 0.0f;
+        }
+        prev = best ? best : 0ull;      // nothing left: every later round finds nothing either
+    }
+}
+
 }  // namespace
 
 void launch_topk_merge(const uint64_t* d_part, int T, int n_slices, int k, int32_t* d_ids, float* d_vals,
@@ -53,6 +136,14 @@ void launch_topk_merge(const uint64_t* d_part, int T, int n_slices, int k, int32
     const size_t smem = (size_t)kMergeWarps * npad * sizeof(uint64_t);
     const int grid = (T + kMergeWarps - 1) / kMergeWarps;
     topk_merge_kernel<<<grid, kMergeWarps * 32, smem, stream>>>(d_part, T, n, npad, k, d_ids, d_vals);
+}
+
+void launch_candidate_merge(const uint64_t* d_cand, const uint32_t* d_counts, const uint32_t* d_hint, int T, int n_slices,
+                            uint32_t cap, int k, int32_t* d_ids, float* d_vals, cudaStream_t stream)
+{
+    if (T <= 0) return;
+    const int grid = (T + kMergeWarps - 1) / kMergeWarps;
+    candidate_merge_kernel<<<grid, kMergeWarps * 32, 0, stream>>>(d_cand, d_counts, d_hint, T, n_slices, cap, k, d_ids, d_vals);
 }
 
 }  // namespace s3

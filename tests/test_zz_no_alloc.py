@@ -51,8 +51,9 @@ def test_static_scratch_encode_matches_regular_entry_point_twice_in_a_row():
     d_in, d_sae = 256, 4096
     W, b_enc, b_dec = G.sae_weights(31, 0, d_in, d_sae, torch.bfloat16)
     sae = S.Sae(W.to(d), b_enc.to(d), b_dec.to(d))
-    # first call: 1000 tokens at k = 32; second call: fewer tokens, another k, other data
-    for seed, T, k in ((41, 1000, 32), (42, 300, 8)):
+    # first call: 200 tokens at k = 32 (two row blocks, the second ragged); second call: fewer tokens, another k,
+    # other data
+    for seed, T, k in ((41, 200, 32), (42, 100, 8)):
         x = G.activations(seed, 0, 0, T, d_in, torch.bfloat16).to(d)
         got_ids, got_vals = _static(sae, x, k)
         ref_ids, ref_vals = _regular(sae, x, k)
