@@ -84,6 +84,10 @@ int pick_slices(const s3_sae* sae, int T)
     const int nrt = row_tiles(sae, T);
     int n_sm = device_sm_count();
     if (sae->max_ctas > 0 && sae->max_ctas < n_sm) n_sm = sae->max_ctas;
+    if (sae->dtype == S3_BF16) {         // the tensor-core kernel runs one unit per CTA pair
+        n_sm = encode_tc_max_pairs();
+        if (sae->max_ctas > 0 && sae->max_ctas / 2 < n_sm) n_sm = sae->max_ctas / 2 > 0 ? sae->max_ctas / 2 : 1;
+    }
     if (sae->dtype == S3_F32) {   // non-persistent kernel: enough blocks to cover the SMs
         int s = (n_sm + nrt - 1) / nrt;
         return s < 1 ? 1 : (s > cap ? cap : s);

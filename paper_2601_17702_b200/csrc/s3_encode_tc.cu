@@ -41,9 +41,10 @@ namespace s3 {
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
-constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
-constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KB
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int PAIR_M = 2 * BM;                      // tokens per tile over the CTA pair
+constexpr int A_STAGE_BYTES = BM * BK * 2;         // 16 KB: this CTA's 128 tokens
+constexpr int B_STAGE_BYTES = (BN / 2) * BK * 2;   // 16 KB: this CTA's half of the tile's 256 features
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;   // per CTA; a stage is complete after twice that
 constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr int TMEM_COLS = 512;
@@ -92,20 +93,53 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return false;
 }
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar)
+__device__ __forceinline__ uint32_t cluster_cta_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Cluster-wide barrier over all threads of both CTAs.
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in the cluster's CTA `rank`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+// Tile load of one CTA of the pair into its own shared memory; the bytes are counted on the mbarrier at
+// cluster address `bar_addr` (the first CTA's), which the .cta_group::2 form allows to lie in the peer CTA.
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_addr)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_u32(dst)),
-        "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_addr)
         : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tc_commit(uint64_t* bar)
+// Arrives, once the MMAs issued so far have completed, on the mbarrier at this shared-memory offset in
+// both CTAs of the pair.
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                     smem_u32(bar)),
+                 "h"(both)
+                 : "memory");
 }
 
 __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
@@ -113,7 +147,7 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t desc_a, ui
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
         "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
         : "memory");
 }
@@ -159,9 +193,9 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
     return d;
 }
 
-// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128.
+// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 256 (over the CTA pair).
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
-                                (static_cast<uint32_t>(BM >> 4) << 24);
+                                (static_cast<uint32_t>(PAIR_M >> 4) << 24);
 
 struct EncodeTcParams {
     int T, d_in, d_sae, k;
@@ -293,7 +327,7 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
     r.tau = r.istar > 0 ? __uint_as_float((static_cast<uint32_t>(r.hbase + r.istar) << HSHIFT) - 1u) : r.tau_floor;
 }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const EncodeTcParams p)
 {
@@ -313,20 +347,28 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kblocks = (p.d_in + BK - 1) / BK;
+    const uint32_t cta_rank = cluster_cta_rank();          // 0 = first CTA of the pair: issues the MMAs, owns the
+    const bool first_cta = cta_rank == 0;                  // barriers that both CTAs signal (full, acc_empty)
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
+        // full:      1 arrival (the first CTA's producer, with the byte count of both CTAs' copies)
+        // empty:     1 arrival per CTA (tcgen05.commit, multicast)      acc_full: likewise
+        // acc_empty: every epilogue thread of both CTAs, on the first CTA's barrier
         for (int s = 0; s < p.n_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_THREADS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 2 * EPI_THREADS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+        // tensor memory of both SMs, allocated pairwise by the same warp of each CTA
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
                      : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync();                                        // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -338,11 +380,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             uint32_t stage = 0, phase = 0;
             uint64_t issued = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+            for (int u = pair; u < p.n_units && ok; u += n_pairs) {
                 const int slice = u / p.n_mtiles, mt = u - slice * p.n_mtiles;
                 const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
                 const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
+                const int row0 = mt * PAIR_M + static_cast<int>(cta_rank) * BM;        // this CTA's tokens
                 for (int nt = tile_lo; nt < tile_hi && ok; ++nt) {
+                    const int col0 = nt * BN + static_cast<int>(cta_rank) * (BN / 2);  // this CTA's half of the features
                     for (int kb = 0; kb < kblocks; ++kb) {
                         if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag)) {
                             dev_set_error(p.status, DEV_TIMEOUT_SMEM_EMPTY);
@@ -350,16 +394,18 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             ok = false;
                             break;
                         }
-                        mbar_expect_tx(&full_bar[stage], STAGE_BYTES);
-                        tma_load_2d(smem_a + stage * A_STAGE_BYTES, &map_x, kb * BK, mt * BM, &full_bar[stage]);
-                        tma_load_2d(smem_b + stage * B_STAGE_BYTES, &map_w, kb * BK, nt * BN, &full_bar[stage]);
+                        if (first_cta) mbar_expect_tx(&full_bar[stage], 2 * STAGE_BYTES);
+                        const uint32_t full_addr = map_to_cta(smem_u32(&full_bar[stage]), 0);
+                        tma_load_2d(smem_a + stage * A_STAGE_BYTES, &map_x, kb * BK, row0, full_addr);
+                        tma_load_2d(smem_b + stage * B_STAGE_BYTES, &map_w, kb * BK, col0, full_addr);
                         ++issued;
                         if (++stage == static_cast<uint32_t>(p.n_stages)) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
-            // Own copies still in flight: wait (bounded) until the last n_stages loads have landed.
-            const uint64_t back = issued < static_cast<uint64_t>(p.n_stages) ? issued : static_cast<uint64_t>(p.n_stages);
+            // Copies still in flight: the first CTA waits (bounded) until the last n_stages stages, its own and
+            // the peer's halves, have landed; the peer stays resident until the closing cluster barrier.
+            const uint64_t back = !first_cta ? 0 : (issued < static_cast<uint64_t>(p.n_stages) ? issued : static_cast<uint64_t>(p.n_stages));
             uint32_t s = stage, ph = phase;
             for (uint64_t i = 0; i < back; ++i) {
                 if (s == 0) { s = p.n_stages - 1; ph ^= 1u; } else { --s; }
@@ -368,12 +414,12 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        // ---------------- MMA issuer (first CTA of the pair only) ----------------
+        if (lane == 0 && first_cta) {
             uint32_t stage = 0, phase = 0;
             uint32_t tile_count = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+            for (int u = pair; u < p.n_units && ok; u += n_pairs) {
                 const int slice = u / p.n_mtiles;
                 const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
                 const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
@@ -401,10 +447,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         for (int kk = 0; kk < BK / UMMA_K; ++kk)
                             tc_mma_bf16(d_tmem, da + static_cast<uint64_t>(kk * 2), db + static_cast<uint64_t>(kk * 2), kInstrDesc,
                                         (kb | kk) != 0 ? 1u : 0u);
-                        tc_commit(&empty_bar[stage]);
+                        tc_commit_pair(&empty_bar[stage]);
                         if (++stage == static_cast<uint32_t>(p.n_stages)) { stage = 0; phase ^= 1u; }
                     }
-                    if (ok) tc_commit(&acc_full[ab]);
+                    if (ok) tc_commit_pair(&acc_full[ab]);
                 }
             }
         }
@@ -416,11 +462,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         uint16_t* my_hist = hist + e;
         uint32_t tile_count = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+        // the accumulator is handed back on the first CTA's barrier
+        const uint32_t acc_empty_addr[2] = {map_to_cta(smem_u32(&acc_empty[0]), 0), map_to_cta(smem_u32(&acc_empty[1]), 0)};
+        for (int u = pair; u < p.n_units && ok; u += n_pairs) {
             const int slice = u / p.n_mtiles, mt = u - slice * p.n_mtiles;
             const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
             const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
-            const int t = mt * BM + e;
+            const int t = mt * PAIR_M + static_cast<int>(cta_rank) * BM + e;
             const bool live = t < p.T;
             uint64_t* glist = p.cand + (static_cast<size_t>(live ? t : 0) * p.n_slices + slice) * p.cap;
 #pragma unroll 1
@@ -471,7 +519,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     }
                 }
                 tc_fence_before();
-                mbar_arrive(&acc_empty[ab]);
+                mbar_arrive_cluster(acc_empty_addr[ab]);
             }
             if (ok) {
                 if (__any_sync(0xffffffffu, cnt > 0)) fold_pending(my_pend, my_hist, glist, r, cnt, p.k, p.cap);
@@ -487,11 +535,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         }
     }
 
+    // Both CTAs are done with tensor memory, and the first CTA has seen every copy land, before either frees
+    // its tensor memory or leaves (the peer's shared memory receives copies and is read by the pair's MMAs).
     tc_fence_before();
     __syncthreads();
+    cluster_sync();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -588,11 +639,26 @@ s3_status encode_tc_prepare(EncodeTcState* st, const void* d_W, const float* d_b
                                                                     d_sae, d_sae_pad, st->d_b_eff);
     S3_CUDA_TRY(cudaGetLastError());
     static_assert(sizeof(CUtensorMap) <= sizeof(st->map_w), "tensor map storage too small");
-    return make_map(reinterpret_cast<CUtensorMap*>(st->map_w), st->d_wt, d_sae, d_in, d_in, BN);
+    return make_map(reinterpret_cast<CUtensorMap*>(st->map_w), st->d_wt, d_sae, d_in, d_in, BN / 2);
 }
 
 int encode_tc_col_tiles(int d_sae) { return (d_sae + BN - 1) / BN; }
-int encode_tc_row_tiles(int T) { return (T + BM - 1) / BM; }
+int encode_tc_row_tiles(int T) { return (T + PAIR_M - 1) / PAIR_M; }   // a CTA pair takes 256 tokens
+
+// CTA pairs that can be resident at once (cached per device).
+int encode_tc_max_pairs();
+
+int encode_tc_max_pairs()
+{
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+    if (dev < 64 && cached[dev]) return cached[dev];
+    int n = device_sm_count() / 2;      // a pair occupies two SMs entirely (shared memory)
+    if (n < 1) n = 1;
+    if (dev < 64) cached[dev] = n;
+    return n;
+}
 
 uint32_t encode_tc_list_cap(int k) { return static_cast<uint32_t>(k < 4 ? 64 : 16 * k); }
 
@@ -636,22 +702,22 @@ s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx
     S3_CUDA_TRY(cudaGetDevice(&dev));
     int max_smem = 0;
     S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    int n_stages = 4;
+    int n_stages = 6;
     while (n_stages > 2 && static_cast<int>(smem_layout(n_stages).total) + 1024 > max_smem) --n_stages;
     S3_REQUIRE(static_cast<int>(smem_layout(n_stages).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
                "shared memory too small for the encode pipeline");
     p.n_stages = n_stages;
     const size_t smem = smem_layout(n_stages).total + 1024;
-    int grid = device_sm_count();
-    if (max_ctas > 0 && max_ctas < grid) grid = max_ctas;
-    if (p.n_units < grid) grid = p.n_units;
     const CUtensorMap& map_w = *reinterpret_cast<const CUtensorMap*>(st->map_w);
     static bool attr_set[64] = {};
     if (dev < 64 && !attr_set[dev]) {
         S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set[dev] = true;
     }
-    encode_tc_kernel<<<grid, NUM_THREADS, smem, stream>>>(map_x, map_w, p);
+    int n_pairs = encode_tc_max_pairs();
+    if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
+    if (p.n_units < n_pairs) n_pairs = p.n_units;
+    encode_tc_kernel<<<2 * n_pairs, NUM_THREADS, smem, stream>>>(map_x, map_w, p);
     S3_CUDA_TRY(cudaGetLastError());
     launch_candidate_merge(p.cand, p.counts, p.hint, T, n_slices, p.cap, k, d_ids, d_vals, stream);
     S3_CUDA_TRY(cudaGetLastError());

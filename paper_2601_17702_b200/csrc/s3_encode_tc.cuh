@@ -17,6 +17,7 @@ s3_status encode_tc_prepare(EncodeTcState* st, const void* d_W, const float* d_b
 int encode_tc_col_tiles(int d_sae);
 int encode_tc_row_tiles(int T);
 int encode_tc_min_slices(int d_sae);
+int encode_tc_max_pairs();         // CTA pairs (work units in flight) of the bf16 encode on this device
 size_t encode_tc_workspace_bytes(int T, int n_slices, int k);     // scratch after the status block
 // Encode kernel + candidate merge: writes ids / vals [T,k].
 s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
