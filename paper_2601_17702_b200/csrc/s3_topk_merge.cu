@@ -62,18 +62,30 @@ candidate_merge_kernel(const uint64_t* __restrict__ cand, const uint32_t* __rest
     const float tau = __uint_as_float(hint[t]);
     uint32_t n = 0;            // survivors so far (warp-uniform)
     bool overflow = false;
-    for (int s = 0; s < n_slices && !overflow; ++s) {
-        const uint32_t cnt = counts[(size_t)t * n_slices + s];
-        const uint64_t* list = cand + ((size_t)t * n_slices + s) * cap;
-        for (uint32_t i0 = 0; i0 < cnt; i0 += 32) {
-            const uint32_t i = i0 + lane;
-            const uint64_t key = i < cnt ? list[i] : 0ull;
-            const bool keep = i < cnt && __uint_as_float(static_cast<uint32_t>(key >> 32)) > tau;
-            const uint32_t m = __ballot_sync(0xffffffffu, keep);
-            const uint32_t at = n + __popc(m & ((1u << lane) - 1u));
-            if (n + __popc(m) > kCandBuf) { overflow = true; break; }
-            if (keep) buf[at] = key;
-            n += __popc(m);
+    // list lengths of up to 32 slices at once; longer rows of slices in rounds
+    for (int s0 = 0; s0 < n_slices && !overflow; s0 += 32) {
+        const uint32_t my_cnt = (s0 + lane < n_slices) ? counts[(size_t)t * n_slices + s0 + lane] : 0u;
+        const int ns = n_slices - s0 < 32 ? n_slices - s0 : 32;
+        for (int s = 0; s < ns && !overflow; ++s) {
+            const uint32_t cnt = __shfl_sync(0xffffffffu, my_cnt, s);
+            const uint64_t* list = cand + ((size_t)t * n_slices + s0 + s) * cap;
+            // 128 entries per step: four independent loads per lane before any of them is used
+            for (uint32_t i0 = 0; i0 < cnt && !overflow; i0 += 128) {
+                uint64_t key[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t i = i0 + q * 32 + lane;
+                    key[q] = i < cnt ? list[i] : 0ull;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const bool keep = __uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > tau;   // key 0: value 0, never kept
+                    const uint32_t m = __ballot_sync(0xffffffffu, keep);
+                    if (n + __popc(m) > kCandBuf) { overflow = true; break; }
+                    if (keep) buf[n + __popc(m & ((1u << lane) - 1u))] = key[q];
+                    n += __popc(m);
+                }
+            }
         }
     }
     if (!overflow) {
