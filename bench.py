@@ -95,6 +95,31 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def workload_config(cfg, rcfg, L_idx, ns):
+    """The `config` object of the JSON line (same for both arms)."""
+    return {"workload": cfg.name, "context_tokens": cfg.L, "chunk": cfg.chunk, "layers": cfg.n_layers,
+            "key_sae": [cfg.key.d_in, cfg.key.d_sae, cfg.key.k], "query_sae": [cfg.query.d_in, cfg.query.d_sae, cfg.query.k],
+            "retrieval_per_step": {"queries": rcfg.Q, "query_tokens": rcfg.nq, "k": rcfg.kq, "index_tokens": L_idx,
+                                   "spans": ns, "width": rcfg.width, "stride": rcfg.stride, "top": rcfg.s},
+            "l2_policy": "inputs larger than L2: every step reads a different 80 MB activation chunk and 1.1 GB of encoder weights",
+            "parallelism": "independent context replicas per GPU, no collectives"}
+
+
+def max_over_ranks(seconds_or_ms: float, world: int, device=None) -> float:
+    """The slowest rank's time (every rank returns it). The path has no exchange step, so this reduction of one
+    timing scalar is the only collective of a multi-GPU run."""
+    if world <= 1:
+        return float(seconds_or_ms)
+    t = torch.tensor([seconds_or_ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank_step: int, steps: int, world: int, slowest_seconds: float) -> float:
+    """Units all ranks processed divided by the slowest rank's time (weak scaling: every rank does the same work)."""
+    return units_per_rank_step * steps * world / slowest_seconds
+
+
 # ------------------------------------------------------------------------------------------ our arm
 
 def run_ours(args, rank, world, local_rank):
@@ -205,12 +230,8 @@ def run_ours(args, rank, world, local_rank):
     pipe.finish()
     assert S.s3_workspace_status(q_ws) == 0 and S.s3_workspace_status(s_ws) == 0
 
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
-    tokens = args.steps * chunk * world
-    value = tokens / (ms * 1e-3)
+    ms = max_over_ranks(ms, world, dev)
+    value = whole_job_rate(chunk, args.steps, world, ms * 1e-3)
 
     # ---- end to end: the step's inputs come from pinned host memory, its result goes back to the host
     n_host = min(4, n_distinct)
@@ -241,11 +262,8 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - w0
     pipe.finish()
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = e2e_steps * chunk * world / e2e_s
+    e2e_s = max_over_ranks(e2e_s, world, dev)
+    e2e_value = whole_job_rate(chunk, e2e_steps, world, e2e_s)
 
     if rank != 0:
         return None
@@ -257,12 +275,7 @@ def run_ours(args, rank, world, local_rank):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "context_tokens": cfg.L, "chunk": chunk, "layers": nl,
-                   "key_sae": [cfg.key.d_in, cfg.key.d_sae, cfg.key.k], "query_sae": [cfg.query.d_in, cfg.query.d_sae, cfg.query.k],
-                   "retrieval_per_step": {"queries": rcfg.Q, "query_tokens": rcfg.nq, "k": rcfg.kq, "index_tokens": L_idx,
-                                          "spans": ns, "width": rcfg.width, "stride": rcfg.stride, "top": rcfg.s},
-                   "l2_policy": "inputs larger than L2: every step reads a different 80 MB activation chunk and 1.1 GB of encoder weights",
-                   "parallelism": "independent context replicas per GPU, no collectives"},
+        "config": workload_config(cfg, rcfg, L_idx, ns),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "note": "host->device copies of the chunk's activations and the read-back of the selected spans are inside the timed region; postings also travel device->host (index append) in both numbers"},
         "gpu_launches": gpu_launches,
@@ -325,7 +338,7 @@ def run_reference(args, cpu_only_sample=None):
     return {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": warm,
             "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic", "impl": "reference",
-            "config": {"workload": cfg.name, "context_tokens": cfg.L, "chunk": cfg.chunk, "layers": cfg.n_layers},
+            "config": workload_config(cfg, rcfg, rcfg.scan.L, C.n_spans(rcfg.scan.L, rcfg.width, rcfg.stride)),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
