@@ -1,0 +1,145 @@
+"""GPU parity at the benchmark's full sizes and in its launch configuration (a whole 8192-token chunk of the
+128K-token workload per call, the batched postings build of all layers and both SAEs, the 256-query retrieval
+over a 32K-token index), checked on sampled outputs the CPU oracle can compute one by one and on properties
+that hold at any size. Integer results bit-exact; encode within the bf16 tolerance (see test_gpu_parity.py)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2601_17702_b200 as S
+from paper_2601_17702_b200.scan import SaeSlot, ScanPipeline, stage_index_on_device
+from parity import check_topk_against_preact, csr_equal
+from workloads import configs as C, generators as G
+
+pytestmark = pytest.mark.gpu
+TOL_BF16 = 2e-2
+
+
+def _dev():
+    assert torch.cuda.is_available()
+    return torch.device("cuda:0")
+
+
+def _sample_rows(T, n=48):
+    return np.unique(np.concatenate([np.arange(0, n), np.arange(T // 2 - n // 2, T // 2 + n // 2), np.arange(T - n, T),
+                                     np.arange(255, 258), np.arange(127, 130)]))
+
+
+@pytest.mark.parametrize("which,layer,chunk_idx", [("key", 0, 0), ("key", 3, 15), ("query", 2, 7)])
+def test_cfg3_full_chunk_encode_sampled_rows(which, layer, chunk_idx):
+    cfg = C.CFG3
+    shp = cfg.key if which == "key" else cfg.query
+    inp = C.ScanInputs(cfg)
+    W, b_enc, b_dec = inp.sae(which, layer)
+    x = inp.x(which, layer, chunk_idx * cfg.chunk, cfg.chunk)
+    d = _dev()
+    sae = S.Sae(W.to(d), b_enc.to(d), b_dec.to(d))
+    ws = S.new_workspace(sae.encode_workspace_bytes(cfg.chunk, shp.k))
+    ids = torch.full((cfg.chunk, shp.k), -7, dtype=torch.int32, device=d)
+    vals = torch.full((cfg.chunk, shp.k), -7.0, dtype=torch.float32, device=d)
+    S.s3_sae_encode_topk(sae, x.to(d), shp.k, ids, vals, ws)
+    assert S.s3_workspace_status(ws) == 0
+    ids, vals = ids.cpu().numpy(), vals.cpu().numpy()
+    rows = _sample_rows(cfg.chunk)
+    pre = O.preact(x[rows].float().numpy(), W.float().numpy(), b_enc.numpy(), b_dec.numpy())
+    check_topk_against_preact(pre, ids[rows], vals[rows], shp.k, TOL_BF16)
+    # properties of every row: k distinct ids in range, values positive and descending
+    assert (ids >= 0).all() and (ids < shp.d_sae).all()
+    assert (np.sort(ids, axis=1)[:, 1:] != np.sort(ids, axis=1)[:, :-1]).all()
+    assert (vals > 0).all() and (np.diff(vals, axis=1) <= 0).all()
+
+
+def test_cfg3_batched_postings_and_index_full_chunk():
+    """All 8 chunk-layers of one benchmark step through the batched postings build and the host index; two
+    chunks, so that the merged CSR spans a chunk boundary. Bit-exact against the oracle on the same ids."""
+    cfg = C.CFG3
+    d = _dev()
+    T = cfg.chunk
+    rng = np.random.default_rng(5)
+    shapes = [(cfg.key.k, cfg.key.d_sae)] * 4 + [(cfg.query.k, cfg.query.d_sae)] * 4
+    indexes = [S.Index(1, D, 8 << 20) for _, D in shapes]
+    bufs = [(torch.zeros(D + 1, dtype=torch.int32, device=d), torch.zeros(T * k, dtype=torch.int32, device=d)) for k, D in shapes]
+    ws = S.new_workspace(sum(S.s3_postings_workspace_bytes(T, k, D) for k, D in shapes))
+    ref = [[] for _ in shapes]
+    for c in range(2):
+        ids_h = []
+        for k, D in shapes:      # k distinct ids per token: random start + distinct strides modulo D
+            start = rng.integers(0, D, size=(T, 1))
+            ids_h.append(((start + np.arange(k)[None, :] * 257) % D).astype(np.int32))
+        ids_d = [torch.as_tensor(a).to(d) for a in ids_h]
+        for ix in indexes:
+            ix.stream_wait()
+        items = [S.make_postings_item(ids_d[i], D, c * T, bufs[i][0], bufs[i][1]) for i, (k, D) in enumerate(shapes)]
+        S.s3_postings_build_batched(items, ws)
+        for i, (k, D) in enumerate(shapes):
+            indexes[i].append(0, bufs[i][0], bufs[i][1], T, k, c * T)
+            ref[i].append(O.postings(ids_h[i], D, c * T)[:2])
+    assert S.s3_workspace_status(ws) == 0
+    for i, (k, D) in enumerate(shapes):
+        rp, ps, _ = indexes[i].export_csr(0)
+        orp, opos = O.index_merge(ref[i], D)
+        csr_equal(rp.numpy(), ps.numpy(), orp, opos)
+        assert indexes[i].stats()["n_postings"] == 2 * T * k      # P = L * layers * k (Sec. 3.4)
+        indexes[i].close()
+
+
+def test_cfg4_retrieval_sampled_queries():
+    """The benchmark's retrieval call (256 queries x 64 tokens, k 64, 2045 overlapping spans over a 32K-token
+    index, 0.5/0.5 fusion, top 16): every output of 12 sampled queries against the oracle, bit-exact."""
+    r = C.CFG4
+    d = _dev()
+    L, k, D = r.scan.L, r.scan.key.k, r.scan.key.d_sae
+    rng = np.random.default_rng(11)
+    start = rng.integers(0, D, size=(L, 1))
+    start[rng.random((L, 1)) < 0.3] = 7                  # feature 7 is popular: a posting list of ~10K entries
+    ctx = ((start + np.arange(k)[None, :] * 131) % D).astype(np.int32)      # k distinct ids per token
+    qs = rng.integers(0, D, size=(r.Q * r.nq, 1))
+    qs[::r.nq] = 7                                       # every query has the popular feature in its first token
+    q = ((qs + np.arange(r.kq)[None, :] * 67) % D).astype(np.int32).reshape(1, r.Q, r.nq, r.kq)
+    qv = rng.random(q.shape).astype(np.float32)
+    ns = C.n_spans(L, r.width, r.stride)
+    bm = G.gamma21(r.bm25_seed, r.Q, ns)
+    rp, pos, _ = O.postings(ctx, D, 0)
+    layers = [(torch.as_tensor(rp.astype(np.int64)).to(d), torch.as_tensor(pos).to(d))]
+    alls = torch.zeros((r.Q, ns), dtype=torch.float32, device=d)
+    ws = S.new_workspace(64)
+    ti, ts = S.s3_coactivation_score_topspans(layers, D, L, torch.as_tensor(q).to(d), torch.as_tensor(qv).to(d), r.width, r.stride,
+                                              r.s, r.alpha, r.beta, ws, bm.to(d), all_scores=alls)
+    assert S.s3_workspace_status(ws) == 0
+    ti, ts, alls = ti.cpu().numpy(), ts.cpu().numpy(), alls.cpu().numpy()
+    sample = [0, 1, 2, 63, 64, 127, 128, 200, 253, 254, 255, 100]
+    co = O.score_spans(ctx[None], q[:, sample], qv[:, sample], D, r.width, r.stride, 0)
+    oi, os_, oall = O.fuse_select(co, bm.numpy()[sample], r.alpha, r.beta, r.s)
+    np.testing.assert_array_equal(alls[sample], oall)
+    np.testing.assert_array_equal(ti[sample], oi)
+    np.testing.assert_array_equal(ts[sample], os_)
+    # every query: the selected spans are the best of its own scores, in order
+    for qi in range(r.Q):
+        order = np.lexsort((np.arange(ns), -alls[qi]))[:r.s]
+        assert ti[qi].tolist() == order.tolist()
+
+
+def test_scan_device_memory_is_flat_across_chunks():
+    """Sec. 3.4 / memory-complexity proposition: device memory is bounded by the chunk, not by the context.
+    After the first chunk, scanning more chunks allocates nothing on the device; the index grows on the host."""
+    cfg = C.CFG2
+    d = _dev()
+    inp = C.ScanInputs(cfg, device=d)
+    sae = S.Sae(*inp.sae("key", 0))
+    pipe = ScanPipeline([SaeSlot("key", [sae], cfg.key.k, cfg.chunk)])
+    pipe.reserve_index(cfg.L)
+    xs = [inp.x("key", 0, c * cfg.chunk, cfg.chunk) for c in range(2)]
+    pipe.scan_chunk(0, {"key": [xs[0]]})
+    torch.cuda.synchronize()
+    base = torch.cuda.memory_allocated()
+    torch.cuda.reset_peak_memory_stats()
+    for c in range(1, cfg.n_chunks):
+        pipe.scan_chunk(c * cfg.chunk, {"key": [xs[c % 2]]})
+    pipe.finish()
+    assert torch.cuda.max_memory_allocated() == base and torch.cuda.memory_allocated() == base
+    st = pipe.slots[0].index.stats()
+    assert st["n_postings"] == cfg.L * cfg.key.k and st["n_positions"] == cfg.L
+    csr = stage_index_on_device(pipe.slots[0].index, d)
+    assert int(csr[0][0][-1].item()) == cfg.L * cfg.key.k
+    pipe.close()
