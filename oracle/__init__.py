@@ -131,3 +131,23 @@ def fuse_select(base, bm25, alpha: float, beta: float, s: int):
                           C.c_int(Q), C.c_int64(ns), C.c_int(s), _p(top_idx, C.c_int32), _p(top_score, C.c_float),
                           _p(allsc, C.c_float))
     return top_idx, top_score, allsc[:, :ns]
+
+
+def position_density(ctx_ids, q_ids, q_vals, d_sae: int, conv_kernel: int, nms_radius: int, n_centers: int,
+                     stop_freq: int = 0):
+    """Per-position relevance S (Eq. 6), its box-smoothed density S' and the NMS peak positions.
+    ctx_ids [n_layers, L, k]; q_ids/q_vals [n_layers, Q, nq, kq].
+    Returns (S fp64 [Q,L], D fp64 [Q,L], centers int32 [Q,n_centers] (-1 = none), center_density fp32 [Q,n_centers])."""
+    ctx_ids, q_ids, q_vals = _i32(ctx_ids), _i32(q_ids), _f32(q_vals)
+    n_layers, L, k = ctx_ids.shape
+    _, Q, nq, kq = q_ids.shape
+    assert q_ids.shape[0] == n_layers and q_vals.shape == q_ids.shape
+    S = np.zeros((Q, L), dtype=np.float64)
+    D = np.zeros((Q, L), dtype=np.float64)
+    centers = np.empty((Q, n_centers), dtype=np.int32)
+    dens = np.empty((Q, n_centers), dtype=np.float32)
+    lib().s3o_position_density(_p(ctx_ids, C.c_int32), C.c_int64(L), C.c_int(k), C.c_int(d_sae), C.c_int(n_layers),
+                               _p(q_ids, C.c_int32), _p(q_vals, C.c_float), C.c_int(Q), C.c_int(nq), C.c_int(kq),
+                               C.c_int(conv_kernel), C.c_int(nms_radius), C.c_int(n_centers), C.c_int64(stop_freq),
+                               _p(S, C.c_double), _p(D, C.c_double), _p(centers, C.c_int32), _p(dens, C.c_float))
+    return S, D, centers, dens

@@ -229,6 +229,86 @@ void s3o_fuse_select(const int64_t* coact, const double* wscore, const float* bm
     }
 }
 
+// Sec. 3.5, "Semantic Density Estimation" and "Adaptive Granularity" (Eq. 6; Alg. 1, Phase 2: S <- accumulate,
+// S' <- Conv1D(S), Idx <- NMS_Select(S', top_k)), straight from the tokens' feature sets.
+//
+//   S[t]  = sum_l sum_{f in F_t^(l)} w_l(f),   w_l(f) = aQ_l(f) * IDF_l(f) for the query's features (else 0)
+//   S'[t] = sum_{d=0}^{K-1} S[t - floor(K/2) + d]          (positions outside [0, L) count as 0)
+//   centres: repeat n_centers times: the alive position with the largest S' (ties: lowest position); stop
+//            when nothing alive has S' > 0; positions within nms_radius of a centre are no longer alive.
+// Readings (the paper leaves these open): the query's tokens are aggregated as in s3o_score_spans, with
+// aQ_l(f) summed in fp32 in query-token order; the smoothing kernel is a box of K unit taps centred on t;
+// suppression is by distance to the chosen centres. So that the peak positions (an argmax) do not depend
+// on summation order, every weight is taken in fixed point, w = rint(aQ * IDF * 2^24) / 2^24, and S, S' are
+// then exact integer sums; this is the precision the selection is made in.
+// Features with freq > stop_freq are skipped when stop_freq > 0.
+void s3o_position_density(const int32_t* ctx_ids, int64_t L, int k, int d_sae, int n_layers,
+                          const int32_t* q_ids, const float* q_vals, int Q, int nq, int kq,
+                          int conv_kernel, int nms_radius, int n_centers, int64_t stop_freq,
+                          double* S /*[Q,L] or null*/, double* D /*[Q,L] or null*/,
+                          int32_t* centers /*[Q,n_centers]*/, float* center_density /*[Q,n_centers]*/)
+{
+    std::vector<std::vector<int64_t>> freq(n_layers, std::vector<int64_t>(d_sae, 0));
+    for (int l = 0; l < n_layers; ++l)
+        for (int64_t t = 0; t < L; ++t)
+            for (int j = 0; j < k; ++j) {
+                const int32_t f = ctx_ids[((int64_t)l * L + t) * k + j];
+                if (f >= 0) freq[l][f] += 1;
+            }
+    const double scale = 16777216.0;   // 2^24
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int q = 0; q < Q; ++q) {
+        std::vector<int64_t> s_fix(L, 0), d_fix(L, 0);
+        std::vector<int64_t> w(d_sae);
+        std::vector<float> aQ(d_sae);
+        std::vector<char> inq(d_sae);
+        for (int l = 0; l < n_layers; ++l) {
+            std::fill(aQ.begin(), aQ.end(), 0.0f);
+            std::fill(inq.begin(), inq.end(), 0);
+            for (int u = 0; u < nq; ++u)
+                for (int j = 0; j < kq; ++j) {
+                    const int64_t o = (((int64_t)l * Q + q) * nq + u) * kq + j;
+                    const int32_t f = q_ids[o];
+                    if (f >= 0) { volatile float sum = aQ[f] + q_vals[o]; aQ[f] = sum; inq[f] = 1; }
+                }
+            for (int f = 0; f < d_sae; ++f) {
+                w[f] = 0;
+                if (!inq[f]) continue;
+                if (stop_freq > 0 && freq[l][f] > stop_freq) continue;
+                w[f] = (int64_t)std::llrint((double)aQ[f] * s3o_idf((double)freq[l][f]) * scale);
+            }
+            for (int64_t t = 0; t < L; ++t)
+                for (int j = 0; j < k; ++j) {
+                    const int32_t f = ctx_ids[((int64_t)l * L + t) * k + j];
+                    if (f >= 0) s_fix[t] += w[f];
+                }
+        }
+        const int64_t half = conv_kernel / 2;
+        for (int64_t t = 0; t < L; ++t) {
+            int64_t sum = 0;
+            for (int64_t d = 0; d < conv_kernel; ++d) {
+                const int64_t u = t - half + d;
+                if (u >= 0 && u < L) sum += s_fix[u];
+            }
+            d_fix[t] = sum;
+        }
+        for (int64_t t = 0; t < L; ++t) {
+            if (S) S[q * L + t] = (double)s_fix[t] / scale;
+            if (D) D[q * L + t] = (double)d_fix[t] / scale;
+        }
+        std::vector<char> alive(L, 1);
+        for (int i = 0; i < n_centers; ++i) {
+            int64_t best = -1;
+            for (int64_t t = 0; t < L; ++t)
+                if (alive[t] && d_fix[t] > 0 && (best < 0 || d_fix[t] > d_fix[best])) best = t;
+            if (best < 0) { centers[q * n_centers + i] = -1; center_density[q * n_centers + i] = 0.0f; continue; }
+            centers[q * n_centers + i] = (int32_t)best;
+            center_density[q * n_centers + i] = (float)((double)d_fix[best] / scale);
+            for (int64_t t = std::max<int64_t>(0, best - nms_radius); t <= std::min<int64_t>(L - 1, best + nms_radius); ++t) alive[t] = 0;
+        }
+    }
+}
+
 int s3o_num_threads(void)
 {
     int n = 1;
