@@ -250,6 +250,42 @@ s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_laye
                                          float* d_all_scores /*[Q,n_spans] nullable*/,
                                          void* d_ws, size_t ws_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Per-position relevance, semantic density and peak selection
+ *            (paper Sec. 3.5 Eq. 6 "Semantic Density Estimation" and "Adaptive Granularity";
+ *             Alg. 1 Phase 2: S <- accumulate, S' <- Conv1D(S), Idx <- NMS_Select(S', top_k))
+ *
+ * Per query q, with the query aggregation of s3_coactivation_score_topspans (aQ_l(f) = the query tokens'
+ * activations of f summed in fp32 in token order; IDF_l(f) = 1/(ln(1+freq_l(f))+1), freq = posting-list
+ * length; lists longer than stop_freq > 0 are skipped):
+ *   S[t]  = sum_l sum_{f in query} [t in I_l[f]] * w_l(f),     w_l(f) = rint(aQ_l(f) * IDF_l(f) * 2^24) / 2^24
+ *   S'[t] = sum_{d=0}^{K-1} S[t - floor(K/2) + d]               (box of K = conv_kernel unit taps centred on t,
+ *                                                                 positions outside [0, L) count as 0)
+ *   centres: n_centers rounds of "alive position with the largest S' (ties: lowest position)"; a round finds
+ *            nothing once no alive position has S' > 0 (centre -1, density 0); positions within nms_radius
+ *            of a chosen centre are no longer alive.
+ * The fixed-point weights make S and S' exact integer sums, so the peaks do not depend on the order in
+ * which postings are visited and are bit-identical to the CPU definition. The shape of the smoothing
+ * kernel, the suppression rule and the multi-token aggregation are readings of points the paper leaves open.
+ *
+ * h_layers as for s3_coactivation_score_topspans. Outputs: d_centers [Q, n_centers] int32, d_center_density
+ * [Q, n_centers] fp32 (S' at the centre); d_S / d_density (nullable) [Q, L] fp32 copies of S and S'.
+ * Limits: n_layers <= S3_MAX_SCORE_LAYERS; nq*k <= 4096; 1 <= conv_kernel <= 1024; nms_radius >= 0;
+ *         1 <= n_centers <= 1024; L <= 4194304. Workspace: s3_density_workspace_bytes(Q, L)
+ *         (two 64-bit words per query and position, plus the status block).
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t conv_kernel, nms_radius, n_centers, reserved;
+    int64_t stop_freq; /* 0 = off */
+} s3_density_params;
+
+size_t s3_density_workspace_bytes(int Q, int64_t L);
+s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L,
+                                         const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
+                                         const s3_density_params* params, int32_t* d_centers /*[Q,n_centers]*/,
+                                         float* d_center_density /*[Q,n_centers]*/, float* d_S /*[Q,L] nullable*/,
+                                         float* d_density /*[Q,L] nullable*/, void* d_ws, size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

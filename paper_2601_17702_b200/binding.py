@@ -27,6 +27,7 @@ EXPORTS = [
     "s3_index_create", "s3_index_reserve", "s3_index_append", "s3_index_stream_wait", "s3_index_sync",
     "s3_index_stats", "s3_index_layer_postings", "s3_index_export_csr", "s3_index_destroy",
     "s3_score_workspace_bytes", "s3_coactivation_score_topspans",
+    "s3_density_workspace_bytes", "s3_position_density_topcenters",
 ]
 
 
@@ -51,6 +52,11 @@ class ScoreParams(C.Structure):
                 ("alpha", C.c_float), ("beta", C.c_float), ("stop_freq", C.c_int64)]
 
 
+class DensityParams(C.Structure):
+    _fields_ = [("conv_kernel", C.c_int32), ("nms_radius", C.c_int32), ("n_centers", C.c_int32), ("reserved", C.c_int32),
+                ("stop_freq", C.c_int64)]
+
+
 class IndexStats(C.Structure):
     _fields_ = [("n_chunks", C.c_int64), ("n_postings", C.c_int64), ("host_bytes", C.c_int64),
                 ("host_bytes_reserved", C.c_int64), ("max_list_len", C.c_int64), ("n_positions", C.c_int64)]
@@ -69,7 +75,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.s3_last_error.restype = C.c_char_p
         for name in ("s3_sae_prepared_bytes", "s3_sae_encode_workspace_bytes", "s3_postings_workspace_bytes",
-                     "s3_score_workspace_bytes"):
+                     "s3_score_workspace_bytes", "s3_density_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.s3_sae_prepared_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_sae_create.argtypes = [C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
@@ -101,6 +107,10 @@ def lib():
                                                      C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(ScoreParams),
                                                      C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                                      C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_density_workspace_bytes.argtypes = [C.c_int, C.c_int64]
+        L.s3_position_density_topcenters.argtypes = [C.POINTER(CsrView), C.c_int, C.c_int, C.c_int64, C.c_void_p, C.c_void_p,
+                                                     C.c_int, C.c_int, C.c_int, C.POINTER(DensityParams), C.c_void_p,
+                                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         _lib = L
     return _lib
 
@@ -303,3 +313,29 @@ def s3_coactivation_score_topspans(layers, d_sae: int, L: int, q_ids: torch.Tens
                                                 C.byref(params), _ptr(bm25), ld, _ptr(top_idx), _ptr(top_score),
                                                 _ptr(all_scores), _ptr(ws), ws.numel(), _stream(stream)))
     return top_idx, top_score
+
+
+def s3_density_workspace_bytes(Q: int, L: int) -> int:
+    return int(lib().s3_density_workspace_bytes(Q, L))
+
+
+def s3_position_density_topcenters(layers, d_sae: int, L: int, q_ids: torch.Tensor, q_vals: torch.Tensor, conv_kernel: int,
+                                   nms_radius: int, n_centers: int, ws: torch.Tensor, stop_freq: int = 0,
+                                   S_out: torch.Tensor | None = None, density_out: torch.Tensor | None = None, stream=None):
+    """layers: list of (row_ptr int64 [d_sae+1], pos int32) device tensors; q_ids/q_vals [n_layers, Q, nq, k].
+    Returns (centers int32 [Q, n_centers], center_density fp32 [Q, n_centers]); S_out / density_out (optional,
+    fp32 [Q, L]) receive the per-position relevance and its smoothed density."""
+    n_layers, Q, nq, k = q_ids.shape
+    assert len(layers) == n_layers and q_ids.dtype == torch.int32 and q_vals.dtype == torch.float32
+    assert q_ids.is_contiguous() and q_vals.is_contiguous()
+    views = (CsrView * n_layers)(*[CsrView(rp.data_ptr(), ps.data_ptr()) for rp, ps in layers])
+    for rp, ps in layers:
+        assert rp.dtype == torch.int64 and ps.dtype == torch.int32 and rp.numel() == d_sae + 1
+    dev = q_ids.device
+    centers = torch.empty((Q, n_centers), dtype=torch.int32, device=dev)
+    dens = torch.empty((Q, n_centers), dtype=torch.float32, device=dev)
+    params = DensityParams(conv_kernel, nms_radius, n_centers, 0, stop_freq)
+    _check(lib().s3_position_density_topcenters(views, n_layers, d_sae, L, _ptr(q_ids), _ptr(q_vals), Q, nq, k,
+                                                C.byref(params), _ptr(centers), _ptr(dens), _ptr(S_out), _ptr(density_out),
+                                                _ptr(ws), ws.numel(), _stream(stream)))
+    return centers, dens

@@ -308,4 +308,38 @@ s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_laye
                         d_top_score, d_all_scores, static_cast<cudaStream_t>(stream));
 }
 
+// ---------------------------------------------------------------------------------------------- density
+size_t s3_density_workspace_bytes(int Q, int64_t L)
+{
+    if (Q < 0 || L < 0) return 0;
+    return 256 + density_workspace_bytes(Q, L);
+}
+
+s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L,
+                                         const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
+                                         const s3_density_params* p, int32_t* d_centers, float* d_center_density, float* d_S,
+                                         float* d_density, void* d_ws, size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(h_layers && p, S3_ERR_INVALID_ARG, "null argument");
+    S3_REQUIRE(n_layers >= 1 && n_layers <= S3_MAX_SCORE_LAYERS, S3_ERR_UNSUPPORTED, "n_layers = %d out of [1, %d]", n_layers,
+               S3_MAX_SCORE_LAYERS);
+    S3_REQUIRE(d_sae >= 1 && d_sae <= (1 << 20), S3_ERR_INVALID_ARG, "d_sae = %d out of range", d_sae);
+    S3_REQUIRE(L >= 0, S3_ERR_INVALID_ARG, "L is negative");
+    S3_REQUIRE(L <= 4194304, S3_ERR_UNSUPPORTED, "L = %lld exceeds 4194304", (long long)L);
+    S3_REQUIRE(Q >= 0 && nq >= 1 && k >= 1, S3_ERR_INVALID_ARG, "Q = %d, nq = %d, k = %d out of range", Q, nq, k);
+    S3_REQUIRE((int64_t)nq * k <= 4096, S3_ERR_UNSUPPORTED, "nq*k = %lld exceeds 4096", (long long)nq * k);
+    S3_REQUIRE(p->conv_kernel >= 1 && p->nms_radius >= 0 && p->n_centers >= 1, S3_ERR_INVALID_ARG,
+               "conv_kernel = %d, nms_radius = %d, n_centers = %d out of range", p->conv_kernel, p->nms_radius, p->n_centers);
+    S3_REQUIRE(p->conv_kernel <= 1024 && p->n_centers <= 1024, S3_ERR_UNSUPPORTED, "conv_kernel and n_centers may not exceed 1024");
+    if (Q == 0) return S3_OK;
+    S3_REQUIRE(d_q_ids && d_q_vals && d_centers && d_center_density, S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE(d_ws != nullptr && ws_bytes >= s3_density_workspace_bytes(Q, L), S3_ERR_CAPACITY,
+               "workspace holds %zu bytes, %zu needed", ws_bytes, s3_density_workspace_bytes(Q, L));
+    for (int l = 0; l < n_layers; ++l)
+        S3_REQUIRE(h_layers[l].d_row_ptr && h_layers[l].d_pos, S3_ERR_INVALID_ARG, "layer %d: null CSR pointer", l);
+    return launch_density(h_layers, n_layers, d_sae, L, d_q_ids, d_q_vals, Q, nq, k, p->conv_kernel, p->nms_radius, p->n_centers,
+                          p->stop_freq, d_centers, d_center_density, d_S, d_density, static_cast<unsigned char*>(d_ws) + 256,
+                          static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"

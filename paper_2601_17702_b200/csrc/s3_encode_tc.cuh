@@ -39,4 +39,10 @@ s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, con
                        const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
                        float* d_all_scores, cudaStream_t stream);
 
+size_t density_workspace_bytes(int Q, int64_t L);
+s3_status launch_density(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L, const int32_t* d_q_ids,
+                         const float* d_q_vals, int Q, int nq, int k, int conv_kernel, int nms_radius, int n_centers,
+                         int64_t stop_freq, int32_t* d_centers, float* d_center_density, float* d_s_out, float* d_d_out,
+                         void* d_scratch, cudaStream_t stream);
+
 }  // namespace s3

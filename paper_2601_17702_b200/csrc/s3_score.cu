@@ -107,6 +107,96 @@ __device__ __forceinline__ void posting_range(const ScoreArgs& a, int p, int p_p
     j_hi = j_hi < a.n_spans - 1 ? j_hi : a.n_spans - 1;
 }
 
+// Phase a, shared by the scoring kernels: the query's nk (id, value) entries -> unique features. Sorts
+// (id, entry) keys ascending (invalid ids last), detects runs: ufeat[u] = id, ustart[u]..ustart[u+1] = its
+// entries in keys[] (so cQ = ustart[u+1] - ustart[u]), and, if wanted, uaq[u] = the entries' activations summed
+// in query-token order in fp32. Returns the number of unique features. Called by the whole block.
+__device__ __forceinline__ int aggregate_query(const int32_t* qi, const float* qv, int nk, int npad, int d_sae, bool want_aq,
+                                               uint32_t* keys, int32_t* ufeat, int32_t* ustart, float* uaq, uint32_t* ws,
+                                               int* n_unique_s)
+{
+    const int tid = threadIdx.x;
+    for (int i = tid; i < npad; i += ST) {
+        uint32_t key = 0xFFFFFFFFu;
+        if (i < nk) {
+            const int32_t f = qi[i];
+            if (f >= 0 && f < d_sae) key = (static_cast<uint32_t>(f) << 12) | static_cast<uint32_t>(i);
+        }
+        keys[i] = key;
+    }
+    __syncthreads();
+    for (int size = 2; size <= npad; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int i = tid; i < (npad >> 1); i += ST) {
+                const int pos = 2 * i - (i & (stride - 1));   // stride is a power of two
+                const bool asc = (pos & size) == 0;
+                const uint32_t x = keys[pos], y = keys[pos + stride];
+                if ((x > y) == asc) { keys[pos] = y; keys[pos + stride] = x; }
+            }
+            __syncthreads();
+        }
+    }
+    uint32_t carry = 0;
+    for (int i0 = 0; i0 < nk; i0 += ST) {
+        const int i = i0 + tid;
+        uint32_t head = 0;
+        if (i < nk && keys[i] != 0xFFFFFFFFu)
+            head = (i == 0) || ((keys[i] >> 12) != (keys[i - 1] >> 12));
+        uint32_t total;
+        const uint32_t u = block_exclusive_scan(head, ws, total) + carry;
+        if (head) { ufeat[u] = static_cast<int32_t>(keys[i] >> 12); ustart[u] = i; }
+        carry += total;
+    }
+    if (tid == 0) {
+        int lo = 0, hi = nk;   // first invalid key (keys sorted, invalid last)
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (keys[mid] == 0xFFFFFFFFu) hi = mid; else lo = mid + 1; }
+        ustart[carry] = lo;
+        *n_unique_s = static_cast<int>(carry);
+    }
+    __syncthreads();
+    const int U = *n_unique_s;
+    for (int u = tid; want_aq && u < U; u += ST) {   // aQ: activations summed in query-token order (fp32)
+        float s = 0.0f;
+        for (int i = ustart[u]; i < ustart[u + 1]; ++i) s = __fadd_rn(s, qv[keys[i] & 0xFFFu]);
+        uaq[u] = s;
+    }
+    __syncthreads();
+    return U;
+}
+
+// Phase b head, shared by the scoring kernels: list bounds of the U unique features (ulo, ulen; a list longer
+// than stop_freq > 0 counts as empty) and the exclusive prefix cstart[0..U] of their 32-posting pieces. ulen
+// may share storage with keys, cstart with ufeat (a thread reads ufeat[u] before it writes cstart[u]).
+// Returns the number of pieces. Called by the whole block.
+__device__ __forceinline__ uint32_t cut_lists(const uint64_t* __restrict__ row_ptr, int U, int64_t stop_freq,
+                                              const int32_t* ufeat, unsigned long long* ulo, uint32_t* ulen,
+                                              uint32_t* cstart, uint32_t* ws)
+{
+    const int tid = threadIdx.x;
+    uint32_t piece_carry = 0;
+    for (int u0 = 0; u0 < U; u0 += ST) {
+        const int u = u0 + tid;
+        uint32_t n_pieces = 0;
+        if (u < U) {
+            const int f = ufeat[u];
+            const uint64_t lo = __ldg(row_ptr + f), hi = __ldg(row_ptr + f + 1);
+            uint64_t len = hi - lo;
+            if (len > 0x7FFFFFFFull) len = 0x7FFFFFFFull;          // positions are int32: a list cannot be longer
+            if (stop_freq > 0 && static_cast<int64_t>(len) > stop_freq) len = 0;   // stop feature
+            ulo[u] = lo;
+            ulen[u] = static_cast<uint32_t>(len);
+            n_pieces = static_cast<uint32_t>((len + PIECE - 1) / PIECE);
+        }
+        uint32_t total;
+        const uint32_t ex = block_exclusive_scan(n_pieces, ws, total) + piece_carry;
+        if (u < U) cstart[u] = ex;
+        piece_carry += total;
+    }
+    if (tid == 0) cstart[U] = piece_carry;
+    __syncthreads();
+    return piece_carry;
+}
+
 __global__ void __launch_bounds__(ST)
 score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__ ScoreArgs a)
 {
@@ -138,81 +228,13 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
     for (int l = 0; l < a.n_layers; ++l) {
         const int32_t* qi = a.q_ids + ((size_t)l * a.Q + q) * a.nk;
         const float* qv = a.q_vals + ((size_t)l * a.Q + q) * a.nk;
-        // a. sort (id, entry) keys ascending; invalid ids sort last
-        for (int i = tid; i < a.npad; i += ST) {
-            uint32_t key = 0xFFFFFFFFu;
-            if (i < a.nk) {
-                const int32_t f = qi[i];
-                if (f >= 0 && f < a.d_sae) key = (static_cast<uint32_t>(f) << 12) | static_cast<uint32_t>(i);
-            }
-            keys[i] = key;
-        }
-        __syncthreads();
-        for (int size = 2; size <= a.npad; size <<= 1) {
-            for (int stride = size >> 1; stride > 0; stride >>= 1) {
-                for (int i = tid; i < (a.npad >> 1); i += ST) {
-                    const int pos = 2 * i - (i & (stride - 1));   // stride is a power of two
-                    const bool asc = (pos & size) == 0;
-                    const uint32_t x = keys[pos], y = keys[pos + stride];
-                    if ((x > y) == asc) { keys[pos] = y; keys[pos + stride] = x; }
-                }
-                __syncthreads();
-            }
-        }
-        // run detection -> unique features
-        uint32_t carry = 0;
-        for (int i0 = 0; i0 < a.nk; i0 += ST) {
-            const int i = i0 + tid;
-            uint32_t head = 0;
-            if (i < a.nk && keys[i] != 0xFFFFFFFFu)
-                head = (i == 0) || ((keys[i] >> 12) != (keys[i - 1] >> 12));
-            uint32_t total;
-            const uint32_t u = block_exclusive_scan(head, ws, total) + carry;
-            if (head) { ufeat[u] = static_cast<int32_t>(keys[i] >> 12); ustart[u] = i; }
-            carry += total;
-        }
-        if (tid == 0) {
-            int lo = 0, hi = a.nk;   // first invalid key (keys sorted, invalid last)
-            while (lo < hi) { const int mid = (lo + hi) >> 1; if (keys[mid] == 0xFFFFFFFFu) hi = mid; else lo = mid + 1; }
-            ustart[carry] = lo;
-            n_unique_s = static_cast<int>(carry);
-        }
-        __syncthreads();
-        const int U = n_unique_s;
-        for (int u = tid; weighted && u < U; u += ST) {   // aQ: activations summed in query-token order (fp32)
-            float s = 0.0f;
-            for (int i = ustart[u]; i < ustart[u + 1]; ++i) s = __fadd_rn(s, qv[keys[i] & 0xFFFu]);
-            uaq[u] = s;
-        }
-        __syncthreads();
-
+        const int U = aggregate_query(qi, qv, a.nk, a.npad, a.d_sae, weighted, keys, ufeat, ustart, uaq, ws, &n_unique_s);
         // b. list bounds of every unique feature (independent loads), then the pieces' prefix sum
-        const uint64_t* __restrict__ row_ptr = layers.v[l].d_row_ptr;
         const int32_t* __restrict__ pos = layers.v[l].d_pos;
-        uint32_t piece_carry = 0;
-        for (int u0 = 0; u0 < U; u0 += ST) {
-            const int u = u0 + tid;
-            uint32_t n_pieces = 0;
-            if (u < U) {
-                const int f = ufeat[u];
-                const uint64_t lo = __ldg(row_ptr + f), hi = __ldg(row_ptr + f + 1);
-                uint64_t len = hi - lo;
-                if (len > 0x7FFFFFFFull) len = 0x7FFFFFFFull;          // positions are int32: a list cannot be longer
-                if (weighted && a.stop_freq > 0 && static_cast<int64_t>(len) > a.stop_freq) len = 0;   // stop feature
-                ulo[u] = lo;
-                ulen[u] = static_cast<uint32_t>(len);
-                n_pieces = static_cast<uint32_t>((len + PIECE - 1) / PIECE);
-            }
-            uint32_t total;
-            const uint32_t ex = block_exclusive_scan(n_pieces, ws, total) + piece_carry;
-            if (u < U) cstart[u] = ex;
-            piece_carry += total;
-        }
-        if (tid == 0) cstart[U] = piece_carry;
-        __syncthreads();
+        const uint32_t piece_total = cut_lists(layers.v[l].d_row_ptr, U, weighted ? a.stop_freq : 0, ufeat, ulo, ulen, cstart, ws);
 
         // each warp takes an equal share of consecutive pieces and walks them with a running feature cursor
-        const uint32_t n_pieces_total = piece_carry;
+        const uint32_t n_pieces_total = piece_total;
         const uint32_t c_begin = static_cast<uint32_t>(static_cast<uint64_t>(n_pieces_total) * warp / SW);
         const uint32_t c_end = static_cast<uint32_t>(static_cast<uint64_t>(n_pieces_total) * (warp + 1) / SW);
         if (c_begin < c_end) {
@@ -321,6 +343,175 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
     }
 }
 
+// ---- per-position relevance, smoothed density, peak selection (Sec. 3.5 Eq. 6, "Adaptive Granularity") --------
+// One block per query. Weights are taken in fixed point (2^-24) so that S, the density and therefore the
+// peaks are exact integer results whatever order the postings are visited in:
+//   1. S[t] += w_l(f) for every posting t of every query feature (64-bit integer atomics in global memory);
+//   2. density D[t] = sum of S over the K positions starting at t - K/2 (zero outside [0, L));
+//   3. greedy non-maximum suppression over D with per-segment maxima in shared memory: a round reduces the
+//      segment maxima, takes the best position (ties: lowest), clears D within the radius and redoes only
+//      the touched segments.
+constexpr int SEG = 2048;            // positions per segment of the maxima table
+constexpr int MAX_SEGS = 2048;       // L <= SEG * MAX_SEGS
+
+struct DensityArgs {
+    const int32_t* q_ids;
+    const float* q_vals;
+    long long* s_fix;        // [Q][L]
+    long long* d_fix;        // [Q][L]
+    int32_t* centers;        // [Q][n_centers]
+    float* center_density;   // [Q][n_centers]
+    float* s_out;            // [Q][L] or null
+    float* d_out;            // [Q][L] or null
+    long long L;
+    int n_layers, d_sae, Q, nk, npad, conv_kernel, nms_radius, n_centers;
+    int64_t stop_freq;
+};
+
+__device__ __forceinline__ bool better(long long v, long long p, long long bv, long long bp)
+{
+    return v > bv || (v == bv && v > 0 && p < bp);
+}
+
+// Maximum (value, lowest position) of d[lo..hi) over the calling warp.
+__device__ __forceinline__ void warp_segment_max(const long long* d, long long lo, long long hi, int lane, long long& bv, long long& bp)
+{
+    bv = 0; bp = -1;
+    for (long long t = lo + lane; t < hi; t += 32) {
+        const long long v = d[t];
+        if (better(v, t, bv, bp)) { bv = v; bp = t; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const long long ov = __shfl_xor_sync(0xffffffffu, bv, o), op = __shfl_xor_sync(0xffffffffu, bp, o);
+        if (better(ov, op, bv, bp)) { bv = ov; bp = op; }
+    }
+}
+
+__global__ void __launch_bounds__(ST)
+density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__ DensityArgs a)
+{
+    extern __shared__ __align__(16) unsigned char score_smem_raw[];
+    const ScoreSmem SL = score_smem(a.nk, a.npad, 0, true);
+    unsigned long long* ulo = reinterpret_cast<unsigned long long*>(score_smem_raw + SL.ulo_off);
+    uint32_t* keys = reinterpret_cast<uint32_t*>(score_smem_raw + SL.keys_off);
+    uint32_t* ulen = keys;
+    int32_t* ufeat = reinterpret_cast<int32_t*>(score_smem_raw + SL.ufeat_off);
+    int32_t* ustart = reinterpret_cast<int32_t*>(score_smem_raw + SL.ustart_off);
+    float* uaq = reinterpret_cast<float*>(score_smem_raw + SL.uaq_off);
+    uint32_t* cstart = reinterpret_cast<uint32_t*>(score_smem_raw + SL.cstart_off);
+    long long* uw = reinterpret_cast<long long*>(score_smem_raw + ((SL.total + 15u) & ~15u));     // [nk] fixed-point weights
+    long long* seg_val = uw + a.nk;                                                               // [n_segs]
+    long long* seg_pos = seg_val + MAX_SEGS;
+    __shared__ uint32_t ws[SW + 1];
+    __shared__ int n_unique_s;
+    __shared__ long long red_v[SW], red_p[SW], pick_s;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int q = blockIdx.x;
+    const long long L = a.L;
+    long long* S = a.s_fix + (size_t)q * L;
+    long long* D = a.d_fix + (size_t)q * L;
+
+    for (long long t = tid; t < L; t += ST) S[t] = 0;
+    __syncthreads();
+
+    for (int l = 0; l < a.n_layers; ++l) {
+        const int32_t* qi = a.q_ids + ((size_t)l * a.Q + q) * a.nk;
+        const float* qv = a.q_vals + ((size_t)l * a.Q + q) * a.nk;
+        const int U = aggregate_query(qi, qv, a.nk, a.npad, a.d_sae, true, keys, ufeat, ustart, uaq, ws, &n_unique_s);
+        const int32_t* __restrict__ pos = layers.v[l].d_pos;
+        const uint32_t n_pieces_total = cut_lists(layers.v[l].d_row_ptr, U, a.stop_freq, ufeat, ulo, ulen, cstart, ws);
+        for (int u = tid; u < U; u += ST)      // w = rint(aQ * IDF(freq) * 2^24), IDF = 1 / (ln(1 + freq) + 1)
+            uw[u] = __double2ll_rn(static_cast<double>(uaq[u]) * (1.0 / (log(1.0 + static_cast<double>(ulen[u])) + 1.0)) * 16777216.0);
+        __syncthreads();
+        const uint32_t c_begin = static_cast<uint32_t>(static_cast<uint64_t>(n_pieces_total) * warp / SW);
+        const uint32_t c_end = static_cast<uint32_t>(static_cast<uint64_t>(n_pieces_total) * (warp + 1) / SW);
+        if (c_begin < c_end) {
+            int lo_u = 0, hi_u = U;              // last u with cstart[u] <= c_begin
+            while (hi_u - lo_u > 1) { const int mid = (lo_u + hi_u) >> 1; if (cstart[mid] <= c_begin) lo_u = mid; else hi_u = mid; }
+            int u = lo_u;
+            for (uint32_t c0 = c_begin; c0 < c_end; c0 += BATCH) {
+                int p[BATCH], ub[BATCH];
+#pragma unroll
+                for (int b = 0; b < BATCH; ++b) {
+                    const uint32_t c = c0 + b;
+                    p[b] = -1; ub[b] = 0;
+                    if (c < c_end) {
+                        while (cstart[u + 1] <= c) ++u;
+                        ub[b] = u;
+                        const uint32_t i = (c - cstart[u]) * PIECE + lane;
+                        if (i < ulen[u]) p[b] = __ldg(pos + ulo[u] + i);
+                    }
+                }
+#pragma unroll
+                for (int b = 0; b < BATCH; ++b)
+                    if (p[b] >= 0 && p[b] < L)
+                        atomicAdd(reinterpret_cast<unsigned long long*>(S + p[b]), static_cast<unsigned long long>(uw[ub[b]]));
+            }
+        }
+        __syncthreads();
+    }
+
+    // density: K taps starting at t - K/2
+    const long long half = a.conv_kernel / 2;
+    for (long long t = tid; t < L; t += ST) {
+        long long sum = 0;
+        const long long lo = t - half < 0 ? 0 : t - half;
+        const long long hi = t - half + a.conv_kernel > L ? L : t - half + a.conv_kernel;
+        for (long long u = lo; u < hi; ++u) sum += S[u];
+        D[t] = sum;
+        if (a.d_out) a.d_out[(size_t)q * L + t] = static_cast<float>(static_cast<double>(sum) * (1.0 / 16777216.0));
+        if (a.s_out) a.s_out[(size_t)q * L + t] = static_cast<float>(static_cast<double>(S[t]) * (1.0 / 16777216.0));
+    }
+    __syncthreads();
+
+    // segment maxima
+    const int n_segs = static_cast<int>((L + SEG - 1) / SEG);
+    for (int sg = warp; sg < n_segs; sg += SW) {
+        long long bv, bp;
+        const long long lo = (long long)sg * SEG, hi = lo + SEG < L ? lo + SEG : L;
+        warp_segment_max(D, lo, hi, lane, bv, bp);
+        if (lane == 0) { seg_val[sg] = bv; seg_pos[sg] = bp; }
+    }
+    __syncthreads();
+
+    for (int r = 0; r < a.n_centers; ++r) {
+        long long bv = 0, bp = -1;
+        for (int sg = tid; sg < n_segs; sg += ST)
+            if (better(seg_val[sg], seg_pos[sg], bv, bp)) { bv = seg_val[sg]; bp = seg_pos[sg]; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const long long ov = __shfl_xor_sync(0xffffffffu, bv, o), op = __shfl_xor_sync(0xffffffffu, bp, o);
+            if (better(ov, op, bv, bp)) { bv = ov; bp = op; }
+        }
+        if (lane == 0) { red_v[warp] = bv; red_p[warp] = bp; }
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 1; w < SW; ++w)
+                if (better(red_v[w], red_p[w], bv, bp)) { bv = red_v[w]; bp = red_p[w]; }
+            a.centers[(size_t)q * a.n_centers + r] = bv > 0 ? static_cast<int32_t>(bp) : -1;
+            a.center_density[(size_t)q * a.n_centers + r] = bv > 0 ? static_cast<float>(static_cast<double>(bv) * (1.0 / 16777216.0)) : 0.0f;
+            pick_s = bv > 0 ? bp : -1;
+        }
+        __syncthreads();
+        const long long c = pick_s;
+        if (c < 0) continue;               // nothing left above zero: the remaining rounds pad (uniform for the block)
+        const long long k_lo = c - a.nms_radius < 0 ? 0 : c - a.nms_radius;
+        const long long k_hi = c + a.nms_radius >= L ? L - 1 : c + a.nms_radius;
+        for (long long t = k_lo + tid; t <= k_hi; t += ST) D[t] = 0;
+        __syncthreads();
+        const int sg_lo = static_cast<int>(k_lo / SEG), sg_hi = static_cast<int>(k_hi / SEG);
+        for (int sg = sg_lo + warp; sg <= sg_hi; sg += SW) {
+            long long sv, sp;
+            const long long lo = (long long)sg * SEG, hi = lo + SEG < L ? lo + SEG : L;
+            warp_segment_max(D, lo, hi, lane, sv, sp);
+            if (lane == 0) { seg_val[sg] = sv; seg_pos[sg] = sp; }
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace
 
 s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
@@ -353,6 +544,46 @@ s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, con
                "n_spans = %d with nq*k = %d needs %zu bytes of shared memory per query, %d available", n_spans, a.nk, smem,
                max_smem - 2048);
     score_kernel<<<Q, ST, smem, stream>>>(layers, a);
+    S3_CUDA_TRY(cudaGetLastError());
+    return S3_OK;
+}
+
+}  // namespace s3
+
+namespace s3 {
+
+size_t density_workspace_bytes(int Q, int64_t L) { return 2 * static_cast<size_t>(Q) * static_cast<size_t>(L) * sizeof(long long); }
+
+s3_status launch_density(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L, const int32_t* d_q_ids,
+                         const float* d_q_vals, int Q, int nq, int k, int conv_kernel, int nms_radius, int n_centers,
+                         int64_t stop_freq, int32_t* d_centers, float* d_center_density, float* d_s_out, float* d_d_out,
+                         void* d_scratch, cudaStream_t stream)
+{
+    static int max_smem_dev[64] = {};
+    int dev = 0;
+    S3_CUDA_TRY(cudaGetDevice(&dev));
+    int max_smem = dev < 64 ? max_smem_dev[dev] : 0;
+    if (max_smem == 0) {
+        S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        S3_CUDA_TRY(cudaFuncSetAttribute(density_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+        if (dev < 64) max_smem_dev[dev] = max_smem;
+    }
+    S3_REQUIRE(L <= static_cast<int64_t>(SEG) * MAX_SEGS, S3_ERR_UNSUPPORTED, "L = %lld exceeds %lld positions", (long long)L,
+               (long long)SEG * MAX_SEGS);
+    ScoreLayers layers;
+    for (int l = 0; l < n_layers; ++l) layers.v[l] = h_layers[l];
+    DensityArgs a;
+    a.q_ids = d_q_ids; a.q_vals = d_q_vals;
+    a.s_fix = static_cast<long long*>(d_scratch);
+    a.d_fix = a.s_fix + static_cast<size_t>(Q) * static_cast<size_t>(L);
+    a.centers = d_centers; a.center_density = d_center_density; a.s_out = d_s_out; a.d_out = d_d_out;
+    a.L = L; a.n_layers = n_layers; a.d_sae = d_sae; a.Q = Q; a.nk = nq * k;
+    int npad = 32;
+    while (npad < a.nk) npad <<= 1;
+    a.npad = npad; a.conv_kernel = conv_kernel; a.nms_radius = nms_radius; a.n_centers = n_centers; a.stop_freq = stop_freq;
+    const size_t smem = ((score_smem(a.nk, npad, 0, true).total + 15u) & ~15u) + static_cast<size_t>(a.nk) * 8 + 2 * MAX_SEGS * 8;
+    S3_REQUIRE(smem + 2048 <= static_cast<size_t>(max_smem), S3_ERR_UNSUPPORTED, "nq*k = %d needs %zu bytes of shared memory", a.nk, smem);
+    density_kernel<<<Q, ST, smem, stream>>>(layers, a);
     S3_CUDA_TRY(cudaGetLastError());
     return S3_OK;
 }

@@ -1,0 +1,113 @@
+"""GPU parity of the per-position relevance / density / peak selection (Sec. 3.5 Eq. 6, "Adaptive Granularity";
+Alg. 1 Phase 2) against the CPU oracle. Both sides take the weights in 2^-24 fixed point, so S, the density
+and the selected centres must agree exactly (fp32 copies of exact integers); the oracle walks the tokens'
+feature sets, the GPU walks posting lists."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2601_17702_b200 as S
+from conftest import read_golden
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev():
+    assert torch.cuda.is_available()
+    return torch.device("cuda:0")
+
+
+def _rand_sets(T, k, D, rng, hot=0):
+    if D <= 4096:
+        keys = rng.random((T, D))
+        if hot:
+            keys[:, :hot] *= 0.05
+        return np.argsort(keys, axis=1)[:, :k].astype(np.int32)
+    start = rng.integers(0, D, size=(T, 1))
+    if hot:
+        start[rng.random((T, 1)) < 0.3] = 5
+    return ((start + np.arange(k)[None, :] * 131) % D).astype(np.int32)
+
+
+def gpu_density(ctx, q, qv, D, K, R, N, stop_freq=0):
+    d = _dev()
+    n_layers, L, k = ctx.shape
+    layers = []
+    for l in range(n_layers):
+        rp, pos, _ = O.postings(ctx[l], D, 0)
+        pos = pos if len(pos) else np.zeros(1, np.int32)
+        layers.append((torch.as_tensor(rp.astype(np.int64)).to(d), torch.as_tensor(pos).to(d)))
+    Q = q.shape[1]
+    ws = S.new_workspace(S.s3_density_workspace_bytes(Q, L))
+    S_out = torch.full((Q, max(L, 1)), -1.0, dtype=torch.float32, device=d)
+    D_out = torch.full((Q, max(L, 1)), -1.0, dtype=torch.float32, device=d)
+    c, dens = S.s3_position_density_topcenters(layers, D, L, torch.as_tensor(q).to(d).contiguous(),
+                                               torch.as_tensor(qv).to(d).contiguous(), K, R, N, ws, stop_freq, S_out, D_out)
+    assert S.s3_workspace_status(ws) == 0
+    return S_out.cpu().numpy()[:, :L], D_out.cpu().numpy()[:, :L], c.cpu().numpy(), dens.cpu().numpy()
+
+
+def _check(ctx, q, qv, D, K, R, N, stop_freq=0):
+    oS, oD, oc, odens = O.position_density(ctx, q, qv, D, K, R, N, stop_freq)
+    gS, gD, gc, gdens = gpu_density(ctx, q, qv, D, K, R, N, stop_freq)
+    np.testing.assert_array_equal(gS, oS.astype(np.float32))
+    np.testing.assert_array_equal(gD, oD.astype(np.float32))
+    np.testing.assert_array_equal(gc, oc)
+    np.testing.assert_array_equal(gdens, odens)
+
+
+def test_hand_example_on_gpu(golden_dir):
+    g = read_golden(os.path.join(golden_dir, "position_density_hand_example.txt"))
+    toks = np.array(g["tokens"], np.int32).reshape(1, -1, 2)
+    q = np.array(g["query"], np.int32).reshape(1, 1, -1, 2)
+    qv = np.array(g["query_vals"], np.float32).reshape(1, 1, -1, 2)
+    _, _, c, _ = gpu_density(toks, q, qv, 8, 3, 1, 3)
+    assert c[0].tolist() == [int(v) for v in g["centers"]]
+    _check(toks, q, qv, 8, 3, 1, 3)
+
+
+@pytest.mark.parametrize("L,k,D,n_layers,Q,nq,kq,K,R,N,stop", [
+    (300, 4, 64, 1, 2, 3, 4, 8, 4, 6, 0),
+    (5000, 8, 256, 3, 4, 7, 8, 48, 24, 40, 0),        # the paper's kernel 48 and 40 centres; several segments
+    (4100, 4, 32, 2, 3, 5, 4, 1, 0, 16, 0),           # no smoothing, no suppression radius
+    (2500, 8, 16, 1, 2, 40, 8, 9, 300, 64, 0),        # radius wider than a segment boundary; runs out of peaks
+    (3000, 4, 64, 2, 2, 6, 4, 48, 10, 8, 900),        # stop features
+    (20, 4, 64, 1, 2, 3, 4, 48, 5, 4, 0),             # kernel wider than the context
+])
+def test_density_and_centres_exact(L, k, D, n_layers, Q, nq, kq, K, R, N, stop):
+    rng = np.random.default_rng(L + K)
+    ctx = np.stack([_rand_sets(L, k, D, rng, hot=2) for _ in range(n_layers)])
+    q = np.stack([_rand_sets(Q * nq, kq, D, rng, hot=2).reshape(Q, nq, kq) for _ in range(n_layers)])
+    q[0, 0, 0, -1] = -1
+    qv = (rng.random(q.shape) * 3).astype(np.float32)
+    _check(ctx, q, qv, D, K, R, N, stop)
+
+
+def test_density_long_context_sampled_queries():
+    # 128K positions, dictionary of 16384, k = 32, 64-token queries with k = 64: the paper's stress length
+    L, k, D, Q, nq, kq = 131072, 32, 16384, 8, 64, 64
+    rng = np.random.default_rng(3)
+    ctx = _rand_sets(L, k, D, rng, hot=1)[None]
+    q = _rand_sets(Q * nq, kq, D, rng, hot=1).reshape(1, Q, nq, kq)
+    qv = rng.random(q.shape).astype(np.float32)
+    _check(ctx, q, qv, D, 48, 24, 40)
+
+
+def test_density_empty_query_and_error_paths():
+    d = _dev()
+    ctx = _rand_sets(100, 4, 32, np.random.default_rng(1))[None]
+    q = np.full((1, 1, 2, 4), -1, np.int32)
+    _check(ctx, q, np.ones(q.shape, np.float32), 32, 8, 2, 3)
+    rp = torch.zeros(33, dtype=torch.int64, device=d)
+    ps = torch.zeros(1, dtype=torch.int32, device=d)
+    qi = torch.zeros((1, 1, 2, 4), dtype=torch.int32, device=d)
+    qf = torch.zeros((1, 1, 2, 4), dtype=torch.float32, device=d)
+    with pytest.raises(S.S3Error) as e:
+        S.s3_position_density_topcenters([(rp, ps)], 32, 100, qi, qf, 8, 2, 3, S.new_workspace(64))
+    assert e.value.code == S.binding.S3_ERR_CAPACITY
+    with pytest.raises(S.S3Error) as e:
+        S.s3_position_density_topcenters([(rp, ps)], 32, 100, qi, qf, 0, 2, 3, S.new_workspace(1 << 16))
+    assert e.value.code == S.binding.S3_ERR_INVALID_ARG
