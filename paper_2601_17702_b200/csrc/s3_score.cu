@@ -19,6 +19,7 @@ constexpr int ST = 512;          // threads per block
 constexpr int SW = ST / 32;      // warps
 constexpr int PIECE = 32;        // postings per work item
 constexpr int BATCH = 8;         // work items a warp keeps in flight
+constexpr int WIN = 8192;        // pieces whose owning feature is tabulated at a time
 
 struct ScoreLayers {
     s3_csr_view v[S3_MAX_SCORE_LAYERS];
@@ -36,11 +37,12 @@ struct ScoreArgs {
     float alpha, beta;
     int64_t stop_freq;
     int stride_shift;   // log2(stride) when the stride is a power of two, else -1
+    unsigned long long stride_magic;   // ceil(2^64 / stride) (stride >= 2)
 };
 
 // Shared-memory carve-up, identical on host and device.
 struct ScoreSmem {
-    uint32_t acc_off, keys_off, ufeat_off, ustart_off, uaq_off, ulo_off, cstart_off, total;
+    uint32_t acc_off, keys_off, ufeat_off, ustart_off, uaq_off, ulo_off, cstart_off, owner_off, total;
 };
 __host__ __device__ inline ScoreSmem score_smem(int nk, int npad, int n_spans, bool weighted)
 {
@@ -52,6 +54,8 @@ __host__ __device__ inline ScoreSmem score_smem(int nk, int npad, int n_spans, b
     L.ufeat_off = o;  L.cstart_off = o;  o += (static_cast<uint32_t>(nk) + 1u) * 4u;   // cstart[u] replaces ufeat[u]
     L.ustart_off = o; o += (static_cast<uint32_t>(nk) + 1u) * 4u;
     L.uaq_off = o;    o += weighted ? static_cast<uint32_t>(nk) * 4u : 0u;
+    o = (o + 3u) & ~3u;
+    L.owner_off = o;  o += WIN * 2u;                                   // owning feature of each piece of the window
     L.total = o + 16u;
     return L;
 }
@@ -85,10 +89,13 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* w
     return res;
 }
 
-// floor(p / stride) for p >= 0 (shift when the stride is a power of two).
+// floor(p / stride) for 0 <= p < 2^31: a shift when the stride is a power of two (POW2), else the high word
+// of p * ceil(2^64 / stride), which is exact for every 32-bit p.
+template <bool POW2>
 __device__ __forceinline__ int div_stride(int p, const ScoreArgs& a)
 {
-    return a.stride_shift >= 0 ? (p >> a.stride_shift) : (p / a.stride);
+    if (POW2) return p >> a.stride_shift;
+    return static_cast<int>(__umul64hi(static_cast<unsigned long long>(p), a.stride_magic));
 }
 
 // Spans that posting i of a list (position p, ascending positions) still adds to. The posting lies in
@@ -96,12 +103,13 @@ __device__ __forceinline__ int div_stride(int p, const ScoreArgs& a)
 // In min-count mode span j already holds cQ earlier postings of the feature exactly when posting i-cQ
 // lies in it, i.e. when j <= hi(p_{i-cQ}); so the posting adds one to spans max(lo(p), hi(p_{i-cQ})+1)
 // .. hi(p) only, and the totals come out as min(cQ, cS(f, j)). p_prev < 0 means "no such posting".
+template <bool POW2>
 __device__ __forceinline__ void posting_range(const ScoreArgs& a, int p, int p_prev, int& j_lo, int& j_hi)
 {
-    j_hi = div_stride(p, a);
-    j_lo = p >= a.width ? div_stride(p - a.width, a) + 1 : 0;
+    j_hi = div_stride<POW2>(p, a);
+    j_lo = p >= a.width ? div_stride<POW2>(p - a.width, a) + 1 : 0;
     if (p_prev >= 0) {
-        const int j_prev = div_stride(p_prev, a) + 1;
+        const int j_prev = div_stride<POW2>(p_prev, a) + 1;
         j_lo = j_prev > j_lo ? j_prev : j_lo;
     }
     j_hi = j_hi < a.n_spans - 1 ? j_hi : a.n_spans - 1;
@@ -197,6 +205,19 @@ __device__ __forceinline__ uint32_t cut_lists(const uint64_t* __restrict__ row_p
     return piece_carry;
 }
 
+// Owning feature of each piece win0 .. win1-1 (binary search in the pieces' prefix, one piece per thread and
+// step), so that the walk below needs no running cursor and its loads are independent of each other.
+__device__ __forceinline__ void tabulate_owners(const uint32_t* cstart, int U, uint32_t win0, uint32_t win1, uint16_t* owner)
+{
+    for (uint32_t c = win0 + threadIdx.x; c < win1; c += ST) {
+        int lo = 0, hi = U;                  // last u with cstart[u] <= c (pieces of empty lists share a start)
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (cstart[mid] <= c) lo = mid; else hi = mid; }
+        owner[c - win0] = static_cast<uint16_t>(lo);
+    }
+    __syncthreads();
+}
+
+template <bool POW2>
 __global__ void __launch_bounds__(ST)
 score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__ ScoreArgs a)
 {
@@ -212,6 +233,7 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
     int32_t* ufeat = reinterpret_cast<int32_t*>(score_smem_raw + SL.ufeat_off);
     int32_t* ustart = reinterpret_cast<int32_t*>(score_smem_raw + SL.ustart_off);
     float* uaq = reinterpret_cast<float*>(score_smem_raw + SL.uaq_off);
+    uint16_t* owner = reinterpret_cast<uint16_t*>(score_smem_raw + SL.owner_off);
     uint32_t* cstart = reinterpret_cast<uint32_t*>(score_smem_raw + SL.cstart_off);   // same storage as ufeat: a thread
                                                                                         // reads ufeat[u], then writes cstart[u]
     __shared__ uint32_t ws[SW + 1];
@@ -233,16 +255,15 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
         const int32_t* __restrict__ pos = layers.v[l].d_pos;
         const uint32_t piece_total = cut_lists(layers.v[l].d_row_ptr, U, weighted ? a.stop_freq : 0, ufeat, ulo, ulen, cstart, ws);
 
-        // each warp takes an equal share of consecutive pieces and walks them with a running feature cursor
-        const uint32_t n_pieces_total = piece_total;
-        const uint32_t c_begin = static_cast<uint32_t>(static_cast<uint64_t>(n_pieces_total) * warp / SW);
-        const uint32_t c_end = static_cast<uint32_t>(static_cast<uint64_t>(n_pieces_total) * (warp + 1) / SW);
-        if (c_begin < c_end) {
-            int lo_u = 0, hi_u = U;              // last u with cstart[u] <= c_begin
-            while (hi_u - lo_u > 1) { const int mid = (lo_u + hi_u) >> 1; if (cstart[mid] <= c_begin) lo_u = mid; else hi_u = mid; }
-            int u = lo_u;
-            // BATCH pieces per round: first all their loads are issued, then their updates, so that a warp
-            // has BATCH independent memory round trips in flight instead of one.
+        // The pieces are walked a window at a time; inside a window every warp takes an equal share. BATCH
+        // pieces per round: first all their loads are issued, then their updates, so that a warp has BATCH
+        // independent memory round trips in flight instead of one.
+        for (uint32_t win0 = 0; win0 < piece_total; win0 += WIN) {
+            const uint32_t win1 = piece_total - win0 < WIN ? piece_total : win0 + WIN;
+            tabulate_owners(cstart, U, win0, win1, owner);
+            const uint32_t n_win = win1 - win0;
+            const uint32_t c_begin = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * warp / SW);
+            const uint32_t c_end = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * (warp + 1) / SW);
             for (uint32_t c0 = c_begin; c0 < c_end; c0 += BATCH) {
                 int p[BATCH], p_prev[BATCH], ub[BATCH];
 #pragma unroll
@@ -250,7 +271,7 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
                     const uint32_t c = c0 + b;
                     p[b] = -1; p_prev[b] = -1; ub[b] = 0;
                     if (c < c_end) {
-                        while (cstart[u + 1] <= c) ++u;
+                        const int u = owner[c - win0];
                         ub[b] = u;
                         const int32_t* __restrict__ list = pos + ulo[u];
                         const uint32_t i = (c - cstart[u]) * PIECE + lane;
@@ -267,7 +288,7 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
                 for (int b = 0; b < BATCH; ++b) {
                     if (p[b] < 0) continue;
                     int j_lo, j_hi;
-                    posting_range(a, p[b], p_prev[b], j_lo, j_hi);
+                    posting_range<POW2>(a, p[b], p_prev[b], j_lo, j_hi);
                     if (weighted) {
                         const double w = static_cast<double>(uaq[ub[b]]) *
                                          (1.0 / (log(1.0 + static_cast<double>(ulen[ub[b]])) + 1.0));
@@ -278,8 +299,8 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
                     }
                 }
             }
+            __syncthreads();
         }
-        __syncthreads();
     }
 
     // min-count mode: difference array -> per-span totals (inclusive prefix sum, in place)
@@ -400,6 +421,7 @@ density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant
     int32_t* ustart = reinterpret_cast<int32_t*>(score_smem_raw + SL.ustart_off);
     float* uaq = reinterpret_cast<float*>(score_smem_raw + SL.uaq_off);
     uint32_t* cstart = reinterpret_cast<uint32_t*>(score_smem_raw + SL.cstart_off);
+    uint16_t* owner = reinterpret_cast<uint16_t*>(score_smem_raw + SL.owner_off);
     long long* uw = reinterpret_cast<long long*>(score_smem_raw + ((SL.total + 15u) & ~15u));     // [nk] fixed-point weights
     long long* seg_val = uw + a.nk;                                                               // [n_segs]
     long long* seg_pos = seg_val + MAX_SEGS;
@@ -425,12 +447,12 @@ density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant
         for (int u = tid; u < U; u += ST)      // w = rint(aQ * IDF(freq) * 2^24), IDF = 1 / (ln(1 + freq) + 1)
             uw[u] = __double2ll_rn(static_cast<double>(uaq[u]) * (1.0 / (log(1.0 + static_cast<double>(ulen[u])) + 1.0)) * 16777216.0);
         __syncthreads();
-        const uint32_t c_begin = static_cast<uint32_t>(static_cast<uint64_t>(n_pieces_total) * warp / SW);
-        const uint32_t c_end = static_cast<uint32_t>(static_cast<uint64_t>(n_pieces_total) * (warp + 1) / SW);
-        if (c_begin < c_end) {
-            int lo_u = 0, hi_u = U;              // last u with cstart[u] <= c_begin
-            while (hi_u - lo_u > 1) { const int mid = (lo_u + hi_u) >> 1; if (cstart[mid] <= c_begin) lo_u = mid; else hi_u = mid; }
-            int u = lo_u;
+        for (uint32_t win0 = 0; win0 < n_pieces_total; win0 += WIN) {
+            const uint32_t win1 = n_pieces_total - win0 < WIN ? n_pieces_total : win0 + WIN;
+            tabulate_owners(cstart, U, win0, win1, owner);
+            const uint32_t n_win = win1 - win0;
+            const uint32_t c_begin = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * warp / SW);
+            const uint32_t c_end = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * (warp + 1) / SW);
             for (uint32_t c0 = c_begin; c0 < c_end; c0 += BATCH) {
                 int p[BATCH], ub[BATCH];
 #pragma unroll
@@ -438,7 +460,7 @@ density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant
                     const uint32_t c = c0 + b;
                     p[b] = -1; ub[b] = 0;
                     if (c < c_end) {
-                        while (cstart[u + 1] <= c) ++u;
+                        const int u = owner[c - win0];
                         ub[b] = u;
                         const uint32_t i = (c - cstart[u]) * PIECE + lane;
                         if (i < ulen[u]) p[b] = __ldg(pos + ulo[u] + i);
@@ -449,8 +471,8 @@ density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant
                     if (p[b] >= 0 && p[b] < L)
                         atomicAdd(reinterpret_cast<unsigned long long*>(S + p[b]), static_cast<unsigned long long>(uw[ub[b]]));
             }
+            __syncthreads();
         }
-        __syncthreads();
     }
 
     // density: K taps starting at t - K/2
@@ -525,7 +547,8 @@ s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, con
     int max_smem = dev < 64 ? max_smem_dev[dev] : 0;
     if (max_smem == 0) {
         S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
         if (dev < 64) max_smem_dev[dev] = max_smem;
     }
     ScoreLayers layers;
@@ -539,11 +562,13 @@ s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, con
     a.npad = npad; a.n_spans = n_spans; a.width = p->width; a.stride = p->stride; a.mode = p->mode; a.s = p->s;
     a.alpha = p->alpha; a.beta = p->beta; a.stop_freq = p->stop_freq;
     a.stride_shift = (p->stride & (p->stride - 1)) == 0 ? __builtin_ctz(static_cast<unsigned>(p->stride)) : -1;
+    a.stride_magic = p->stride >= 2 ? ~0ull / static_cast<unsigned long long>(p->stride) + 1ull : 0ull;
     const size_t smem = score_smem(a.nk, npad, n_spans, p->mode == S3_SCORE_WEIGHTED).total;
     S3_REQUIRE(smem + 2048 <= static_cast<size_t>(max_smem), S3_ERR_UNSUPPORTED,
                "n_spans = %d with nq*k = %d needs %zu bytes of shared memory per query, %d available", n_spans, a.nk, smem,
                max_smem - 2048);
-    score_kernel<<<Q, ST, smem, stream>>>(layers, a);
+    if (a.stride_shift >= 0) score_kernel<true><<<Q, ST, smem, stream>>>(layers, a);
+    else score_kernel<false><<<Q, ST, smem, stream>>>(layers, a);
     S3_CUDA_TRY(cudaGetLastError());
     return S3_OK;
 }
