@@ -131,53 +131,44 @@ postings_colscan_kernel(const __grid_constant__ PostingsPlan pl)
 }
 
 // ---- 3. row_ptr = exclusive scan of the list lengths, in place ------------------------------------------------
-// Thread t owns entries [t*per, (t+1)*per): a first sweep sums them (independent loads), a block scan
-// of the 1024 sums gives each thread its starting offset, a second sweep writes the offsets.
+// One block per item walks the array in tiles of 1024 consecutive entries (coalesced): warp scans, a scan of
+// the 32 warp sums, and a running carry from tile to tile.
 __global__ void __launch_bounds__(PT)
 postings_rowscan_kernel(const __grid_constant__ PostingsPlan pl)
 {
-    __shared__ uint32_t warp_sums[33];
+    __shared__ uint32_t warp_sums[2][33];
     const s3_postings_item& it = pl.items[blockIdx.x];
     uint32_t* rp = it.d_row_ptr;
     const int n = it.d_sae;
-    const int per = (n + PT - 1) / PT;
-    const int lo = min(n, (int)threadIdx.x * per), hi = min(n, lo + per);
-    uint32_t sum = 0;
-#pragma unroll 8
-    for (int i = lo; i < hi; ++i) sum += rp[i];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t inc = sum;
+    uint32_t carry = 0;
+    int buf = 0;
+    uint32_t v_next = threadIdx.x < n ? rp[threadIdx.x] : 0u;
+    for (int i0 = 0; i0 < n; i0 += PT, buf ^= 1) {
+        const int i = i0 + threadIdx.x;
+        const uint32_t v = v_next;
+        v_next = (i + PT < n) ? rp[i + PT] : 0u;            // next tile's load overlaps this tile's scan
+        uint32_t inc = v;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += v;
-    }
-    if (lane == 31) warp_sums[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        const uint32_t w = warp_sums[lane];
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += u;
+        }
+        if (lane == 31) warp_sums[buf][warp] = inc;
+        __syncthreads();
+        uint32_t w = warp_sums[buf][lane];                   // every warp scans the 32 warp sums itself
         uint32_t winc = w;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xffffffffu, winc, o);
-            if (lane >= o) winc += v;
+            const uint32_t u = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += u;
         }
-        warp_sums[lane] = winc - w;
-        if (lane == 31) warp_sums[32] = winc;
+        const uint32_t before_warp = __shfl_sync(0xffffffffu, winc - w, warp);
+        const uint32_t tile_total = __shfl_sync(0xffffffffu, winc, 31);
+        if (i < n) rp[i] = carry + before_warp + inc - v;
+        carry += tile_total;
     }
-    __syncthreads();
-    uint32_t run = warp_sums[warp] + inc - sum;
-    for (int i0 = lo; i0 < hi; i0 += 8) {
-        uint32_t c[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) c[j] = (i0 + j < hi) ? rp[i0 + j] : 0u;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (i0 + j < hi) rp[i0 + j] = run;
-            run += c[j];
-        }
-    }
-    if (threadIdx.x == 0) rp[n] = warp_sums[32];
+    if (threadIdx.x == 0) rp[n] = carry;
 }
 
 // ---- 4. ordered scatter ---------------------------------------------------------------------------------
