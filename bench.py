@@ -488,7 +488,7 @@ def main():
     out = run_ours(args, rank, world, local_rank)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            out["cpu_baseline"] = run_reference(args, cpu_only_sample=32)
+            out["cpu_baseline"] = run_reference(args, cpu_only_sample=512)
         print(json.dumps(out), flush=True)
     if world > 1:
         torch.distributed.destroy_process_group()
