@@ -55,6 +55,7 @@ candidate_merge_kernel(const uint64_t* __restrict__ cand, const uint32_t* __rest
                        int32_t* __restrict__ ids, float* __restrict__ vals)
 {
     __shared__ uint64_t cand_buf[kMergeWarps][kCandBuf];
+    __shared__ uint32_t cand_hist[kMergeWarps][64];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * kMergeWarps + warp;
     if (t >= T) return;
@@ -86,6 +87,50 @@ candidate_merge_kernel(const uint64_t* __restrict__ cand, const uint32_t* __rest
                     n += __popc(m);
                 }
             }
+        }
+    }
+    if (!overflow && n > 2u * static_cast<uint32_t>(k)) {
+        // Many more survivors than k: tighten the bound once more before sorting. A 64-bucket histogram over the
+        // float bits above the bound's bucket (16 buckets per octave) shows the highest bucket edge that k
+        // survivors still reach; what lies below it is dropped.
+        uint32_t* hist = cand_hist[warp];
+        hist[lane] = 0; hist[lane + 32] = 0;
+        __syncwarp();
+        const int base = static_cast<int>(__float_as_uint(tau) >> 19);
+        for (uint32_t i = lane; i < n; i += 32) {
+            int idx = static_cast<int>(static_cast<uint32_t>(buf[i] >> 32) >> 19) - base;
+            idx = idx < 0 ? 0 : (idx > 63 ? 63 : idx);
+            atomicAdd(&hist[idx], 1u);
+        }
+        __syncwarp();
+        // lane l holds buckets 2l and 2l+1; suffix sums over the lanes by shuffles
+        const uint32_t h0 = hist[2 * lane], h1 = hist[2 * lane + 1];
+        uint32_t suf = h0 + h1;                                  // buckets >= 2l, after the scan
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t up = __shfl_down_sync(0xffffffffu, suf, o);
+            if (lane + o < 32) suf += up;
+        }
+        // highest bucket b with (number of survivors in buckets >= b) >= k
+        int best = (suf - h0 >= static_cast<uint32_t>(k)) ? 2 * lane + 1 : ((suf >= static_cast<uint32_t>(k)) ? 2 * lane : 0);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const int other = __shfl_xor_sync(0xffffffffu, best, o);
+            best = other > best ? other : best;
+        }
+        if (best > 0) {
+            const float tau2 = __uint_as_float((static_cast<uint32_t>(base + best) << 19) - 1u);   // value >= edge
+            uint32_t w = 0;
+            for (uint32_t i0 = 0; i0 < n; i0 += 32) {
+                const uint32_t i = i0 + lane;
+                const uint64_t key = i < n ? buf[i] : 0ull;
+                const bool keep = i < n && __uint_as_float(static_cast<uint32_t>(key >> 32)) > tau2;
+                const uint32_t m = __ballot_sync(0xffffffffu, keep);
+                if (keep) buf[w + __popc(m & ((1u << lane) - 1u))] = key;      // w <= i0: never an unread slot
+                w += __popc(m);
+            }
+            __syncwarp();
+            n = w;
         }
     }
     if (!overflow) {
