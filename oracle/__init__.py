@@ -151,3 +151,26 @@ def position_density(ctx_ids, q_ids, q_vals, d_sae: int, conv_kernel: int, nms_r
                                C.c_int(conv_kernel), C.c_int(nms_radius), C.c_int(n_centers), C.c_int64(stop_freq),
                                _p(S, C.c_double), _p(D, C.c_double), _p(centers, C.c_int32), _p(dens, C.c_float))
     return S, D, centers, dens
+
+
+def fuse_index_sets(centers, span_width: int, lexical, lead: int, tail: int, L: int):
+    """Sec. 3.6, Eq. 7: M_final = M_S3 U M_BM25 U M_Bias, per query, as ascending unique positions in [0, L).
+    M_S3   = union over the selected centres c >= 0 of the window [c - span_width//2, c - span_width//2 + span_width)
+             (reading: the paper's variable-length span rule is not given; a fixed window centred on the peak stands in),
+    M_BM25 = the supplied lexical positions (entries < 0 are padding; entries >= L are ignored),
+    M_Bias = the first `lead` and the last `tail` positions.
+    centers [Q, N] int, lexical [Q, n_lex] int or None. Returns a list of Q int32 arrays. Plain Python sets."""
+    centers = np.asarray(centers)
+    out = []
+    for q in range(centers.shape[0]):
+        m = set()
+        for c in centers[q].tolist():
+            if c >= 0:
+                lo = c - span_width // 2
+                m.update(t for t in range(lo, lo + span_width) if 0 <= t < L)
+        if lexical is not None:
+            m.update(int(t) for t in np.asarray(lexical)[q].tolist() if 0 <= t < L)
+        m.update(range(0, min(lead, L)))
+        m.update(range(max(0, L - tail), L))
+        out.append(np.array(sorted(m), dtype=np.int32))
+    return out
