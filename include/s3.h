@@ -286,6 +286,27 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
                                          float* d_center_density /*[Q,n_centers]*/, float* d_S /*[Q,L] nullable*/,
                                          float* d_density /*[Q,L] nullable*/, void* d_ws, size_t ws_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Hybrid fusion of index sets                  (paper Sec. 3.6 Eq. 7: M_final = M_S3 U M_BM25 U M_Bias;
+ *                                               Alg. 1 Phase 3: Idx_Final <- Idx_S3 U Idx_Lexical U LeadTail)
+ *
+ * Per query q, the ascending, duplicate-free positions in [0, L) of
+ *   M_S3   : the window [c - span_width/2, c - span_width/2 + span_width) around every centre c >= 0 of
+ *            d_centers [Q, n_centers] (as returned by s3_position_density_topcenters; the paper's rule for
+ *            variable-length spans is not given, a fixed window centred on the peak stands in),
+ *   M_BM25 : the supplied lexical positions d_lexical [Q, n_lex] (nullable; entries < 0 are padding,
+ *            entries >= L are ignored),
+ *   M_Bias : the first `lead` and the last `tail` positions.
+ * d_out_idx [Q, cap] int32 receives the positions (-1 after the last one), d_out_count [Q] the size of the
+ * set; when it exceeds cap only the cap lowest positions are written. The caller gathers tokens with them.
+ * Workspace: s3_fuse_workspace_bytes(Q, L) (one bit per query and position, plus the status block).
+ * ---------------------------------------------------------------------------------------------- */
+size_t s3_fuse_workspace_bytes(int Q, int64_t L);
+s3_status s3_fuse_index_sets(const int32_t* d_centers, int Q, int n_centers, int span_width,
+                             const int32_t* d_lexical /*nullable*/, int n_lex, int lead, int tail, int64_t L,
+                             int32_t* d_out_idx /*[Q,cap]*/, int cap, int32_t* d_out_count /*[Q]*/,
+                             void* d_ws, size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

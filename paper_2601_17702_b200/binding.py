@@ -28,6 +28,7 @@ EXPORTS = [
     "s3_index_stats", "s3_index_layer_postings", "s3_index_export_csr", "s3_index_destroy",
     "s3_score_workspace_bytes", "s3_coactivation_score_topspans",
     "s3_density_workspace_bytes", "s3_position_density_topcenters",
+    "s3_fuse_workspace_bytes", "s3_fuse_index_sets",
 ]
 
 
@@ -75,7 +76,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.s3_last_error.restype = C.c_char_p
         for name in ("s3_sae_prepared_bytes", "s3_sae_encode_workspace_bytes", "s3_postings_workspace_bytes",
-                     "s3_score_workspace_bytes", "s3_density_workspace_bytes"):
+                     "s3_score_workspace_bytes", "s3_density_workspace_bytes", "s3_fuse_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.s3_sae_prepared_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_sae_create.argtypes = [C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
@@ -111,6 +112,9 @@ def lib():
         L.s3_position_density_topcenters.argtypes = [C.POINTER(CsrView), C.c_int, C.c_int, C.c_int64, C.c_void_p, C.c_void_p,
                                                      C.c_int, C.c_int, C.c_int, C.POINTER(DensityParams), C.c_void_p,
                                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_fuse_workspace_bytes.argtypes = [C.c_int, C.c_int64]
+        L.s3_fuse_index_sets.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64,
+                                         C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         _lib = L
     return _lib
 
@@ -339,3 +343,24 @@ def s3_position_density_topcenters(layers, d_sae: int, L: int, q_ids: torch.Tens
                                                 C.byref(params), _ptr(centers), _ptr(dens), _ptr(S_out), _ptr(density_out),
                                                 _ptr(ws), ws.numel(), _stream(stream)))
     return centers, dens
+
+
+def s3_fuse_workspace_bytes(Q: int, L: int) -> int:
+    return int(lib().s3_fuse_workspace_bytes(Q, L))
+
+
+def s3_fuse_index_sets(centers: torch.Tensor, span_width: int, lexical: torch.Tensor | None, lead: int, tail: int, L: int,
+                       cap: int, ws: torch.Tensor, stream=None):
+    """centers int32 [Q, N] (-1 = none), lexical int32 [Q, n_lex] or None. Returns (idx int32 [Q, cap] ascending,
+    -1 padded; count int32 [Q])."""
+    assert centers.dtype == torch.int32 and centers.is_contiguous() and centers.dim() == 2
+    Q, N = centers.shape
+    n_lex = 0
+    if lexical is not None:
+        assert lexical.dtype == torch.int32 and lexical.is_contiguous() and lexical.shape[0] == Q
+        n_lex = lexical.shape[1]
+    idx = torch.empty((Q, cap), dtype=torch.int32, device=centers.device)
+    count = torch.empty((Q,), dtype=torch.int32, device=centers.device)
+    _check(lib().s3_fuse_index_sets(_ptr(centers), Q, N, span_width, _ptr(lexical), n_lex, lead, tail, L, _ptr(idx), cap,
+                                    _ptr(count), _ptr(ws), ws.numel(), _stream(stream)))
+    return idx, count

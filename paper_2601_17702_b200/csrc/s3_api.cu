@@ -342,4 +342,29 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
                           static_cast<cudaStream_t>(stream));
 }
 
+// ---------------------------------------------------------------------------------------------- index-set fusion
+size_t s3_fuse_workspace_bytes(int Q, int64_t L)
+{
+    if (Q < 0 || L < 0) return 0;
+    return 256 + fuse_workspace_bytes(Q, L);
+}
+
+s3_status s3_fuse_index_sets(const int32_t* d_centers, int Q, int n_centers, int span_width, const int32_t* d_lexical, int n_lex,
+                             int lead, int tail, int64_t L, int32_t* d_out_idx, int cap, int32_t* d_out_count, void* d_ws,
+                             size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(Q >= 0 && n_centers >= 0 && n_lex >= 0, S3_ERR_INVALID_ARG, "Q = %d, n_centers = %d, n_lex = %d out of range", Q,
+               n_centers, n_lex);
+    S3_REQUIRE(span_width >= 0 && lead >= 0 && tail >= 0 && cap >= 0, S3_ERR_INVALID_ARG,
+               "span_width = %d, lead = %d, tail = %d, cap = %d must not be negative", span_width, lead, tail, cap);
+    S3_REQUIRE(L >= 0 && L <= INT32_MAX, S3_ERR_INVALID_ARG, "L out of range");
+    if (Q == 0) return S3_OK;
+    S3_REQUIRE(d_out_count != nullptr && (cap == 0 || d_out_idx != nullptr), S3_ERR_INVALID_ARG, "null output pointer");
+    S3_REQUIRE(n_centers == 0 || d_centers != nullptr, S3_ERR_INVALID_ARG, "d_centers is null");
+    S3_REQUIRE(d_ws != nullptr && ws_bytes >= s3_fuse_workspace_bytes(Q, L), S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed",
+               ws_bytes, s3_fuse_workspace_bytes(Q, L));
+    return launch_fuse_sets(d_centers, Q, n_centers, span_width, d_lexical, d_lexical ? n_lex : 0, lead, tail, L, d_out_idx, cap,
+                            d_out_count, static_cast<unsigned char*>(d_ws) + 256, static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"

@@ -39,6 +39,10 @@ s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, con
                        const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
                        float* d_all_scores, cudaStream_t stream);
 
+size_t fuse_workspace_bytes(int Q, int64_t L);
+s3_status launch_fuse_sets(const int32_t* d_centers, int Q, int n_centers, int span_width, const int32_t* d_lexical, int n_lex,
+                           int lead, int tail, int64_t L, int32_t* d_out_idx, int cap, int32_t* d_out_count, void* d_scratch,
+                           cudaStream_t stream);
 size_t density_workspace_bytes(int Q, int64_t L);
 s3_status launch_density(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L, const int32_t* d_q_ids,
                          const float* d_q_vals, int Q, int nq, int k, int conv_kernel, int nms_radius, int n_centers,
