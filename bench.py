@@ -443,6 +443,38 @@ def run_case(args):
                                                          bm25, top_idx=top_idx, top_score=top_score)
         out.update(L=L, d_sae=D, k=k, Q=r.Q, nq=r.nq, kq=r.kq, spans=ns, stride=stride, gathered_postings=gathered,
                    index_bytes=int(ps.numel()) * 4, bytes=gathered * 4 + r.Q * ns * 4 + r.Q * r.s * 8)
+    elif args.case == "density":
+        # the paper's Phase 2 tail alone: per-position relevance (Eq. 6), box-smoothed density (48 taps), greedy NMS
+        # with 40 centres, then the index-set union of Eq. 7 (256-token windows, 64 lexical hits, 64 lead / tail);
+        # same random index and queries as the score case
+        r = C.CFG4
+        L = args.tokens or r.scan.L
+        k, D = (r.scan.key.k, r.scan.key.d_sae) if not args.tokens else (16, 8192)
+        g = torch.Generator(device=dev).manual_seed(1)
+        ids = torch.cat([torch.rand((min(65536, L - t0), D), device=dev, generator=g).topk(k, dim=1).indices.to(torch.int32)
+                         for t0 in range(0, L, 65536)])
+        rp32 = torch.zeros(D + 1, dtype=torch.int32, device=dev)
+        pos = torch.zeros(L * k, dtype=torch.int32, device=dev)
+        ws = S.new_workspace(S.s3_postings_workspace_bytes(L, k, D), dev)
+        S.s3_postings_build(ids, D, 0, rp32, pos, ws)
+        layers = [(rp32.to(torch.int64), pos)]
+        q_ids = torch.rand((r.Q * r.nq, D), device=dev, generator=g).topk(r.kq, dim=1).indices.to(torch.int32).view(1, r.Q, r.nq, r.kq)
+        q_vals = torch.rand(q_ids.shape, dtype=torch.float32, device=dev, generator=g)
+        lexical = torch.randint(0, L, (r.Q, 64), device=dev, generator=g, dtype=torch.int32)
+        dws = S.new_workspace(S.s3_density_workspace_bytes(r.Q, L), dev)
+        fws = S.new_workspace(S.s3_fuse_workspace_bytes(r.Q, L), dev)
+        cap = 40 * 256 + 64 + 128
+        lens = (rp32[1:] - rp32[:-1])
+        gathered = 0
+        for q in range(r.Q):
+            gathered += int(lens[torch.unique(q_ids[0, q].flatten().long())].sum().item())
+
+        def run(i):
+            c, _ = S.s3_position_density_topcenters(layers, D, L, q_ids, q_vals, 48, 24, 40, dws)
+            if not args.no_union:
+                S.s3_fuse_index_sets(c, 256, lexical, 64, 64, L, cap, fws)
+        out.update(L=L, d_sae=D, k=k, Q=r.Q, nq=r.nq, kq=r.kq, conv_kernel=48, nms_radius=24, n_centers=40,
+                   gathered_postings=gathered, bytes=gathered * 4 + r.Q * L * 16)
     else:
         raise SystemExit(f"unknown case {args.case}")
     for i in range(2):
@@ -465,11 +497,12 @@ def run_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score")
+    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)
     ap.add_argument("--items", type=int, default=8)
+    ap.add_argument("--no-union", action="store_true", help="density case: leave out the index-set union")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=96)
     ap.add_argument("--warmup", type=int, default=3)
