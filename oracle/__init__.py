@@ -174,3 +174,87 @@ def fuse_index_sets(centers, span_width: int, lexical, lead: int, tail: int, L: 
         m.update(range(max(0, L - tail), L))
         out.append(np.array(sorted(m), dtype=np.int32))
     return out
+
+
+# ---------------------------------------------------------------------------------------------- compact index
+# Sec. 3.4 (memory analysis) asks a production index for contiguous integer arrays with delta encoding and optional
+# stop-feature pruning; the layout itself is this library's (the paper fixes none). Per layer, from the merged CSR:
+#   pruning   : a feature whose list is longer than stop_freq > 0 keeps no postings;
+#   row_ptr   : uint64 [D+1], prefix sum of the kept list lengths;
+#   blocks    : a kept list is cut into blocks of 32 postings (the last one shorter); blk_ptr uint32 [D+1] is the prefix
+#               sum of the lists' block counts;
+#   per block : blk_first = its first position; width = bit length of the largest (gap - 1) between consecutive
+#               positions inside the block (0 when all gaps are 1 or the block holds one posting);
+#               blk_desc = (word offset of its payload << 6) | width;
+#   payload   : uint32 words; a block of c postings stores its c - 1 values (gap - 1), `width` bits each, back to
+#               back starting at bit 0 of its first word, least significant bit first, in ceil((c-1)*width/32)
+#               words; blocks follow each other in order; one zero word closes the array.
+
+def compact_encode(row_ptr, pos, stop_freq: int = 0):
+    """Returns dict(row_ptr uint64 [D+1], blk_ptr uint32 [D+1], blk_first int32 [B], blk_desc uint64 [B],
+    payload uint32 [W+1]). Python integers as bit buffers: slow and plain."""
+    row_ptr = np.asarray(row_ptr, dtype=np.uint64)
+    pos = np.asarray(pos, dtype=np.int64)
+    D = len(row_ptr) - 1
+    out_rp, blk_ptr, firsts, descs, words = [0], [0], [], [], []
+    for f in range(D):
+        lst = pos[int(row_ptr[f]):int(row_ptr[f + 1])].tolist()
+        if stop_freq > 0 and len(lst) > stop_freq:
+            lst = []
+        out_rp.append(out_rp[-1] + len(lst))
+        blk_ptr.append(blk_ptr[-1] + (len(lst) + 31) // 32)
+        for b0 in range(0, len(lst), 32):
+            blk = lst[b0:b0 + 32]
+            gaps = [blk[i] - blk[i - 1] - 1 for i in range(1, len(blk))]
+            assert all(g >= 0 for g in gaps), "positions of a list must ascend strictly"
+            width = max(gaps).bit_length() if gaps else 0
+            bits = 0
+            for i, g in enumerate(gaps):
+                bits |= g << (i * width)
+            n_words = (len(gaps) * width + 31) // 32
+            firsts.append(blk[0])
+            descs.append((len(words) << 6) | width)
+            words.extend((bits >> (32 * w)) & 0xFFFFFFFF for w in range(n_words))
+    words.append(0)
+    return dict(row_ptr=np.array(out_rp, dtype=np.uint64), blk_ptr=np.array(blk_ptr, dtype=np.uint32),
+                blk_first=np.array(firsts, dtype=np.int32), blk_desc=np.array(descs, dtype=np.uint64),
+                payload=np.array(words, dtype=np.uint32))
+
+
+def compact_decode(c):
+    """Inverse of compact_encode on the kept postings: (row_ptr uint64 [D+1], pos int32). Reads the payload bit by
+    bit (written without reference to the encoder's buffer arithmetic)."""
+    rp, bp = c["row_ptr"], c["blk_ptr"]
+    payload = c["payload"]
+    pos = []
+    for f in range(len(rp) - 1):
+        n = int(rp[f + 1]) - int(rp[f])
+        for j, b in enumerate(range(int(bp[f]), int(bp[f + 1]))):
+            cnt = min(32, n - 32 * j)
+            desc = int(c["blk_desc"][b])
+            width, bit = desc & 63, (desc >> 6) * 32
+            p = int(c["blk_first"][b])
+            pos.append(p)
+            for _ in range(cnt - 1):
+                g = 0
+                for i in range(width):
+                    g |= ((int(payload[(bit + i) // 32]) >> ((bit + i) % 32)) & 1) << i
+                bit += width
+                p += g + 1
+                pos.append(p)
+    return np.asarray(rp, dtype=np.uint64), np.array(pos, dtype=np.int32)
+
+
+def prune_stop_features(row_ptr, pos, stop_freq: int):
+    """The CSR with every list longer than stop_freq > 0 emptied (Sec. 3.4 stop-feature pruning; the appendix's
+    hard frequency threshold applied when the index is built)."""
+    row_ptr = np.asarray(row_ptr, dtype=np.uint64)
+    pos = np.asarray(pos)
+    keep, out_rp = [], [0]
+    for f in range(len(row_ptr) - 1):
+        lo, hi = int(row_ptr[f]), int(row_ptr[f + 1])
+        if stop_freq > 0 and hi - lo > stop_freq:
+            hi = lo
+        keep.append(pos[lo:hi])
+        out_rp.append(out_rp[-1] + hi - lo)
+    return np.array(out_rp, dtype=np.uint64), (np.concatenate(keep) if keep else pos[:0]).astype(np.int32)
