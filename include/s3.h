@@ -287,6 +287,73 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
                                          float* d_density /*[Q,L] nullable*/, void* d_ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * Compact inverted index        (paper Sec. 3.4, memory analysis: contiguous integer arrays with delta
+ *                                encoding and optional stop-feature pruning; the appendix's hard frequency
+ *                                threshold for stop features. The layout is this library's.)
+ *
+ * One layer's merged CSR (row_ptr uint64 [d_sae+1], pos int32 strictly ascending per feature) becomes
+ *   row_ptr   uint64 [d_sae+1] : prefix sum of the KEPT list lengths; a feature whose list is longer than
+ *                                stop_freq > 0 keeps no postings (it then counts as absent in every
+ *                                scoring mode, and the kept features' freq, hence IDF, is unchanged);
+ *   blk_ptr   uint32 [d_sae+1] : prefix sum of the lists' block counts, a list of n postings having
+ *                                ceil(n/32) blocks of 32 postings (the last one shorter);
+ *   blk_first int32  [n_blocks]: first position of the block;
+ *   blk_desc  uint64 [n_blocks]: (word offset of the block's payload << 6) | width, width = bit length of
+ *                                the largest (gap - 1) between consecutive positions inside the block;
+ *   payload   uint32 [n_words] : per block of c postings its c-1 values (gap - 1), `width` bits each, back
+ *                                to back from bit 0 of the block's first word, least significant bit first,
+ *                                in ceil((c-1)*width/32) words; one zero word closes the array.
+ * A full block takes 12 bytes plus ceil(31*width/32) words instead of 128 bytes.
+ *
+ * s3_compact_bound gives capacities that always suffice (blocks <= n/32 + min(n, d_sae), words <= n + 1).
+ * s3_compact_build runs five small kernels on `stream`; d_sizes (device, 4 x uint64) receives
+ * {kept postings, n_blocks, n_words, 0}. If a capacity is too small nothing beyond it is written, the
+ * workspace status is set (s3_workspace_status returns S3_ERR_CAPACITY) and d_sizes holds what is needed
+ * as far as it was computed. Workspace: s3_compact_workspace_bytes(n_postings, d_sae).
+ *
+ * s3_coactivation_score_topspans_compact is s3_coactivation_score_topspans reading this form: a warp
+ * decodes a block with one prefix sum; results are identical to scoring the pruned CSR.
+ *
+ * s3_compact_save / s3_compact_file_info / s3_compact_load move HOST copies of the arrays to and from a
+ * file (checksummed per layer; load verifies the checksum and that every offset stays inside its array,
+ * and refuses the file otherwise with S3_ERR_INVALID_ARG). In s3_compact_load the caller provides
+ * buffers with capacities in n_blocks / n_words (from s3_compact_file_info); the actual sizes are written
+ * back. I/O failures return S3_ERR_STATE.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    const uint64_t* d_row_ptr;
+    const uint32_t* d_blk_ptr;
+    const int32_t* d_blk_first;
+    const uint64_t* d_blk_desc;
+    const uint32_t* d_payload;
+} s3_compact_view;
+
+typedef struct {
+    uint64_t* h_row_ptr;
+    uint32_t* h_blk_ptr;
+    int32_t* h_blk_first;
+    uint64_t* h_blk_desc;
+    uint32_t* h_payload;
+    uint64_t n_blocks, n_words;
+} s3_compact_host_layer;
+
+s3_status s3_compact_bound(uint64_t n_postings, int d_sae, uint64_t* max_blocks, uint64_t* max_words);
+size_t s3_compact_workspace_bytes(uint64_t n_postings, int d_sae);
+s3_status s3_compact_build(const uint64_t* d_row_ptr, const int32_t* d_pos, uint64_t n_postings, int d_sae,
+                           int64_t stop_freq, uint64_t* d_out_row_ptr, uint32_t* d_blk_ptr, int32_t* d_blk_first,
+                           uint64_t* d_blk_desc, uint64_t cap_blocks, uint32_t* d_payload, uint64_t cap_words,
+                           uint64_t* d_sizes /*[4]*/, void* d_ws, size_t ws_bytes, void* stream);
+s3_status s3_coactivation_score_topspans_compact(const s3_compact_view* h_layers, int n_layers, int d_sae, int64_t L,
+                                                 const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
+                                                 const s3_score_params* params, const float* d_bm25, int64_t ld_bm25,
+                                                 int32_t* d_top_idx, float* d_top_score, float* d_all_scores,
+                                                 void* d_ws, size_t ws_bytes, void* stream);
+s3_status s3_compact_save(const char* path, int n_layers, int d_sae, const s3_compact_host_layer* h_layers);
+s3_status s3_compact_file_info(const char* path, int* n_layers, int* d_sae, uint64_t* h_n_blocks, uint64_t* h_n_words,
+                               int cap_layers);
+s3_status s3_compact_load(const char* path, int n_layers, int d_sae, s3_compact_host_layer* h_layers);
+
+/* ------------------------------------------------------------------------------------------------
  * Hybrid fusion of index sets                  (paper Sec. 3.6 Eq. 7: M_final = M_S3 U M_BM25 U M_Bias;
  *                                               Alg. 1 Phase 3: Idx_Final <- Idx_S3 U Idx_Lexical U LeadTail)
  *

@@ -29,6 +29,8 @@ EXPORTS = [
     "s3_score_workspace_bytes", "s3_coactivation_score_topspans",
     "s3_density_workspace_bytes", "s3_position_density_topcenters",
     "s3_fuse_workspace_bytes", "s3_fuse_index_sets",
+    "s3_compact_bound", "s3_compact_workspace_bytes", "s3_compact_build", "s3_coactivation_score_topspans_compact",
+    "s3_compact_save", "s3_compact_file_info", "s3_compact_load",
 ]
 
 
@@ -46,6 +48,16 @@ class PostingsItem(C.Structure):
 
 class CsrView(C.Structure):
     _fields_ = [("d_row_ptr", C.c_void_p), ("d_pos", C.c_void_p)]
+
+
+class CompactView(C.Structure):
+    _fields_ = [("d_row_ptr", C.c_void_p), ("d_blk_ptr", C.c_void_p), ("d_blk_first", C.c_void_p),
+                ("d_blk_desc", C.c_void_p), ("d_payload", C.c_void_p)]
+
+
+class CompactHostLayer(C.Structure):
+    _fields_ = [("h_row_ptr", C.c_void_p), ("h_blk_ptr", C.c_void_p), ("h_blk_first", C.c_void_p),
+                ("h_blk_desc", C.c_void_p), ("h_payload", C.c_void_p), ("n_blocks", C.c_uint64), ("n_words", C.c_uint64)]
 
 
 class ScoreParams(C.Structure):
@@ -76,7 +88,8 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.s3_last_error.restype = C.c_char_p
         for name in ("s3_sae_prepared_bytes", "s3_sae_encode_workspace_bytes", "s3_postings_workspace_bytes",
-                     "s3_score_workspace_bytes", "s3_density_workspace_bytes", "s3_fuse_workspace_bytes"):
+                     "s3_score_workspace_bytes", "s3_density_workspace_bytes", "s3_fuse_workspace_bytes",
+                     "s3_compact_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.s3_sae_prepared_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_sae_create.argtypes = [C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
@@ -115,6 +128,16 @@ def lib():
         L.s3_fuse_workspace_bytes.argtypes = [C.c_int, C.c_int64]
         L.s3_fuse_index_sets.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64,
                                          C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_compact_bound.argtypes = [C.c_uint64, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+        L.s3_compact_workspace_bytes.argtypes = [C.c_uint64, C.c_int]
+        L.s3_compact_build.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_int, C.c_int64, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p,
+                                       C.c_size_t, C.c_void_p]
+        L.s3_coactivation_score_topspans_compact.argtypes = [C.POINTER(CompactView)] + L.s3_coactivation_score_topspans.argtypes[1:]
+        L.s3_compact_save.argtypes = [C.c_char_p, C.c_int, C.c_int, C.POINTER(CompactHostLayer)]
+        L.s3_compact_file_info.argtypes = [C.c_char_p, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_uint64),
+                                           C.POINTER(C.c_uint64), C.c_int]
+        L.s3_compact_load.argtypes = [C.c_char_p, C.c_int, C.c_int, C.POINTER(CompactHostLayer)]
         _lib = L
     return _lib
 
@@ -364,3 +387,124 @@ def s3_fuse_index_sets(centers: torch.Tensor, span_width: int, lexical: torch.Te
     _check(lib().s3_fuse_index_sets(_ptr(centers), Q, N, span_width, _ptr(lexical), n_lex, lead, tail, L, _ptr(idx), cap,
                                     _ptr(count), _ptr(ws), ws.numel(), _stream(stream)))
     return idx, count
+
+
+# ------------------------------------------------------------------------------------------------ compact index
+COMPACT_FIELDS = ("row_ptr", "blk_ptr", "blk_first", "blk_desc", "payload")
+_COMPACT_DTYPES = dict(row_ptr=torch.int64, blk_ptr=torch.int32, blk_first=torch.int32, blk_desc=torch.int64,
+                       payload=torch.int32)
+
+
+class CompactLayer:
+    """The five arrays of one layer's compact index as tensors (unsigned contents in same-width signed dtypes):
+    row_ptr int64 [d_sae+1], blk_ptr int32 [d_sae+1], blk_first int32 [n_blocks], blk_desc int64 [n_blocks],
+    payload int32 [n_words]."""
+
+    def __init__(self, row_ptr, blk_ptr, blk_first, blk_desc, payload):
+        self.row_ptr, self.blk_ptr, self.blk_first, self.blk_desc, self.payload = row_ptr, blk_ptr, blk_first, blk_desc, payload
+        for name in COMPACT_FIELDS:
+            t = getattr(self, name)
+            assert t.dtype == _COMPACT_DTYPES[name] and t.is_contiguous(), name
+
+    def view(self) -> CompactView:
+        return CompactView(*[getattr(self, n).data_ptr() for n in COMPACT_FIELDS])
+
+    def host_layer(self) -> CompactHostLayer:
+        assert self.row_ptr.device.type == "cpu"
+        return CompactHostLayer(*[getattr(self, n).data_ptr() for n in COMPACT_FIELDS], self.blk_first.numel(),
+                                self.payload.numel())
+
+    def to(self, device):
+        return CompactLayer(*[getattr(self, n).to(device) for n in COMPACT_FIELDS])
+
+    def nbytes(self) -> int:
+        return sum(getattr(self, n).numel() * getattr(self, n).element_size() for n in COMPACT_FIELDS)
+
+
+def s3_compact_bound(n_postings: int, d_sae: int):
+    b, w = C.c_uint64(), C.c_uint64()
+    _check(lib().s3_compact_bound(n_postings, d_sae, C.byref(b), C.byref(w)))
+    return b.value, w.value
+
+
+def s3_compact_workspace_bytes(n_postings: int, d_sae: int) -> int:
+    return int(lib().s3_compact_workspace_bytes(n_postings, d_sae))
+
+
+def s3_compact_build(row_ptr: torch.Tensor, pos: torch.Tensor, d_sae: int, stop_freq: int = 0, ws: torch.Tensor | None = None,
+                     cap_blocks: int | None = None, cap_words: int | None = None, stream=None) -> CompactLayer:
+    """row_ptr int64 [d_sae+1], pos int32: one layer's merged CSR on the device. Allocates the outputs at the
+    bound (or the given capacities), runs the build, waits for it and returns the arrays cut to their sizes."""
+    assert row_ptr.dtype == torch.int64 and pos.dtype == torch.int32 and row_ptr.numel() == d_sae + 1
+    dev = row_ptr.device
+    n = pos.numel()
+    mb, mw = s3_compact_bound(n, d_sae)
+    cap_blocks = mb if cap_blocks is None else cap_blocks
+    cap_words = mw if cap_words is None else cap_words
+    if ws is None:
+        ws = torch.zeros(s3_compact_workspace_bytes(n, d_sae), dtype=torch.uint8, device=dev)
+    out_rp = torch.empty(d_sae + 1, dtype=torch.int64, device=dev)
+    blk_ptr = torch.empty(d_sae + 1, dtype=torch.int32, device=dev)
+    blk_first = torch.empty(max(cap_blocks, 1), dtype=torch.int32, device=dev)
+    blk_desc = torch.empty(max(cap_blocks, 1), dtype=torch.int64, device=dev)
+    payload = torch.empty(max(cap_words, 1), dtype=torch.int32, device=dev)
+    sizes = torch.zeros(4, dtype=torch.int64, device=dev)
+    _check(lib().s3_compact_build(_ptr(row_ptr), _ptr(pos), n, d_sae, stop_freq, _ptr(out_rp), _ptr(blk_ptr), _ptr(blk_first),
+                                  _ptr(blk_desc), cap_blocks, _ptr(payload), cap_words, _ptr(sizes), _ptr(ws), ws.numel(),
+                                  _stream(stream)))
+    code = C.c_uint32(0)
+    _check(lib().s3_workspace_status(_ptr(ws), _stream(stream), C.byref(code)))
+    _, n_blocks, n_words, _ = sizes.tolist()
+    return CompactLayer(out_rp, blk_ptr, blk_first[:n_blocks].contiguous(), blk_desc[:n_blocks].contiguous(),
+                        payload[:n_words].contiguous())
+
+
+def s3_coactivation_score_topspans_compact(layers, d_sae: int, L: int, q_ids: torch.Tensor, q_vals: torch.Tensor,
+                                           width: int, stride: int, s: int, alpha: float, beta: float, ws: torch.Tensor,
+                                           bm25: torch.Tensor | None = None, mode: int = S3_SCORE_MINCOUNT, stop_freq: int = 0,
+                                           top_idx: torch.Tensor | None = None, top_score: torch.Tensor | None = None,
+                                           all_scores: torch.Tensor | None = None, stream=None):
+    """As s3_coactivation_score_topspans, with `layers` a list of CompactLayer on the device."""
+    n_layers, Q, nq, k = q_ids.shape
+    assert len(layers) == n_layers and q_ids.dtype == torch.int32 and q_vals.dtype == torch.float32
+    assert q_ids.is_contiguous() and q_vals.is_contiguous()
+    for c in layers:
+        assert c.row_ptr.numel() == d_sae + 1 and c.payload.numel() >= 1
+    views = (CompactView * n_layers)(*[c.view() for c in layers])
+    dev = q_ids.device
+    if top_idx is None:
+        top_idx = torch.empty((Q, s), dtype=torch.int32, device=dev)
+    if top_score is None:
+        top_score = torch.empty((Q, s), dtype=torch.float32, device=dev)
+    params = ScoreParams(width, stride, mode, s, alpha, beta, stop_freq)
+    ld = 0 if bm25 is None else bm25.stride(0)
+    _check(lib().s3_coactivation_score_topspans_compact(views, n_layers, d_sae, L, _ptr(q_ids), _ptr(q_vals), Q, nq, k,
+                                                        C.byref(params), _ptr(bm25), ld, _ptr(top_idx), _ptr(top_score),
+                                                        _ptr(all_scores), _ptr(ws), ws.numel(), _stream(stream)))
+    return top_idx, top_score
+
+
+def s3_compact_save(path: str, layers, d_sae: int):
+    """layers: list of CompactLayer on the HOST."""
+    arr = (CompactHostLayer * len(layers))(*[c.host_layer() for c in layers])
+    _check(lib().s3_compact_save(path.encode(), len(layers), d_sae, arr))
+
+
+def s3_compact_file_info(path: str):
+    """Returns (n_layers, d_sae, [n_blocks per layer], [n_words per layer])."""
+    n_layers, d_sae = C.c_int(), C.c_int()
+    nb = (C.c_uint64 * 16)()
+    nw = (C.c_uint64 * 16)()
+    _check(lib().s3_compact_file_info(path.encode(), C.byref(n_layers), C.byref(d_sae), nb, nw, 16))
+    return n_layers.value, d_sae.value, list(nb[:n_layers.value]), list(nw[:n_layers.value])
+
+
+def s3_compact_load(path: str):
+    """Returns (list of CompactLayer on the host, d_sae)."""
+    n_layers, d_sae, nb, nw = s3_compact_file_info(path)
+    layers = [CompactLayer(torch.empty(d_sae + 1, dtype=torch.int64), torch.empty(d_sae + 1, dtype=torch.int32),
+                           torch.empty(nb[l], dtype=torch.int32), torch.empty(nb[l], dtype=torch.int64),
+                           torch.empty(nw[l], dtype=torch.int32)) for l in range(n_layers)]
+    arr = (CompactHostLayer * n_layers)(*[c.host_layer() for c in layers])
+    _check(lib().s3_compact_load(path.encode(), n_layers, d_sae, arr))
+    return layers, d_sae

@@ -120,6 +120,7 @@ s3_status s3_workspace_status(const void* d_ws, void* stream, uint32_t* code_out
     if (code_out) *code_out = code;
     if (code == DEV_OK) return S3_OK;
     if (code == DEV_BAD_FEATURE_ID) return fail(S3_ERR_INVALID_ARG, "a feature id >= d_sae was met on the device (code %u)", code);
+    if (code == DEV_COMPACT_CAPACITY) return fail(S3_ERR_CAPACITY, "compact index: block or payload buffer too small (code %u)", code);
     return fail(S3_ERR_TIMEOUT, "a bounded device-side wait ran out (code %u)", code);
 }
 
@@ -280,10 +281,14 @@ size_t s3_score_workspace_bytes(int Q, int nq, int k, int n_layers, int n_spans,
     return S3_WS_HEADER_BYTES;
 }
 
-s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L,
-                                         const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
-                                         const s3_score_params* p, const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx,
-                                         float* d_top_score, float* d_all_scores, void* d_ws, size_t ws_bytes, void* stream)
+}  // extern "C"
+
+namespace {
+
+// Argument checks shared by the two scoring entry points; *n_spans_out receives the span count.
+s3_status check_score_args(const void* h_layers, int n_layers, int d_sae, int64_t L, const int32_t* d_q_ids, const float* d_q_vals,
+                           int Q, int nq, int k, const s3_score_params* p, const float* d_bm25, int64_t ld_bm25,
+                           const int32_t* d_top_idx, const float* d_top_score, const void* d_ws, size_t ws_bytes, int64_t* n_spans_out)
 {
     S3_REQUIRE(h_layers && p, S3_ERR_INVALID_ARG, "null argument");
     S3_REQUIRE(n_layers >= 1 && n_layers <= S3_MAX_SCORE_LAYERS, S3_ERR_UNSUPPORTED, "n_layers = %d out of [1, %d]", n_layers,
@@ -297,15 +302,87 @@ s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_laye
     S3_REQUIRE(p->s >= 1 && p->s <= 64, S3_ERR_UNSUPPORTED, "s = %d out of [1, 64]", p->s);
     const int64_t n_spans = (L >= p->width) ? (L - p->width) / p->stride + 1 : 0;
     S3_REQUIRE(n_spans <= 16384, S3_ERR_UNSUPPORTED, "n_spans = %lld exceeds 16384", (long long)n_spans);
+    *n_spans_out = n_spans;
     if (Q == 0) return S3_OK;
     S3_REQUIRE(d_q_ids && d_q_vals && d_top_idx && d_top_score, S3_ERR_INVALID_ARG, "null device pointer");
     S3_REQUIRE(d_ws != nullptr && ws_bytes >= S3_WS_HEADER_BYTES, S3_ERR_CAPACITY, "workspace missing or smaller than %d bytes",
                S3_WS_HEADER_BYTES);
     S3_REQUIRE(d_bm25 == nullptr || ld_bm25 >= n_spans, S3_ERR_INVALID_ARG, "ld_bm25 smaller than n_spans");
+    return S3_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L,
+                                         const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
+                                         const s3_score_params* p, const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx,
+                                         float* d_top_score, float* d_all_scores, void* d_ws, size_t ws_bytes, void* stream)
+{
+    int64_t n_spans = 0;
+    const s3_status st = check_score_args(h_layers, n_layers, d_sae, L, d_q_ids, d_q_vals, Q, nq, k, p, d_bm25, ld_bm25, d_top_idx,
+                                          d_top_score, d_ws, ws_bytes, &n_spans);
+    if (st != S3_OK || Q == 0) return st;
     for (int l = 0; l < n_layers; ++l)
         S3_REQUIRE(h_layers[l].d_row_ptr && (h_layers[l].d_pos || n_spans == 0), S3_ERR_INVALID_ARG, "layer %d: null CSR pointer", l);
     return launch_score(h_layers, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, (int)n_spans, p, d_bm25, ld_bm25, d_top_idx,
                         d_top_score, d_all_scores, static_cast<cudaStream_t>(stream));
+}
+
+s3_status s3_coactivation_score_topspans_compact(const s3_compact_view* h_layers, int n_layers, int d_sae, int64_t L,
+                                                 const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
+                                                 const s3_score_params* p, const float* d_bm25, int64_t ld_bm25,
+                                                 int32_t* d_top_idx, float* d_top_score, float* d_all_scores, void* d_ws,
+                                                 size_t ws_bytes, void* stream)
+{
+    int64_t n_spans = 0;
+    const s3_status st = check_score_args(h_layers, n_layers, d_sae, L, d_q_ids, d_q_vals, Q, nq, k, p, d_bm25, ld_bm25, d_top_idx,
+                                          d_top_score, d_ws, ws_bytes, &n_spans);
+    if (st != S3_OK || Q == 0) return st;
+    for (int l = 0; l < n_layers; ++l)
+        S3_REQUIRE(h_layers[l].d_row_ptr && h_layers[l].d_blk_ptr && h_layers[l].d_blk_first && h_layers[l].d_blk_desc &&
+                       h_layers[l].d_payload,
+                   S3_ERR_INVALID_ARG, "layer %d: null pointer in the compact view", l);
+    return launch_score_compact(h_layers, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, (int)n_spans, p, d_bm25, ld_bm25,
+                                d_top_idx, d_top_score, d_all_scores, static_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------------------------- compact index
+s3_status s3_compact_bound(uint64_t n_postings, int d_sae, uint64_t* max_blocks, uint64_t* max_words)
+{
+    S3_REQUIRE(max_blocks && max_words, S3_ERR_INVALID_ARG, "null output pointer");
+    S3_REQUIRE(d_sae >= 1 && d_sae <= (1 << 20), S3_ERR_INVALID_ARG, "d_sae = %d out of range", d_sae);
+    S3_REQUIRE(n_postings <= (1ull << 36), S3_ERR_UNSUPPORTED, "more than 2^36 postings in one layer");
+    compact_bound(n_postings, d_sae, max_blocks, max_words);
+    return S3_OK;
+}
+
+size_t s3_compact_workspace_bytes(uint64_t n_postings, int d_sae)
+{
+    if (d_sae < 1 || d_sae > (1 << 20) || n_postings > (1ull << 36)) return 0;
+    return 256 + compact_workspace_bytes(n_postings, d_sae);
+}
+
+s3_status s3_compact_build(const uint64_t* d_row_ptr, const int32_t* d_pos, uint64_t n_postings, int d_sae, int64_t stop_freq,
+                           uint64_t* d_out_row_ptr, uint32_t* d_blk_ptr, int32_t* d_blk_first, uint64_t* d_blk_desc,
+                           uint64_t cap_blocks, uint32_t* d_payload, uint64_t cap_words, uint64_t* d_sizes, void* d_ws,
+                           size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(d_sae >= 1 && d_sae <= (1 << 20), S3_ERR_INVALID_ARG, "d_sae = %d out of range", d_sae);
+    S3_REQUIRE(n_postings <= (1ull << 36), S3_ERR_UNSUPPORTED, "more than 2^36 postings in one layer");
+    S3_REQUIRE(stop_freq >= 0, S3_ERR_INVALID_ARG, "stop_freq must not be negative");
+    S3_REQUIRE(d_row_ptr && (d_pos || n_postings == 0) && d_out_row_ptr && d_blk_ptr && d_sizes, S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE((d_blk_first && d_blk_desc) || cap_blocks == 0, S3_ERR_INVALID_ARG, "null block arrays");
+    S3_REQUIRE(d_payload != nullptr && cap_words >= 1, S3_ERR_CAPACITY, "the payload needs at least its closing word");
+    uint64_t need_blocks, need_words;
+    compact_bound(n_postings, d_sae, &need_blocks, &need_words);
+    const uint64_t scratch_blocks = cap_blocks < need_blocks ? cap_blocks : need_blocks;
+    S3_REQUIRE(d_ws != nullptr && ws_bytes >= 256 + (scratch_blocks + 1) * 8, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed",
+               ws_bytes, static_cast<size_t>(256 + (scratch_blocks + 1) * 8));
+    return launch_compact_build(d_row_ptr, d_pos, d_sae, stop_freq, d_out_row_ptr, d_blk_ptr, d_blk_first, d_blk_desc, scratch_blocks,
+                                d_payload, cap_words, d_sizes, static_cast<uint32_t*>(d_ws),
+                                static_cast<unsigned char*>(d_ws) + 256, static_cast<cudaStream_t>(stream));
 }
 
 // ---------------------------------------------------------------------------------------------- density

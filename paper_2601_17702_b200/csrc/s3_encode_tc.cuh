@@ -39,6 +39,16 @@ s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, con
                        const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
                        float* d_all_scores, cudaStream_t stream);
 
+s3_status launch_score_compact(const s3_compact_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
+                               const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
+                               const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
+                               float* d_all_scores, cudaStream_t stream);
+void compact_bound(uint64_t n_postings, int d_sae, uint64_t* max_blocks, uint64_t* max_words);
+size_t compact_workspace_bytes(uint64_t n_postings, int d_sae);
+s3_status launch_compact_build(const uint64_t* d_row_ptr, const int32_t* d_pos, int d_sae, int64_t stop_freq,
+                               uint64_t* d_out_row_ptr, uint32_t* d_blk_ptr, int32_t* d_blk_first, uint64_t* d_blk_desc,
+                               uint64_t cap_blocks, uint32_t* d_payload, uint64_t cap_words, uint64_t* d_sizes,
+                               uint32_t* d_status, void* d_scratch, cudaStream_t stream);
 size_t fuse_workspace_bytes(int Q, int64_t L);
 s3_status launch_fuse_sets(const int32_t* d_centers, int Q, int n_centers, int span_width, const int32_t* d_lexical, int n_lex,
                            int lead, int tail, int64_t L, int32_t* d_out_idx, int cap, int32_t* d_out_count, void* d_scratch,

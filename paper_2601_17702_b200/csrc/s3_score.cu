@@ -24,6 +24,10 @@ constexpr int WIN = 8192;        // pieces whose owning feature is tabulated at 
 struct ScoreLayers {
     s3_csr_view v[S3_MAX_SCORE_LAYERS];
 };
+struct CompactLayers {
+    s3_compact_view v[S3_MAX_SCORE_LAYERS];
+};
+constexpr int CBATCH = 4;        // compact index: blocks of 32 postings a warp decodes side by side
 
 struct ScoreArgs {
     const int32_t* q_ids;
@@ -178,7 +182,7 @@ __device__ __forceinline__ int aggregate_query(const int32_t* qi, const float* q
 // Returns the number of pieces. Called by the whole block.
 __device__ __forceinline__ uint32_t cut_lists(const uint64_t* __restrict__ row_ptr, int U, int64_t stop_freq,
                                               const int32_t* ufeat, unsigned long long* ulo, uint32_t* ulen,
-                                              uint32_t* cstart, uint32_t* ws)
+                                              uint32_t* cstart, uint32_t* ws, const uint32_t* __restrict__ blk_ptr = nullptr)
 {
     const int tid = threadIdx.x;
     uint32_t piece_carry = 0;
@@ -191,7 +195,7 @@ __device__ __forceinline__ uint32_t cut_lists(const uint64_t* __restrict__ row_p
             uint64_t len = hi - lo;
             if (len > 0x7FFFFFFFull) len = 0x7FFFFFFFull;          // positions are int32: a list cannot be longer
             if (stop_freq > 0 && static_cast<int64_t>(len) > stop_freq) len = 0;   // stop feature
-            ulo[u] = lo;
+            ulo[u] = blk_ptr ? static_cast<unsigned long long>(__ldg(blk_ptr + f)) : lo;   // compact index: first block
             ulen[u] = static_cast<uint32_t>(len);
             n_pieces = static_cast<uint32_t>((len + PIECE - 1) / PIECE);
         }
@@ -217,9 +221,47 @@ __device__ __forceinline__ void tabulate_owners(const uint32_t* cstart, int U, u
     __syncthreads();
 }
 
-template <bool POW2>
+// Compact index: the positions of block `blk` (cnt postings) in three steps, so that a warp can have the loads of
+// several blocks in flight: header, payload words of the lane's value, then value -> gap -> 32-lane prefix sum.
+struct BlockHead {
+    int first;
+    uint32_t width;
+    const uint32_t* words;
+};
+__device__ __forceinline__ BlockHead block_head(const s3_compact_view& v, uint32_t blk)
+{
+    BlockHead h;
+    h.first = __ldg(v.d_blk_first + blk);
+    const unsigned long long desc = __ldg(reinterpret_cast<const unsigned long long*>(v.d_blk_desc) + blk);
+    h.width = static_cast<uint32_t>(desc & 63u);
+    h.words = v.d_payload + (desc >> 6);
+    return h;
+}
+__device__ __forceinline__ void block_value_words(const BlockHead& h, uint32_t cnt, int lane, uint32_t& lo, uint32_t& hi)
+{
+    lo = 0; hi = 0;
+    if (lane >= 1 && lane < static_cast<int>(cnt) && h.width) {
+        const uint32_t* w = h.words + (((lane - 1) * h.width) >> 5);
+        lo = __ldg(w);
+        hi = __ldg(w + 1);                    // the payload's closing word keeps this in bounds
+    }
+}
+__device__ __forceinline__ int block_positions(const BlockHead& h, uint32_t cnt, int lane, uint32_t lo, uint32_t hi)
+{
+    const uint32_t v = __funnelshift_r(lo, hi, ((lane - 1) * h.width) & 31) & ((1u << h.width) - 1u);
+    int d = lane == 0 ? h.first : (lane < static_cast<int>(cnt) ? static_cast<int>(v) + 1 : 0);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, d, o);
+        if (lane >= o) d += y;
+    }
+    return lane < static_cast<int>(cnt) ? d : -1;
+}
+
+template <bool POW2, bool COMPACT>
 __global__ void __launch_bounds__(ST)
-score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__ ScoreArgs a)
+score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__ CompactLayers clayers,
+             const __grid_constant__ ScoreArgs a)
 {
     extern __shared__ __align__(16) unsigned char score_smem_raw[];
     const bool weighted = a.mode == S3_SCORE_WEIGHTED;
@@ -253,7 +295,8 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
         const int U = aggregate_query(qi, qv, a.nk, a.npad, a.d_sae, weighted, keys, ufeat, ustart, uaq, ws, &n_unique_s);
         // b. list bounds of every unique feature (independent loads), then the pieces' prefix sum
         const int32_t* __restrict__ pos = layers.v[l].d_pos;
-        const uint32_t piece_total = cut_lists(layers.v[l].d_row_ptr, U, weighted ? a.stop_freq : 0, ufeat, ulo, ulen, cstart, ws);
+        const uint32_t piece_total = cut_lists(layers.v[l].d_row_ptr, U, weighted ? a.stop_freq : 0, ufeat, ulo, ulen, cstart, ws,
+                                               COMPACT ? clayers.v[l].d_blk_ptr : nullptr);
 
         // The pieces are walked a window at a time; inside a window every warp takes an equal share. BATCH
         // pieces per round: first all their loads are issued, then their updates, so that a warp has BATCH
@@ -264,6 +307,76 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
             const uint32_t n_win = win1 - win0;
             const uint32_t c_begin = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * warp / SW);
             const uint32_t c_end = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * (warp + 1) / SW);
+            if constexpr (COMPACT) {
+                // A piece is one block of the compact index. In min-count mode posting i also needs the position of
+                // posting i - cQ of its list: the 32 lanes' targets lie in at most two blocks, floor((32 j - cQ)/32)
+                // and the next one; whichever of them is not block j itself is decoded too (jobs 1 and 2).
+                const s3_compact_view& cv = clayers.v[l];
+                for (uint32_t c0 = c_begin; c0 < c_end; c0 += CBATCH) {
+                    BlockHead h[CBATCH][3];
+                    uint32_t cnt[CBATCH][3], lo[CBATCH][3], hi[CBATCH][3];
+                    int ub[CBATCH], jb[CBATCH], ta[CBATCH], cqb[CBATCH];
+#pragma unroll
+                    for (int b = 0; b < CBATCH; ++b) {
+                        const uint32_t c = c0 + b;
+                        cnt[b][0] = cnt[b][1] = cnt[b][2] = 0;
+                        ub[b] = 0; jb[b] = 0; ta[b] = 0; cqb[b] = 0;
+                        if (c < c_end) {
+                            const int u = owner[c - win0];
+                            const int j = static_cast<int>(c - cstart[u]);
+                            const uint32_t blk0 = static_cast<uint32_t>(ulo[u]);
+                            const uint32_t left = ulen[u] - 32u * static_cast<uint32_t>(j);
+                            ub[b] = u; jb[b] = j;
+                            cnt[b][0] = left < 32u ? left : 32u;
+                            h[b][0] = block_head(cv, blk0 + j);
+                            if (!weighted) {
+                                const int cq = ustart[u + 1] - ustart[u];
+                                const int tb = (32 * j - cq) >> 5;           // floor, may be negative
+                                cqb[b] = cq; ta[b] = tb;
+                                if (tb >= 0 && tb < j) { cnt[b][1] = 32u; h[b][1] = block_head(cv, blk0 + tb); }
+                                if (tb + 1 >= 0 && tb + 1 < j) { cnt[b][2] = 32u; h[b][2] = block_head(cv, blk0 + tb + 1); }
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int b = 0; b < CBATCH; ++b)
+#pragma unroll
+                        for (int r = 0; r < 3; ++r) {
+                            lo[b][r] = 0; hi[b][r] = 0;
+                            if (cnt[b][r]) block_value_words(h[b][r], cnt[b][r], lane, lo[b][r], hi[b][r]);
+                        }
+#pragma unroll
+                    for (int b = 0; b < CBATCH; ++b) {
+                        if (cnt[b][0] == 0) continue;                      // uniform over the warp
+                        const int p = block_positions(h[b][0], cnt[b][0], lane, lo[b][0], hi[b][0]);
+                        int p_prev = -1;
+                        if (!weighted) {
+                            const int p1 = cnt[b][1] ? block_positions(h[b][1], 32u, lane, lo[b][1], hi[b][1]) : -1;
+                            const int p2 = cnt[b][2] ? block_positions(h[b][2], 32u, lane, lo[b][2], hi[b][2]) : -1;
+                            const int src = (lane - cqb[b]) & 31;
+                            const int v0 = __shfl_sync(0xffffffffu, p, src);
+                            const int v1 = __shfl_sync(0xffffffffu, p1, src);
+                            const int v2 = __shfl_sync(0xffffffffu, p2, src);
+                            const int t = 32 * jb[b] + lane - cqb[b];      // list index of the earlier posting
+                            if (t >= 0) {
+                                const int tb = t >> 5;
+                                p_prev = tb == jb[b] ? v0 : (tb == ta[b] ? v1 : v2);
+                            }
+                        }
+                        if (p < 0) continue;
+                        int j_lo, j_hi;
+                        posting_range<POW2>(a, p, p_prev, j_lo, j_hi);
+                        if (weighted) {
+                            const double w = static_cast<double>(uaq[ub[b]]) *
+                                             (1.0 / (log(1.0 + static_cast<double>(ulen[ub[b]])) + 1.0));
+                            for (int j = j_lo; j <= j_hi; ++j) atomicAdd(&acc_d[j], w);
+                        } else if (j_lo <= j_hi) {
+                            atomicAdd(&acc_i[j_lo], 1);
+                            atomicAdd(&acc_i[j_hi + 1], -1);
+                        }
+                    }
+                }
+            } else
             for (uint32_t c0 = c_begin; c0 < c_end; c0 += BATCH) {
                 int p[BATCH], p_prev[BATCH], ub[BATCH];
 #pragma unroll
@@ -536,10 +649,12 @@ density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant
 
 }  // namespace
 
-s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
-                       const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
-                       const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
-                       float* d_all_scores, cudaStream_t stream)
+namespace {
+
+s3_status launch_score_impl(const ScoreLayers& layers, const CompactLayers* clayers, int n_layers, int d_sae, const int32_t* d_q_ids,
+                            const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
+                            const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
+                            float* d_all_scores, cudaStream_t stream)
 {
     static int max_smem_dev[64] = {};
     int dev = 0;
@@ -547,12 +662,12 @@ s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, con
     int max_smem = dev < 64 ? max_smem_dev[dev] : 0;
     if (max_smem == 0) {
         S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
-        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
         if (dev < 64) max_smem_dev[dev] = max_smem;
     }
-    ScoreLayers layers;
-    for (int l = 0; l < n_layers; ++l) layers.v[l] = h_layers[l];
     ScoreArgs a;
     a.q_ids = d_q_ids; a.q_vals = d_q_vals; a.bm25 = d_bm25; a.ld_bm25 = ld_bm25;
     a.top_idx = d_top_idx; a.top_score = d_top_score; a.all_scores = d_all_scores;
@@ -567,10 +682,45 @@ s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, con
     S3_REQUIRE(smem + 2048 <= static_cast<size_t>(max_smem), S3_ERR_UNSUPPORTED,
                "n_spans = %d with nq*k = %d needs %zu bytes of shared memory per query, %d available", n_spans, a.nk, smem,
                max_smem - 2048);
-    if (a.stride_shift >= 0) score_kernel<true><<<Q, ST, smem, stream>>>(layers, a);
-    else score_kernel<false><<<Q, ST, smem, stream>>>(layers, a);
+    if (clayers) {
+        if (a.stride_shift >= 0) score_kernel<true, true><<<Q, ST, smem, stream>>>(layers, *clayers, a);
+        else score_kernel<false, true><<<Q, ST, smem, stream>>>(layers, *clayers, a);
+    } else {
+        CompactLayers none = {};
+        if (a.stride_shift >= 0) score_kernel<true, false><<<Q, ST, smem, stream>>>(layers, none, a);
+        else score_kernel<false, false><<<Q, ST, smem, stream>>>(layers, none, a);
+    }
     S3_CUDA_TRY(cudaGetLastError());
     return S3_OK;
+}
+
+}  // namespace
+
+s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
+                       const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
+                       const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
+                       float* d_all_scores, cudaStream_t stream)
+{
+    ScoreLayers layers = {};
+    for (int l = 0; l < n_layers; ++l) layers.v[l] = h_layers[l];
+    return launch_score_impl(layers, nullptr, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, n_spans, p, d_bm25, ld_bm25,
+                             d_top_idx, d_top_score, d_all_scores, stream);
+}
+
+s3_status launch_score_compact(const s3_compact_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
+                               const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
+                               const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
+                               float* d_all_scores, cudaStream_t stream)
+{
+    ScoreLayers layers = {};
+    CompactLayers cl = {};
+    for (int l = 0; l < n_layers; ++l) {
+        cl.v[l] = h_layers[l];
+        layers.v[l].d_row_ptr = h_layers[l].d_row_ptr;
+        layers.v[l].d_pos = nullptr;
+    }
+    return launch_score_impl(layers, &cl, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, n_spans, p, d_bm25, ld_bm25,
+                             d_top_idx, d_top_score, d_all_scores, stream);
 }
 
 }  // namespace s3
