@@ -441,6 +441,23 @@ def run_case(args):
             gathered += int(lens[torch.unique(q_ids[0, q].flatten().long())].sum().item())
         run = lambda i: S.s3_coactivation_score_topspans(csr, D, L, q_ids, q_vals, r.width, stride, r.s, r.alpha, r.beta, ws,
                                                          bm25, top_idx=top_idx, top_score=top_score)
+        if args.compact:
+            # the same index in block-delta form: build timed once, then the scorer decodes blocks in its gather
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            cws = S.new_workspace(S.s3_compact_workspace_bytes(csr[0][1].numel(), D), dev)
+            S.s3_compact_build(csr[0][0], csr[0][1], D, 0, cws)
+            e0.record()
+            comp = S.s3_compact_build(csr[0][0], csr[0][1], D, 0, cws)
+            e1.record()
+            torch.cuda.synchronize()
+            ref_idx, ref_score = run(0)
+            ref_idx, ref_score = ref_idx.clone(), ref_score.clone()
+            run = lambda i: S.s3_coactivation_score_topspans_compact([comp], D, L, q_ids, q_vals, r.width, stride, r.s, r.alpha,
+                                                                     r.beta, ws, bm25, top_idx=top_idx, top_score=top_score)
+            run(0)
+            torch.cuda.synchronize()
+            out.update(compact_bytes=comp.nbytes(), compact_build_ms=e0.elapsed_time(e1),
+                       same_result=bool(torch.equal(ref_idx, top_idx) and torch.equal(ref_score, top_score)))
         out.update(L=L, d_sae=D, k=k, Q=r.Q, nq=r.nq, kq=r.kq, spans=ns, stride=stride, gathered_postings=gathered,
                    index_bytes=int(ps.numel()) * 4, bytes=gathered * 4 + r.Q * ns * 4 + r.Q * r.s * 8)
     elif args.case == "density":
@@ -502,6 +519,7 @@ def main():
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)
     ap.add_argument("--items", type=int, default=8)
+    ap.add_argument("--compact", action="store_true", help="score case: read the block-delta compact index")
     ap.add_argument("--no-union", action="store_true", help="density case: leave out the index-set union")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=96)

@@ -1,8 +1,9 @@
 """CPU oracle of the streaming-scan hot path. TEST INFRASTRUCTURE ONLY.
 
 Only tests/, the smoke check and the benchmark's CPU-baseline leg may import this package; the
-product package never does. The arithmetic lives in s3_oracle.cpp (plain C++, fp64); this file only
-marshals numpy arrays into it.
+product package never does. The floating-point arithmetic lives in s3_oracle.cpp (plain C++, fp64), which this file
+marshals numpy arrays into; the pure integer / set steps at the end of the file (index-set union, compact index
+encoding) are plain Python here. No function is "parity unpinned".
 """
 from __future__ import annotations
 

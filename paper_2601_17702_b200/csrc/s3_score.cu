@@ -27,7 +27,7 @@ struct ScoreLayers {
 struct CompactLayers {
     s3_compact_view v[S3_MAX_SCORE_LAYERS];
 };
-constexpr int CBATCH = 4;        // compact index: blocks of 32 postings a warp decodes side by side
+constexpr int CBATCH = 8;        // compact index: blocks of 32 postings a warp decodes side by side
 
 struct ScoreArgs {
     const int32_t* q_ids;
@@ -221,41 +221,50 @@ __device__ __forceinline__ void tabulate_owners(const uint32_t* cstart, int U, u
     __syncthreads();
 }
 
-// Compact index: the positions of block `blk` (cnt postings) in three steps, so that a warp can have the loads of
-// several blocks in flight: header, payload words of the lane's value, then value -> gap -> 32-lane prefix sum.
-struct BlockHead {
+// Compact index: the positions of a block of cnt postings in three steps, so that a warp can have the loads of
+// several blocks in flight: header, the payload words of the lane's value, then value -> gap -> 32-lane prefix sum.
+struct PieceHead {
     int first;
-    uint32_t width;
-    const uint32_t* words;
+    unsigned long long desc;     // (payload word offset << 6) | width
+    uint32_t cnt;                // postings in the block; 0 = no block
 };
-__device__ __forceinline__ BlockHead block_head(const s3_compact_view& v, uint32_t blk)
+__device__ __forceinline__ PieceHead block_head(const s3_compact_view& v, uint32_t blk, uint32_t cnt)
 {
-    BlockHead h;
+    PieceHead h;
     h.first = __ldg(v.d_blk_first + blk);
-    const unsigned long long desc = __ldg(reinterpret_cast<const unsigned long long*>(v.d_blk_desc) + blk);
-    h.width = static_cast<uint32_t>(desc & 63u);
-    h.words = v.d_payload + (desc >> 6);
+    h.desc = __ldg(reinterpret_cast<const unsigned long long*>(v.d_blk_desc) + blk);
+    h.cnt = cnt;
     return h;
 }
-__device__ __forceinline__ void block_value_words(const BlockHead& h, uint32_t cnt, int lane, uint32_t& lo, uint32_t& hi)
+__device__ __forceinline__ void block_value_words(const s3_compact_view& v, const PieceHead& h, int lane, uint32_t& lo, uint32_t& hi)
 {
     lo = 0; hi = 0;
-    if (lane >= 1 && lane < static_cast<int>(cnt) && h.width) {
-        const uint32_t* w = h.words + (((lane - 1) * h.width) >> 5);
+    const uint32_t width = static_cast<uint32_t>(h.desc & 63u);
+    if (lane >= 1 && lane < static_cast<int>(h.cnt) && width) {
+        const uint32_t* w = v.d_payload + (h.desc >> 6) + (((lane - 1) * width) >> 5);
         lo = __ldg(w);
         hi = __ldg(w + 1);                    // the payload's closing word keeps this in bounds
     }
 }
-__device__ __forceinline__ int block_positions(const BlockHead& h, uint32_t cnt, int lane, uint32_t lo, uint32_t hi)
+__device__ __forceinline__ int block_positions(const PieceHead& h, int lane, uint32_t lo, uint32_t hi)
 {
-    const uint32_t v = __funnelshift_r(lo, hi, ((lane - 1) * h.width) & 31) & ((1u << h.width) - 1u);
-    int d = lane == 0 ? h.first : (lane < static_cast<int>(cnt) ? static_cast<int>(v) + 1 : 0);
+    const uint32_t width = static_cast<uint32_t>(h.desc & 63u);
+    const uint32_t v = __funnelshift_r(lo, hi, ((lane - 1) * width) & 31) & ((1u << width) - 1u);
+    int d = lane == 0 ? h.first : (lane < static_cast<int>(h.cnt) ? static_cast<int>(v) + 1 : 0);
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int y = __shfl_up_sync(0xffffffffu, d, o);
         if (lane >= o) d += y;
     }
-    return lane < static_cast<int>(cnt) ? d : -1;
+    return lane < static_cast<int>(h.cnt) ? d : -1;
+}
+// A full block decoded on the spot (three dependent steps; the rare path of the scorer).
+__device__ __noinline__ int block_positions_now(const s3_compact_view& v, uint32_t blk, int lane)
+{
+    const PieceHead h = block_head(v, blk, 32u);
+    uint32_t lo, hi;
+    block_value_words(v, h, lane, lo, hi);
+    return block_positions(h, lane, lo, hi);
 }
 
 template <bool POW2, bool COMPACT>
@@ -308,73 +317,91 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
             const uint32_t c_begin = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * warp / SW);
             const uint32_t c_end = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * (warp + 1) / SW);
             if constexpr (COMPACT) {
-                // A piece is one block of the compact index. In min-count mode posting i also needs the position of
-                // posting i - cQ of its list: the 32 lanes' targets lie in at most two blocks, floor((32 j - cQ)/32)
-                // and the next one; whichever of them is not block j itself is decoded too (jobs 1 and 2).
+                // A piece is one block of the compact index. The headers of the next CBATCH blocks are fetched while
+                // the payload words of the current ones are in flight, so a batch waits for one memory round trip.
+                // In min-count mode posting i also needs the position of posting i - cQ of its list: the 32 lanes'
+                // targets lie in at most two blocks, x = floor((32 j - cQ)/32) and x + 1. Block j itself is at hand; an
+                // earlier block j - d is piece b - d of this warp (its pieces are consecutive) and is taken from the
+                // batch or from the last two blocks of the previous batch; only when it lies further back (the start
+                // of the warp's share, cQ > 64) is it decoded on the spot.
                 const s3_compact_view& cv = clayers.v[l];
+                auto fetch_head = [&](uint32_t c) {
+                    PieceHead h;
+                    h.first = 0; h.desc = 0; h.cnt = 0;
+                    if (c < c_end) {
+                        const int u = owner[c - win0];
+                        const uint32_t j = c - cstart[u];
+                        const uint32_t left = ulen[u] - 32u * j;
+                        h = block_head(cv, static_cast<uint32_t>(ulo[u]) + j, left < 32u ? left : 32u);
+                    }
+                    return h;
+                };
+                PieceHead hn[CBATCH];
+#pragma unroll
+                for (int b = 0; b < CBATCH; ++b) hn[b] = fetch_head(c_begin + b);
+                int carry1 = -1, carry2 = -1;                              // positions of pieces c0 - 1 and c0 - 2
                 for (uint32_t c0 = c_begin; c0 < c_end; c0 += CBATCH) {
-                    BlockHead h[CBATCH][3];
-                    uint32_t cnt[CBATCH][3], lo[CBATCH][3], hi[CBATCH][3];
-                    int ub[CBATCH], jb[CBATCH], ta[CBATCH], cqb[CBATCH];
+                    PieceHead hc[CBATCH];
+                    uint32_t lo[CBATCH], hi[CBATCH];
+                    int hist[CBATCH + 2];
 #pragma unroll
                     for (int b = 0; b < CBATCH; ++b) {
-                        const uint32_t c = c0 + b;
-                        cnt[b][0] = cnt[b][1] = cnt[b][2] = 0;
-                        ub[b] = 0; jb[b] = 0; ta[b] = 0; cqb[b] = 0;
-                        if (c < c_end) {
-                            const int u = owner[c - win0];
-                            const int j = static_cast<int>(c - cstart[u]);
-                            const uint32_t blk0 = static_cast<uint32_t>(ulo[u]);
-                            const uint32_t left = ulen[u] - 32u * static_cast<uint32_t>(j);
-                            ub[b] = u; jb[b] = j;
-                            cnt[b][0] = left < 32u ? left : 32u;
-                            h[b][0] = block_head(cv, blk0 + j);
-                            if (!weighted) {
-                                const int cq = ustart[u + 1] - ustart[u];
-                                const int tb = (32 * j - cq) >> 5;           // floor, may be negative
-                                cqb[b] = cq; ta[b] = tb;
-                                if (tb >= 0 && tb < j) { cnt[b][1] = 32u; h[b][1] = block_head(cv, blk0 + tb); }
-                                if (tb + 1 >= 0 && tb + 1 < j) { cnt[b][2] = 32u; h[b][2] = block_head(cv, blk0 + tb + 1); }
-                            }
-                        }
+                        hc[b] = hn[b];
+                        block_value_words(cv, hc[b], lane, lo[b], hi[b]);
                     }
 #pragma unroll
-                    for (int b = 0; b < CBATCH; ++b)
-#pragma unroll
-                        for (int r = 0; r < 3; ++r) {
-                            lo[b][r] = 0; hi[b][r] = 0;
-                            if (cnt[b][r]) block_value_words(h[b][r], cnt[b][r], lane, lo[b][r], hi[b][r]);
-                        }
+                    for (int b = 0; b < CBATCH; ++b) hn[b] = fetch_head(c0 + CBATCH + b);
+                    hist[0] = carry2; hist[1] = carry1;
+                    const int avail = c0 - c_begin < 2u ? static_cast<int>(c0 - c_begin) : 2;
 #pragma unroll
                     for (int b = 0; b < CBATCH; ++b) {
-                        if (cnt[b][0] == 0) continue;                      // uniform over the warp
-                        const int p = block_positions(h[b][0], cnt[b][0], lane, lo[b][0], hi[b][0]);
+                        hist[b + 2] = -1;
+                        if (hc[b].cnt == 0) continue;                      // uniform over the warp
+                        const int p = block_positions(hc[b], lane, lo[b], hi[b]);
+                        hist[b + 2] = p;
+                        const int u = owner[c0 + b - win0];
                         int p_prev = -1;
                         if (!weighted) {
-                            const int p1 = cnt[b][1] ? block_positions(h[b][1], 32u, lane, lo[b][1], hi[b][1]) : -1;
-                            const int p2 = cnt[b][2] ? block_positions(h[b][2], 32u, lane, lo[b][2], hi[b][2]) : -1;
-                            const int src = (lane - cqb[b]) & 31;
-                            const int v0 = __shfl_sync(0xffffffffu, p, src);
-                            const int v1 = __shfl_sync(0xffffffffu, p1, src);
-                            const int v2 = __shfl_sync(0xffffffffu, p2, src);
-                            const int t = 32 * jb[b] + lane - cqb[b];      // list index of the earlier posting
+                            const int j = static_cast<int>(c0 + b - cstart[u]);
+                            const int cq = ustart[u + 1] - ustart[u];
+                            const int x = (32 * j - cq) >> 5;              // floor, may be negative
+                            int pr[3] = {p, -1, -1};
+#pragma unroll
+                            for (int r = 1; r <= 2; ++r) {
+                                const int xb = x + r - 1;
+                                if (xb >= 0 && xb < j) {
+                                    const int d = j - xb;
+                                    if (d <= b + avail) {
+#pragma unroll
+                                        for (int e = 1; e <= b + 2; ++e)
+                                            if (d == e) pr[r] = hist[b + 2 - e];
+                                    } else {
+                                        pr[r] = block_positions_now(cv, static_cast<uint32_t>(ulo[u]) + xb, lane);
+                                    }
+                                }
+                            }
+                            const int src = (lane - cq) & 31;
+                            const int v0 = __shfl_sync(0xffffffffu, pr[0], src);
+                            const int v1 = __shfl_sync(0xffffffffu, pr[1], src);
+                            const int v2 = __shfl_sync(0xffffffffu, pr[2], src);
+                            const int t = 32 * j + lane - cq;              // list index of the earlier posting
                             if (t >= 0) {
                                 const int tb = t >> 5;
-                                p_prev = tb == jb[b] ? v0 : (tb == ta[b] ? v1 : v2);
+                                p_prev = tb == j ? v0 : (tb == x ? v1 : v2);
                             }
                         }
                         if (p < 0) continue;
                         int j_lo, j_hi;
                         posting_range<POW2>(a, p, p_prev, j_lo, j_hi);
                         if (weighted) {
-                            const double w = static_cast<double>(uaq[ub[b]]) *
-                                             (1.0 / (log(1.0 + static_cast<double>(ulen[ub[b]])) + 1.0));
-                            for (int j = j_lo; j <= j_hi; ++j) atomicAdd(&acc_d[j], w);
+                            const double w = static_cast<double>(uaq[u]) * (1.0 / (log(1.0 + static_cast<double>(ulen[u])) + 1.0));
+                            for (int jj = j_lo; jj <= j_hi; ++jj) atomicAdd(&acc_d[jj], w);
                         } else if (j_lo <= j_hi) {
                             atomicAdd(&acc_i[j_lo], 1);
                             atomicAdd(&acc_i[j_hi + 1], -1);
                         }
                     }
+                    carry2 = hist[CBATCH]; carry1 = hist[CBATCH + 1];
                 }
             } else
             for (uint32_t c0 = c_begin; c0 < c_end; c0 += BATCH) {
