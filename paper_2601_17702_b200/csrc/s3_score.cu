@@ -508,12 +508,15 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
 // One block per query. Weights are taken in fixed point (2^-24) so that S, the density and therefore the
 // peaks are exact integer results whatever order the postings are visited in:
 //   1. S[t] += w_l(f) for every posting t of every query feature (64-bit integer atomics in global memory);
-//   2. density D[t] = sum of S over the K positions starting at t - K/2 (zero outside [0, L));
+//   2. density D[t] = sum of S over the K positions starting at t - K/2 (zero outside [0, L)): a tile of S plus its
+//      halo is prefix-summed in shared memory and D[t] is the difference of two prefix values;
 //   3. greedy non-maximum suppression over D with per-segment maxima in shared memory: a round reduces the
 //      segment maxima, takes the best position (ties: lowest), clears D within the radius and redoes only
 //      the touched segments.
-constexpr int SEG = 2048;            // positions per segment of the maxima table
-constexpr int MAX_SEGS = 2048;       // L <= SEG * MAX_SEGS
+constexpr int MIN_SEG_SHIFT = 8;      // a segment of the maxima table holds 2^seg_shift >= 256 positions,
+constexpr int MAX_SEGS = 2048;       // the smallest power of two that covers L with MAX_SEGS segments
+constexpr int CONV_TILE = 2048;      // positions smoothed per pass through shared memory
+constexpr int MAX_CONV_KERNEL = 1024;
 
 struct DensityArgs {
     const int32_t* q_ids;
@@ -525,7 +528,7 @@ struct DensityArgs {
     float* s_out;            // [Q][L] or null
     float* d_out;            // [Q][L] or null
     long long L;
-    int n_layers, d_sae, Q, nk, npad, conv_kernel, nms_radius, n_centers;
+    int n_layers, d_sae, Q, nk, npad, conv_kernel, nms_radius, n_centers, seg_shift;
     int64_t stop_freq;
 };
 
@@ -565,9 +568,10 @@ density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant
     long long* uw = reinterpret_cast<long long*>(score_smem_raw + ((SL.total + 15u) & ~15u));     // [nk] fixed-point weights
     long long* seg_val = uw + a.nk;                                                               // [n_segs]
     long long* seg_pos = seg_val + MAX_SEGS;
+    long long* tile = seg_pos + MAX_SEGS;                                                         // [CONV_TILE + MAX_CONV_KERNEL]
     __shared__ uint32_t ws[SW + 1];
     __shared__ int n_unique_s;
-    __shared__ long long red_v[SW], red_p[SW], pick_s;
+    __shared__ long long red_v[SW], red_p[SW], pick_s, scan_tot[SW + 1];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = blockIdx.x;
@@ -615,24 +619,54 @@ density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant
         }
     }
 
-    // density: K taps starting at t - K/2
+    // density: K taps starting at t - K/2. Per tile of CONV_TILE positions: S[t0 - K/2 .. t0 + CONV_TILE + K - K/2) goes
+    // to shared memory, is replaced by its inclusive prefix sum P (each thread scans a run of consecutive entries, the
+    // runs' totals are scanned across the block), and D[t0 + i] = P[i + K - 1] - P[i - 1].
     const long long half = a.conv_kernel / 2;
-    for (long long t = tid; t < L; t += ST) {
+    const int n_tile = CONV_TILE + a.conv_kernel - 1;                     // entries staged per tile
+    const int run = (n_tile + ST - 1) / ST;
+    for (long long t0 = 0; t0 < L; t0 += CONV_TILE) {
+        for (int i = tid; i < n_tile; i += ST) {
+            const long long t = t0 - half + i;
+            tile[i] = (t >= 0 && t < L) ? S[t] : 0;
+        }
+        __syncthreads();
+        const int i_lo = tid * run, i_hi = i_lo + run < n_tile ? i_lo + run : n_tile;
         long long sum = 0;
-        const long long lo = t - half < 0 ? 0 : t - half;
-        const long long hi = t - half + a.conv_kernel > L ? L : t - half + a.conv_kernel;
-        for (long long u = lo; u < hi; ++u) sum += S[u];
-        D[t] = sum;
-        if (a.d_out) a.d_out[(size_t)q * L + t] = static_cast<float>(static_cast<double>(sum) * (1.0 / 16777216.0));
-        if (a.s_out) a.s_out[(size_t)q * L + t] = static_cast<float>(static_cast<double>(S[t]) * (1.0 / 16777216.0));
+        for (int i = i_lo; i < i_hi; ++i) { sum += tile[i]; tile[i] = sum; }
+        long long inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        if (lane == 31) scan_tot[warp] = inc;
+        __syncthreads();
+        if (tid == 0) {
+            long long acc = 0;
+            for (int w = 0; w < SW; ++w) { const long long v = scan_tot[w]; scan_tot[w] = acc; acc += v; }
+        }
+        __syncthreads();
+        const long long base = scan_tot[warp] + inc - sum;
+        for (int i = i_lo; i < i_hi; ++i) tile[i] += base;
+        __syncthreads();
+        for (int i = tid; i < CONV_TILE; i += ST) {
+            const long long t = t0 + i;
+            if (t >= L) break;
+            const long long d = tile[i + a.conv_kernel - 1] - (i > 0 ? tile[i - 1] : 0);
+            D[t] = d;
+            if (a.d_out) a.d_out[(size_t)q * L + t] = static_cast<float>(static_cast<double>(d) * (1.0 / 16777216.0));
+            if (a.s_out) a.s_out[(size_t)q * L + t] = static_cast<float>(static_cast<double>(S[t]) * (1.0 / 16777216.0));
+        }
+        __syncthreads();
     }
-    __syncthreads();
 
     // segment maxima
-    const int n_segs = static_cast<int>((L + SEG - 1) / SEG);
+    const int seg = 1 << a.seg_shift;
+    const int n_segs = static_cast<int>((L + seg - 1) >> a.seg_shift);
     for (int sg = warp; sg < n_segs; sg += SW) {
         long long bv, bp;
-        const long long lo = (long long)sg * SEG, hi = lo + SEG < L ? lo + SEG : L;
+        const long long lo = (long long)sg << a.seg_shift, hi = lo + seg < L ? lo + seg : L;
         warp_segment_max(D, lo, hi, lane, bv, bp);
         if (lane == 0) { seg_val[sg] = bv; seg_pos[sg] = bp; }
     }
@@ -663,10 +697,10 @@ density_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant
         const long long k_hi = c + a.nms_radius >= L ? L - 1 : c + a.nms_radius;
         for (long long t = k_lo + tid; t <= k_hi; t += ST) D[t] = 0;
         __syncthreads();
-        const int sg_lo = static_cast<int>(k_lo / SEG), sg_hi = static_cast<int>(k_hi / SEG);
+        const int sg_lo = static_cast<int>(k_lo >> a.seg_shift), sg_hi = static_cast<int>(k_hi >> a.seg_shift);
         for (int sg = sg_lo + warp; sg <= sg_hi; sg += SW) {
             long long sv, sp;
-            const long long lo = (long long)sg * SEG, hi = lo + SEG < L ? lo + SEG : L;
+            const long long lo = (long long)sg << a.seg_shift, hi = lo + seg < L ? lo + seg : L;
             warp_segment_max(D, lo, hi, lane, sv, sp);
             if (lane == 0) { seg_val[sg] = sv; seg_pos[sg] = sp; }
         }
@@ -770,8 +804,9 @@ s3_status launch_density(const s3_csr_view* h_layers, int n_layers, int d_sae, i
         S3_CUDA_TRY(cudaFuncSetAttribute(density_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
         if (dev < 64) max_smem_dev[dev] = max_smem;
     }
-    S3_REQUIRE(L <= static_cast<int64_t>(SEG) * MAX_SEGS, S3_ERR_UNSUPPORTED, "L = %lld exceeds %lld positions", (long long)L,
-               (long long)SEG * MAX_SEGS);
+    int seg_shift = MIN_SEG_SHIFT;
+    while (((L + (1ll << seg_shift) - 1) >> seg_shift) > MAX_SEGS) ++seg_shift;
+    S3_REQUIRE(conv_kernel <= MAX_CONV_KERNEL, S3_ERR_UNSUPPORTED, "conv_kernel = %d exceeds %d", conv_kernel, MAX_CONV_KERNEL);
     ScoreLayers layers;
     for (int l = 0; l < n_layers; ++l) layers.v[l] = h_layers[l];
     DensityArgs a;
@@ -782,8 +817,9 @@ s3_status launch_density(const s3_csr_view* h_layers, int n_layers, int d_sae, i
     a.L = L; a.n_layers = n_layers; a.d_sae = d_sae; a.Q = Q; a.nk = nq * k;
     int npad = 32;
     while (npad < a.nk) npad <<= 1;
-    a.npad = npad; a.conv_kernel = conv_kernel; a.nms_radius = nms_radius; a.n_centers = n_centers; a.stop_freq = stop_freq;
-    const size_t smem = ((score_smem(a.nk, npad, 0, true).total + 15u) & ~15u) + static_cast<size_t>(a.nk) * 8 + 2 * MAX_SEGS * 8;
+    a.npad = npad; a.conv_kernel = conv_kernel; a.nms_radius = nms_radius; a.n_centers = n_centers; a.stop_freq = stop_freq; a.seg_shift = seg_shift;
+    const size_t smem = ((score_smem(a.nk, npad, 0, true).total + 15u) & ~15u) + static_cast<size_t>(a.nk) * 8 + 2 * MAX_SEGS * 8 +
+                        static_cast<size_t>(CONV_TILE + MAX_CONV_KERNEL) * 8;
     S3_REQUIRE(smem + 2048 <= static_cast<size_t>(max_smem), S3_ERR_UNSUPPORTED, "nq*k = %d needs %zu bytes of shared memory", a.nk, smem);
     density_kernel<<<Q, ST, smem, stream>>>(layers, a);
     S3_CUDA_TRY(cudaGetLastError());
