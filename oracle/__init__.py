@@ -68,6 +68,22 @@ def encode_topk(x, W, b_enc, b_dec, k: int):
     return topk(preact(x, W, b_enc, b_dec), k)
 
 
+def decode(ids, vals, W_dec, b_dec, x=None):
+    """x_hat = z_hat W_dec + b_dec (Sec. 3.3, after Eq. 2), fp64 [T, d_in]; with x also the per-token squared
+    reconstruction error, fp64 [T]. ids int32 [T,k] (-1 = padding), vals fp32 [T,k], W_dec [d_sae, d_in]."""
+    ids, vals, W_dec, b_dec = _i32(ids), _f32(vals), _f32(W_dec), _f32(b_dec)
+    T, k = ids.shape
+    d_sae, d_in = W_dec.shape
+    assert vals.shape == ids.shape and b_dec.shape == (d_in,) and ids.max(initial=-1) < d_sae
+    x_hat = np.empty((T, d_in), dtype=np.float64)
+    xx = None if x is None else _f32(x)
+    err = None if x is None else np.empty(T, dtype=np.float64)
+    lib().s3o_decode(_p(ids, C.c_int32), _p(vals, C.c_float), C.c_int64(T), C.c_int(k), _p(W_dec, C.c_float),
+                     _p(b_dec, C.c_float), C.c_int(d_in), C.c_int(d_sae), _p(xx, C.c_float), _p(x_hat, C.c_double),
+                     _p(err, C.c_double))
+    return x_hat if x is None else (x_hat, err)
+
+
 def postings(ids, d_sae: int, pos_base: int = 0, vals=None):
     """Eq. 4 for one chunk: (row_ptr uint32 [d_sae+1], pos int32 [nnz], pval fp32 [nnz] or None)."""
     ids = _i32(ids)

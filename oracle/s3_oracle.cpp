@@ -309,6 +309,37 @@ void s3o_position_density(const int32_t* ctx_ids, int64_t L, int k, int d_sae, i
     }
 }
 
+// Sec. 3.3, the reconstruction stated after Eq. 2: x_hat = z_hat W_dec + b_dec, with z_hat the Top-k code given as
+// (id, value) pairs per token (id < 0 = padding). W_dec is [d_sae, d_in] row-major: row f is feature f's direction.
+// fp64; the k terms are added in the order given, b_dec last. sqerr[t] (nullable) = sum_i (x[t,i] - x_hat[t,i])^2,
+// the per-token reconstruction error whose batch mean is the quantity an SAE is trained to reduce.
+void s3o_decode(const int32_t* ids, const float* vals, int64_t T, int k, const float* W_dec, const float* b_dec,
+                int d_in, int d_sae, const float* x /*[T,d_in] or null*/, double* x_hat /*[T,d_in]*/, double* sqerr /*[T] or null*/)
+{
+    (void)d_sae;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        double* out = x_hat + t * (int64_t)d_in;
+        for (int i = 0; i < d_in; ++i) out[i] = 0.0;
+        for (int j = 0; j < k; ++j) {
+            const int32_t f = ids[t * k + j];
+            if (f < 0) continue;
+            const double z = (double)vals[t * k + j];
+            const float* row = W_dec + (int64_t)f * d_in;
+            for (int i = 0; i < d_in; ++i) out[i] += z * (double)row[i];
+        }
+        for (int i = 0; i < d_in; ++i) out[i] += (double)b_dec[i];
+        if (sqerr && x) {
+            double e = 0.0;
+            for (int i = 0; i < d_in; ++i) {
+                const double d = (double)x[t * (int64_t)d_in + i] - out[i];
+                e += d * d;
+            }
+            sqerr[t] = e;
+        }
+    }
+}
+
 int s3o_num_threads(void)
 {
     int n = 1;
