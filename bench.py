@@ -460,6 +460,21 @@ def run_case(args):
                        same_result=bool(torch.equal(ref_idx, top_idx) and torch.equal(ref_score, top_score)))
         out.update(L=L, d_sae=D, k=k, Q=r.Q, nq=r.nq, kq=r.kq, spans=ns, stride=stride, gathered_postings=gathered,
                    index_bytes=int(ps.numel()) * 4, bytes=gathered * 4 + r.Q * ns * 4 + r.Q * r.s * 8)
+    elif args.case == "decode":
+        # SAE decode alone on the key SAE's shape: x_hat = z_hat W_dec + b_dec and the squared reconstruction error.
+        # bytes = the k gathered dictionary rows per token (mostly L2 hits: the dictionary is 32 MB) + x read + x_hat written
+        shp = cfg.key
+        T, k = args.tokens or cfg.chunk, shp.k
+        g = torch.Generator(device=dev).manual_seed(1)
+        W_dec = (torch.randn((shp.d_sae, shp.d_in), device=dev, generator=g) / shp.d_in ** 0.5).to(torch.bfloat16)
+        b_dec = torch.zeros(shp.d_in, device=dev)
+        xs = [torch.randn((T, shp.d_in), device=dev, generator=g).to(torch.bfloat16) for _ in range(2)]
+        idss = [torch.cat([torch.rand((2048, shp.d_sae), device=dev, generator=g).topk(k, dim=1).indices.to(torch.int32)
+                           for _ in range(0, T, 2048)])[:T].contiguous() for _ in range(2)]
+        vals = torch.rand((T, k), device=dev, generator=g)
+        run = lambda i: S.s3_sae_decode(W_dec, b_dec, idss[i % 2], vals, xs[i % 2])
+        out.update(T=T, d_in=shp.d_in, d_sae=shp.d_sae, k=k, bytes=T * k * shp.d_in * 2 + T * shp.d_in * (2 + 4),
+                   hbm_bytes=shp.d_sae * shp.d_in * 2 + T * shp.d_in * (2 + 4))
     elif args.case == "density":
         # the paper's Phase 2 tail alone: per-position relevance (Eq. 6), box-smoothed density (48 taps), greedy NMS
         # with 40 centres, then the index-set union of Eq. 7 (256-token windows, 64 lexical hits, 64 lead / tail);
@@ -514,7 +529,7 @@ def run_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density")
+    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)

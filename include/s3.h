@@ -287,6 +287,24 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
                                          float* d_density /*[Q,L] nullable*/, void* d_ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * SAE decode                     (paper Sec. 3.3, the reconstruction stated after Eq. 2:
+ *                                 x_hat = z_hat W_dec + b_dec)
+ *
+ * z_hat is the Top-k code as returned by s3_sae_encode_topk: d_ids / d_vals [T, k], id < 0 (padding) or
+ * id >= d_sae contributing nothing. W_dec is [d_sae, d_in] row-major (row f = direction of feature f), bf16
+ * or fp32; b_dec fp32 [d_in]. Per token the k scaled rows are added in the order given with fp32 FMAs
+ * starting from 0, b_dec last.
+ *   d_xhat  (nullable) fp32 [T, ld_xhat]  : the reconstruction;
+ *   d_sqerr (nullable) fp32 [T]           : sum_i (x[t,i] - x_hat[t,i])^2 against d_x [T, ldx] (same dtype as
+ *                                           W_dec), the per-token reconstruction error (fp32, fixed order).
+ * At least one of the two is required. Limits: 1 <= k <= S3_MAX_K; d_in a multiple of 8 (bf16) or 4 (fp32);
+ * pitches multiples of 4 (x_hat) and of 8 / 4 (x). No workspace. T == 0 is a no-op.
+ * ---------------------------------------------------------------------------------------------- */
+s3_status s3_sae_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int d_sae, s3_dtype dtype,
+                        const int32_t* d_ids, const float* d_vals, int T, int k,
+                        float* d_xhat, int64_t ld_xhat, const void* d_x, int64_t ldx, float* d_sqerr, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * Compact inverted index        (paper Sec. 3.4, memory analysis: contiguous integer arrays with delta
  *                                encoding and optional stop-feature pruning; the appendix's hard frequency
  *                                threshold for stop features. The layout is this library's.)

@@ -31,6 +31,7 @@ EXPORTS = [
     "s3_fuse_workspace_bytes", "s3_fuse_index_sets",
     "s3_compact_bound", "s3_compact_workspace_bytes", "s3_compact_build", "s3_coactivation_score_topspans_compact",
     "s3_compact_save", "s3_compact_file_info", "s3_compact_load",
+    "s3_sae_decode",
 ]
 
 
@@ -138,6 +139,8 @@ def lib():
         L.s3_compact_file_info.argtypes = [C.c_char_p, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_uint64),
                                            C.POINTER(C.c_uint64), C.c_int]
         L.s3_compact_load.argtypes = [C.c_char_p, C.c_int, C.c_int, C.POINTER(CompactHostLayer)]
+        L.s3_sae_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                    C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -508,3 +511,25 @@ def s3_compact_load(path: str):
     arr = (CompactHostLayer * n_layers)(*[c.host_layer() for c in layers])
     _check(lib().s3_compact_load(path.encode(), n_layers, d_sae, arr))
     return layers, d_sae
+
+
+def s3_sae_decode(W_dec: torch.Tensor, b_dec: torch.Tensor, ids: torch.Tensor, vals: torch.Tensor, x: torch.Tensor | None = None,
+                  want_xhat: bool = True, stream=None):
+    """W_dec [d_sae, d_in] bf16 or fp32, b_dec fp32 [d_in], ids int32 / vals fp32 [T, k]. Returns (x_hat fp32 [T, d_in] or
+    None, sqerr fp32 [T] or None); sqerr is computed when x [T, d_in] (dtype of W_dec) is given."""
+    assert W_dec.is_contiguous() and b_dec.dtype == torch.float32 and ids.dtype == torch.int32 and vals.dtype == torch.float32
+    assert ids.is_contiguous() and vals.is_contiguous() and ids.shape == vals.shape
+    d_sae, d_in = W_dec.shape
+    T, k = ids.shape
+    dtype = {torch.bfloat16: S3_BF16, torch.float32: S3_F32}[W_dec.dtype]
+    dev = W_dec.device
+    x_hat = torch.empty((T, d_in), dtype=torch.float32, device=dev) if want_xhat else None
+    sqerr = None
+    ldx = 0
+    if x is not None:
+        assert x.dtype == W_dec.dtype and x.shape == (T, d_in) and x.stride(1) == 1
+        sqerr = torch.empty((T,), dtype=torch.float32, device=dev)
+        ldx = x.stride(0)
+    _check(lib().s3_sae_decode(_ptr(W_dec), _ptr(b_dec), d_in, d_sae, dtype, _ptr(ids), _ptr(vals), T, k, _ptr(x_hat), d_in,
+                               _ptr(x), ldx, _ptr(sqerr), _stream(stream)))
+    return x_hat, sqerr

@@ -419,6 +419,28 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
                           static_cast<cudaStream_t>(stream));
 }
 
+// ---------------------------------------------------------------------------------------------- SAE decode
+s3_status s3_sae_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int d_sae, s3_dtype dtype, const int32_t* d_ids,
+                        const float* d_vals, int T, int k, float* d_xhat, int64_t ld_xhat, const void* d_x, int64_t ldx,
+                        float* d_sqerr, void* stream)
+{
+    S3_REQUIRE(dtype == S3_BF16 || dtype == S3_F32, S3_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
+    const int vec = dtype == S3_BF16 ? 8 : 4;
+    S3_REQUIRE(d_in >= 1 && d_sae >= 1 && d_in % vec == 0, S3_ERR_INVALID_ARG, "d_in = %d must be a positive multiple of %d", d_in, vec);
+    S3_REQUIRE(k >= 1 && k <= S3_MAX_K, S3_ERR_UNSUPPORTED, "k = %d out of [1, %d]", k, S3_MAX_K);
+    S3_REQUIRE(T >= 0, S3_ERR_INVALID_ARG, "T is negative");
+    if (T == 0) return S3_OK;
+    S3_REQUIRE(d_W_dec && d_b_dec && d_ids && d_vals, S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE(d_xhat || d_sqerr, S3_ERR_INVALID_ARG, "neither x_hat nor sqerr is wanted");
+    S3_REQUIRE(aligned16(d_W_dec) && aligned16(d_b_dec), S3_ERR_INVALID_ARG, "W_dec and b_dec must be 16-byte aligned");
+    if (d_xhat) S3_REQUIRE(aligned16(d_xhat) && ld_xhat >= d_in && ld_xhat % 4 == 0, S3_ERR_INVALID_ARG,
+                           "x_hat must be 16-byte aligned with a row pitch that is a multiple of 4 and >= d_in");
+    if (d_sqerr) S3_REQUIRE(d_x && aligned16(d_x) && ldx >= d_in && ldx % vec == 0, S3_ERR_INVALID_ARG,
+                            "sqerr needs x, 16-byte aligned with a row pitch that is a multiple of %d and >= d_in", vec);
+    return launch_decode(d_W_dec, d_b_dec, d_in, d_sae, dtype, d_ids, d_vals, T, k, d_xhat, ld_xhat, d_x, ldx, d_sqerr,
+                         static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------------------- index-set fusion
 size_t s3_fuse_workspace_bytes(int Q, int64_t L)
 {

@@ -49,6 +49,9 @@ s3_status launch_compact_build(const uint64_t* d_row_ptr, const int32_t* d_pos, 
                                uint64_t* d_out_row_ptr, uint32_t* d_blk_ptr, int32_t* d_blk_first, uint64_t* d_blk_desc,
                                uint64_t cap_blocks, uint32_t* d_payload, uint64_t cap_words, uint64_t* d_sizes,
                                uint32_t* d_status, void* d_scratch, cudaStream_t stream);
+s3_status launch_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int d_sae, s3_dtype dtype, const int32_t* d_ids,
+                        const float* d_vals, int T, int k, float* d_xhat, int64_t ld_xhat, const void* d_x, int64_t ldx,
+                        float* d_sqerr, cudaStream_t stream);
 size_t fuse_workspace_bytes(int Q, int64_t L);
 s3_status launch_fuse_sets(const int32_t* d_centers, int Q, int n_centers, int span_width, const int32_t* d_lexical, int n_lex,
                            int lead, int tail, int64_t L, int32_t* d_out_idx, int cap, int32_t* d_out_count, void* d_scratch,
