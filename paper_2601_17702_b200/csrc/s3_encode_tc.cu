@@ -524,11 +524,24 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (ok) {
                 if (__any_sync(0xffffffffu, cnt > 0)) fold_pending(my_pend, my_hist, glist, r, cnt, p.k, p.cap);
                 if (live) {
-                    p.counts[static_cast<size_t>(t) * p.n_slices + slice] = r.gcnt;
-                    // Publish the bound: at least k values of this slice exceed it. An exact k-th value
+                    // The bound to publish: at least k values of this slice exceed it. An exact k-th value
                     // only bounds from below after stepping to the next float down.
                     uint32_t out = __float_as_uint(r.tau);
                     if (r.istar == 0 && r.floor_exact && out > 0u) out -= 1u;
+                    // The list was filled under bounds that rose along the slice (about k (1 + ln(columns / k))
+                    // entries); only what beats the final bound can still matter, so the list is compacted once
+                    // here and the merge reads a fraction of it.
+                    const float cut = __uint_as_float(out);
+                    uint32_t w = 0;
+                    for (uint32_t i0 = 0; i0 < r.gcnt; i0 += 16) {
+                        uint64_t key[16];                        // read first: the writes land at or before i0
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) key[q] = i0 + q < r.gcnt ? glist[i0 + q] : 0ull;
+#pragma unroll
+                        for (int q = 0; q < 16; ++q)
+                            if (__uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > cut) glist[w++] = key[q];
+                    }
+                    p.counts[static_cast<size_t>(t) * p.n_slices + slice] = w;
                     if (out > hint_in) atomicMax(p.hint + t, out);
                 }
             }

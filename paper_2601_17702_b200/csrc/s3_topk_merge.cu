@@ -56,6 +56,7 @@ candidate_merge_kernel(const uint64_t* __restrict__ cand, const uint32_t* __rest
 {
     __shared__ uint64_t cand_buf[kMergeWarps][kCandBuf];
     __shared__ uint32_t cand_hist[kMergeWarps][64];
+    __shared__ uint32_t cand_start[kMergeWarps][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * kMergeWarps + warp;
     if (t >= T) return;
@@ -63,29 +64,47 @@ candidate_merge_kernel(const uint64_t* __restrict__ cand, const uint32_t* __rest
     const float tau = __uint_as_float(hint[t]);
     uint32_t n = 0;            // survivors so far (warp-uniform)
     bool overflow = false;
-    // list lengths of up to 32 slices at once; longer rows of slices in rounds
+    // Up to 32 slices at a time (more in rounds): the lists' lengths are prefix-summed over the lanes, and the
+    // entries of all those lists form one flat range that the warp walks 128 at a time, so the loads of different
+    // slices are in flight together instead of one list after the other.
+    uint32_t* start = cand_start[warp];
     for (int s0 = 0; s0 < n_slices && !overflow; s0 += 32) {
-        const uint32_t my_cnt = (s0 + lane < n_slices) ? counts[(size_t)t * n_slices + s0 + lane] : 0u;
         const int ns = n_slices - s0 < 32 ? n_slices - s0 : 32;
-        for (int s = 0; s < ns && !overflow; ++s) {
-            const uint32_t cnt = __shfl_sync(0xffffffffu, my_cnt, s);
-            const uint64_t* list = cand + ((size_t)t * n_slices + s0 + s) * cap;
-            // 128 entries per step: four independent loads per lane before any of them is used
-            for (uint32_t i0 = 0; i0 < cnt && !overflow; i0 += 128) {
-                uint64_t key[4];
+        const uint32_t my_cnt = lane < ns ? counts[(size_t)t * n_slices + s0 + lane] : 0u;
+        uint32_t inc = my_cnt;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t i = i0 + q * 32 + lane;
-                    key[q] = i < cnt ? list[i] : 0ull;
-                }
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
+        __syncwarp();
+        start[lane] = inc - my_cnt;                            // first flat index of slice s0 + lane
+        __syncwarp();
+        const uint64_t* lists = cand + ((size_t)t * n_slices + s0) * cap;
+        for (uint32_t i0 = 0; i0 < total && !overflow; i0 += 128) {
+            uint64_t key[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const bool keep = __uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > tau;   // key 0: value 0, never kept
-                    const uint32_t m = __ballot_sync(0xffffffffu, keep);
-                    if (n + __popc(m) > kCandBuf) { overflow = true; break; }
-                    if (keep) buf[n + __popc(m & ((1u << lane) - 1u))] = key[q];
-                    n += __popc(m);
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t i = i0 + q * 32 + lane;
+                key[q] = 0ull;
+                if (i < total) {
+                    int lo = 0, hi = 32;                       // last slice whose start is <= i (empty lists share a start)
+#pragma unroll
+                    for (int step = 0; step < 5; ++step) {
+                        const int mid = (lo + hi) >> 1;
+                        if (start[mid] <= i) lo = mid; else hi = mid;
+                    }
+                    key[q] = lists[(size_t)lo * cap + (i - start[lo])];
                 }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const bool keep = __uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > tau;   // key 0: value 0, never kept
+                const uint32_t m = __ballot_sync(0xffffffffu, keep);
+                if (n + __popc(m) > kCandBuf) { overflow = true; break; }
+                if (keep) buf[n + __popc(m & ((1u << lane) - 1u))] = key[q];
+                n += __popc(m);
             }
         }
     }
