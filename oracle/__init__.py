@@ -275,3 +275,28 @@ def prune_stop_features(row_ptr, pos, stop_freq: int):
         keep.append(pos[lo:hi])
         out_rp.append(out_rp[-1] + hi - lo)
     return np.array(out_rp, dtype=np.uint64), (np.concatenate(keep) if keep else pos[:0]).astype(np.int32)
+
+
+# ---------------------------------------------------------------------------------------------- head aggregation
+def head_aggregate(ids, vals, k_out: int):
+    """Sec. 3.3 / 3.4: the SAE reads one head's projection (x in R^d_head) and the index keeps "the Top-k sparsity per
+    token after head aggregation"; the aggregation rule is not given. Reading: all heads share one feature-ID space;
+    a token's activation of feature f is the sum over the heads whose Top-k holds f (fp32, heads in ascending order,
+    which is the precision the selection is made in), and the token keeps the k_out largest sums > 0, ordered by
+    (sum descending, id ascending), padded with id -1 / value 0.
+    ids int32 [T, H, k] (-1 = padding), vals fp32 [T, H, k]. Returns (ids int32 [T, k_out], vals fp32 [T, k_out])."""
+    ids, vals = _i32(ids), _f32(vals)
+    T, H, k = ids.shape
+    out_i = np.full((T, k_out), -1, dtype=np.int32)
+    out_v = np.zeros((T, k_out), dtype=np.float32)
+    for t in range(T):
+        acc = {}
+        for h in range(H):
+            for j in range(k):
+                f = int(ids[t, h, j])
+                if f >= 0:
+                    acc[f] = np.float32(acc.get(f, np.float32(0.0)) + vals[t, h, j])
+        best = sorted(((f, v) for f, v in acc.items() if v > 0), key=lambda fv: (-float(fv[1]), fv[0]))[:k_out]
+        for r, (f, v) in enumerate(best):
+            out_i[t, r], out_v[t, r] = f, v
+    return out_i, out_v
