@@ -460,6 +460,24 @@ def run_case(args):
                        same_result=bool(torch.equal(ref_idx, top_idx) and torch.equal(ref_score, top_score)))
         out.update(L=L, d_sae=D, k=k, Q=r.Q, nq=r.nq, kq=r.kq, spans=ns, stride=stride, gathered_postings=gathered,
                    index_bytes=int(ps.numel()) * 4, bytes=gathered * 4 + r.Q * ns * 4 + r.Q * r.s * 8)
+    elif args.case == "heads":
+        # per-head SAE as in Sec. 3.3 (x in R^d_head, one feature-ID space): the key SAE's dictionary width and k with
+        # d_head = 128 inputs, 8 KV heads per token, then head aggregation back to k features per token
+        H, d_head, D, k = 8, 128, cfg.key.d_sae, cfg.key.k
+        T = args.tokens or cfg.chunk
+        g = torch.Generator(device=dev).manual_seed(1)
+        W = (torch.randn((d_head, D), device=dev, generator=g) / d_head ** 0.5).to(torch.bfloat16)
+        sae = S.Sae(W, torch.zeros(D, device=dev), torch.zeros(d_head, device=dev))
+        xs = [torch.randn((T * H, d_head), device=dev, generator=g).to(torch.bfloat16) for _ in range(2)]
+        ids = torch.empty((T * H, k), dtype=torch.int32, device=dev)
+        vals = torch.empty((T * H, k), dtype=torch.float32, device=dev)
+        ws = S.new_workspace(sae.encode_workspace_bytes(T * H, k), dev)
+
+        def run(i):
+            S.s3_sae_encode_topk(sae, xs[i % 2], k, ids, vals, ws)
+            if not args.no_union:
+                S.s3_head_aggregate_topk(ids.view(T, H, k), vals.view(T, H, k), D, k)
+        out.update(T=T, H=H, d_head=d_head, d_sae=D, k=k, flop=2.0 * T * H * d_head * D)
     elif args.case == "decode":
         # SAE decode alone on the key SAE's shape: x_hat = z_hat W_dec + b_dec and the squared reconstruction error.
         # bytes = the k gathered dictionary rows per token (mostly L2 hits: the dictionary is 32 MB) + x read + x_hat written
@@ -529,13 +547,13 @@ def run_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode")
+    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)
     ap.add_argument("--items", type=int, default=8)
     ap.add_argument("--compact", action="store_true", help="score case: read the block-delta compact index")
-    ap.add_argument("--no-union", action="store_true", help="density case: leave out the index-set union")
+    ap.add_argument("--no-union", action="store_true", help="density case: leave out the index-set union; heads case: leave out the aggregation")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=96)
     ap.add_argument("--warmup", type=int, default=3)

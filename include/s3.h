@@ -287,6 +287,21 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
                                          float* d_density /*[Q,L] nullable*/, void* d_ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * Head aggregation + Top-k       (paper Sec. 3.3: the SAE reads one head's projection, x in R^d_head, with one
+ *                                 feature-ID space for all of them; Sec. 3.4: k is "the Top-k sparsity per token
+ *                                 after head aggregation". The rule itself is not given; this is the reading.)
+ *
+ * d_ids / d_vals [T, H, k] hold, per token, the Top-k codes of its H heads (e.g. s3_sae_encode_topk on the
+ * [T*H, d_head] view of the projections). Per token: a(f) = sum of f's activations over the heads whose code
+ * holds it (fp32, heads in ascending order; id < 0 or >= d_sae skipped); output the k_out features with the
+ * largest a(f) > 0 by (a descending, id ascending), padded with id -1 / value 0. The result has the layout
+ * of an encode result and feeds s3_postings_build.
+ * Limits: H*k <= 4096; k_out <= 4096; d_sae <= 2^20. No workspace. T == 0 is a no-op.
+ * ---------------------------------------------------------------------------------------------- */
+s3_status s3_head_aggregate_topk(const int32_t* d_ids, const float* d_vals, int T, int H, int k, int d_sae, int k_out,
+                                 int32_t* d_out_ids /*[T,k_out]*/, float* d_out_vals /*[T,k_out]*/, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * SAE decode                     (paper Sec. 3.3, the reconstruction stated after Eq. 2:
  *                                 x_hat = z_hat W_dec + b_dec)
  *

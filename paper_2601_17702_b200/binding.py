@@ -31,7 +31,7 @@ EXPORTS = [
     "s3_fuse_workspace_bytes", "s3_fuse_index_sets",
     "s3_compact_bound", "s3_compact_workspace_bytes", "s3_compact_build", "s3_coactivation_score_topspans_compact",
     "s3_compact_save", "s3_compact_file_info", "s3_compact_load",
-    "s3_sae_decode",
+    "s3_sae_decode", "s3_head_aggregate_topk",
 ]
 
 
@@ -141,6 +141,8 @@ def lib():
         L.s3_compact_load.argtypes = [C.c_char_p, C.c_int, C.c_int, C.POINTER(CompactHostLayer)]
         L.s3_sae_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                     C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+        L.s3_head_aggregate_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                             C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -533,3 +535,15 @@ def s3_sae_decode(W_dec: torch.Tensor, b_dec: torch.Tensor, ids: torch.Tensor, v
     _check(lib().s3_sae_decode(_ptr(W_dec), _ptr(b_dec), d_in, d_sae, dtype, _ptr(ids), _ptr(vals), T, k, _ptr(x_hat), d_in,
                                _ptr(x), ldx, _ptr(sqerr), _stream(stream)))
     return x_hat, sqerr
+
+
+def s3_head_aggregate_topk(ids: torch.Tensor, vals: torch.Tensor, d_sae: int, k_out: int, stream=None):
+    """ids int32 / vals fp32 [T, H, k]: the heads' Top-k codes of every token. Returns (ids int32 [T, k_out],
+    vals fp32 [T, k_out]): the features with the largest activation summed over the heads."""
+    assert ids.dtype == torch.int32 and vals.dtype == torch.float32 and ids.shape == vals.shape and ids.dim() == 3
+    assert ids.is_contiguous() and vals.is_contiguous()
+    T, H, k = ids.shape
+    out_i = torch.empty((T, k_out), dtype=torch.int32, device=ids.device)
+    out_v = torch.empty((T, k_out), dtype=torch.float32, device=ids.device)
+    _check(lib().s3_head_aggregate_topk(_ptr(ids), _ptr(vals), T, H, k, d_sae, k_out, _ptr(out_i), _ptr(out_v), _stream(stream)))
+    return out_i, out_v

@@ -419,6 +419,20 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
                           static_cast<cudaStream_t>(stream));
 }
 
+// ---------------------------------------------------------------------------------------------- head aggregation
+s3_status s3_head_aggregate_topk(const int32_t* d_ids, const float* d_vals, int T, int H, int k, int d_sae, int k_out,
+                                 int32_t* d_out_ids, float* d_out_vals, void* stream)
+{
+    S3_REQUIRE(T >= 0 && H >= 1 && k >= 1 && k_out >= 1, S3_ERR_INVALID_ARG, "T = %d, H = %d, k = %d, k_out = %d out of range", T, H, k,
+               k_out);
+    S3_REQUIRE((int64_t)H * k <= 4096, S3_ERR_UNSUPPORTED, "H*k = %lld exceeds 4096", (long long)H * k);
+    S3_REQUIRE(k_out <= 4096, S3_ERR_UNSUPPORTED, "k_out = %d exceeds 4096", k_out);
+    S3_REQUIRE(d_sae >= 1 && d_sae <= (1 << 20), S3_ERR_INVALID_ARG, "d_sae = %d out of range", d_sae);
+    if (T == 0) return S3_OK;
+    S3_REQUIRE(d_ids && d_vals && d_out_ids && d_out_vals, S3_ERR_INVALID_ARG, "null device pointer");
+    return launch_head_aggregate(d_ids, d_vals, T, H, k, d_sae, k_out, d_out_ids, d_out_vals, static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------------------- SAE decode
 s3_status s3_sae_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int d_sae, s3_dtype dtype, const int32_t* d_ids,
                         const float* d_vals, int T, int k, float* d_xhat, int64_t ld_xhat, const void* d_x, int64_t ldx,

@@ -112,9 +112,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
     return r;
 }
+// Arrival on a barrier of the first CTA (cluster address). The default CTA-scope release is enough: what the waiting
+// MMA warp must not overtake are this thread's tensor-memory loads, which tcgen05.wait::ld and the tcgen05 fences
+// order; a cluster-scope release would also make every thread wait here for its outstanding global stores.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
 // Tile load of one CTA of the pair into its own shared memory; the bytes are counted on the mbarrier at

@@ -52,6 +52,8 @@ s3_status launch_compact_build(const uint64_t* d_row_ptr, const int32_t* d_pos, 
 s3_status launch_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int d_sae, s3_dtype dtype, const int32_t* d_ids,
                         const float* d_vals, int T, int k, float* d_xhat, int64_t ld_xhat, const void* d_x, int64_t ldx,
                         float* d_sqerr, cudaStream_t stream);
+s3_status launch_head_aggregate(const int32_t* d_ids, const float* d_vals, int T, int H, int k, int d_sae, int k_out,
+                                int32_t* d_out_ids, float* d_out_vals, cudaStream_t stream);
 size_t fuse_workspace_bytes(int Q, int64_t L);
 s3_status launch_fuse_sets(const int32_t* d_centers, int Q, int n_centers, int span_width, const int32_t* d_lexical, int n_lex,
                            int lead, int tail, int64_t L, int32_t* d_out_idx, int cap, int32_t* d_out_count, void* d_scratch,
