@@ -168,20 +168,6 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "r"(taddr)
         : "memory");
 }
-// Named barrier 1 over the 128 epilogue threads with an AND-reduction of `pred`.
-__device__ __forceinline__ bool epi_all(bool pred)
-{
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 1, %2, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out)
-        : "r"(static_cast<uint32_t>(pred)), "n"(128)
-        : "memory");
-    return out != 0;
-}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major tile, 128-byte rows, 128-byte swizzle, 8-row groups 1024 B apart.
@@ -490,8 +476,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     dev_set_error(p.status, DEV_TIMEOUT_ACC_FULL);
                     *abort_flag = 1;
                 }
-                // Make the go/no-go decision uniform across the four epilogue warps.
-                if (!epi_all(arrived)) { ok = false; break; }
+                // The go/no-go decision is taken per warp: the four epilogue warps share nothing but the abort flag,
+                // which ends the others' waits soon after one of them gave up, so they need not move in step.
+                if (!__all_sync(0xffffffffu, arrived)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ab * BN + (static_cast<uint32_t>(quarter * 32) << 16);
                 const float4* bias4 = reinterpret_cast<const float4*>(p.b_eff + static_cast<size_t>(nt) * BN);
