@@ -497,13 +497,26 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 #pragma unroll
                     for (int h = 0; h < BATCH / STEP; ++h) {
 #pragma unroll
-                        for (int j = 0; j < STEP; ++j) {
-                            // Branch-free append: the slot after the list is always written and only
-                            // kept (by advancing cnt) when the value beats the bound.
-                            const float v = __uint_as_float(acc[h * STEP + j]) + bias[h * STEP + j];
-                            my_pend[cnt * EPI_THREADS] =
-                                (static_cast<uint64_t>(__float_as_uint(v)) << 32) | (ncol0 - static_cast<uint32_t>(h * STEP + j));
-                            cnt += (v > r.tau) ? 1 : 0;
+                        for (int j = 0; j < STEP; j += 4) {
+                            // Branch-free append, four values at a time: a value is written to the slot after the
+                            // entries kept so far and stays only if it beats the bound (the next one lands on the
+                            // same slot otherwise). The slots inside the group come from the group's own flags, so
+                            // the count is a dependent chain of one addition per four values.
+                            float v[4];
+                            int keep[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                v[q] = __uint_as_float(acc[h * STEP + j + q]) + bias[h * STEP + j + q];
+                                keep[q] = (v[q] > r.tau) ? 1 : 0;
+                            }
+                            const int o1 = keep[0], o2 = o1 + keep[1], o3 = o2 + keep[2];
+                            uint64_t* slot = my_pend + cnt * EPI_THREADS;
+                            const uint32_t nc = ncol0 - static_cast<uint32_t>(h * STEP + j);
+                            slot[0] = (static_cast<uint64_t>(__float_as_uint(v[0])) << 32) | nc;
+                            slot[o1 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[1])) << 32) | (nc - 1u);
+                            slot[o2 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[2])) << 32) | (nc - 2u);
+                            slot[o3 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[3])) << 32) | (nc - 3u);
+                            cnt += o3 + keep[3];
                         }
                         if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) fold_pending(my_pend, my_hist, glist, r, cnt, p.k, p.cap);
                     }
