@@ -463,7 +463,7 @@ def run_case(args):
     elif args.case == "heads":
         # per-head SAE as in Sec. 3.3 (x in R^d_head, one feature-ID space): the key SAE's dictionary width and k with
         # d_head = 128 inputs, 8 KV heads per token, then head aggregation back to k features per token
-        H, d_head, D, k = 8, 128, cfg.key.d_sae, cfg.key.k
+        H, d_head, D, k = 8, 128, cfg.key.d_sae, args.k or cfg.key.k
         T = args.tokens or cfg.chunk
         g = torch.Generator(device=dev).manual_seed(1)
         W = (torch.randn((d_head, D), device=dev, generator=g) / d_head ** 0.5).to(torch.bfloat16)
@@ -552,6 +552,7 @@ def main():
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)
     ap.add_argument("--items", type=int, default=8)
+    ap.add_argument("--k", type=int, default=0, help="heads case: Top-k per head and per token (default: the key SAE's)")
     ap.add_argument("--compact", action="store_true", help="score case: read the block-delta compact index")
     ap.add_argument("--no-union", action="store_true", help="density case: leave out the index-set union; heads case: leave out the aggregation")
     ap.add_argument("--gpus", type=int, default=1)

@@ -44,7 +44,7 @@ enum {
 
 typedef enum { S3_BF16 = 0, S3_F32 = 1 } s3_dtype;
 
-#define S3_MAX_K 64            /* largest Top-k per token                                           */
+#define S3_MAX_K 128           /* largest Top-k per token                                           */
 #define S3_MAX_POSTINGS_ITEMS 32
 #define S3_MAX_SCORE_LAYERS 16
 #define S3_WS_HEADER_BYTES 64

@@ -126,9 +126,12 @@ s3_status launch_encode_simt(const float* d_x, int64_t ldx, const float* d_W, co
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 64 && !attr_set[dev]) {
-        S3_CUDA_TRY(cudaFuncSetAttribute(encode_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        int max_smem = 0;
+        S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set[dev] = true;
     }
+    S3_REQUIRE(smem <= 227u * 1024u, S3_ERR_UNSUPPORTED, "k = %d needs %zu bytes of shared memory per block", k, smem);
     const int grid = n_slices * encode_simt_row_tiles(T);
     encode_simt_kernel<<<grid, THREADS, smem, stream>>>(d_x, ldx, d_W, d_b_enc, d_b_dec, T, d_in, d_sae, k, n_slices,
                                                        encode_simt_col_tiles(d_sae), d_part);

@@ -104,6 +104,6 @@ def test_decode_error_paths():
     b = torch.zeros(16, device=dev)
     with pytest.raises(S.S3Error):
         S.s3_sae_decode(W, b, ids, vals, None, want_xhat=False)         # nothing wanted
-    big = torch.zeros((2, 65), dtype=torch.int32, device=dev)
+    big = torch.zeros((2, 129), dtype=torch.int32, device=dev)
     with pytest.raises(S.S3Error):
-        S.s3_sae_decode(W, b, big, torch.zeros((2, 65), device=dev))
+        S.s3_sae_decode(W, b, big, torch.zeros((2, 129), device=dev))

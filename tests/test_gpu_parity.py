@@ -69,7 +69,8 @@ def test_cfg1_encode_fp32_full():
     assert (ids == oi).mean() > 0.999          # fp32 vs fp64: practically always the very same ids
 
 
-@pytest.mark.parametrize("T,d_in,d_sae,k", [(1, 8, 16, 1), (130, 24, 200, 5), (257, 100, 1000, 64), (64, 128, 129, 17)])
+@pytest.mark.parametrize("T,d_in,d_sae,k", [(1, 8, 16, 1), (130, 24, 200, 5), (257, 100, 1000, 64), (64, 128, 129, 17),
+                                            (100, 32, 600, 128)])
 def test_encode_fp32_shapes(T, d_in, d_sae, k):
     rng = np.random.default_rng(T + d_in)
     x = torch.from_numpy(rng.standard_normal((T, d_in)).astype(np.float32))
@@ -109,6 +110,9 @@ def test_encode_fp32_degenerate_rows():
     (640, 512, 8192, 16, 5),
     (257, 256, 2048, 64, 3),
     (96, 72, 264, 1, 0),           # smaller than every tile; d_in, d_sae only multiples of 8
+    (300, 128, 16384, 128, 0),     # the paper's per-head SAE: d_head 128, expansion 128, k = 128
+    (260, 256, 4096, 128, 3),      # k = 128, the largest supported, over several slices
+    (64, 64, 136, 128, 0),         # k close to d_sae
 ])
 def test_encode_bf16_shapes(T, d_in, d_sae, k, n_slices):
     x = G.activations(11, 0, 0, T, d_in, torch.bfloat16)
