@@ -511,7 +511,7 @@ def run_case(args):
         q_ids = torch.rand((r.Q * r.nq, D), device=dev, generator=g).topk(r.kq, dim=1).indices.to(torch.int32).view(1, r.Q, r.nq, r.kq)
         q_vals = torch.rand(q_ids.shape, dtype=torch.float32, device=dev, generator=g)
         lexical = torch.randint(0, L, (r.Q, 64), device=dev, generator=g, dtype=torch.int32)
-        dws = S.new_workspace(S.s3_density_workspace_bytes(r.Q, L), dev)
+        dws = S.new_workspace(S.s3_density_workspace_bytes(r.Q, L, 1, D, r.nq, r.kq), dev)
         fws = S.new_workspace(S.s3_fuse_workspace_bytes(r.Q, L), dev)
         cap = 40 * 256 + 64 + 128
         lens = (rp32[1:] - rp32[:-1])

@@ -271,15 +271,17 @@ s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_laye
  * h_layers as for s3_coactivation_score_topspans. Outputs: d_centers [Q, n_centers] int32, d_center_density
  * [Q, n_centers] fp32 (S' at the centre); d_S / d_density (nullable) [Q, L] fp32 copies of S and S'.
  * Limits: n_layers <= S3_MAX_SCORE_LAYERS; nq*k <= 4096; 1 <= conv_kernel <= 1024; nms_radius >= 0;
- *         1 <= n_centers <= 1024; L <= 4194304. Workspace: s3_density_workspace_bytes(Q, L)
- *         (two 64-bit words per query and position, plus the status block).
+ *         1 <= n_centers <= 1024; L <= 4194304.
+ * Workspace: s3_density_workspace_bytes(Q, L, n_layers, d_sae, nq, k): two 64-bit words per query and
+ *         position, the queries' unique features and weights (12 bytes per query entry and layer), one 32-bit
+ *         offset per layer, feature and tile of 8192 positions, plus the status block.
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
     int32_t conv_kernel, nms_radius, n_centers, reserved;
     int64_t stop_freq; /* 0 = off */
 } s3_density_params;
 
-size_t s3_density_workspace_bytes(int Q, int64_t L);
+size_t s3_density_workspace_bytes(int Q, int64_t L, int n_layers, int d_sae, int nq, int k);
 s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L,
                                          const int32_t* d_q_ids, const float* d_q_vals, int Q, int nq, int k,
                                          const s3_density_params* params, int32_t* d_centers /*[Q,n_centers]*/,

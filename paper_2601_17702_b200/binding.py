@@ -122,7 +122,7 @@ def lib():
                                                      C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(ScoreParams),
                                                      C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                                      C.c_void_p, C.c_size_t, C.c_void_p]
-        L.s3_density_workspace_bytes.argtypes = [C.c_int, C.c_int64]
+        L.s3_density_workspace_bytes.argtypes = [C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int]
         L.s3_position_density_topcenters.argtypes = [C.POINTER(CsrView), C.c_int, C.c_int, C.c_int64, C.c_void_p, C.c_void_p,
                                                      C.c_int, C.c_int, C.c_int, C.POINTER(DensityParams), C.c_void_p,
                                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -347,8 +347,8 @@ def s3_coactivation_score_topspans(layers, d_sae: int, L: int, q_ids: torch.Tens
     return top_idx, top_score
 
 
-def s3_density_workspace_bytes(Q: int, L: int) -> int:
-    return int(lib().s3_density_workspace_bytes(Q, L))
+def s3_density_workspace_bytes(Q: int, L: int, n_layers: int, d_sae: int, nq: int, k: int) -> int:
+    return int(lib().s3_density_workspace_bytes(Q, L, n_layers, d_sae, nq, k))
 
 
 def s3_position_density_topcenters(layers, d_sae: int, L: int, q_ids: torch.Tensor, q_vals: torch.Tensor, conv_kernel: int,

@@ -386,10 +386,10 @@ s3_status s3_compact_build(const uint64_t* d_row_ptr, const int32_t* d_pos, uint
 }
 
 // ---------------------------------------------------------------------------------------------- density
-size_t s3_density_workspace_bytes(int Q, int64_t L)
+size_t s3_density_workspace_bytes(int Q, int64_t L, int n_layers, int d_sae, int nq, int k)
 {
-    if (Q < 0 || L < 0) return 0;
-    return 256 + density_workspace_bytes(Q, L);
+    if (Q < 0 || L < 0 || n_layers < 1 || d_sae < 1 || nq < 1 || k < 1) return 0;
+    return 256 + density_workspace_bytes(Q, L, n_layers, d_sae, nq, k);
 }
 
 s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L,
@@ -410,8 +410,8 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
     S3_REQUIRE(p->conv_kernel <= 1024 && p->n_centers <= 1024, S3_ERR_UNSUPPORTED, "conv_kernel and n_centers may not exceed 1024");
     if (Q == 0) return S3_OK;
     S3_REQUIRE(d_q_ids && d_q_vals && d_centers && d_center_density, S3_ERR_INVALID_ARG, "null device pointer");
-    S3_REQUIRE(d_ws != nullptr && ws_bytes >= s3_density_workspace_bytes(Q, L), S3_ERR_CAPACITY,
-               "workspace holds %zu bytes, %zu needed", ws_bytes, s3_density_workspace_bytes(Q, L));
+    S3_REQUIRE(d_ws != nullptr && ws_bytes >= s3_density_workspace_bytes(Q, L, n_layers, d_sae, nq, k), S3_ERR_CAPACITY,
+               "workspace holds %zu bytes, %zu needed", ws_bytes, s3_density_workspace_bytes(Q, L, n_layers, d_sae, nq, k));
     for (int l = 0; l < n_layers; ++l)
         S3_REQUIRE(h_layers[l].d_row_ptr && h_layers[l].d_pos, S3_ERR_INVALID_ARG, "layer %d: null CSR pointer", l);
     return launch_density(h_layers, n_layers, d_sae, L, d_q_ids, d_q_vals, Q, nq, k, p->conv_kernel, p->nms_radius, p->n_centers,

@@ -58,7 +58,7 @@ size_t fuse_workspace_bytes(int Q, int64_t L);
 s3_status launch_fuse_sets(const int32_t* d_centers, int Q, int n_centers, int span_width, const int32_t* d_lexical, int n_lex,
                            int lead, int tail, int64_t L, int32_t* d_out_idx, int cap, int32_t* d_out_count, void* d_scratch,
                            cudaStream_t stream);
-size_t density_workspace_bytes(int Q, int64_t L);
+size_t density_workspace_bytes(int Q, int64_t L, int n_layers, int d_sae, int nq, int k);
 s3_status launch_density(const s3_csr_view* h_layers, int n_layers, int d_sae, int64_t L, const int32_t* d_q_ids,
                          const float* d_q_vals, int Q, int nq, int k, int conv_kernel, int nms_radius, int n_centers,
                          int64_t stop_freq, int32_t* d_centers, float* d_center_density, float* d_s_out, float* d_d_out,

@@ -41,7 +41,7 @@ def gpu_density(ctx, q, qv, D, K, R, N, stop_freq=0):
         pos = pos if len(pos) else np.zeros(1, np.int32)
         layers.append((torch.as_tensor(rp.astype(np.int64)).to(d), torch.as_tensor(pos).to(d)))
     Q = q.shape[1]
-    ws = S.new_workspace(S.s3_density_workspace_bytes(Q, L))
+    ws = S.new_workspace(S.s3_density_workspace_bytes(Q, L, n_layers, D, q.shape[2], q.shape[3]))
     S_out = torch.full((Q, max(L, 1)), -1.0, dtype=torch.float32, device=d)
     D_out = torch.full((Q, max(L, 1)), -1.0, dtype=torch.float32, device=d)
     c, dens = S.s3_position_density_topcenters(layers, D, L, torch.as_tensor(q).to(d).contiguous(),
@@ -109,5 +109,5 @@ def test_density_empty_query_and_error_paths():
         S.s3_position_density_topcenters([(rp, ps)], 32, 100, qi, qf, 8, 2, 3, S.new_workspace(64))
     assert e.value.code == S.binding.S3_ERR_CAPACITY
     with pytest.raises(S.S3Error) as e:
-        S.s3_position_density_topcenters([(rp, ps)], 32, 100, qi, qf, 0, 2, 3, S.new_workspace(1 << 16))
+        S.s3_position_density_topcenters([(rp, ps)], 32, 100, qi, qf, 0, 2, 3, S.new_workspace(1 << 20))
     assert e.value.code == S.binding.S3_ERR_INVALID_ARG
