@@ -524,6 +524,7 @@ constexpr int MAX_CONV_KERNEL = 1024;
 constexpr int POS_TILE = 8192;       // positions accumulated per block (64 KB of 64-bit sums)
 constexpr int FCHUNK = 1024;         // query features handled per pass of the accumulate kernel
 constexpr int AWIN = 4096;           // pieces whose owning feature is tabulated at a time there
+constexpr int APIECE = 16;           // postings per piece there: a tile holds a fraction of a list, so half a warp per piece
 
 struct DensityArgs {
     const int32_t* q_ids;
@@ -654,7 +655,7 @@ density_accumulate_kernel(const __grid_constant__ ScoreLayers layers, const __gr
                     ulo[i] = __ldg(row_ptr + f) + first;
                     ulen[i] = len;
                     uw[i] = w;
-                    n_pieces = (len + PIECE - 1) / PIECE;
+                    n_pieces = (len + APIECE - 1) / APIECE;
                 }
                 uint32_t total;
                 const uint32_t ex = block_exclusive_scan(n_pieces, ws, total) + carry;
@@ -675,16 +676,16 @@ density_accumulate_kernel(const __grid_constant__ ScoreLayers layers, const __gr
                 const uint32_t n_win = win1 - win0;
                 const uint32_t c_begin = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * warp / SW);
                 const uint32_t c_end = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * (warp + 1) / SW);
-                for (uint32_t c0 = c_begin; c0 < c_end; c0 += BATCH) {
+                for (uint32_t c0 = c_begin; c0 < c_end; c0 += 2 * BATCH) {
                     int p[BATCH], ub[BATCH];
 #pragma unroll
                     for (int b = 0; b < BATCH; ++b) {
-                        const uint32_t c = c0 + b;
+                        const uint32_t c = c0 + 2 * b + (lane >> 4);          // each half of the warp takes a piece
                         p[b] = -1; ub[b] = 0;
                         if (c < c_end) {
                             const int i = owner[c - win0];
                             ub[b] = i;
-                            const uint32_t j = (c - cstart[i]) * PIECE + lane;
+                            const uint32_t j = (c - cstart[i]) * APIECE + (lane & 15);
                             if (j < ulen[i]) p[b] = __ldg(pos + ulo[i] + j);
                         }
                     }
