@@ -120,6 +120,91 @@ def test_cfg4_retrieval_sampled_queries():
         assert ti[qi].tolist() == order.tolist()
 
 
+def _cfg4_inputs():
+    r = C.CFG4
+    L, k, D = r.scan.L, r.scan.key.k, r.scan.key.d_sae
+    rng = np.random.default_rng(11)
+    start = rng.integers(0, D, size=(L, 1))
+    start[rng.random((L, 1)) < 0.3] = 7                  # feature 7 is popular: a posting list of ~10K entries
+    ctx = ((start + np.arange(k)[None, :] * 131) % D).astype(np.int32)      # k distinct ids per token
+    qs = rng.integers(0, D, size=(r.Q * r.nq, 1))
+    qs[::r.nq] = 7                                       # every query has the popular feature in its first token
+    q = ((qs + np.arange(r.kq)[None, :] * 67) % D).astype(np.int32).reshape(1, r.Q, r.nq, r.kq)
+    qv = rng.random(q.shape).astype(np.float32)
+    return r, L, k, D, ctx, q, qv
+
+
+def test_cfg4_compact_index_scores_like_the_raw_one():
+    """The retrieval call of the benchmark on the compact form of its index: all 256 queries give the very spans and
+    scores of the raw CSR, sampled queries match the oracle, and with the popular feature pruned at build time the
+    sampled queries match the oracle on the context without it."""
+    r, L, k, D, ctx, q, qv = _cfg4_inputs()
+    d = _dev()
+    ns = C.n_spans(L, r.width, r.stride)
+    bm = G.gamma21(r.bm25_seed, r.Q, ns)
+    rp, pos, _ = O.postings(ctx, D, 0)
+    rp_t, pos_t = torch.as_tensor(rp.astype(np.int64)).to(d), torch.as_tensor(pos).to(d)
+    qi_t, qv_t = torch.as_tensor(q).to(d), torch.as_tensor(qv).to(d)
+    ws = S.new_workspace(64)
+    ti0, ts0 = S.s3_coactivation_score_topspans([(rp_t, pos_t)], D, L, qi_t, qv_t, r.width, r.stride, r.s, r.alpha, r.beta, ws, bm.to(d))
+    comp = S.s3_compact_build(rp_t, pos_t, D)
+    assert comp.nbytes() < 0.75 * (pos_t.numel() * 4 + rp_t.numel() * 8)
+    ti1, ts1 = S.s3_coactivation_score_topspans_compact([comp], D, L, qi_t, qv_t, r.width, r.stride, r.s, r.alpha, r.beta, ws, bm.to(d))
+    assert torch.equal(ti0, ti1) and torch.equal(ts0, ts1)
+    stop = 5000                                          # the appendix's hard threshold: drops feature 7's ~10K postings
+    pruned = S.s3_compact_build(rp_t, pos_t, D, stop)
+    assert int(pruned.row_ptr[-1]) < pos_t.numel()
+    alls = torch.zeros((r.Q, ns), dtype=torch.float32, device=d)
+    ti2, ts2 = S.s3_coactivation_score_topspans_compact([pruned], D, L, qi_t, qv_t, r.width, r.stride, r.s, r.alpha, r.beta, ws,
+                                                        bm.to(d), all_scores=alls)
+    assert S.s3_workspace_status(ws) == 0
+    sample = [0, 1, 64, 128, 255]
+    freq = np.bincount(ctx.ravel(), minlength=D)
+    ctx_p = ctx.copy()
+    ctx_p[np.isin(ctx, np.nonzero(freq > stop)[0])] = -1
+    co = O.score_spans(ctx_p[None], q[:, sample], qv[:, sample], D, r.width, r.stride, 0)
+    oi, os_, oall = O.fuse_select(co, bm.numpy()[sample], r.alpha, r.beta, r.s)
+    np.testing.assert_array_equal(alls.cpu().numpy()[sample], oall)
+    np.testing.assert_array_equal(ti2.cpu().numpy()[sample], oi)
+    np.testing.assert_array_equal(ts2.cpu().numpy()[sample], os_)
+
+
+def test_cfg4_position_density_sampled_queries():
+    """The paper's Phase 2 tail at the retrieval workload's size (256 queries, 32K positions, 48 taps, 40 centres):
+    relevance, density and centres of sampled queries against the oracle, exactly; every query's centres are valid
+    (distinct, at least the radius apart, densities descending)."""
+    r, L, k, D, ctx, q, qv = _cfg4_inputs()
+    d = _dev()
+    K, R, N = 48, 24, 40
+    rp, pos, _ = O.postings(ctx, D, 0)
+    layers = [(torch.as_tensor(rp.astype(np.int64)).to(d), torch.as_tensor(pos).to(d))]
+    ws = S.new_workspace(S.s3_density_workspace_bytes(r.Q, L, 1, D, r.nq, r.kq))
+    S_out = torch.empty((r.Q, L), dtype=torch.float32, device=d)
+    D_out = torch.empty((r.Q, L), dtype=torch.float32, device=d)
+    c, dens = S.s3_position_density_topcenters(layers, D, L, torch.as_tensor(q).to(d), torch.as_tensor(qv).to(d), K, R, N, ws, 5000,
+                                               S_out, D_out)
+    assert S.s3_workspace_status(ws) == 0
+    c, dens = c.cpu().numpy(), dens.cpu().numpy()
+    sample = [0, 1, 127, 128, 255]
+    oS, oD, oc, odens = O.position_density(ctx[None], q[:, sample], qv[:, sample], D, K, R, N, 5000)
+    np.testing.assert_array_equal(S_out.cpu().numpy()[sample], oS.astype(np.float32))
+    np.testing.assert_array_equal(D_out.cpu().numpy()[sample], oD.astype(np.float32))
+    np.testing.assert_array_equal(c[sample], oc)
+    np.testing.assert_array_equal(dens[sample], odens)
+    for qi in range(r.Q):
+        got = c[qi][c[qi] >= 0]
+        assert len(set(got.tolist())) == len(got)
+        if len(got) > 1:
+            assert np.abs(got[:, None] - got[None, :])[~np.eye(len(got), dtype=bool)].min() > R
+        assert (np.diff(dens[qi][: len(got)]) <= 0).all()
+    idx, cnt = S.s3_fuse_index_sets(torch.as_tensor(c[sample]).to(d), 256, None, 64, 64, L, N * 256 + 128,
+                                    S.new_workspace(S.s3_fuse_workspace_bytes(len(sample), L)))
+    want = O.fuse_index_sets(oc, 256, None, 64, 64, L)
+    for i, m in enumerate(want):
+        assert int(cnt[i]) == len(m)
+        np.testing.assert_array_equal(idx[i, : len(m)].cpu().numpy(), m)
+
+
 def test_scan_device_memory_is_flat_across_chunks():
     """Sec. 3.4 / memory-complexity proposition: device memory is bounded by the chunk, not by the context.
     After the first chunk, scanning more chunks allocates nothing on the device; the index grows on the host."""
