@@ -383,6 +383,11 @@ s3_status s3_coactivation_score_topspans_compact(const s3_compact_view* h_layers
                                                  const s3_score_params* params, const float* d_bm25, int64_t ld_bm25,
                                                  int32_t* d_top_idx, float* d_top_score, float* d_all_scores,
                                                  void* d_ws, size_t ws_bytes, void* stream);
+/* Writes the kept postings back as a plain position array (d_pos, cap_postings entries; the CSR's row_ptr is the
+ * view's own d_row_ptr): the inverse of s3_compact_build on the pruned index. A d_pos that is too small sets the
+ * workspace status (S3_ERR_CAPACITY from s3_workspace_status) and writes nothing. *h_view holds device pointers. */
+s3_status s3_compact_expand(const s3_compact_view* h_view, int d_sae, int32_t* d_pos, uint64_t cap_postings,
+                            void* d_ws, size_t ws_bytes, void* stream);
 s3_status s3_compact_save(const char* path, int n_layers, int d_sae, const s3_compact_host_layer* h_layers);
 s3_status s3_compact_file_info(const char* path, int* n_layers, int* d_sae, uint64_t* h_n_blocks, uint64_t* h_n_words,
                                int cap_layers);

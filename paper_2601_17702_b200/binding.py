@@ -31,7 +31,7 @@ EXPORTS = [
     "s3_fuse_workspace_bytes", "s3_fuse_index_sets",
     "s3_compact_bound", "s3_compact_workspace_bytes", "s3_compact_build", "s3_coactivation_score_topspans_compact",
     "s3_compact_save", "s3_compact_file_info", "s3_compact_load",
-    "s3_sae_decode", "s3_head_aggregate_topk",
+    "s3_sae_decode", "s3_head_aggregate_topk", "s3_compact_expand",
 ]
 
 
@@ -143,6 +143,7 @@ def lib():
                                     C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
         L.s3_head_aggregate_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                              C.c_void_p, C.c_void_p]
+        L.s3_compact_expand.argtypes = [C.POINTER(CompactView), C.c_int, C.c_void_p, C.c_uint64, C.c_void_p, C.c_size_t, C.c_void_p]
         _lib = L
     return _lib
 
@@ -547,3 +548,17 @@ def s3_head_aggregate_topk(ids: torch.Tensor, vals: torch.Tensor, d_sae: int, k_
     out_v = torch.empty((T, k_out), dtype=torch.float32, device=ids.device)
     _check(lib().s3_head_aggregate_topk(_ptr(ids), _ptr(vals), T, H, k, d_sae, k_out, _ptr(out_i), _ptr(out_v), _stream(stream)))
     return out_i, out_v
+
+
+def s3_compact_expand(layer: CompactLayer, d_sae: int, ws: torch.Tensor | None = None, stream=None):
+    """The compact layer's kept postings as a raw CSR on the device: (row_ptr int64 [d_sae+1], pos int32)."""
+    dev = layer.row_ptr.device
+    n = int(layer.row_ptr[-1])
+    pos = torch.empty(max(n, 1), dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = torch.zeros(64, dtype=torch.uint8, device=dev)
+    view = layer.view()
+    _check(lib().s3_compact_expand(C.byref(view), d_sae, _ptr(pos), n, _ptr(ws), ws.numel(), _stream(stream)))
+    code = C.c_uint32(0)
+    _check(lib().s3_workspace_status(_ptr(ws), _stream(stream), C.byref(code)))
+    return layer.row_ptr, pos[:n]

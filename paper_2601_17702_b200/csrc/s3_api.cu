@@ -419,6 +419,18 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
                           static_cast<cudaStream_t>(stream));
 }
 
+s3_status s3_compact_expand(const s3_compact_view* h_view, int d_sae, int32_t* d_pos, uint64_t cap_postings, void* d_ws,
+                            size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(h_view != nullptr, S3_ERR_INVALID_ARG, "h_view is null");
+    S3_REQUIRE(d_sae >= 1 && d_sae <= (1 << 20), S3_ERR_INVALID_ARG, "d_sae = %d out of range", d_sae);
+    S3_REQUIRE(h_view->d_row_ptr && h_view->d_blk_ptr && h_view->d_payload, S3_ERR_INVALID_ARG, "null pointer in the compact view");
+    S3_REQUIRE(d_pos != nullptr || cap_postings == 0, S3_ERR_INVALID_ARG, "d_pos is null");
+    S3_REQUIRE(d_ws != nullptr && ws_bytes >= S3_WS_HEADER_BYTES, S3_ERR_CAPACITY, "workspace missing or smaller than %d bytes",
+               S3_WS_HEADER_BYTES);
+    return launch_compact_expand(*h_view, d_sae, d_pos, cap_postings, static_cast<uint32_t*>(d_ws), static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------------------- head aggregation
 s3_status s3_head_aggregate_topk(const int32_t* d_ids, const float* d_vals, int T, int H, int k, int d_sae, int k_out,
                                  int32_t* d_out_ids, float* d_out_vals, void* stream)

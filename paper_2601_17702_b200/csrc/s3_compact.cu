@@ -186,6 +186,49 @@ __global__ void __launch_bounds__(CT) compact_pack_kernel(const __grid_constant_
     }
 }
 
+// The inverse of the build: every block's positions written back as a plain position array (one warp per block:
+// gaps unpacked, 32-lane prefix sum), so that a consumer of the raw CSR can be fed from the compact form.
+struct ExpandArgs {
+    s3_compact_view v;
+    int32_t* pos;
+    uint64_t cap_postings;
+    uint32_t* status;
+    int d_sae;
+};
+
+__global__ void __launch_bounds__(CT) compact_expand_kernel(const __grid_constant__ ExpandArgs a)
+{
+    const uint32_t n_blocks = a.v.d_blk_ptr[a.d_sae];
+    if (a.v.d_row_ptr[a.d_sae] > a.cap_postings) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) dev_set_error(a.status, DEV_COMPACT_CAPACITY);
+        return;
+    }
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp0 = (blockIdx.x * CT + threadIdx.x) >> 5, n_warps = gridDim.x * (CT / 32);
+    for (uint32_t b = warp0; b < n_blocks; b += n_warps) {
+        const int f = owner_of_block(a.v.d_blk_ptr, a.d_sae, b);
+        const uint64_t base = a.v.d_row_ptr[f], kept = a.v.d_row_ptr[f + 1] - base;
+        const uint64_t j = b - a.v.d_blk_ptr[f];
+        const uint64_t left = kept - 32 * j;
+        const int cnt = left < 32 ? static_cast<int>(left) : 32;
+        const uint64_t desc = a.v.d_blk_desc[b];
+        const uint32_t width = static_cast<uint32_t>(desc & 63u);
+        uint32_t val = 0;
+        if (lane >= 1 && lane < cnt && width) {
+            const uint32_t bit = (lane - 1) * width;
+            const uint32_t* w = a.v.d_payload + (desc >> 6) + (bit >> 5);
+            val = __funnelshift_r(w[0], w[1], bit & 31) & ((1u << width) - 1u);     // the closing word keeps w[1] in bounds
+        }
+        int d = lane == 0 ? a.v.d_blk_first[b] : (lane < cnt ? static_cast<int>(val) + 1 : 0);
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, d, o);
+            if (lane >= o) d += y;
+        }
+        if (lane < cnt) a.pos[base + 32 * j + lane] = d;
+    }
+}
+
 }  // namespace
 
 void compact_bound(uint64_t n_postings, int d_sae, uint64_t* max_blocks, uint64_t* max_words)
@@ -218,6 +261,16 @@ s3_status launch_compact_build(const uint64_t* d_row_ptr, const int32_t* d_pos, 
     compact_measure_kernel<<<grid, CT, 0, stream>>>(a);
     compact_scan_words_kernel<<<1, SCAN_T, 0, stream>>>(a);
     compact_pack_kernel<<<grid, CT, 0, stream>>>(a);
+    S3_CUDA_TRY(cudaGetLastError());
+    return S3_OK;
+}
+
+s3_status launch_compact_expand(const s3_compact_view& v, int d_sae, int32_t* d_pos, uint64_t cap_postings, uint32_t* d_status,
+                                cudaStream_t stream)
+{
+    ExpandArgs a;
+    a.v = v; a.pos = d_pos; a.cap_postings = cap_postings; a.status = d_status; a.d_sae = d_sae;
+    compact_expand_kernel<<<device_sm_count() * 8, CT, 0, stream>>>(a);
     S3_CUDA_TRY(cudaGetLastError());
     return S3_OK;
 }

@@ -54,6 +54,8 @@ s3_status launch_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int
                         float* d_sqerr, cudaStream_t stream);
 s3_status launch_head_aggregate(const int32_t* d_ids, const float* d_vals, int T, int H, int k, int d_sae, int k_out,
                                 int32_t* d_out_ids, float* d_out_vals, cudaStream_t stream);
+s3_status launch_compact_expand(const s3_compact_view& v, int d_sae, int32_t* d_pos, uint64_t cap_postings, uint32_t* d_status,
+                                cudaStream_t stream);
 size_t fuse_workspace_bytes(int Q, int64_t L);
 s3_status launch_fuse_sets(const int32_t* d_centers, int Q, int n_centers, int span_width, const int32_t* d_lexical, int n_lex,
                            int lead, int tail, int64_t L, int32_t* d_out_idx, int cap, int32_t* d_out_count, void* d_scratch,

@@ -79,6 +79,29 @@ def test_build_on_scan_sized_index():
     assert c.nbytes() < 0.6 * (pos.nbytes + rp.nbytes)        # gaps of about 8 bits plus headers: well under 4 B per posting
 
 
+def test_expand_is_the_inverse_of_build():
+    rng = np.random.default_rng(9)
+    lists = [np.sort(rng.choice(1 << 20, size=int(rng.choice([0, 1, 31, 32, 33, 100, 700])), replace=False)).tolist()
+             for _ in range(400)]
+    lists[3] = [0, 2**31 - 1]
+    rp, pos = _csr(lists)
+    for stop in (0, 90):
+        c = gpu_build(rp, pos, stop)
+        want_rp, want_pos = O.compact_decode(O.compact_encode(rp, pos, stop))          # the oracle's own decoder
+        got_rp, got_pos = S.s3_compact_expand(c, len(rp) - 1)
+        np.testing.assert_array_equal(got_rp.cpu().numpy().astype(np.uint64), want_rp)
+        np.testing.assert_array_equal(got_pos.cpu().numpy(), want_pos)
+        np.testing.assert_array_equal(want_pos, O.prune_stop_features(rp, pos, stop)[1])
+    d = _dev()
+    view = c.view()
+    ws = torch.zeros(64, dtype=torch.uint8, device=d)
+    small = torch.empty(4, dtype=torch.int32, device=d)
+    S.binding._check(S.binding.lib().s3_compact_expand(S.binding.C.byref(view), len(rp) - 1, small.data_ptr(), 4, ws.data_ptr(), 64,
+                                                       S.binding._stream()))
+    with pytest.raises(S.S3Error):
+        S.s3_workspace_status(ws)
+
+
 def test_empty_index_and_capacity_error():
     c = gpu_build(np.zeros(9, np.uint64), np.zeros(0, np.int32))
     assert c.blk_first.numel() == 0 and c.payload.tolist() == [0] and c.row_ptr.tolist() == [0] * 9
