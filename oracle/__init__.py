@@ -300,3 +300,48 @@ def head_aggregate(ids, vals, k_out: int):
         for r, (f, v) in enumerate(best):
             out_i[t, r], out_v[t, r] = f, v
     return out_i, out_v
+
+
+# ---------------------------------------------------------------------------------------------- SAE training step
+# The paper trains its Top-K SAEs with Adam (appendix table: learning rate 1e-3, batches of 4096 tokens) and gives no loss;
+# reading: the mean over the batch of the squared reconstruction error of Sec. 3.3's x_hat, differentiated through the
+# Top-k code with the active set held fixed (the selection is piecewise constant, so this is the gradient wherever it
+# exists). Adam as published (Kingma & Ba): m = b1 m + (1-b1) g, v = b2 v + (1-b2) g^2, p -= lr * m_hat / (sqrt(v_hat) + eps)
+# with m_hat = m / (1 - b1^step), v_hat = v / (1 - b2^step). Plain numpy, fp64.
+
+def sae_loss_and_grads(x, W_enc, b_enc, W_dec, b_dec, ids):
+    """x [T, d_in], W_enc [d_in, d_sae], b_enc [d_sae], W_dec [d_sae, d_in], b_dec [d_in], ids int32 [T, k] (the active
+    set, -1 = padding). z[t,j] = W_enc[:, f]·(x_t - b_dec) + b_enc[f] for f = ids[t,j] (the pre-activation of a selected
+    feature, which the ReLU passes), x_hat = z W_dec + b_dec, loss = mean_t ||x_hat_t - x_t||^2.
+    Returns (loss, gW_enc, gb_enc, gW_dec, gb_dec), all fp64."""
+    x = np.asarray(x, np.float64)
+    W_enc, b_enc = np.asarray(W_enc, np.float64), np.asarray(b_enc, np.float64)
+    W_dec, b_dec = np.asarray(W_dec, np.float64), np.asarray(b_dec, np.float64)
+    ids = np.asarray(ids)
+    T, d_in = x.shape
+    gW_enc, gb_enc = np.zeros_like(W_enc), np.zeros_like(b_enc)
+    gW_dec, gb_dec = np.zeros_like(W_dec), np.zeros_like(b_dec)
+    loss = 0.0
+    for t in range(T):
+        f = ids[t][ids[t] >= 0]
+        xc = x[t] - b_dec
+        z = xc @ W_enc[:, f] + b_enc[f]
+        r = z @ W_dec[f] + b_dec - x[t]
+        loss += float(r @ r) / T
+        g = 2.0 * r / T                                  # d loss / d x_hat_t
+        gz = W_dec[f] @ g                                # d loss / d z
+        np.add.at(gW_dec, f, np.outer(z, g))
+        np.add.at(gb_enc, f, gz)
+        np.add.at(gW_enc.T, f, np.outer(gz, xc))
+        gb_dec += g - W_enc[:, f] @ gz                   # directly, and through (x - b_dec) in the encoder
+    return loss, gW_enc, gb_enc, gW_dec, gb_dec
+
+
+def adam_update(p, m, v, g, lr, beta1, beta2, eps, step):
+    """One Adam update (step counted from 1). Returns (p, m, v), fp64."""
+    p, m, v, g = (np.asarray(a, np.float64) for a in (p, m, v, g))
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    m_hat = m / (1.0 - beta1 ** step)
+    v_hat = v / (1.0 - beta2 ** step)
+    return p - lr * m_hat / (np.sqrt(v_hat) + eps), m, v
