@@ -478,6 +478,30 @@ def run_case(args):
             if not args.no_union:
                 S.s3_head_aggregate_topk(ids.view(T, H, k), vals.view(T, H, k), D, k)
         out.update(T=T, H=H, d_head=d_head, d_sae=D, k=k, flop=2.0 * T * H * d_head * D)
+    elif args.case == "train":
+        # one fp32 training step of the paper's SAE shape (appendix: batches of 4096 tokens, expansion 128 over d_head = 128,
+        # k = 128, Adam at 1e-3): encode + Top-k, backward through the code, Adam on the four parameter tensors
+        T, d_in, D, k = args.tokens or 4096, 128, 16384, args.k or 128
+        g = torch.Generator(device=dev).manual_seed(1)
+        W_enc = torch.randn((d_in, D), device=dev, generator=g) / d_in ** 0.5
+        params = [W_enc, torch.zeros(D, device=dev), W_enc.t().contiguous(), torch.zeros(d_in, device=dev)]
+        moments = [(torch.zeros_like(p), torch.zeros_like(p)) for p in params]
+        xs = [torch.randn((T, d_in), device=dev, generator=g) for _ in range(2)]
+        ids = torch.empty((T, k), dtype=torch.int32, device=dev)
+        vals = torch.empty((T, k), dtype=torch.float32, device=dev)
+        sae = S.Sae(params[0], params[1], params[3])          # fp32: the handle reads the parameters in place
+        ws = S.new_workspace(sae.encode_workspace_bytes(T, k), dev)
+        bws = S.new_workspace(S.s3_sae_backward_workspace_bytes(T), dev)
+        state = {"step": 0}
+
+        def run(i):
+            state["step"] += 1
+            x = xs[i % 2]
+            S.s3_sae_encode_topk(sae, x, k, ids, vals, ws)
+            _, gWe, gbe, gWd, gbd = S.s3_sae_backward(params[0], params[2], params[3], x, ids, vals, bws)
+            for p, (m, v), gr in zip(params, moments, (gWe, gbe, gWd, gbd)):
+                S.s3_adam_update(p, m, v, gr, 1e-3, 0.9, 0.999, 1e-8, state["step"])
+        out.update(T=T, d_in=d_in, d_sae=D, k=k, flop=2.0 * T * d_in * D, adam_bytes=(2 * d_in * D + D + d_in) * 28)
     elif args.case == "decode":
         # SAE decode alone on the key SAE's shape: x_hat = z_hat W_dec + b_dec and the squared reconstruction error.
         # bytes = the k gathered dictionary rows per token (mostly L2 hits: the dictionary is 32 MB) + x read + x_hat written
@@ -547,7 +571,7 @@ def run_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads")
+    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads | train")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)

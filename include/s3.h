@@ -322,6 +322,38 @@ s3_status s3_sae_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int
                         float* d_xhat, int64_t ld_xhat, const void* d_x, int64_t ldx, float* d_sqerr, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * SAE training step on fp32 parameters      (paper appendix, training configuration: Top-K SAEs trained with
+ *                                             Adam, learning rate 1e-3, batches of 4096 tokens; Sec. 3.3 for the
+ *                                             model. The loss is not printed; reading below.)
+ *
+ * s3_sae_backward: with z_hat the Top-k code of the batch (d_ids / d_vals [T, k] from s3_sae_encode_topk on the
+ * same parameters; id < 0 = padding) and x_hat = z_hat W_dec + b_dec,
+ *     loss = (1/T) sum_t ||x_hat_t - x_t||^2,
+ * and its gradients through the code with the active set held fixed (z[t,j] = W_enc[:,f].(x_t - b_dec) + b_enc[f]
+ * for the selected f):  gW_enc [d_in, d_sae], gb_enc [d_sae], gW_dec [d_sae, d_in], gb_dec [d_in], all fp32 and
+ * overwritten. The sums over tokens are fp32 atomics (no fixed order); the loss is added in a fixed order.
+ * All arrays fp32, x with row pitch ldx. Limits: 1 <= k <= S3_MAX_K, d_in <= 4096, T >= 1.
+ * Workspace: s3_sae_backward_workspace_bytes(T).
+ *
+ * s3_adam_update: one Adam step on n parameters, in place (Kingma & Ba):
+ *     m = beta1 m + (1-beta1) g;  v = beta2 v + (1-beta2) g^2;
+ *     p -= lr * (m / (1-beta1^step)) / (sqrt(v / (1-beta2^step)) + eps),        step counted from 1.
+ * A training step is: encode -> backward -> one update per parameter tensor (-> s3_sae_create again for bf16 use).
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    float lr, beta1, beta2, eps;
+    int32_t step, reserved;
+} s3_adam_params;
+
+size_t s3_sae_backward_workspace_bytes(int T);
+s3_status s3_sae_backward(const float* d_W_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
+                          const int32_t* d_ids, const float* d_vals, int T, int k, int d_in, int d_sae,
+                          float* d_gW_enc, float* d_gb_enc, float* d_gW_dec, float* d_gb_dec, float* d_loss,
+                          void* d_ws, size_t ws_bytes, void* stream);
+s3_status s3_adam_update(float* d_param, float* d_m, float* d_v, const float* d_grad, size_t n,
+                         const s3_adam_params* params, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * Compact inverted index        (paper Sec. 3.4, memory analysis: contiguous integer arrays with delta
  *                                encoding and optional stop-feature pruning; the appendix's hard frequency
  *                                threshold for stop features. The layout is this library's.)

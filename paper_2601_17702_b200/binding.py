@@ -32,6 +32,7 @@ EXPORTS = [
     "s3_compact_bound", "s3_compact_workspace_bytes", "s3_compact_build", "s3_coactivation_score_topspans_compact",
     "s3_compact_save", "s3_compact_file_info", "s3_compact_load",
     "s3_sae_decode", "s3_head_aggregate_topk", "s3_compact_expand",
+    "s3_sae_backward_workspace_bytes", "s3_sae_backward", "s3_adam_update",
 ]
 
 
@@ -59,6 +60,11 @@ class CompactView(C.Structure):
 class CompactHostLayer(C.Structure):
     _fields_ = [("h_row_ptr", C.c_void_p), ("h_blk_ptr", C.c_void_p), ("h_blk_first", C.c_void_p),
                 ("h_blk_desc", C.c_void_p), ("h_payload", C.c_void_p), ("n_blocks", C.c_uint64), ("n_words", C.c_uint64)]
+
+
+class AdamParams(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("step", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class ScoreParams(C.Structure):
@@ -90,7 +96,7 @@ def lib():
         L.s3_last_error.restype = C.c_char_p
         for name in ("s3_sae_prepared_bytes", "s3_sae_encode_workspace_bytes", "s3_postings_workspace_bytes",
                      "s3_score_workspace_bytes", "s3_density_workspace_bytes", "s3_fuse_workspace_bytes",
-                     "s3_compact_workspace_bytes"):
+                     "s3_compact_workspace_bytes", "s3_sae_backward_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.s3_sae_prepared_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_sae_create.argtypes = [C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
@@ -144,6 +150,11 @@ def lib():
         L.s3_head_aggregate_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                              C.c_void_p, C.c_void_p]
         L.s3_compact_expand.argtypes = [C.POINTER(CompactView), C.c_int, C.c_void_p, C.c_uint64, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_sae_backward_workspace_bytes.argtypes = [C.c_int]
+        L.s3_sae_backward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int,
+                                      C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_adam_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(AdamParams), C.c_void_p]
         _lib = L
     return _lib
 
@@ -562,3 +573,39 @@ def s3_compact_expand(layer: CompactLayer, d_sae: int, ws: torch.Tensor | None =
     code = C.c_uint32(0)
     _check(lib().s3_workspace_status(_ptr(ws), _stream(stream), C.byref(code)))
     return layer.row_ptr, pos[:n]
+
+
+def s3_sae_backward(W_enc: torch.Tensor, W_dec: torch.Tensor, b_dec: torch.Tensor, x: torch.Tensor, ids: torch.Tensor,
+                    vals: torch.Tensor, ws: torch.Tensor | None = None, stream=None):
+    """fp32 tensors: W_enc [d_in, d_sae], W_dec [d_sae, d_in], b_dec [d_in], x [T, d_in]; ids int32 / vals fp32 [T, k] from the
+    encode. Returns (loss [1], gW_enc, gb_enc, gW_dec, gb_dec)."""
+    for t in (W_enc, W_dec, b_dec, x, vals):
+        assert t.dtype == torch.float32
+    assert W_enc.is_contiguous() and W_dec.is_contiguous() and ids.is_contiguous() and vals.is_contiguous() and x.stride(1) == 1
+    d_in, d_sae = W_enc.shape
+    T, k = ids.shape
+    assert W_dec.shape == (d_sae, d_in) and x.shape == (T, d_in) and ids.dtype == torch.int32
+    dev = x.device
+    if ws is None:
+        ws = torch.zeros(s3_sae_backward_workspace_bytes(T), dtype=torch.uint8, device=dev)
+    gW_enc, gW_dec = torch.empty_like(W_enc), torch.empty_like(W_dec)
+    gb_enc = torch.empty(d_sae, dtype=torch.float32, device=dev)
+    gb_dec = torch.empty(d_in, dtype=torch.float32, device=dev)
+    loss = torch.empty(1, dtype=torch.float32, device=dev)
+    _check(lib().s3_sae_backward(_ptr(W_enc), _ptr(W_dec), _ptr(b_dec), _ptr(x), x.stride(0), _ptr(ids), _ptr(vals), T, k, d_in, d_sae,
+                                 _ptr(gW_enc), _ptr(gb_enc), _ptr(gW_dec), _ptr(gb_dec), _ptr(loss), _ptr(ws), ws.numel(),
+                                 _stream(stream)))
+    return loss, gW_enc, gb_enc, gW_dec, gb_dec
+
+
+def s3_sae_backward_workspace_bytes(T: int) -> int:
+    return int(lib().s3_sae_backward_workspace_bytes(T))
+
+
+def s3_adam_update(param: torch.Tensor, m: torch.Tensor, v: torch.Tensor, grad: torch.Tensor, lr: float, beta1: float, beta2: float,
+                   eps: float, step: int, stream=None):
+    """In-place Adam step on a contiguous fp32 tensor and its moments."""
+    for t in (param, m, v, grad):
+        assert t.dtype == torch.float32 and t.is_contiguous() and t.numel() == param.numel()
+    params = AdamParams(lr, beta1, beta2, eps, step, 0)
+    _check(lib().s3_adam_update(_ptr(param), _ptr(m), _ptr(v), _ptr(grad), param.numel(), C.byref(params), _stream(stream)))

@@ -467,6 +467,44 @@ s3_status s3_sae_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int
                          static_cast<cudaStream_t>(stream));
 }
 
+// ---------------------------------------------------------------------------------------------- SAE training step
+size_t s3_sae_backward_workspace_bytes(int T)
+{
+    if (T < 0) return 0;
+    return 256 + round_up(static_cast<size_t>(T) * 4, 256);
+}
+
+s3_status s3_sae_backward(const float* d_W_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
+                          const int32_t* d_ids, const float* d_vals, int T, int k, int d_in, int d_sae, float* d_gW_enc,
+                          float* d_gb_enc, float* d_gW_dec, float* d_gb_dec, float* d_loss, void* d_ws, size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(T >= 1 && d_in >= 1 && d_sae >= 1, S3_ERR_INVALID_ARG, "T = %d, d_in = %d, d_sae = %d out of range", T, d_in, d_sae);
+    S3_REQUIRE(k >= 1 && k <= S3_MAX_K, S3_ERR_UNSUPPORTED, "k = %d out of [1, %d]", k, S3_MAX_K);
+    S3_REQUIRE(d_in <= 4096, S3_ERR_UNSUPPORTED, "d_in = %d exceeds 4096", d_in);
+    S3_REQUIRE(ldx >= d_in, S3_ERR_INVALID_ARG, "ldx = %lld is smaller than d_in = %d", (long long)ldx, d_in);
+    S3_REQUIRE(d_W_enc && d_W_dec && d_b_dec && d_x && d_ids && d_vals && d_gW_enc && d_gb_enc && d_gW_dec && d_gb_dec && d_loss,
+               S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE(d_ws != nullptr && ws_bytes >= s3_sae_backward_workspace_bytes(T), S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed",
+               ws_bytes, s3_sae_backward_workspace_bytes(T));
+    return launch_sae_backward(d_W_enc, d_W_dec, d_b_dec, d_x, ldx, d_ids, d_vals, T, k, d_in, d_sae, d_gW_enc, d_gb_enc, d_gW_dec,
+                               d_gb_dec, d_loss, reinterpret_cast<float*>(static_cast<unsigned char*>(d_ws) + 256),
+                               static_cast<cudaStream_t>(stream));
+}
+
+s3_status s3_adam_update(float* d_param, float* d_m, float* d_v, const float* d_grad, size_t n, const s3_adam_params* p, void* stream)
+{
+    S3_REQUIRE(p != nullptr, S3_ERR_INVALID_ARG, "params is null");
+    S3_REQUIRE(p->step >= 1, S3_ERR_INVALID_ARG, "step = %d must count from 1", p->step);
+    S3_REQUIRE(p->beta1 >= 0.0f && p->beta1 < 1.0f && p->beta2 >= 0.0f && p->beta2 < 1.0f && p->eps >= 0.0f, S3_ERR_INVALID_ARG,
+               "beta1 = %g, beta2 = %g must lie in [0, 1) and eps = %g must not be negative", p->beta1, p->beta2, p->eps);
+    if (n == 0) return S3_OK;
+    S3_REQUIRE(d_param && d_m && d_v && d_grad, S3_ERR_INVALID_ARG, "null device pointer");
+    const double c1 = 1.0 / (1.0 - pow(static_cast<double>(p->beta1), p->step));
+    const double c2 = 1.0 / (1.0 - pow(static_cast<double>(p->beta2), p->step));
+    return launch_adam(d_param, d_m, d_v, d_grad, n, p->lr, p->beta1, p->beta2, p->eps, static_cast<float>(c1), static_cast<float>(c2),
+                       static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------------------- index-set fusion
 size_t s3_fuse_workspace_bytes(int Q, int64_t L)
 {
