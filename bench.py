@@ -489,19 +489,38 @@ def run_case(args):
         xs = [torch.randn((T, d_in), device=dev, generator=g) for _ in range(2)]
         ids = torch.empty((T, k), dtype=torch.int32, device=dev)
         vals = torch.empty((T, k), dtype=torch.float32, device=dev)
-        sae = S.Sae(params[0], params[1], params[3])          # fp32: the handle reads the parameters in place
-        ws = S.new_workspace(sae.encode_workspace_bytes(T, k), dev)
         bws = S.new_workspace(S.s3_sae_backward_workspace_bytes(T), dev)
         state = {"step": 0}
+        if args.fp32_forward:
+            sae = S.Sae(params[0], params[1], params[3])      # fp32: the handle reads the parameters in place
+            ws = S.new_workspace(sae.encode_workspace_bytes(T, k), dev)
+        else:
+            W16 = torch.empty((d_in, D), dtype=torch.bfloat16, device=dev)
+            x16 = torch.empty((T, d_in), dtype=torch.bfloat16, device=dev)
+            ws = None
 
         def run(i):
+            nonlocal ws
             state["step"] += 1
             x = xs[i % 2]
-            S.s3_sae_encode_topk(sae, x, k, ids, vals, ws)
-            _, gWe, gbe, gWd, gbd = S.s3_sae_backward(params[0], params[2], params[3], x, ids, vals, bws)
+            if args.fp32_forward:
+                S.s3_sae_encode_topk(sae, x, k, ids, vals, ws)
+                code = vals
+            else:
+                # the tensor cores select the active set from bf16 copies; the gradient below is taken in fp32
+                S.s3_cast_f32_to_bf16(params[0], W16)
+                S.s3_cast_f32_to_bf16(x, x16)
+                sae16 = S.Sae(W16, params[1], params[3])
+                if ws is None:
+                    ws = S.new_workspace(sae16.encode_workspace_bytes(T, k), dev)
+                S.s3_sae_encode_topk(sae16, x16, k, ids, vals, ws)
+                code = None
+            _, gWe, gbe, gWd, gbd = S.s3_sae_backward(params[0], params[2], params[3], x, ids, code, bws, b_enc=params[1])
             for p, (m, v), gr in zip(params, moments, (gWe, gbe, gWd, gbd)):
                 S.s3_adam_update(p, m, v, gr, 1e-3, 0.9, 0.999, 1e-8, state["step"])
-        out.update(T=T, d_in=d_in, d_sae=D, k=k, flop=2.0 * T * d_in * D, adam_bytes=(2 * d_in * D + D + d_in) * 28)
+            if not args.fp32_forward:
+                sae16.close()                                 # its buffers return to torch's allocator in stream order
+        out.update(T=T, d_in=d_in, d_sae=D, k=k, forward="fp32" if args.fp32_forward else "bf16", flop=2.0 * T * d_in * D, adam_bytes=(2 * d_in * D + D + d_in) * 28)
     elif args.case == "decode":
         # SAE decode alone on the key SAE's shape: x_hat = z_hat W_dec + b_dec and the squared reconstruction error.
         # bytes = the k gathered dictionary rows per token (mostly L2 hits: the dictionary is 32 MB) + x read + x_hat written
@@ -577,6 +596,7 @@ def main():
     ap.add_argument("--max-ctas", type=int, default=0)
     ap.add_argument("--items", type=int, default=8)
     ap.add_argument("--k", type=int, default=0, help="heads case: Top-k per head and per token (default: the key SAE's)")
+    ap.add_argument("--fp32-forward", action="store_true", help="train case: fp32 FFMA forward pass instead of the bf16 one")
     ap.add_argument("--compact", action="store_true", help="score case: read the block-delta compact index")
     ap.add_argument("--no-union", action="store_true", help="density case: leave out the index-set union; heads case: leave out the aggregation")
     ap.add_argument("--gpus", type=int, default=1)

@@ -332,6 +332,9 @@ s3_status s3_sae_decode(const void* d_W_dec, const float* d_b_dec, int d_in, int
  * and its gradients through the code with the active set held fixed (z[t,j] = W_enc[:,f].(x_t - b_dec) + b_enc[f]
  * for the selected f):  gW_enc [d_in, d_sae], gb_enc [d_sae], gW_dec [d_sae, d_in], gb_dec [d_in], all fp32 and
  * overwritten. The sums over tokens are fp32 atomics (no fixed order); the loss is added in a fixed order.
+ * d_vals may be NULL: z is then recomputed in fp32 from W_enc, b_enc, b_dec and x for the given ids, which is the
+ * form to use when the ids come from a bf16 forward pass over a bf16 copy of the parameters (s3_cast_f32_to_bf16,
+ * s3_sae_create with S3_BF16): the tensor cores pick the active set, the gradient is taken in fp32.
  * All arrays fp32, x with row pitch ldx. Limits: 1 <= k <= S3_MAX_K, d_in <= 4096, T >= 1.
  * Workspace: s3_sae_backward_workspace_bytes(T).
  *
@@ -346,10 +349,12 @@ typedef struct {
 } s3_adam_params;
 
 size_t s3_sae_backward_workspace_bytes(int T);
-s3_status s3_sae_backward(const float* d_W_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
+s3_status s3_sae_backward(const float* d_W_enc, const float* d_b_enc /*nullable with d_vals*/, const float* d_W_dec,
+                          const float* d_b_dec, const float* d_x, int64_t ldx,
                           const int32_t* d_ids, const float* d_vals, int T, int k, int d_in, int d_sae,
                           float* d_gW_enc, float* d_gb_enc, float* d_gW_dec, float* d_gb_dec, float* d_loss,
                           void* d_ws, size_t ws_bytes, void* stream);
+s3_status s3_cast_f32_to_bf16(const float* d_src, void* d_dst, size_t n, void* stream);   /* round to nearest even */
 s3_status s3_adam_update(float* d_param, float* d_m, float* d_v, const float* d_grad, size_t n,
                          const s3_adam_params* params, void* stream);
 

@@ -32,7 +32,7 @@ EXPORTS = [
     "s3_compact_bound", "s3_compact_workspace_bytes", "s3_compact_build", "s3_coactivation_score_topspans_compact",
     "s3_compact_save", "s3_compact_file_info", "s3_compact_load",
     "s3_sae_decode", "s3_head_aggregate_topk", "s3_compact_expand",
-    "s3_sae_backward_workspace_bytes", "s3_sae_backward", "s3_adam_update",
+    "s3_sae_backward_workspace_bytes", "s3_sae_backward", "s3_adam_update", "s3_cast_f32_to_bf16",
 ]
 
 
@@ -151,7 +151,8 @@ def lib():
                                              C.c_void_p, C.c_void_p]
         L.s3_compact_expand.argtypes = [C.POINTER(CompactView), C.c_int, C.c_void_p, C.c_uint64, C.c_void_p, C.c_size_t, C.c_void_p]
         L.s3_sae_backward_workspace_bytes.argtypes = [C.c_int]
-        L.s3_sae_backward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int,
+        L.s3_cast_f32_to_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_sae_backward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int,
                                       C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_size_t, C.c_void_p]
         L.s3_adam_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(AdamParams), C.c_void_p]
@@ -576,12 +577,14 @@ def s3_compact_expand(layer: CompactLayer, d_sae: int, ws: torch.Tensor | None =
 
 
 def s3_sae_backward(W_enc: torch.Tensor, W_dec: torch.Tensor, b_dec: torch.Tensor, x: torch.Tensor, ids: torch.Tensor,
-                    vals: torch.Tensor, ws: torch.Tensor | None = None, stream=None):
-    """fp32 tensors: W_enc [d_in, d_sae], W_dec [d_sae, d_in], b_dec [d_in], x [T, d_in]; ids int32 / vals fp32 [T, k] from the
-    encode. Returns (loss [1], gW_enc, gb_enc, gW_dec, gb_dec)."""
-    for t in (W_enc, W_dec, b_dec, x, vals):
-        assert t.dtype == torch.float32
-    assert W_enc.is_contiguous() and W_dec.is_contiguous() and ids.is_contiguous() and vals.is_contiguous() and x.stride(1) == 1
+                    vals: torch.Tensor | None, ws: torch.Tensor | None = None, b_enc: torch.Tensor | None = None, stream=None):
+    """fp32 tensors: W_enc [d_in, d_sae], W_dec [d_sae, d_in], b_dec [d_in], x [T, d_in]; ids int32 [T, k] and either the
+    fp32 vals [T, k] of the same encode or None with b_enc [d_sae] (the code is then recomputed in fp32).
+    Returns (loss [1], gW_enc, gb_enc, gW_dec, gb_dec)."""
+    for t in (W_enc, W_dec, b_dec, x, vals, b_enc):
+        assert t is None or t.dtype == torch.float32
+    assert W_enc.is_contiguous() and W_dec.is_contiguous() and ids.is_contiguous() and x.stride(1) == 1
+    assert vals is None or vals.is_contiguous()
     d_in, d_sae = W_enc.shape
     T, k = ids.shape
     assert W_dec.shape == (d_sae, d_in) and x.shape == (T, d_in) and ids.dtype == torch.int32
@@ -592,7 +595,7 @@ def s3_sae_backward(W_enc: torch.Tensor, W_dec: torch.Tensor, b_dec: torch.Tenso
     gb_enc = torch.empty(d_sae, dtype=torch.float32, device=dev)
     gb_dec = torch.empty(d_in, dtype=torch.float32, device=dev)
     loss = torch.empty(1, dtype=torch.float32, device=dev)
-    _check(lib().s3_sae_backward(_ptr(W_enc), _ptr(W_dec), _ptr(b_dec), _ptr(x), x.stride(0), _ptr(ids), _ptr(vals), T, k, d_in, d_sae,
+    _check(lib().s3_sae_backward(_ptr(W_enc), _ptr(b_enc), _ptr(W_dec), _ptr(b_dec), _ptr(x), x.stride(0), _ptr(ids), _ptr(vals), T, k, d_in, d_sae,
                                  _ptr(gW_enc), _ptr(gb_enc), _ptr(gW_dec), _ptr(gb_dec), _ptr(loss), _ptr(ws), ws.numel(),
                                  _stream(stream)))
     return loss, gW_enc, gb_enc, gW_dec, gb_dec
@@ -609,3 +612,12 @@ def s3_adam_update(param: torch.Tensor, m: torch.Tensor, v: torch.Tensor, grad: 
         assert t.dtype == torch.float32 and t.is_contiguous() and t.numel() == param.numel()
     params = AdamParams(lr, beta1, beta2, eps, step, 0)
     _check(lib().s3_adam_update(_ptr(param), _ptr(m), _ptr(v), _ptr(grad), param.numel(), C.byref(params), _stream(stream)))
+
+
+def s3_cast_f32_to_bf16(src: torch.Tensor, dst: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    assert src.dtype == torch.float32 and src.is_contiguous()
+    if dst is None:
+        dst = torch.empty(src.shape, dtype=torch.bfloat16, device=src.device)
+    assert dst.dtype == torch.bfloat16 and dst.is_contiguous() and dst.numel() == src.numel()
+    _check(lib().s3_cast_f32_to_bf16(_ptr(src), _ptr(dst), src.numel(), _stream(stream)))
+    return dst

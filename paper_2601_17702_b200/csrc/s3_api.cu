@@ -474,7 +474,7 @@ size_t s3_sae_backward_workspace_bytes(int T)
     return 256 + round_up(static_cast<size_t>(T) * 4, 256);
 }
 
-s3_status s3_sae_backward(const float* d_W_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
+s3_status s3_sae_backward(const float* d_W_enc, const float* d_b_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
                           const int32_t* d_ids, const float* d_vals, int T, int k, int d_in, int d_sae, float* d_gW_enc,
                           float* d_gb_enc, float* d_gW_dec, float* d_gb_dec, float* d_loss, void* d_ws, size_t ws_bytes, void* stream)
 {
@@ -482,13 +482,21 @@ s3_status s3_sae_backward(const float* d_W_enc, const float* d_W_dec, const floa
     S3_REQUIRE(k >= 1 && k <= S3_MAX_K, S3_ERR_UNSUPPORTED, "k = %d out of [1, %d]", k, S3_MAX_K);
     S3_REQUIRE(d_in <= 4096, S3_ERR_UNSUPPORTED, "d_in = %d exceeds 4096", d_in);
     S3_REQUIRE(ldx >= d_in, S3_ERR_INVALID_ARG, "ldx = %lld is smaller than d_in = %d", (long long)ldx, d_in);
-    S3_REQUIRE(d_W_enc && d_W_dec && d_b_dec && d_x && d_ids && d_vals && d_gW_enc && d_gb_enc && d_gW_dec && d_gb_dec && d_loss,
+    S3_REQUIRE(d_W_enc && d_W_dec && d_b_dec && d_x && d_ids && d_gW_enc && d_gb_enc && d_gW_dec && d_gb_dec && d_loss,
                S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE(d_vals != nullptr || d_b_enc != nullptr, S3_ERR_INVALID_ARG, "without d_vals the code is recomputed and needs d_b_enc");
     S3_REQUIRE(d_ws != nullptr && ws_bytes >= s3_sae_backward_workspace_bytes(T), S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed",
                ws_bytes, s3_sae_backward_workspace_bytes(T));
-    return launch_sae_backward(d_W_enc, d_W_dec, d_b_dec, d_x, ldx, d_ids, d_vals, T, k, d_in, d_sae, d_gW_enc, d_gb_enc, d_gW_dec,
+    return launch_sae_backward(d_W_enc, d_b_enc, d_W_dec, d_b_dec, d_x, ldx, d_ids, d_vals, T, k, d_in, d_sae, d_gW_enc, d_gb_enc, d_gW_dec,
                                d_gb_dec, d_loss, reinterpret_cast<float*>(static_cast<unsigned char*>(d_ws) + 256),
                                static_cast<cudaStream_t>(stream));
+}
+
+s3_status s3_cast_f32_to_bf16(const float* d_src, void* d_dst, size_t n, void* stream)
+{
+    if (n == 0) return S3_OK;
+    S3_REQUIRE(d_src && d_dst, S3_ERR_INVALID_ARG, "null device pointer");
+    return launch_cast_bf16(d_src, d_dst, n, static_cast<cudaStream_t>(stream));
 }
 
 s3_status s3_adam_update(float* d_param, float* d_m, float* d_v, const float* d_grad, size_t n, const s3_adam_params* p, void* stream)

@@ -56,7 +56,8 @@ s3_status launch_head_aggregate(const int32_t* d_ids, const float* d_vals, int T
                                 int32_t* d_out_ids, float* d_out_vals, cudaStream_t stream);
 s3_status launch_compact_expand(const s3_compact_view& v, int d_sae, int32_t* d_pos, uint64_t cap_postings, uint32_t* d_status,
                                 cudaStream_t stream);
-s3_status launch_sae_backward(const float* d_W_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
+s3_status launch_cast_bf16(const float* d_src, void* d_dst, size_t n, cudaStream_t stream);
+s3_status launch_sae_backward(const float* d_W_enc, const float* d_b_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
                               const int32_t* d_ids, const float* d_vals, int T, int k, int d_in, int d_sae, float* d_gW_enc,
                               float* d_gb_enc, float* d_gW_dec, float* d_gb_dec, float* d_loss, float* d_sqerr, cudaStream_t stream);
 s3_status launch_adam(float* d_p, float* d_m, float* d_v, const float* d_g, size_t n, float lr, float beta1, float beta2, float eps,

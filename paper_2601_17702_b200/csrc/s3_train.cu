@@ -10,6 +10,8 @@
 //   accumulated with fp32 atomics (the sums over tokens have no fixed order; the tests allow for that). The per-token
 //   squared errors go to scratch and are summed by one block in a fixed order.
 // adam: elementwise, bias corrections passed in.
+#include <cuda_bf16.h>
+
 #include "s3_common.cuh"
 #include "s3_encode_tc.cuh"
 
@@ -22,10 +24,11 @@ constexpr int TT = 128;      // threads per block
 struct BackwardArgs {
     const float* W_enc;      // [d_in, d_sae]
     const float* W_dec;      // [d_sae, d_in]
+    const float* b_enc;      // read only when vals is null
     const float* b_dec;
     const float* x;
     const int32_t* ids;
-    const float* vals;
+    const float* vals;       // null: z is recomputed in fp32 from the parameters
     float* gW_enc;
     float* gb_enc;
     float* gW_dec;
@@ -50,7 +53,21 @@ __global__ void __launch_bounds__(TT) sae_backward_kernel(const __grid_constant_
             int32_t f = a.ids[(size_t)t * a.k + tid];
             if (f >= a.d_sae) f = -1;
             s_id[tid] = f;
-            s_z[tid] = f >= 0 ? a.vals[(size_t)t * a.k + tid] : 0.0f;
+            s_z[tid] = (f >= 0 && a.vals) ? a.vals[(size_t)t * a.k + tid] : 0.0f;
+        }
+        if (a.vals == nullptr) {
+            // z[j] = W_enc[:, f_j] . (x - b_dec) + b_enc[f_j] in fp32 (the ids may come from a bf16 forward pass)
+            for (int c = tid; c < a.d_in; c += TT) xc_s[c] = a.x[(size_t)t * a.ldx + c] - __ldg(a.b_dec + c);
+            __syncthreads();
+            for (int j = warp; j < a.k; j += TT / 32) {
+                const int32_t f = s_id[j];
+                float dot = 0.0f;
+                if (f >= 0)
+                    for (int c = lane; c < a.d_in; c += 32) dot = __fmaf_rn(__ldg(a.W_enc + (size_t)c * a.d_sae + f), xc_s[c], dot);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                if (lane == 0) s_z[j] = f >= 0 ? dot + __ldg(a.b_enc + f) : 0.0f;
+            }
         }
         __syncthreads();
         float err = 0.0f;
@@ -131,9 +148,23 @@ __global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ p, float*
     }
 }
 
+__global__ void __launch_bounds__(256) cast_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t n)
+{
+    for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (size_t)gridDim.x * 256) dst[i] = __float2bfloat16_rn(src[i]);
+}
+
 }  // namespace
 
-s3_status launch_sae_backward(const float* d_W_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
+s3_status launch_cast_bf16(const float* d_src, void* d_dst, size_t n, cudaStream_t stream)
+{
+    const size_t want = (n + 255) / 256;
+    const size_t cap = static_cast<size_t>(device_sm_count()) * 16;
+    cast_bf16_kernel<<<static_cast<unsigned>(want < cap ? want : cap), 256, 0, stream>>>(d_src, static_cast<__nv_bfloat16*>(d_dst), n);
+    S3_CUDA_TRY(cudaGetLastError());
+    return S3_OK;
+}
+
+s3_status launch_sae_backward(const float* d_W_enc, const float* d_b_enc, const float* d_W_dec, const float* d_b_dec, const float* d_x, int64_t ldx,
                               const int32_t* d_ids, const float* d_vals, int T, int k, int d_in, int d_sae, float* d_gW_enc,
                               float* d_gb_enc, float* d_gW_dec, float* d_gb_dec, float* d_loss, float* d_sqerr, cudaStream_t stream)
 {
@@ -143,7 +174,7 @@ s3_status launch_sae_backward(const float* d_W_enc, const float* d_W_dec, const 
     S3_CUDA_TRY(cudaMemsetAsync(d_gb_enc, 0, static_cast<size_t>(d_sae) * 4, stream));
     S3_CUDA_TRY(cudaMemsetAsync(d_gb_dec, 0, static_cast<size_t>(d_in) * 4, stream));
     BackwardArgs a;
-    a.W_enc = d_W_enc; a.W_dec = d_W_dec; a.b_dec = d_b_dec; a.x = d_x; a.ids = d_ids; a.vals = d_vals;
+    a.W_enc = d_W_enc; a.b_enc = d_b_enc; a.W_dec = d_W_dec; a.b_dec = d_b_dec; a.x = d_x; a.ids = d_ids; a.vals = d_vals;
     a.gW_enc = d_gW_enc; a.gb_enc = d_gb_enc; a.gW_dec = d_gW_dec; a.gb_dec = d_gb_dec; a.sqerr = d_sqerr;
     a.ldx = ldx; a.T = T; a.k = k; a.d_in = d_in; a.d_sae = d_sae;
     const int max_grid = device_sm_count() * 16;

@@ -66,6 +66,30 @@ def test_backward_matches_oracle(T, d_in, d_sae, k):
         close(got, w, 1e-4)
 
 
+@pytest.mark.parametrize("T,d_in,d_sae,k", [(300, 128, 1024, 32), (100, 64, 4096, 128)])
+def test_backward_with_a_bf16_forward_pass(T, d_in, d_sae, k):
+    """The tensor cores pick the active set from bf16 copies of the parameters; the gradient is taken in fp32 on the
+    fp32 parameters with the code recomputed for that set, which is what the oracle does with the same ids."""
+    d = _dev()
+    params = [p.to(d) for p in _params(T + 7, d_in, d_sae)]
+    x = torch.randn((T, d_in), generator=torch.Generator().manual_seed(T)).to(d)
+    W16 = S.s3_cast_f32_to_bf16(params[0])
+    assert torch.equal(W16, params[0].to(torch.bfloat16))                   # round to nearest even, like the library cast
+    sae = S.Sae(W16, params[1], params[3])
+    ids = torch.empty((T, k), dtype=torch.int32, device=d)
+    vals = torch.empty((T, k), dtype=torch.float32, device=d)
+    ws = S.new_workspace(sae.encode_workspace_bytes(T, k), d)
+    S.s3_sae_encode_topk(sae, S.s3_cast_f32_to_bf16(x), k, ids, vals, ws)
+    loss, gWe, gbe, gWd, gbd = S.s3_sae_backward(params[0], params[2], params[3], x, ids, None, b_enc=params[1])
+    torch.cuda.synchronize()
+    want = O.sae_loss_and_grads(x.cpu().numpy(), *[p.cpu().numpy() for p in params], ids.cpu().numpy())
+    assert abs(float(loss) - want[0]) <= 1e-5 * want[0]
+    for got, w in zip((gWe, gbe, gWd, gbd), want[1:]):
+        close(got, w, 1e-4)
+    with pytest.raises(S.S3Error):
+        S.s3_sae_backward(params[0], params[2], params[3], x, ids, None)     # neither vals nor b_enc
+
+
 def test_adam_matches_oracle_over_steps():
     d = _dev()
     rng = np.random.default_rng(0)
