@@ -2,6 +2,8 @@
 128K-token workload per call, the batched postings build of all layers and both SAEs, the 256-query retrieval
 over a 32K-token index), checked on sampled outputs the CPU oracle can compute one by one and on properties
 that hold at any size. Integer results bit-exact; encode within the bf16 tolerance (see test_gpu_parity.py)."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -217,12 +219,13 @@ def test_scan_device_memory_is_flat_across_chunks():
     xs = [inp.x("key", 0, c * cfg.chunk, cfg.chunk) for c in range(2)]
     pipe.scan_chunk(0, {"key": [xs[0]]})
     torch.cuda.synchronize()
+    gc.collect()                                         # tensors of earlier tests must not be freed in mid-measurement
     base = torch.cuda.memory_allocated()
     torch.cuda.reset_peak_memory_stats()
     for c in range(1, cfg.n_chunks):
         pipe.scan_chunk(c * cfg.chunk, {"key": [xs[c % 2]]})
     pipe.finish()
-    assert torch.cuda.max_memory_allocated() == base and torch.cuda.memory_allocated() == base
+    assert torch.cuda.max_memory_allocated() <= base and torch.cuda.memory_allocated() <= base      # nothing was allocated
     st = pipe.slots[0].index.stats()
     assert st["n_postings"] == cfg.L * cfg.key.k and st["n_positions"] == cfg.L
     csr = stage_index_on_device(pipe.slots[0].index, d)

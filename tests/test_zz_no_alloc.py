@@ -9,6 +9,8 @@ within the encode tolerance the other GPU tests use). It also checks that an inp
 array is refused with a capacity error instead of being run.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run every other test."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -37,9 +39,10 @@ def _static(sae, x, k):
     ids = torch.full((T, k), -9, dtype=torch.int32, device=x.device)
     vals = torch.full((T, k), -9.0, dtype=torch.float32, device=x.device)
     status = torch.full((1,), 77, dtype=torch.int32, device=x.device)
+    gc.collect()                                            # no tensor of an earlier test is freed inside the window
     before = torch.cuda.memory_allocated()
     S.s3_sae_encode_topk_static(sae, x, k, ids, vals, status)
-    assert torch.cuda.memory_allocated() == before          # nothing was allocated through torch either
+    assert torch.cuda.memory_allocated() <= before          # nothing was allocated through torch either
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     return ids.cpu().numpy(), vals.cpu().numpy()
