@@ -76,6 +76,8 @@ def test_hand_example_on_gpu(golden_dir):
     (2500, 8, 16, 1, 2, 40, 8, 9, 300, 64, 0),        # radius wider than a segment boundary; runs out of peaks
     (3000, 4, 64, 2, 2, 6, 4, 48, 10, 8, 900),        # stop features
     (20, 4, 64, 1, 2, 3, 4, 48, 5, 4, 0),             # kernel wider than the context
+    (20001, 4, 64, 2, 3, 6, 4, 48, 24, 40, 0),        # three position tiles, the last one ragged; two layers
+    (8193, 8, 4096, 1, 2, 40, 64, 8, 4, 40, 3),       # one position past a tile; 2560 query entries (several feature passes); most lists are stop features
 ])
 def test_density_and_centres_exact(L, k, D, n_layers, Q, nq, kq, K, R, N, stop):
     rng = np.random.default_rng(L + K)
