@@ -4,7 +4,7 @@
 
 #include <new>
 
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 #include "s3_topk.cuh"
 
 namespace s3 {

@@ -10,7 +10,7 @@
 //   pack    : one warp per block: values OR-ed into a shared-memory image of the block, copied out; descriptor
 //             = (word offset << 6) | width. A zero word closes the payload so a two-word read never leaves it.
 #include "s3_common.cuh"
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 
 namespace s3 {
 

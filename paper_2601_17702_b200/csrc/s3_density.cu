@@ -1,6 +1,6 @@
 // Per-position relevance, smoothed density and peak selection (Sec. 3.5 Eq. 6, "Adaptive Granularity"; Alg. 1 Phase 2):
 // the paper's own retrieval tail, beside the fixed-width span scorer of s3_score.cu.
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 #include "s3_query.cuh"
 
 namespace s3 {

@@ -33,7 +33,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 #include "s3_topk.cuh"
 
 namespace s3 {

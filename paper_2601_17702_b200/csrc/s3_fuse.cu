@@ -3,7 +3,7 @@
 // the selected density peaks, the supplied lexical positions, the first `lead` and last `tail` positions; a
 // block scan over the words' population counts then gives every word its place in the output.
 #include "s3_common.cuh"
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 
 namespace s3 {
 

@@ -1,5 +1,5 @@
 // Head aggregation of per-head Top-k codes (Sec. 3.3, Sec. 3.4).
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 #include "s3_query.cuh"
 
 namespace s3 {

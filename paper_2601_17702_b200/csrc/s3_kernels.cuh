@@ -1,4 +1,5 @@
-// Host-side interface of the tensor-core (bf16) and FP32-pipe encode kernels.
+// Host-side interface between the C ABI (s3_api.cu) and the kernel files: launchers, size queries and host state, one group
+// per .cu file.
 #pragma once
 
 #include "s3_common.cuh"

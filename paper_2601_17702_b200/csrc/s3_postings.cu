@@ -16,7 +16,7 @@
 // is bit-identical from run to run. Features are handled in ranges of 32768 per pass (one pass for
 // the usual dictionary sizes).
 #include "s3_common.cuh"
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 
 namespace s3 {
 

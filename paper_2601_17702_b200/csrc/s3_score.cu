@@ -9,7 +9,7 @@
 //      range as +1/-1 in a difference array that one prefix sum turns into min(cQ, cS) totals;
 //      weighted mode adds aQ*IDF to each span of the range in fp64;
 //   c. fuse with the lexical score vector and pick the s best spans (score desc, index asc).
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 #include "s3_query.cuh"
 
 namespace s3 {

@@ -13,7 +13,7 @@
 #include <cuda_bf16.h>
 
 #include "s3_common.cuh"
-#include "s3_encode_tc.cuh"
+#include "s3_kernels.cuh"
 
 namespace s3 {
 
