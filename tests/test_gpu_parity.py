@@ -127,6 +127,34 @@ def test_encode_bf16_shapes(T, d_in, d_sae, k, n_slices):
     assert np.abs(vals[same] - ov[same]).max() < 2e-3
 
 
+def test_encode_bf16_degenerate_rows():
+    """Rows that defeat the streaming bound on the tensor-core path: every feature tied (the candidate lists overflow
+    and fall back to the exact cut), no positive value, fewer positives than k, a plateau of ties around the k-th value.
+    Exactly representable values, so ids and values must equal the oracle's."""
+    d_in, D, k = 64, 4096, 32
+    W = torch.zeros((d_in, D))
+    W[0, :] = 1.0                                         # pre[t, f] = x[t, 0] + b_enc[f]
+    W[1, 100:140] = 1.0                                   # features 100..139 also see x[t, 1]
+    b_enc = torch.zeros(D)
+    b_enc[2000:2100] = 0.5                                # a plateau of 100 tied features above the rest
+    x = torch.zeros((6, d_in))
+    x[0, 0] = 1.0                                         # all 4096 tied at 1.0, plateau at 1.5
+    x[1, 0] = -1.0                                        # plateau at -0.5: nothing positive
+    x[2, 0] = -0.25                                       # only the plateau (0.25) is positive: 100 ties, k = 32 of them
+    x[3, 0] = -1.0
+    x[3, 1] = 1.25                                        # 40 positives (0.25) only through the second input
+    x[4, 0] = 2.0
+    x[4, 1] = -1.0                                        # 40 features one below the rest
+    # row 5: all zero -> pre = b_enc: plateau 0.5, rest 0 (not positive)
+    for n_slices in (0, 1, 4):
+        ids, vals = gpu_encode(W.to(torch.bfloat16), b_enc, torch.zeros(d_in), x.to(torch.bfloat16), k, n_slices)
+        oi, ov = O.encode_topk(x.numpy(), W.numpy(), b_enc.numpy(), np.zeros(d_in, np.float32), k)
+        np.testing.assert_array_equal(ids, oi)
+        np.testing.assert_array_equal(vals, ov)
+    assert ids[0].tolist() == list(range(2000, 2032)) and (ids[1] == -1).all()
+    assert ids[3].tolist() == list(range(100, 132)) and ids[5].tolist() == list(range(2000, 2032))
+
+
 def test_encode_bf16_result_independent_of_schedule():
     T, d_in, d_sae, k = 512, 256, 4096, 32
     x = G.activations(12, 0, 0, T, d_in, torch.bfloat16)
