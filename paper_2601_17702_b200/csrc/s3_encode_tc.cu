@@ -52,6 +52,7 @@ constexpr int BATCH = 32;                    // columns per tcgen05.ld
 constexpr int STEP = 8;                      // columns filtered between two checks of the pending lists
 constexpr int PEND_CAP = 2 * STEP;           // pending-list slots per row
 constexpr int NB = 64;                       // histogram buckets per row
+constexpr int kCompactMinTiles = 32;          // units of at least this many column tiles compact their candidate lists
 constexpr int HSHIFT = 19;                   // bucket = float bits >> 19: 16 buckets per octave
 constexpr uint32_t WAIT_LIMIT = 1u << 26;    // try_wait polls before a wait is declared dead (~1 s)
 
@@ -533,10 +534,11 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     if (r.istar == 0 && r.floor_exact && out > 0u) out -= 1u;
                     // The list was filled under bounds that rose along the slice (about k (1 + ln(columns / k))
                     // entries); only what beats the final bound can still matter, so the list is compacted once
-                    // here and the merge reads a fraction of it.
+                    // here and the merge reads a fraction of it. The pass is a tail of dependent round trips after the
+                    // unit's last tile, so it is taken only when the unit was long enough to make that tail small.
                     const float cut = __uint_as_float(out);
-                    uint32_t w = 0;
-                    for (uint32_t i0 = 0; i0 < r.gcnt; i0 += 16) {
+                    uint32_t w = tile_hi - tile_lo >= kCompactMinTiles ? 0u : r.gcnt;
+                    for (uint32_t i0 = 0; i0 < r.gcnt && tile_hi - tile_lo >= kCompactMinTiles; i0 += 16) {
                         uint64_t key[16];                        // read first: the writes land at or before i0
 #pragma unroll
                         for (int q = 0; q < 16; ++q) key[q] = i0 + q < r.gcnt ? glist[i0 + q] : 0ull;
