@@ -478,6 +478,20 @@ def run_case(args):
             if not args.no_union:
                 S.s3_head_aggregate_topk(ids.view(T, H, k), vals.view(T, H, k), D, k)
         out.update(T=T, H=H, d_head=d_head, d_sae=D, k=k, flop=2.0 * T * H * d_head * D)
+    elif args.case == "project":
+        # the upstream projections of a Llama-3.1-8B layer on one chunk (d_model 4096 -> keys 1024, queries 4096) through the
+        # dense-epilogue form of the encode GEMM, bf16 in and out
+        d_model = 4096
+        d_out = args.k or 1024
+        T = args.tokens or cfg.chunk
+        g = torch.Generator(device=dev).manual_seed(1)
+        Wp = (torch.randn((d_model, d_out), device=dev, generator=g) / d_model ** 0.5).to(torch.bfloat16)
+        proj = S.Sae(Wp, torch.zeros(d_out, device=dev), torch.zeros(d_model, device=dev))
+        hs = [torch.randn((T, d_model), device=dev, generator=g).to(torch.bfloat16) for _ in range(2)]
+        outp = torch.empty((T, d_out), dtype=torch.bfloat16, device=dev)
+        pws = S.new_workspace(64, dev)
+        run = lambda i: S.s3_sae_preact(proj, hs[i % 2], torch.bfloat16, outp, pws)
+        out.update(T=T, d_model=d_model, d_out=d_out, flop=2.0 * T * d_model * d_out)
     elif args.case == "train":
         # one fp32 training step of the paper's SAE shape (appendix: batches of 4096 tokens, expansion 128 over d_head = 128,
         # k = 128, Adam at 1e-3): encode + Top-k, backward through the code, Adam on the four parameter tensors
@@ -590,7 +604,7 @@ def run_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads | train")
+    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads | train | project (--k = output width)")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)

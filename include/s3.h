@@ -92,6 +92,14 @@ size_t s3_sae_encode_workspace_bytes(const s3_sae* sae, int T_max, int k);
 s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, int T, int k,
                              int32_t* d_ids /*[T,k]*/, float* d_vals /*[T,k]*/,
                              void* d_ws, size_t ws_bytes, void* stream);
+/* The same GEMM with a dense epilogue: d_out [T, ld_out] (fp32 or bf16, rounded to nearest even) receives the
+ * pre-activations pre[t,f] of Eq. 1 before the ReLU, nothing is selected. With zero biases this is a plain projection
+ * x W (e.g. the key projection K = W_K h, paper appendix on chunk-independent prefill, whose output feeds
+ * s3_sae_encode_topk on the same stream while it is still in the L2 cache); it also serves to inspect an encoder.
+ * bf16 encoders only (S3_ERR_UNSUPPORTED otherwise). ld_out must be a multiple of 8 (bf16) or 4 (fp32) and >= d_sae;
+ * d_out 16-byte aligned. Workspace: the 64-byte status block only. */
+s3_status s3_sae_preact(const s3_sae* sae, const void* d_x, int64_t ldx, int T, void* d_out, int64_t ld_out,
+                        s3_dtype out_dtype, void* d_ws, size_t ws_bytes, void* stream);
 /* Tuning knob: number of column slices each row block of the encode is split into (0 = automatic)
  * and the largest number of thread blocks a launch may use (0 = all SMs). Results do not depend on
  * either. */

@@ -32,7 +32,7 @@ EXPORTS = [
     "s3_compact_bound", "s3_compact_workspace_bytes", "s3_compact_build", "s3_coactivation_score_topspans_compact",
     "s3_compact_save", "s3_compact_file_info", "s3_compact_load",
     "s3_sae_decode", "s3_head_aggregate_topk", "s3_compact_expand",
-    "s3_sae_backward_workspace_bytes", "s3_sae_backward", "s3_adam_update", "s3_cast_f32_to_bf16",
+    "s3_sae_backward_workspace_bytes", "s3_sae_backward", "s3_adam_update", "s3_cast_f32_to_bf16", "s3_sae_preact",
 ]
 
 
@@ -156,6 +156,8 @@ def lib():
                                       C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_size_t, C.c_void_p]
         L.s3_adam_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(AdamParams), C.c_void_p]
+        L.s3_sae_preact.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_size_t,
+                                    C.c_void_p]
         _lib = L
     return _lib
 
@@ -621,3 +623,18 @@ def s3_cast_f32_to_bf16(src: torch.Tensor, dst: torch.Tensor | None = None, stre
     assert dst.dtype == torch.bfloat16 and dst.is_contiguous() and dst.numel() == src.numel()
     _check(lib().s3_cast_f32_to_bf16(_ptr(src), _ptr(dst), src.numel(), _stream(stream)))
     return dst
+
+
+def s3_sae_preact(sae: "Sae", x: torch.Tensor, out_dtype: torch.dtype = torch.float32, out: torch.Tensor | None = None,
+                  ws: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Dense pre-activations [T, d_sae] of a bf16 encoder (fp32 or bf16 output)."""
+    T = x.shape[0]
+    if out is None:
+        out = torch.empty((T, sae.d_sae), dtype=out_dtype, device=x.device)
+    assert out.dtype == out_dtype and out.stride(1) == 1 and x.stride(1) == 1
+    if ws is None:
+        ws = torch.zeros(64, dtype=torch.uint8, device=x.device)
+    code = {torch.bfloat16: S3_BF16, torch.float32: S3_F32}[out_dtype]
+    _check(lib().s3_sae_preact(sae.handle, _ptr(x), x.stride(0) if T > 1 else max(x.stride(0), sae.d_in), T, _ptr(out), out.stride(0),
+                               code, _ptr(ws), ws.numel(), _stream(stream)))
+    return out

@@ -226,6 +226,25 @@ s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, in
     return S3_OK;
 }
 
+s3_status s3_sae_preact(const s3_sae* sae, const void* d_x, int64_t ldx, int T, void* d_out, int64_t ld_out, s3_dtype out_dtype,
+                        void* d_ws, size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(sae != nullptr, S3_ERR_INVALID_ARG, "sae is null");
+    S3_REQUIRE(sae->dtype == S3_BF16, S3_ERR_UNSUPPORTED, "dense pre-activations are built for bf16 encoders only");
+    S3_REQUIRE(out_dtype == S3_BF16 || out_dtype == S3_F32, S3_ERR_INVALID_ARG, "unknown output dtype %d", (int)out_dtype);
+    S3_REQUIRE(T >= 0, S3_ERR_INVALID_ARG, "T = %d is negative", T);
+    if (T == 0) return S3_OK;
+    S3_REQUIRE(d_x && d_out && d_ws, S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE(ws_bytes >= S3_WS_HEADER_BYTES, S3_ERR_CAPACITY, "workspace smaller than %d bytes", S3_WS_HEADER_BYTES);
+    S3_REQUIRE(aligned16(d_x) && aligned16(d_out), S3_ERR_INVALID_ARG, "misaligned device pointer");
+    S3_REQUIRE(ldx >= sae->d_in && ldx % 8 == 0, S3_ERR_INVALID_ARG, "ldx = %lld must be a multiple of 8 and >= d_in", (long long)ldx);
+    const int vec = out_dtype == S3_BF16 ? 8 : 4;
+    S3_REQUIRE(ld_out >= sae->d_sae && ld_out % vec == 0, S3_ERR_INVALID_ARG, "ld_out = %lld must be a multiple of %d and >= d_sae",
+               (long long)ld_out, vec);
+    return launch_preact_tc(&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, pick_slices(sae, T), sae->max_ctas,
+                            static_cast<uint32_t*>(d_ws), d_out, ld_out, out_dtype == S3_BF16, static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------------------- postings
 size_t s3_postings_workspace_bytes(int T_max, int k, int d_sae)
 {

@@ -195,6 +195,9 @@ struct EncodeTcParams {
     uint64_t* cand;            // [T][n_slices][cap]
     uint32_t* counts;          // [T][n_slices]
     uint32_t* hint;            // [T] float bits of the best published bound
+    void* dense_out;           // dense mode: the pre-activations [T, ld_out], fp32 or bf16
+    long long ld_out;
+    int out_bf16;
     uint32_t* status;
 };
 
@@ -317,6 +320,9 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
     r.tau = r.istar > 0 ? __uint_as_float((static_cast<uint32_t>(r.hbase + r.istar) << HSHIFT) - 1u) : r.tau_floor;
 }
 
+// DENSE: the epilogue writes the pre-activations themselves (row-major, fp32 or bf16) instead of selecting; the rest of
+// the kernel is the same pipeline.
+template <bool DENSE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                  const EncodeTcParams p)
@@ -460,11 +466,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
             const int t = mt * PAIR_M + static_cast<int>(cta_rank) * BM + e;
             const bool live = t < p.T;
-            uint64_t* glist = p.cand + (static_cast<size_t>(live ? t : 0) * p.n_slices + slice) * p.cap;
+            uint64_t* glist = DENSE ? nullptr : p.cand + (static_cast<size_t>(live ? t : 0) * p.n_slices + slice) * p.cap;
+            if (!DENSE) {
 #pragma unroll 1
-            for (int sl = 0; sl < NB; ++sl) my_hist[sl * EPI_THREADS] = 0;
+                for (int sl = 0; sl < NB; ++sl) my_hist[sl * EPI_THREADS] = 0;
+            }
             // start from the best bound another slice of these rows has published so far, if any
-            const uint32_t hint_in = live ? *reinterpret_cast<volatile const uint32_t*>(p.hint + t) : 0u;
+            const uint32_t hint_in = (live && !DENSE) ? *reinterpret_cast<volatile const uint32_t*>(p.hint + t) : 0u;
             RowSel r;
             r.tau_floor = live ? __uint_as_float(hint_in) : INFINITY;    // rows past T select nothing
             r.tau = r.tau_floor;
@@ -494,6 +502,31 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         bias[4 * j4 + 0] = b4.x; bias[4 * j4 + 1] = b4.y; bias[4 * j4 + 2] = b4.z; bias[4 * j4 + 3] = b4.w;
                     }
                     tc_wait_ld();
+                    if constexpr (DENSE) {
+                        // 32 consecutive columns of this thread's row: 128 (fp32) or 64 (bf16) contiguous bytes
+                        const int col0 = nt * BN + cb * BATCH;
+                        if (live) {
+#pragma unroll
+                            for (int g8 = 0; g8 < BATCH / 8; ++g8) {
+                                if (col0 + g8 * 8 >= p.d_sae) break;              // d_sae is a multiple of 8
+                                float v[8];
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(acc[g8 * 8 + q]) + bias[g8 * 8 + q];
+                                if (p.out_bf16) {
+                                    __nv_bfloat162 h2[4];
+#pragma unroll
+                                    for (int q = 0; q < 4; ++q) h2[q] = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+                                    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.dense_out) + static_cast<size_t>(t) * p.ld_out + col0 + g8 * 8;
+                                    *reinterpret_cast<uint4*>(out) = *reinterpret_cast<const uint4*>(h2);
+                                } else {
+                                    float* out = static_cast<float*>(p.dense_out) + static_cast<size_t>(t) * p.ld_out + col0 + g8 * 8;
+                                    *reinterpret_cast<float4*>(out) = make_float4(v[0], v[1], v[2], v[3]);
+                                    *reinterpret_cast<float4*>(out + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                                }
+                            }
+                        }
+                        continue;
+                    }
                     const uint32_t ncol0 = ~static_cast<uint32_t>(nt * BN + cb * BATCH);   // ~(col0 + j) = ncol0 - j
 #pragma unroll
                     for (int h = 0; h < BATCH / STEP; ++h) {
@@ -525,7 +558,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 tc_fence_before();
                 mbar_arrive_cluster(acc_empty_addr[ab]);
             }
-            if (ok) {
+            if (ok && !DENSE) {
                 if (__any_sync(0xffffffffu, cnt > 0)) fold_pending(my_pend, my_hist, glist, r, cnt, p.k, p.cap);
                 if (live) {
                     // The bound to publish: at least k values of this slice exceed it. An exact k-th value
@@ -689,10 +722,14 @@ size_t encode_tc_workspace_bytes(int T, int n_slices, int k)
     return round_up(t * 4, 256) + round_up(t * s * 4, 256) + t * s * encode_tc_list_cap(k) * sizeof(uint64_t);
 }
 
-s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
-                           int n_slices, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals,
-                           cudaStream_t stream)
+namespace {
+
+// Common launch of the two epilogue modes. Selection: d_scratch / d_ids / d_vals set, d_dense null. Dense: the reverse.
+s3_status launch_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k, int n_slices,
+                    int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals, void* d_dense, int64_t ld_out,
+                    bool out_bf16, cudaStream_t stream)
 {
+    const bool dense = d_dense != nullptr;
     alignas(64) CUtensorMap map_x;
     s3_status rc = make_map(&map_x, d_x, static_cast<uint64_t>(T), static_cast<uint64_t>(d_in), static_cast<uint64_t>(ldx), BM);
     if (rc != S3_OK) return rc;
@@ -707,14 +744,18 @@ s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx
     p.n_units = p.n_mtiles * n_slices;
     p.cap = encode_tc_list_cap(k);
     p.b_eff = st->d_b_eff;
-    unsigned char* base = static_cast<unsigned char*>(d_scratch);
-    p.hint = reinterpret_cast<uint32_t*>(base);
-    p.counts = reinterpret_cast<uint32_t*>(base + round_up(static_cast<size_t>(T) * 4, 256));
-    p.cand = reinterpret_cast<uint64_t*>(base + round_up(static_cast<size_t>(T) * 4, 256) +
-                                         round_up(static_cast<size_t>(T) * n_slices * 4, 256));
     p.status = d_status;
-    // no bound is known for any row yet
-    S3_CUDA_TRY(cudaMemsetAsync(p.hint, 0, static_cast<size_t>(T) * 4, stream));
+    p.dense_out = d_dense; p.ld_out = ld_out; p.out_bf16 = out_bf16 ? 1 : 0;
+    p.hint = nullptr; p.counts = nullptr; p.cand = nullptr;
+    if (!dense) {
+        unsigned char* base = static_cast<unsigned char*>(d_scratch);
+        p.hint = reinterpret_cast<uint32_t*>(base);
+        p.counts = reinterpret_cast<uint32_t*>(base + round_up(static_cast<size_t>(T) * 4, 256));
+        p.cand = reinterpret_cast<uint64_t*>(base + round_up(static_cast<size_t>(T) * 4, 256) +
+                                             round_up(static_cast<size_t>(T) * n_slices * 4, 256));
+        // no bound is known for any row yet
+        S3_CUDA_TRY(cudaMemsetAsync(p.hint, 0, static_cast<size_t>(T) * 4, stream));
+    }
 
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
@@ -729,17 +770,39 @@ s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx
     const CUtensorMap& map_w = *reinterpret_cast<const CUtensorMap*>(st->map_w);
     static bool attr_set[64] = {};
     if (dev < 64 && !attr_set[dev]) {
-        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set[dev] = true;
     }
     int n_pairs = encode_tc_max_pairs();
     if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
     if (p.n_units < n_pairs) n_pairs = p.n_units;
-    encode_tc_kernel<<<2 * n_pairs, NUM_THREADS, smem, stream>>>(map_x, map_w, p);
+    if (dense) {
+        encode_tc_kernel<true><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(map_x, map_w, p);
+        S3_CUDA_TRY(cudaGetLastError());
+        return S3_OK;
+    }
+    encode_tc_kernel<false><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(map_x, map_w, p);
     S3_CUDA_TRY(cudaGetLastError());
     launch_candidate_merge(p.cand, p.counts, p.hint, T, n_slices, p.cap, k, d_ids, d_vals, stream);
     S3_CUDA_TRY(cudaGetLastError());
     return S3_OK;
+}
+
+}  // namespace
+
+s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
+                           int n_slices, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals,
+                           cudaStream_t stream)
+{
+    return launch_tc(st, d_x, ldx, T, d_in, d_sae, k, n_slices, max_ctas, d_scratch, d_status, d_ids, d_vals, nullptr, 0, false, stream);
+}
+
+s3_status launch_preact_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int n_slices,
+                           int max_ctas, uint32_t* d_status, void* d_out, int64_t ld_out, bool out_bf16, cudaStream_t stream)
+{
+    return launch_tc(st, d_x, ldx, T, d_in, d_sae, 1, n_slices, max_ctas, nullptr, d_status, nullptr, nullptr, d_out, ld_out, out_bf16,
+                     stream);
 }
 
 }  // namespace s3
