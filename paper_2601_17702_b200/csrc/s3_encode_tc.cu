@@ -53,6 +53,8 @@ constexpr int STEP = 8;                      // columns filtered between two che
 constexpr int PEND_CAP = 2 * STEP;           // pending-list slots per row
 constexpr int NB = 64;                       // histogram buckets per row
 constexpr int kCompactMinTiles = 32;          // units of at least this many column tiles compact their candidate lists
+constexpr int COLD_LEVELS = 6;                // trial bounds of the cold-start pass, as fractions of the first batch's maximum
+__device__ constexpr float kColdFraction[COLD_LEVELS] = {0.80f, 0.65f, 0.52f, 0.40f, 0.30f, 0.20f};
 constexpr int HSHIFT = 19;                   // bucket = float bits >> 19: 16 buckets per octave
 constexpr uint32_t WAIT_LIMIT = 1u << 26;    // try_wait polls before a wait is declared dead (~1 s)
 
@@ -491,6 +493,47 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ab * BN + (static_cast<uint32_t>(quarter * 32) << 16);
                 const float4* bias4 = reinterpret_cast<const float4*>(p.b_eff + static_cast<size_t>(nt) * BN);
+                if (!DENSE && nt == tile_lo && __any_sync(0xffffffffu, live && r.tau == 0.0f)) {
+                    // Cold start: without a bound every second value of the unit's first tile would go through the pending
+                    // lists. A first pass over that tile only counts, per row, how many of its values exceed each of
+                    // COLD_LEVELS fractions of the largest value of the row's first 32 columns; the highest level that at
+                    // least k values exceed is a bound that k values of this slice are known to beat, and the regular pass
+                    // below (the accumulator is still in tensor memory) starts from it.
+                    float level[COLD_LEVELS];
+                    int seen[COLD_LEVELS];
+#pragma unroll 1
+                    for (int cb = 0; cb < BN / BATCH; ++cb) {
+                        uint32_t acc[32];
+                        tc_ld32(taddr + cb * BATCH, acc);
+                        float bias[BATCH];
+#pragma unroll
+                        for (int j4 = 0; j4 < BATCH / 4; ++j4) {
+                            const float4 b4 = __ldg(bias4 + cb * (BATCH / 4) + j4);
+                            bias[4 * j4 + 0] = b4.x; bias[4 * j4 + 1] = b4.y; bias[4 * j4 + 2] = b4.z; bias[4 * j4 + 3] = b4.w;
+                        }
+                        tc_wait_ld();
+                        if (cb == 0) {
+                            float top = 0.0f;
+#pragma unroll
+                            for (int q = 0; q < BATCH; ++q) top = fmaxf(top, __uint_as_float(acc[q]) + bias[q]);
+#pragma unroll
+                            for (int lv = 0; lv < COLD_LEVELS; ++lv) { level[lv] = top * kColdFraction[lv]; seen[lv] = 0; }
+                        }
+#pragma unroll
+                        for (int q = 0; q < BATCH; ++q) {
+                            const float v = __uint_as_float(acc[q]) + bias[q];
+#pragma unroll
+                            for (int lv = 0; lv < COLD_LEVELS; ++lv) seen[lv] += (v > level[lv]) ? 1 : 0;
+                        }
+                    }
+                    if (live && r.tau == 0.0f) {
+                        float bound = 0.0f;
+#pragma unroll
+                        for (int lv = COLD_LEVELS - 1; lv >= 0; --lv)
+                            if (seen[lv] >= p.k && level[lv] > bound) bound = level[lv];       // levels descend with lv ascending
+                        r.tau_floor = r.tau = bound;
+                    }
+                }
 #pragma unroll 1
                 for (int cb = 0; cb < BN / BATCH; ++cb) {
                     uint32_t acc[32];
