@@ -35,7 +35,7 @@ from workloads import configs as C, generators as G  # noqa: E402
 METRIC = "scanned tokens/s (SAE Top-k encode + postings) at 128K ctx"
 # Measured DRAM traffic of one query-SAE encode launch at the benchmark's size (see profiles/); set to None when
 # the encode kernel changes until the counters are taken again.
-ENCODE_QUERY_DRAM_BYTES = 1.32e9
+ENCODE_QUERY_DRAM_BYTES = 1.41e9
 UNIT = "tokens/s"
 
 
@@ -308,7 +308,7 @@ def run_ours(args, rank, world, local_rank):
                      "peak_source": f"{peaks['source']} sustained bf16 matmul", "frac_of_burst": tflops / peaks["bf16_tflops"],
                      "frac_of_nominal_2250": tflops / 2250.0, "launch_ms": enc_avg_ms, "launches_timed": len(enc_ms),
                      # dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of this kernel (ncu, one pass,
-                     # two launches: 1.27 + 0.07 and 1.22 + 0.07 GB); compulsory bytes are 0.34 GB (W_enc^T once + x)
+                     # two launches: 1.29 + 0.07 and 1.40 + 0.07 GB); compulsory bytes are 0.34 GB (W_enc^T once + x)
                      "traffic": ENCODE_QUERY_DRAM_BYTES, "traffic_unit": "bytes per launch"},
         "device_mem": {"allocated_after_warmup_mib": mem_after_warm / 2**20, "peak_in_timed_region_mib": peak_mem / 2**20},
     }
