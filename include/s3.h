@@ -144,15 +144,19 @@ s3_status s3_sae_encode_topk_static(const s3_sae* sae, const void* d_x, int64_t 
  * Groups the (feature, position) pairs of one chunk of one layer into a CSR:
  *   row_ptr[f] = number of pairs with id < f  (row_ptr has d_sae + 1 entries, uint32)
  *   pos[row_ptr[f] .. row_ptr[f+1]) = ascending absolute positions pos_base + t with f in F_t
- * ids [T,k] int32; entries < 0 are padding and are skipped; ids within a token must be distinct.
+ * ids [T,k] int32; entries < 0 are padding and are skipped; ids within a token must be distinct (a repeated id
+ * keeps both of its pairs and is reported through the workspace status as S3_ERR_INVALID_ARG, as is an
+ * id >= d_sae, whose pair is dropped).
  * d_vals / d_pval (both null or both non-null) carry each pair's activation next to its position.
  * d_pos (and d_pval) must hold T*k entries. The result is bit-exact and run-to-run identical.
- * Limits: d_sae <= 2^20, k <= 4096, T*k < 2^31, pos_base + T <= 2^31 - 1 (S3_ERR_CAPACITY: positions are
- *         int32). T == 0 writes zeros to row_ptr.
- * Workspace: the status block plus a table of per-token-run feature counts;
- * s3_postings_workspace_bytes(T, k, d_sae) bounds it for one item, and a batch needs the sum of its
- * items' values. The batched form processes up to S3_MAX_POSTINGS_ITEMS independent chunk-layers in one
- * sequence of launches; `items` is a HOST array.
+ * Limits: d_sae <= 2^20, k <= 4096, T*k <= 2^27, pos_base + T <= 2^31 - 1 (S3_ERR_CAPACITY: positions are
+ *         int32); ceil(log2 T) + ceil(log2(d_sae / 2048)) <= 32 (S3_ERR_UNSUPPORTED; only dictionaries beyond
+ *         65536 features meet it, at more than 2^23 tokens per item). T == 0 writes zeros to row_ptr.
+ * Workspace: the status block, the item's pairs regrouped by feature range (4 bytes per pair, 8 with values)
+ * and a small directory; s3_postings_workspace_bytes(T, k, d_sae) bounds it for one item, and a batch needs
+ * the sum of its items' values. The batched form processes up to S3_MAX_POSTINGS_ITEMS independent
+ * chunk-layers in two launches; `items` is a HOST array. Batches that follow one another on a stream should
+ * share one workspace: the regrouped pairs are then rewritten in place and stay in the L2 cache.
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
     const int32_t* d_ids;

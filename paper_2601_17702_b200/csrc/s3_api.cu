@@ -120,6 +120,7 @@ s3_status s3_workspace_status(const void* d_ws, void* stream, uint32_t* code_out
     if (code_out) *code_out = code;
     if (code == DEV_OK) return S3_OK;
     if (code == DEV_BAD_FEATURE_ID) return fail(S3_ERR_INVALID_ARG, "a feature id >= d_sae was met on the device (code %u)", code);
+    if (code == DEV_DUPLICATE_ID) return fail(S3_ERR_INVALID_ARG, "a token carried the same feature id twice (code %u)", code);
     if (code == DEV_COMPACT_CAPACITY) return fail(S3_ERR_CAPACITY, "compact index: block or payload buffer too small (code %u)", code);
     return fail(S3_ERR_TIMEOUT, "a bounded device-side wait ran out (code %u)", code);
 }
@@ -257,7 +258,7 @@ static s3_status check_item(const s3_postings_item& it, int idx)
                it.k, it.d_sae);
     S3_REQUIRE(it.d_sae <= (1 << 20), S3_ERR_UNSUPPORTED, "item %d: d_sae = %d exceeds 2^20", idx, it.d_sae);
     S3_REQUIRE(it.k <= 4096, S3_ERR_UNSUPPORTED, "item %d: k = %d exceeds 4096", idx, it.k);
-    S3_REQUIRE((int64_t)it.T * it.k <= INT32_MAX, S3_ERR_UNSUPPORTED, "item %d: T*k = %lld must be below 2^31", idx,
+    S3_REQUIRE((int64_t)it.T * it.k <= (1ll << 27), S3_ERR_UNSUPPORTED, "item %d: T*k = %lld exceeds 2^27", idx,
                (long long)it.T * it.k);
     S3_REQUIRE(it.d_row_ptr != nullptr, S3_ERR_INVALID_ARG, "item %d: d_row_ptr is null", idx);
     S3_REQUIRE(it.T == 0 || (it.d_ids && it.d_pos), S3_ERR_INVALID_ARG, "item %d: null device pointer", idx);

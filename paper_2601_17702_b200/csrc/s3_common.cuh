@@ -42,6 +42,7 @@ enum : uint32_t {
     DEV_TIMEOUT_ACC_EMPTY = 4,   // MMA warp: accumulator never drained
     DEV_BAD_FEATURE_ID = 16,     // postings: id >= d_sae met in the input
     DEV_COMPACT_CAPACITY = 17,   // compact index: block or payload buffer too small (sizes[] has the need)
+    DEV_DUPLICATE_ID = 18,       // postings: one token carries the same feature id twice
 };
 
 __device__ __forceinline__ void dev_set_error(uint32_t* status, uint32_t code) { atomicCAS(status, 0u, code); }

@@ -58,7 +58,7 @@ class ScanPipeline:
             s.index.stream_wait()
         for i in range(0, len(items), 32):
             B.s3_postings_build_batched(items[i:i + 32], self.ws_post)
-            self.launches += 4         # count, column scan, row scan, scatter
+            self.launches += 2         # partition by bucket, bucket sort
         for s in self.slots:
             for l in range(self.n_layers):
                 s.index.append(l, s.row_ptr[l], s.pos[l], T, s.k, pos_base, s.pval[l] if s.pval else None)

@@ -276,6 +276,61 @@ def test_postings_skewed_and_giant_list():
     assert rp[8] - rp[7] == T
 
 
+def test_postings_list_longer_than_one_sort_and_values():
+    # 64 features, one per bucket: feature 5 sits in every token (a list of 20000 entries, longer than what one
+    # shared-memory sort holds), the others are short; values travel with the positions
+    T, k, d_sae = 20000, 4, 64
+    rng = np.random.default_rng(11)
+    ids = np.stack([rng.choice(np.delete(np.arange(d_sae), 5), size=k, replace=False) for _ in range(T)]).astype(np.int32)
+    ids[:, 2] = 5
+    ids[17, 3] = -1
+    vals = rng.random((T, k)).astype(np.float32)
+    rp, pos, pval = gpu_postings(ids, d_sae, 4096, vals)
+    orp, opos, opval = O.postings(ids, d_sae, 4096, vals)
+    csr_equal(rp, pos, orp, opos)
+    np.testing.assert_array_equal(pval, opval)
+    assert rp[6] - rp[5] == T
+
+
+def test_postings_skewed_buckets_need_several_sweeps():
+    # 24 hot features inside one bucket of 256, each in a third of the tokens: the bucket holds many times what one
+    # shared-memory sort takes and is sorted by ranges of its features
+    T, k, d_sae = 6000, 16, 4096
+    rng = np.random.default_rng(12)
+    ids = np.full((T, k), -1, np.int32)
+    for t in range(T):
+        hot = 256 + rng.choice(24, size=8, replace=False)
+        cold = rng.choice(np.concatenate([np.arange(256), np.arange(512, d_sae)]), size=8, replace=False)
+        ids[t] = rng.permutation(np.concatenate([hot, cold]))
+    rp, pos, _ = gpu_postings(ids, d_sae, 77)
+    orp, opos, _ = O.postings(ids, d_sae, 77)
+    csr_equal(rp, pos, orp, opos)
+
+
+def test_postings_more_runs_than_the_segment_table():
+    # 17.6 M pairs in one item: more token runs than a bucket block keeps in shared memory
+    T, k, d_sae = 1_100_000, 16, 8192
+    t = np.arange(T, dtype=np.int64)[:, None]
+    j = np.arange(k, dtype=np.int64)[None, :]
+    ids = ((t * 7 + (t // 1000) * 3 + j * 131) % d_sae).astype(np.int32)       # distinct within a token: 131 j < d_sae
+    rp, pos, _ = gpu_postings(ids, d_sae, 5)
+    orp, opos, _ = O.postings(ids, d_sae, 5)
+    csr_equal(rp, pos, orp, opos)
+
+
+def test_postings_repeated_id_in_a_token_is_reported():
+    d = dev()
+    ids = torch.tensor([[3, 3], [1, 2]], dtype=torch.int32, device=d)
+    rp = torch.zeros(9, dtype=torch.int32, device=d)
+    ps = torch.zeros(4, dtype=torch.int32, device=d)
+    ws = S.new_workspace(S.s3_postings_workspace_bytes(2, 2, 8))
+    S.s3_postings_build(ids, 8, 0, rp, ps, ws)
+    with pytest.raises(S.binding.S3Error) as e:
+        S.s3_workspace_status(ws)
+    assert e.value.code == S.binding.S3_ERR_INVALID_ARG
+    assert rp.cpu().tolist()[-1] == 4          # nothing is dropped and nothing is written out of range
+
+
 def test_postings_empty_inputs():
     rp, pos, _ = gpu_postings(np.zeros((0, 4), np.int32), 64, 0)
     assert (rp == 0).all() and len(pos) == 0
