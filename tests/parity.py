@@ -2,17 +2,25 @@
 import numpy as np
 
 
-def check_topk_against_preact(pre, ids, vals, k, tol):
+def check_topk_against_preact(pre, ids, vals, k, tol, stats=None):
     """pre: oracle fp64 pre-activations [T, D]; ids/vals: the implementation's [T, k] output.
 
     Values: |val - pre| / (|pre| + 1) <= tol for every reported id.
     Sets: with thr the oracle's k-th largest positive value (0 if fewer than k are positive) and
     band = tol * (|thr| + 1): every feature above thr + band must be reported, nothing at or below
     thr - band (or <= -band) may be, and when no other feature lies inside the band the reported
-    set equals the oracle's exactly. Rows are value-descending with distinct ids, padded -1 / 0.
-    Returns the number of rows that needed the band."""
+    set equals the oracle's exactly. In a row that needs the band the count is still fixed (k ids when k
+    pre-activations are clearly positive, never more than the possibly positive ones) and no unreported
+    feature may beat the weakest reported one by more than the two values' error bounds.
+    Rows are value-descending with distinct ids, padded -1 / 0.
+    Returns the number of rows that needed the band; `stats` (a dict) accumulates rows, banded rows, rows whose
+    id list equals the oracle's Top-k exactly, and the largest |val - pre| / (|pre| + 1) seen."""
     T, D = pre.shape
     banded = 0
+    if stats is not None:
+        for key in ("rows", "banded", "exact"):
+            stats.setdefault(key, 0)
+        stats.setdefault("max_rel_err", 0.0)
     for t in range(T):
         z = pre[t]
         g = ids[t]
@@ -38,14 +46,36 @@ def check_topk_against_preact(pre, ids, vals, k, tol):
         assert set(must.tolist()) <= Gs, f"row {t}: a feature clearly above the threshold is missing"
         assert Gs <= set(must.tolist()) | set(maybe.tolist()), f"row {t}: a feature clearly below the threshold was reported"
         extra = set(maybe.tolist()) - set(oset.tolist())
+        exact = G.tolist() == oset.tolist()
         if not extra:
             assert Gs == set(oset.tolist()), f"row {t}: id set differs with no near-tie to excuse it"
             # equal values must come out in ascending id order
-            assert G.tolist() == oset.tolist() or _only_value_ties_reordered(z, G, oset, tol)
+            assert exact or _only_value_ties_reordered(z, G, oset, tol)
         else:
             banded += 1
-            assert len(must) <= n <= k
+            lo = min(k, int((z > tol).sum()))
+            hi = min(k, int((z > -tol).sum()))
+            assert lo <= n <= hi, f"row {t}: {n} ids reported, between {lo} and {hi} expected"
+            rest = np.ones(D, dtype=bool)
+            rest[G] = False
+            if rest.any():
+                weakest = z[G].min() if n == k else 0.0
+                slack = tol * (abs(weakest) + 1.0) + tol * (np.abs(z[rest]).max(initial=0.0) + 1.0) if n < k else 2.0 * band
+                assert z[rest].max() <= weakest + slack, f"row {t}: an unreported feature beats the weakest reported one"
+        if stats is not None:
+            stats["rows"] += 1
+            stats["banded"] += 1 if extra else 0
+            stats["exact"] += 1 if exact else 0
+            stats["max_rel_err"] = max(stats["max_rel_err"], float(err.max(initial=0.0)))
     return banded
+
+
+def assert_tight(stats, min_exact=0.98, max_rel_err=2e-4):
+    """The statistic that is much tighter than the acceptance band: nearly every row's id list is the oracle's
+    Top-k in the oracle's order, and the values agree to fp32-accumulation accuracy."""
+    assert stats["rows"] > 0
+    assert stats["exact"] >= min_exact * stats["rows"], f"only {stats['exact']} of {stats['rows']} rows equal the oracle's Top-k"
+    assert stats["max_rel_err"] <= max_rel_err, f"largest relative value error {stats['max_rel_err']}"
 
 
 def _only_value_ties_reordered(z, G, oset, tol):

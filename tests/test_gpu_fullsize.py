@@ -11,7 +11,7 @@ import torch
 import oracle as O
 import paper_2601_17702_b200 as S
 from paper_2601_17702_b200.scan import SaeSlot, ScanPipeline, stage_index_on_device
-from parity import check_topk_against_preact, csr_equal
+from parity import assert_tight, check_topk_against_preact, csr_equal
 from workloads import configs as C, generators as G
 
 pytestmark = pytest.mark.gpu
@@ -45,7 +45,9 @@ def test_cfg3_full_chunk_encode_sampled_rows(which, layer, chunk_idx):
     ids, vals = ids.cpu().numpy(), vals.cpu().numpy()
     rows = _sample_rows(cfg.chunk)
     pre = O.preact(x[rows].float().numpy(), W.float().numpy(), b_enc.numpy(), b_dec.numpy())
-    check_topk_against_preact(pre, ids[rows], vals[rows], shp.k, TOL_BF16)
+    stats = {}
+    check_topk_against_preact(pre, ids[rows], vals[rows], shp.k, TOL_BF16, stats)
+    assert_tight(stats)            # nearly every sampled row IS the oracle's Top-k, values at fp32-accumulation accuracy
     # properties of every row: k distinct ids in range, values positive and descending
     assert (ids >= 0).all() and (ids < shp.d_sae).all()
     assert (np.sort(ids, axis=1)[:, 1:] != np.sort(ids, axis=1)[:, :-1]).all()

@@ -8,7 +8,7 @@ import torch
 
 import oracle as O
 import paper_2601_17702_b200 as S
-from parity import check_topk_against_preact, csr_equal
+from parity import assert_tight, check_topk_against_preact, csr_equal
 from workloads import configs as C, generators as G
 
 pytestmark = pytest.mark.gpu
@@ -199,7 +199,9 @@ def test_cfg2_chunk_encode_sampled_rows():
     ids, vals = gpu_encode(W, b_enc, b_dec, x, cfg.key.k)
     rows = np.unique(np.concatenate([np.arange(0, 130), np.arange(2000, 2064), np.arange(cfg.chunk - 62, cfg.chunk)]))
     pre = O.preact(x[rows].float().numpy(), W.float().numpy(), b_enc.numpy(), b_dec.numpy())
-    check_topk_against_preact(pre, ids[rows], vals[rows], cfg.key.k, TOL_BF16)
+    stats = {}
+    check_topk_against_preact(pre, ids[rows], vals[rows], cfg.key.k, TOL_BF16, stats)
+    assert_tight(stats)
     assert (ids >= 0).all()
 
 
@@ -212,7 +214,9 @@ def test_cfg3_query_sae_sampled_rows():
     ids, vals = gpu_encode(W, b_enc, b_dec, x, cfg.query.k)
     rows = np.concatenate([np.arange(0, 40), np.arange(500, 540), np.arange(T - 40, T)])
     pre = O.preact(x[rows].float().numpy(), W.float().numpy(), b_enc.numpy(), b_dec.numpy())
-    check_topk_against_preact(pre, ids[rows], vals[rows], cfg.query.k, TOL_BF16)
+    stats = {}
+    check_topk_against_preact(pre, ids[rows], vals[rows], cfg.query.k, TOL_BF16, stats)
+    assert_tight(stats)
 
 
 def test_cfg5_zipf_chunk_sampled_rows():
@@ -223,7 +227,9 @@ def test_cfg5_zipf_chunk_sampled_rows():
     ids, vals = gpu_encode(W, b_enc, b_dec, x, cfg.key.k)
     rows = np.concatenate([np.arange(0, 128), np.arange(8000, 8128), np.arange(cfg.chunk - 128, cfg.chunk)])
     pre = O.preact(x[rows].float().numpy(), W.float().numpy(), b_enc.numpy(), b_dec.numpy())
-    check_topk_against_preact(pre, ids[rows], vals[rows], cfg.key.k, TOL_BF16)
+    stats = {}
+    check_topk_against_preact(pre, ids[rows], vals[rows], cfg.key.k, TOL_BF16, stats)
+    assert_tight(stats)
     # full-size postings of the skewed chunk, bit-exact against the oracle on the GPU's own ids
     rp, pos, _ = gpu_postings(ids, cfg.key.d_sae, 7 * cfg.chunk)
     orp, opos, _ = O.postings(ids, cfg.key.d_sae, 7 * cfg.chunk)
