@@ -12,7 +12,8 @@ overlapping 64-token spans against a 32K-token device-staged index, 0.5/0.5 fusi
 vector, top-16), so that every stage of the path runs in every step. metric = scanned context tokens/s.
 
 Prints ONE JSON line (rank 0). `--impl reference` times the CPU oracle (oracle/) on a bounded sample of
-the same workload on the host cores instead.
+the same workload on the host cores instead. `--workload cfg5 | cfg2` runs the other scan configurations (scan only).
+With `--gpus N` and no launcher around it the script starts its own N ranks (one process per GPU).
 """
 from __future__ import annotations
 
@@ -49,63 +50,102 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs: NVML from a thread every few
+    milliseconds (nvidia-smi's own source, without its start-up time), or an nvidia-smi loop if NVML cannot be loaded.
+    Read-only queries."""
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
     Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
+    def __init__(self, device: torch.device):
+        self.device = device
+        self.samples = []          # (wall time, sm MHz, max MHz, set of active reasons)
+        self.thread = None
         self.proc = None
-        self.lines = []
+        self.stop_flag = threading.Event()
+        self.source = None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "50", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            import pynvml as N
+            N.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(self.device).uuid)
+            try:
+                h = N.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+            except Exception:
+                h = N.nvmlDeviceGetHandleByIndex(self.device.index or 0)
+            mx = N.nvmlDeviceGetMaxClockInfo(h, N.NVML_CLOCK_SM)
+            bits = {"hw_slowdown": N.nvmlClocksThrottleReasonHwSlowdown, "hw_thermal_slowdown": N.nvmlClocksThrottleReasonHwThermalSlowdown,
+                    "sw_thermal_slowdown": N.nvmlClocksThrottleReasonSwThermalSlowdown, "sw_power_cap": N.nvmlClocksThrottleReasonSwPowerCap}
+
+            def loop():
+                while not self.stop_flag.is_set():
+                    try:
+                        sm = N.nvmlDeviceGetClockInfo(h, N.NVML_CLOCK_SM)
+                        r = N.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                        self.samples.append((time.time(), float(sm), float(mx), {n for n, b in bits.items() if r & b}))
+                    except Exception:
+                        pass
+                    time.sleep(0.004)
+            self.thread = threading.Thread(target=loop, daemon=True)
             self.thread.start()
+            self.source = "nvml"
+            return
+        except Exception:
+            pass
+        try:
+            idx = self.device.index or 0
+            if "CUDA_VISIBLE_DEVICES" in os.environ:
+                idx = int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[idx])
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "20", "-i", str(idx)], stdout=subprocess.PIPE, text=True)
+
+            def read():
+                for line in self.proc.stdout:
+                    f = [v.strip() for v in line.split(",")][1:]
+                    try:
+                        self.samples.append((time.time(), float(f[0]), float(f[1]),
+                                             {n for n, v in zip(self.NAMES, f[3:7]) if v.lower().startswith("active")}))
+                    except (ValueError, IndexError):
+                        continue
+            self.thread = threading.Thread(target=read, daemon=True)
+            self.thread.start()
+            self.source = "nvidia-smi"
         except Exception:
             self.proc = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append((time.time(), line.strip()))
-
     def stop(self, t_begin=None, t_end=None):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ts, ln in self.lines:
-            if t_begin is not None and not (t_begin <= ts <= t_end + 0.06):
-                continue
-            f = [v.strip() for v in ln.split(",")][1:]
-            if len(f) < 7:
-                continue
+        self.stop_flag.set()
+        if self.proc:
+            self.proc.terminate()
             try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        if self.source is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["no clock source"]}
+        sel = [x for x in self.samples if t_begin is None or t_begin <= x[0] <= t_end]
+        reasons = set()
+        for x in sel:
+            reasons |= x[3]
+        return {"sm_mhz": statistics.median(x[1] for x in sel) if sel else None, "sm_max_mhz": max((x[2] for x in sel), default=None),
+                "samples": len(sel), "reasons": sorted(reasons), "source": self.source}
+
+
+WORKLOADS = {"cfg3": (C.CFG3, C.CFG4), "cfg5": (C.CFG5, None), "cfg2": (C.CFG2, None)}
 
 
 def workload_config(cfg, rcfg, L_idx, ns):
     """The `config` object of the JSON line (same for both arms)."""
-    return {"workload": cfg.name, "context_tokens": cfg.L, "chunk": cfg.chunk, "layers": cfg.n_layers,
-            "key_sae": [cfg.key.d_in, cfg.key.d_sae, cfg.key.k], "query_sae": [cfg.query.d_in, cfg.query.d_sae, cfg.query.k],
-            "retrieval_per_step": {"queries": rcfg.Q, "query_tokens": rcfg.nq, "k": rcfg.kq, "index_tokens": L_idx,
-                                   "spans": ns, "width": rcfg.width, "stride": rcfg.stride, "top": rcfg.s},
-            "l2_policy": "inputs larger than L2: every step reads a different 80 MB activation chunk and 1.1 GB of encoder weights",
-            "parallelism": "independent context replicas per GPU, no collectives"}
+    out = {"workload": cfg.name, "context_tokens": cfg.L, "chunk": cfg.chunk, "layers": cfg.n_layers,
+           "key_sae": [cfg.key.d_in, cfg.key.d_sae, cfg.key.k],
+           "query_sae": [cfg.query.d_in, cfg.query.d_sae, cfg.query.k] if cfg.query else None,
+           "l2_policy": "inputs larger than L2: every step reads a different activation chunk and all layers' encoder weights",
+           "parallelism": "independent context replicas per GPU, no collectives"}
+    if rcfg is not None:
+        out["retrieval_per_step"] = {"queries": rcfg.Q, "query_tokens": rcfg.nq, "k": rcfg.kq, "index_tokens": L_idx,
+                                     "spans": ns, "width": rcfg.width, "stride": rcfg.stride, "top": rcfg.s}
+    return out
 
 
 def max_over_ranks(seconds_or_ms: float, world: int, device=None) -> float:
@@ -123,6 +163,19 @@ def whole_job_rate(units_per_rank_step: int, steps: int, world: int, slowest_sec
     return units_per_rank_step * steps * world / slowest_seconds
 
 
+def pick_tensor_peak(peaks: dict, region_seconds: float):
+    """The measured bf16 rate that applies to a kernel timed inside a region of that length: the burst rate for a
+    region that ends before the power cap has pulled the clocks down (about two seconds), else the sustained one."""
+    if region_seconds < 2.0:
+        return peaks["bf16_tflops"], f"{peaks['source']} burst bf16 matmul (timed region {region_seconds:.2f} s < 2 s)"
+    return peaks["bf16_tflops_sustained"], f"{peaks['source']} sustained bf16 matmul (timed region {region_seconds:.2f} s)"
+
+
+def mean_ms(pairs):
+    v = [a.elapsed_time(b) for a, b in pairs]
+    return sum(v) / len(v) if v else None
+
+
 # ------------------------------------------------------------------------------------------ our arm
 
 def run_ours(args, rank, world, local_rank):
@@ -131,123 +184,154 @@ def run_ours(args, rank, world, local_rank):
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    cfg, rcfg = C.CFG3, C.CFG4
+    cfg, rcfg = WORKLOADS[args.workload]
     peaks = load_peaks()
+    sampler = ClockSampler(dev)
+    if rank == 0:
+        sampler.start()
     inp = C.ScanInputs(cfg, device=dev)
     nl, chunk = cfg.n_layers, cfg.chunk
 
     key_saes = [S.Sae(*inp.sae("key", l)) for l in range(nl)]
-    qry_saes = [S.Sae(*inp.sae("query", l)) for l in range(nl)]
-    pipe = ScanPipeline([SaeSlot("key", key_saes, cfg.key.k, chunk), SaeSlot("query", qry_saes, cfg.query.k, chunk)])
-    total_steps = args.steps + args.warmup
-    pipe.reserve_index((total_steps * 2 + 2) * chunk)
+    slots = [SaeSlot("key", key_saes, cfg.key.k, chunk)]
+    if cfg.query:
+        slots.append(SaeSlot("query", [S.Sae(*inp.sae("query", l)) for l in range(nl)], cfg.query.k, chunk))
+    pipe = ScanPipeline(slots)
+    e2e_steps = max(2, min(args.steps, 8))
+    total_steps = 2 * args.steps + args.warmup + e2e_steps + 4
+    pipe.reserve_index((total_steps + 2) * chunk)
 
-    n_distinct = min(cfg.n_chunks, total_steps)
-    xk = [[inp.x("key", l, c * chunk, chunk) for l in range(nl)] for c in range(n_distinct)]
-    xq = [[inp.x("query", l, c * chunk, chunk) for l in range(nl)] for c in range(n_distinct)]
+    n_distinct = min(cfg.n_chunks, args.steps + args.warmup)
+    xs = [{s.name: [inp.x(s.name, l, c * chunk, chunk) for l in range(nl)] for s in slots} for c in range(n_distinct)]
 
     # retrieval side: a 32K-token key index of layer 0 staged on the device, and the query batch
-    rpipe = ScanPipeline([SaeSlot("key", [key_saes[0]], cfg.key.k, chunk)])
-    for c in range(rcfg.scan.L // chunk):
-        rpipe.scan_chunk(c * chunk, {"key": [xk[c % n_distinct][0]]})
-    rpipe.finish()
-    csr = stage_index_on_device(rpipe.slots[0].index, dev)
-    L_idx = rcfg.scan.L
-    ns = C.n_spans(L_idx, rcfg.width, rcfg.stride)
-    xqry = inp.retrieval_queries(0, rcfg.Q, rcfg.nq)
-    q_ids = torch.empty((rcfg.Q * rcfg.nq, rcfg.kq), dtype=torch.int32, device=dev)
-    q_vals = torch.empty((rcfg.Q * rcfg.nq, rcfg.kq), dtype=torch.float32, device=dev)
-    q_ws = S.new_workspace(key_saes[0].encode_workspace_bytes(rcfg.Q * rcfg.nq, rcfg.kq), dev)
-    s_ws = S.new_workspace(64, dev)
-    bm25 = G.gamma21(rcfg.bm25_seed, rcfg.Q, ns).to(dev)
-    top_idx = torch.empty((rcfg.Q, rcfg.s), dtype=torch.int32, device=dev)
-    top_score = torch.empty((rcfg.Q, rcfg.s), dtype=torch.float32, device=dev)
-    top_idx_h = torch.empty((rcfg.Q, rcfg.s), dtype=torch.int32).pin_memory()
-
     launches = [0]
-    enc_events = []
+    timers = {}
+    retrieval = None
+    L_idx = ns = None
+    if rcfg is not None:
+        rpipe = ScanPipeline([SaeSlot("key", [key_saes[0]], cfg.key.k, chunk)])
+        for c in range(rcfg.scan.L // chunk):
+            rpipe.scan_chunk(c * chunk, {"key": [xs[c % n_distinct]["key"][0]]})
+        rpipe.finish()
+        csr = stage_index_on_device(rpipe.slots[0].index, dev)
+        L_idx = rcfg.scan.L
+        ns = C.n_spans(L_idx, rcfg.width, rcfg.stride)
+        xqry = inp.retrieval_queries(0, rcfg.Q, rcfg.nq)
+        q_ids = torch.empty((rcfg.Q * rcfg.nq, rcfg.kq), dtype=torch.int32, device=dev)
+        q_vals = torch.empty((rcfg.Q * rcfg.nq, rcfg.kq), dtype=torch.float32, device=dev)
+        q_ws = S.new_workspace(key_saes[0].encode_workspace_bytes(rcfg.Q * rcfg.nq, rcfg.kq), dev)
+        s_ws = S.new_workspace(S.s3_score_workspace_bytes(rcfg.Q, rcfg.nq, rcfg.kq, 1, ns, rcfg.s), dev)
+        bm25 = G.gamma21(rcfg.bm25_seed, rcfg.Q, ns).to(dev)
+        top_idx = torch.empty((rcfg.Q, rcfg.s), dtype=torch.int32, device=dev)
+        top_score = torch.empty((rcfg.Q, rcfg.s), dtype=torch.float32, device=dev)
+        top_idx_h = torch.empty((rcfg.Q, rcfg.s), dtype=torch.int32).pin_memory()
 
-    def retrieval(xqry_in):
-        S.s3_sae_encode_topk(key_saes[0], xqry_in, rcfg.kq, q_ids, q_vals, q_ws)
-        S.s3_coactivation_score_topspans(csr, cfg.key.d_sae, L_idx, q_ids.view(1, rcfg.Q, rcfg.nq, rcfg.kq),
-                                         q_vals.view(1, rcfg.Q, rcfg.nq, rcfg.kq), rcfg.width, rcfg.stride, rcfg.s,
-                                         rcfg.alpha, rcfg.beta, s_ws, bm25, top_idx=top_idx, top_score=top_score)
-        launches[0] += 3
-
-    def step(i, xk_c, xq_c, timed_kernel=False, xqry_in=None):
-        if timed_kernel:
-            # the dominant kernel (query-SAE encode) is bracketed by events on the launching stream
-            pipe_scan_with_events(i, xk_c, xq_c)
-        else:
-            pipe.scan_chunk(i * chunk, {"key": xk_c, "query": xq_c})
-        retrieval(xqry if xqry_in is None else xqry_in)
-
-    def pipe_scan_with_events(i, xk_c, xq_c):
-        orig = S.binding.s3_sae_encode_topk
-
-        def wrapped(sae, x, k, ids, vals, ws, stream=None):
-            if sae.d_in == cfg.query.d_in:
+        def retrieval(xqry_in, timed=False):
+            S.s3_sae_encode_topk(key_saes[0], xqry_in, rcfg.kq, q_ids, q_vals, q_ws)
+            if timed:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-                orig(sae, x, k, ids, vals, ws, stream)
+            S.s3_coactivation_score_topspans(csr, cfg.key.d_sae, L_idx, q_ids.view(1, rcfg.Q, rcfg.nq, rcfg.kq),
+                                             q_vals.view(1, rcfg.Q, rcfg.nq, rcfg.kq), rcfg.width, rcfg.stride, rcfg.s,
+                                             rcfg.alpha, rcfg.beta, s_ws, bm25, top_idx=top_idx, top_score=top_score)
+            if timed:
                 e1.record()
-                enc_events.append((e0, e1))
-            else:
-                orig(sae, x, k, ids, vals, ws, stream)
-        import paper_2601_17702_b200.scan as scan_mod
-        scan_mod.B.s3_sae_encode_topk = wrapped
-        try:
-            pipe.scan_chunk(i * chunk, {"key": xk_c, "query": xq_c})
-        finally:
-            scan_mod.B.s3_sae_encode_topk = orig
+                timers.setdefault("score", []).append((e0, e1))
+            launches[0] += 2 + S.SCORE_LAUNCHES
+
+        # algorithmic bytes of the scoring call: every (query, unique feature) pair gathers its list once
+        retrieval(xqry)
+        lens = (csr[0][0][1:] - csr[0][0][:-1])
+        gathered = 0
+        for q in range(rcfg.Q):
+            f = q_ids.view(rcfg.Q, -1)[q].long()
+            gathered += int(lens[torch.unique(f[f >= 0])].sum().item())
+        score_bytes = gathered * 4 + rcfg.Q * ns * 4 + rcfg.Q * rcfg.s * 8
+
+    def step(i, x_c, timed=False, xqry_in=None, append=True):
+        pipe.timers = timers if timed else None
+        pipe.scan_chunk(i * chunk, x_c, append=append)
+        if retrieval is not None:
+            retrieval(xqry if xqry_in is None else xqry_in, timed)
 
     def barrier():
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
-                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
-    if rank == 0:
-        sampler.start()
     # ---- device-resident timing (inputs already in HBM)
     for i in range(args.warmup):
-        step(i, xk[i % n_distinct], xq[i % n_distinct])
+        step(i, xs[i % n_distinct])
     barrier()
     torch.cuda.reset_peak_memory_stats()
     mem_after_warm = torch.cuda.memory_allocated()
+    free_after_warm = torch.cuda.mem_get_info()[0]
     l0 = pipe.launches + launches[0]
     wall0 = time.time()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for j in range(args.steps):
         i = args.warmup + j
-        step(i, xk[i % n_distinct], xq[i % n_distinct], timed_kernel=True)
+        step(i, xs[i % n_distinct], timed=True)
     t1.record()
+    host_enqueue_s = time.time() - wall0            # the host is done queueing here; the device is still working
     barrier()
+    wall1 = time.time()
     ms = t0.elapsed_time(t1)
-    clocks = sampler.stop(wall0, time.time()) if rank == 0 else None
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
     gpu_launches = pipe.launches + launches[0] - l0
     peak_mem = torch.cuda.max_memory_allocated()
-    enc_ms = [a.elapsed_time(b) for a, b in enc_events]
+    free_after_run = torch.cuda.mem_get_info()[0]
+    kernel_ms = {name: mean_ms(p) for name, p in timers.items()}
+    n_timed = {name: len(p) for name, p in timers.items()}
+    pipe.timers = None
     pipe.finish()
-    assert S.s3_workspace_status(q_ws) == 0 and S.s3_workspace_status(s_ws) == 0
+    if retrieval is not None:
+        assert S.s3_workspace_status(q_ws) == 0 and S.s3_workspace_status(s_ws) == 0
 
     ms = max_over_ranks(ms, world, dev)
     value = whole_job_rate(chunk, args.steps, world, ms * 1e-3)
 
+    # ---- the same steps without the hand-over to the host index: what the appends cost on top of the device work
+    base = args.warmup + args.steps
+    barrier()
+    t0.record()
+    for j in range(args.steps):
+        step(base + j, xs[(base + j) % n_distinct], append=False)
+    t1.record()
+    barrier()
+    ms_noappend = t0.elapsed_time(t1)
+    d2h_index = sum(nl * (chunk * s.k * 4 + (s.d_sae + 1) * 4) for s in slots)
+    pinned = torch.empty(d2h_index, dtype=torch.uint8).pin_memory()
+    devbuf = torch.empty(d2h_index, dtype=torch.uint8, device=dev)
+    pinned.copy_(devbuf, non_blocking=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(4):
+        pinned.copy_(devbuf, non_blocking=True)
+    t1.record()
+    torch.cuda.synchronize()
+    d2h_alone_ms = t0.elapsed_time(t1) / 4
+    del pinned, devbuf
+    exposed_ms = max(0.0, (ms - ms_noappend) / args.steps)
+
     # ---- end to end: the step's inputs come from pinned host memory, its result goes back to the host
     n_host = min(4, n_distinct)
-    xk_h = [[t.cpu().pin_memory() for t in xk[c]] for c in range(n_host)]
-    xq_h = [[t.cpu().pin_memory() for t in xq[c]] for c in range(n_host)]
+    x_h = [{n: [t.cpu().pin_memory() for t in ts] for n, ts in xs[c].items()} for c in range(n_host)]
     # two sets of device input buffers: while a step computes on one, the next step's inputs are copied into the
     # other on a copy stream (events order buffer reuse), so the PCIe transfer hides behind the encodes
-    xk_d = [[torch.empty_like(t) for t in xk[0]] for _ in range(2)]
-    xq_d = [[torch.empty_like(t) for t in xq[0]] for _ in range(2)]
-    xqry_d = [torch.empty_like(xqry) for _ in range(2)]
-    h2d = sum(t.numel() * t.element_size() for t in xk_h[0] + xq_h[0]) + xqry.numel() * xqry.element_size()
-    xqry_h = xqry.cpu().pin_memory()
-    d2h = top_idx_h.numel() * 4
+    x_d = [{n: [torch.empty_like(t) for t in ts] for n, ts in xs[0].items()} for _ in range(2)]
+    h2d = sum(t.numel() * t.element_size() for ts in x_h[0].values() for t in ts)
+    d2h = 0
+    if retrieval is not None:
+        xqry_d = [torch.empty_like(xqry) for _ in range(2)]
+        xqry_h = xqry.cpu().pin_memory()
+        h2d += xqry.numel() * xqry.element_size()
+        d2h = top_idx_h.numel() * 4
+    else:
+        stats_h = torch.empty(8, dtype=torch.int32).pin_memory()     # the scan's per-step result: the last list offsets
+        d2h = stats_h.numel() * 4
     copy_stream = torch.cuda.Stream(device=dev)
     ready = [torch.cuda.Event() for _ in range(2)]      # inputs of the buffer set have arrived
     consumed = [torch.cuda.Event() for _ in range(2)]   # the step that read the buffer set has finished
@@ -256,10 +340,11 @@ def run_ours(args, rank, world, local_rank):
         b, c = i % 2, i % n_host
         with torch.cuda.stream(copy_stream):
             copy_stream.wait_event(consumed[b])
-            for l in range(nl):
-                xk_d[b][l].copy_(xk_h[c][l], non_blocking=True)
-                xq_d[b][l].copy_(xq_h[c][l], non_blocking=True)
-            xqry_d[b].copy_(xqry_h, non_blocking=True)
+            for n, ts in x_h[c].items():
+                for l, t in enumerate(ts):
+                    x_d[b][n][l].copy_(t, non_blocking=True)
+            if retrieval is not None:
+                xqry_d[b].copy_(xqry_h, non_blocking=True)
             ready[b].record(copy_stream)
 
     def e2e_step(i, last):
@@ -267,12 +352,14 @@ def run_ours(args, rank, world, local_rank):
         if not last:
             e2e_upload(i + 1)                           # next step's inputs travel while this step computes
         torch.cuda.current_stream().wait_event(ready[b])
-        step(i, xk_d[b], xq_d[b], xqry_in=xqry_d[b])
+        step(i, x_d[b], xqry_in=xqry_d[b] if retrieval is not None else None)
         consumed[b].record()
-        top_idx_h.copy_(top_idx, non_blocking=True)
+        if retrieval is not None:
+            top_idx_h.copy_(top_idx, non_blocking=True)
+        else:
+            stats_h.copy_(slots[0].row_ptr[0][-8:], non_blocking=True)
 
-    base = args.warmup + args.steps
-    e2e_steps = max(2, min(args.steps, 8))
+    base = args.warmup + 2 * args.steps
     for b in range(2):
         consumed[b].record()
     e2e_upload(base)
@@ -290,48 +377,74 @@ def run_ours(args, rank, world, local_rank):
 
     if rank != 0:
         return None
-    enc_avg_ms = sum(enc_ms) / len(enc_ms)
-    flops = 2.0 * chunk * cfg.query.d_in * cfg.query.d_sae
+    # dominant kernel: the encode with the most FLOPs (the query SAE where there is one)
+    dom = slots[-1]
+    shp = cfg.query if cfg.query else cfg.key
+    enc_avg_ms = kernel_ms["encode_" + dom.name]
+    flops = 2.0 * chunk * shp.d_in * shp.d_sae
     tflops = flops / (enc_avg_ms * 1e-3) / 1e12
-    peak = peaks["bf16_tflops_sustained"]
+    peak, peak_source = pick_tensor_peak(peaks, ms * 1e-3)
+    post_bytes = sum(nl * (chunk * s.k * 8 + (s.d_sae + 1) * 4) for s in slots)
+    post_gbs = post_bytes / (kernel_ms["postings"] * 1e-3) / 1e9
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": workload_config(cfg, rcfg, L_idx, ns),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "note": "every step's activations are copied from pinned host memory (double-buffered on a copy stream, overlapping the previous step's kernels) and the selected spans are read back, all inside the timed region; postings also travel device->host (index append) in both numbers"},
+                "steps": e2e_steps, "note": "every step's activations are copied from pinned host memory (double-buffered on a copy stream, overlapping the previous step's kernels) and the step's result is read back, all inside the timed region; postings also travel device->host (index append) in both numbers"},
         "gpu_launches": gpu_launches,
         "clocks": clocks,
-        "roofline": {"bound": "tensor", "kernel": "encode_tc_kernel (query SAE 4096->32768, k=64, T=8192; duration includes the Top-k merge kernel)",
-                     "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
-                     "peak_source": f"{peaks['source']} sustained bf16 matmul", "frac_of_burst": tflops / peaks["bf16_tflops"],
-                     "frac_of_nominal_2250": tflops / 2250.0, "launch_ms": enc_avg_ms, "launches_timed": len(enc_ms),
-                     # dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of this kernel (ncu, one pass,
-                     # two launches: 1.29 + 0.07 and 1.40 + 0.07 GB); compulsory bytes are 0.34 GB (W_enc^T once + x)
-                     "traffic": ENCODE_QUERY_DRAM_BYTES, "traffic_unit": "bytes per launch"},
-        "device_mem": {"allocated_after_warmup_mib": mem_after_warm / 2**20, "peak_in_timed_region_mib": peak_mem / 2**20},
+        "roofline": {"bound": "tensor", "kernel": f"encode_tc_kernel ({dom.name} SAE {shp.d_in}->{shp.d_sae}, k={shp.k}, T={chunk}; duration includes the Top-k merge kernel)",
+                     "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak, "peak_source": peak_source,
+                     "frac_of_measured_burst": tflops / peaks["bf16_tflops"], "frac_of_measured_sustained": tflops / peaks["bf16_tflops_sustained"],
+                     "frac_of_nominal_2250": tflops / 2250.0, "launch_ms": enc_avg_ms, "launches_timed": n_timed["encode_" + dom.name],
+                     # dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of this kernel (ncu, one pass);
+                     # null when the kernel has changed since the counters were taken or the workload has no capture
+                     "traffic": ENCODE_QUERY_DRAM_BYTES if args.workload == "cfg3" else None, "traffic_unit": "bytes per launch"},
+        "roofline_postings": {"bound": "hbm", "kernel": "postings_partition_kernel + postings_bucket_kernel (all chunk-layers of a step in one batch)",
+                              "achieved": post_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": post_gbs / peaks["hbm_gbs"],
+                              "frac_of_nominal_8000": post_gbs / 8000.0, "peak_source": f"{peaks['source']} copy bandwidth",
+                              "bytes_per_launch": post_bytes, "launch_ms": kernel_ms["postings"], "launches_timed": n_timed["postings"],
+                              "traffic": None},
+        "append_overlap": {"ms_per_step": ms / args.steps, "ms_per_step_without_append": ms_noappend / args.steps,
+                           "index_d2h_bytes_per_step": d2h_index, "d2h_alone_ms": d2h_alone_ms, "exposed_ms_per_step": exposed_ms,
+                           "hidden_frac": 1.0 - min(1.0, exposed_ms / d2h_alone_ms)},
+        "host": {"syncs_in_chunk_loop": pipe.host_syncs, "enqueue_ms_per_step": host_enqueue_s * 1e3 / args.steps,
+                 "note": "the host queued all timed steps in enqueue_ms_per_step each, ahead of the device (ms_per_step): nothing in the loop waits for the GPU"},
+        "kernel_ms_in_step": kernel_ms,
+        "device_mem": {"allocated_after_warmup_mib": mem_after_warm / 2**20, "peak_in_timed_region_mib": peak_mem / 2**20,
+                       "cudaMemGetInfo_free_delta_bytes": free_after_warm - free_after_run},
     }
+    if retrieval is not None:
+        sc_gbs = score_bytes / (kernel_ms["score"] * 1e-3) / 1e9
+        out["roofline_scoring"] = {"bound": "hbm", "kernel": "span scoring + fusion + top-s (index L2-resident: gathered bytes, not DRAM bytes)",
+                                   "achieved": sc_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": sc_gbs / peaks["hbm_gbs"],
+                                   "frac_of_nominal_8000": sc_gbs / 8000.0, "peak_source": f"{peaks['source']} copy bandwidth",
+                                   "bytes_per_launch": score_bytes, "gathered_postings": gathered, "launch_ms": kernel_ms["score"],
+                                   "launches_timed": n_timed["score"], "traffic": None}
     return out
 
 
 # ------------------------------------------------------------------------------------------ oracle arm
 
-def oracle_step(n_tok, seed_row, cfg, inp_cpu, weights, rcfg):
+def oracle_step(n_tok, seed_row, cfg, inp_cpu, weights):
     """One bounded sample of the workload through the CPU oracle: n_tok tokens through every layer's key
-    and query SAE (encode, Top-k, postings), then one query scored against the sample's own postings."""
+    (and query) SAE (encode, Top-k, postings), then one query scored against the sample's own postings."""
     import numpy as np
     import oracle as O
     ids_key = []
     for l in range(cfg.n_layers):
         for which, shp in (("key", cfg.key), ("query", cfg.query)):
+            if shp is None:
+                continue
             W, b_enc, b_dec = weights[(which, l)]
             x = inp_cpu.x(which, l, seed_row, n_tok).float().numpy()
             ids, vals = O.encode_topk(x, W, b_enc, b_dec, shp.k)
             O.postings(ids, shp.d_sae, seed_row)
             if which == "key":
                 ids_key.append(ids)
-    w = min(rcfg.width, n_tok)
+    w = min(64, n_tok)
     q = ids_key[0][: min(n_tok, 4)]
     co = O.score_spans(ids_key[0][None], q[None, None], np.ones(q.shape, np.float32)[None, None], cfg.key.d_sae, w, max(1, w // 4), 0)
     O.fuse_select(co, None, 1.0, 0.0, 1)
@@ -339,31 +452,33 @@ def oracle_step(n_tok, seed_row, cfg, inp_cpu, weights, rcfg):
 
 def run_reference(args, cpu_only_sample=None):
     import oracle as O
-    cfg, rcfg = C.CFG3, C.CFG4
+    cfg, rcfg = WORKLOADS[args.workload]
     inp = C.ScanInputs(cfg, device="cpu")
     weights = {}
     for l in range(cfg.n_layers):
-        for which in ("key", "query"):
+        for which in ("key", "query") if cfg.query else ("key",):
             W, b_enc, b_dec = inp.sae(which, l)
             weights[(which, l)] = (W.float().numpy(), b_enc.numpy(), b_dec.numpy())
     n_tok = cpu_only_sample or 16
     steps, warm = (1, 0) if cpu_only_sample else (args.steps, min(args.warmup, 1))
     for i in range(warm):
-        oracle_step(n_tok, i * n_tok, cfg, inp, weights, rcfg)
+        oracle_step(n_tok, i * n_tok, cfg, inp, weights)
     t0 = time.perf_counter()
     for i in range(steps):
-        oracle_step(n_tok, (warm + i) * n_tok, cfg, inp, weights, rcfg)
+        oracle_step(n_tok, (warm + i) * n_tok, cfg, inp, weights)
     dt = time.perf_counter() - t0
     value = steps * n_tok / dt
     cores = O.num_threads()
-    sample = (f"{n_tok} context tokens per step through all {cfg.n_layers} layers' key and query SAEs (encode, Top-k, postings) "
+    sample = (f"{n_tok} context tokens per step through all {cfg.n_layers} layers' SAEs (encode, Top-k, postings) "
               f"plus one query scored on the sample; {steps} steps")
     if cpu_only_sample:
-        return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+        return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": dt}
+    L_idx = rcfg.scan.L if rcfg else None
+    ns = C.n_spans(L_idx, rcfg.width, rcfg.stride) if rcfg else None
     return {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": warm,
             "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic", "impl": "reference",
-            "config": workload_config(cfg, rcfg, rcfg.scan.L, C.n_spans(rcfg.scan.L, rcfg.width, rcfg.stride)),
+            "config": workload_config(cfg, rcfg, L_idx, ns),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
@@ -410,6 +525,7 @@ def run_case(args):
         # retrieval scoring alone: a random index of L tokens (k ids per token out of D features) as one
         # merged CSR, Q queries of nq tokens with kq ids each; bytes = gathered postings + lexical scores + outputs
         r = C.CFG4
+        nQ = args.queries or nQ
         L = args.tokens or r.scan.L
         k, D = (r.scan.key.k, r.scan.key.d_sae) if not args.tokens else (16, 8192)
         stride = r.stride if not args.tokens else 64
@@ -429,15 +545,15 @@ def run_case(args):
         rp, ps, _ = ix.export_csr(0)
         csr = [(rp.to(dev), ps.to(dev))]
         ix.close()
-        q_ids = torch.rand((r.Q * r.nq, D), device=dev, generator=g).topk(r.kq, dim=1).indices.to(torch.int32).view(1, r.Q, r.nq, r.kq)
+        q_ids = torch.rand((nQ * r.nq, D), device=dev, generator=g).topk(r.kq, dim=1).indices.to(torch.int32).view(1, nQ, r.nq, r.kq)
         q_vals = torch.ones(q_ids.shape, dtype=torch.float32, device=dev)
         ns = C.n_spans(L, r.width, stride)
-        bm25 = G.gamma21(r.bm25_seed, r.Q, ns).to(dev)
-        top_idx = torch.empty((r.Q, r.s), dtype=torch.int32, device=dev)
-        top_score = torch.empty((r.Q, r.s), dtype=torch.float32, device=dev)
+        bm25 = G.gamma21(r.bm25_seed, nQ, ns).to(dev)
+        top_idx = torch.empty((nQ, r.s), dtype=torch.int32, device=dev)
+        top_score = torch.empty((nQ, r.s), dtype=torch.float32, device=dev)
         lens = (csr[0][0][1:] - csr[0][0][:-1])
         gathered = 0
-        for q in range(r.Q):
+        for q in range(nQ):
             gathered += int(lens[torch.unique(q_ids[0, q].flatten().long())].sum().item())
         run = lambda i: S.s3_coactivation_score_topspans(csr, D, L, q_ids, q_vals, r.width, stride, r.s, r.alpha, r.beta, ws,
                                                          bm25, top_idx=top_idx, top_score=top_score)
@@ -458,8 +574,8 @@ def run_case(args):
             torch.cuda.synchronize()
             out.update(compact_bytes=comp.nbytes(), compact_build_ms=e0.elapsed_time(e1),
                        same_result=bool(torch.equal(ref_idx, top_idx) and torch.equal(ref_score, top_score)))
-        out.update(L=L, d_sae=D, k=k, Q=r.Q, nq=r.nq, kq=r.kq, spans=ns, stride=stride, gathered_postings=gathered,
-                   index_bytes=int(ps.numel()) * 4, bytes=gathered * 4 + r.Q * ns * 4 + r.Q * r.s * 8)
+        out.update(L=L, d_sae=D, k=k, Q=nQ, nq=r.nq, kq=r.kq, spans=ns, stride=stride, gathered_postings=gathered,
+                   index_bytes=int(ps.numel()) * 4, bytes=gathered * 4 + nQ * ns * 4 + nQ * r.s * 8)
     elif args.case == "heads":
         # per-head SAE as in Sec. 3.3 (x in R^d_head, one feature-ID space): the key SAE's dictionary width and k with
         # d_head = 128 inputs, 8 KV heads per token, then head aggregation back to k features per token
@@ -602,23 +718,63 @@ def run_case(args):
     print(json.dumps(out), flush=True)
 
 
+def spawn_ranks(args) -> int:
+    """`python bench.py --gpus N` without a launcher around it: N child processes of this script, one per GPU, with the
+    rendezvous variables a launcher would set (127.0.0.1). Rank 0's JSON line is the output; returns the worst exit code."""
+    import socket
+    with socket.socket() as sck:
+        sck.bind(("127.0.0.1", 0))
+        port = sck.getsockname()[1]
+    procs = []
+    for r in range(args.gpus):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(args.gpus), LOCAL_WORLD_SIZE=str(args.gpus),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    return max(abs(p.wait()) for p in procs)
+
+
+def run_stub(args, rank, world):
+    """The launch, barrier and max-over-ranks plumbing of a multi-rank run with a sleep in place of the GPU step
+    (backend gloo, no GPU): what the CPU tests drive."""
+    def step():
+        time.sleep(0.002 * (rank + 1))
+    for _ in range(args.warmup):
+        step()
+    torch.distributed.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    torch.distributed.barrier()
+    slowest = max_over_ranks(dt, world)
+    if rank != 0:
+        return None
+    return {"metric": METRIC, "value": whole_job_rate(1, args.steps, world, slowest), "unit": "stub steps/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": slowest / args.steps * 1e3, "impl": "stub"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads | train | project (--k = output width)")
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS), help="cfg3 = the 128K-token 4-layer key+query scan the metric is quoted on (default); cfg5 = the 1M-token 8-layer Zipf scan; cfg2 = the 32K-token one-layer scan")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)
     ap.add_argument("--items", type=int, default=8)
     ap.add_argument("--k", type=int, default=0, help="heads case: Top-k per head and per token (default: the key SAE's)")
+    ap.add_argument("--queries", type=int, default=0, help="score case: number of queries (default: the retrieval workload's 256)")
     ap.add_argument("--fp32-forward", action="store_true", help="train case: fp32 FFMA forward pass instead of the bf16 one")
     ap.add_argument("--compact", action="store_true", help="score case: read the block-delta compact index")
     ap.add_argument("--no-union", action="store_true", help="density case: leave out the index-set union; heads case: leave out the aggregation")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=96)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "stub"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-tokens", type=int, default=2048, help="context tokens the CPU oracle is timed on for cpu_baseline")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.case:
+        sys.exit(spawn_ranks(args))               # no launcher around us: start the ranks ourselves
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -631,12 +787,19 @@ def main():
         if rank == 0:
             print(json.dumps(run_reference(args)), flush=True)
         return
+    if args.impl == "stub":
+        torch.distributed.init_process_group("gloo")
+        out = run_stub(args, rank, world)
+        if rank == 0:
+            print(json.dumps(out), flush=True)
+        torch.distributed.destroy_process_group()
+        return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     out = run_ours(args, rank, world, local_rank)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            out["cpu_baseline"] = run_reference(args, cpu_only_sample=512)
+            out["cpu_baseline"] = run_reference(args, cpu_only_sample=args.cpu_sample_tokens)
         print(json.dumps(out), flush=True)
     if world > 1:
         torch.distributed.destroy_process_group()

@@ -18,6 +18,7 @@ S3_BF16, S3_F32 = 0, 1
 S3_SCORE_MINCOUNT, S3_SCORE_WEIGHTED = 0, 1
 S3_WS_HEADER_BYTES = 64
 S3_STATIC_SCRATCH_BYTES = 16 << 20
+SCORE_LAUNCHES = 1            # kernels one span-scoring call enqueues
 
 EXPORTS = [
     "s3_last_error", "s3_version", "s3_workspace_status",

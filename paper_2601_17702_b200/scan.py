@@ -4,6 +4,8 @@ them to the host-resident index. It only sequences calls of the C ABI on torch-o
 memory is allocated once, for one chunk, and reused for every chunk of the context."""
 from __future__ import annotations
 
+import contextlib
+
 import torch
 
 from . import binding as B
@@ -34,14 +36,28 @@ class ScanPipeline:
         n_post = sum(B.s3_postings_workspace_bytes(s.chunk, s.k, s.d_sae) for s in slots) * self.n_layers
         self.ws_post = B.new_workspace(n_post, slots[0].ids[0].device)
         self.launches = 0          # kernels of this library enqueued so far
+        self.timers = None         # when set to a dict: name -> list of (start, end) CUDA events around each call
+        self.host_syncs = 0        # host-blocking calls made by scan_chunk (none: ordering is by stream and events)
+
+    @contextlib.contextmanager
+    def _timed(self, name: str):
+        if self.timers is None:
+            yield
+            return
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        yield
+        e1.record()
+        self.timers.setdefault(name, []).append((e0, e1))
 
     def reserve_index(self, n_tokens: int):
         for s in self.slots:
             per_layer = n_tokens * s.k * (8 if s.pval else 4) + (n_tokens // s.chunk + 2) * (s.d_sae + 1 + 64) * 4
             s.index.reserve(per_layer * self.n_layers + (1 << 20))
 
-    def scan_chunk(self, pos_base: int, x_by_slot: dict[str, list[torch.Tensor]]):
-        """x_by_slot[name][layer] is the [T, d_in] projection of this chunk for that SAE stream."""
+    def scan_chunk(self, pos_base: int, x_by_slot: dict[str, list[torch.Tensor]], append: bool = True):
+        """x_by_slot[name][layer] is the [T, d_in] projection of this chunk for that SAE stream. append=False leaves
+        out the hand-over to the host index (to time the device work without the copies)."""
         items = []
         T = None
         for s in self.slots:
@@ -49,7 +65,8 @@ class ScanPipeline:
             for l in range(self.n_layers):
                 x = xs[l]
                 T = x.shape[0]
-                B.s3_sae_encode_topk(s.saes[l], x, s.k, s.ids[l][:T], s.vals[l][:T], s.ws)
+                with self._timed("encode_" + s.name):
+                    B.s3_sae_encode_topk(s.saes[l], x, s.k, s.ids[l][:T], s.vals[l][:T], s.ws)
                 self.launches += 2
                 items.append(B.make_postings_item(s.ids[l][:T], s.d_sae, pos_base, s.row_ptr[l], s.pos[l],
                                                   s.vals[l][:T] if s.pval else None, s.pval[l] if s.pval else None))
@@ -57,8 +74,11 @@ class ScanPipeline:
         for s in self.slots:
             s.index.stream_wait()
         for i in range(0, len(items), 32):
-            B.s3_postings_build_batched(items[i:i + 32], self.ws_post)
+            with self._timed("postings"):
+                B.s3_postings_build_batched(items[i:i + 32], self.ws_post)
             self.launches += 2         # partition by bucket, bucket sort
+        if not append:
+            return
         for s in self.slots:
             for l in range(self.n_layers):
                 s.index.append(l, s.row_ptr[l], s.pos[l], T, s.k, pos_base, s.pval[l] if s.pval else None)
