@@ -34,9 +34,9 @@ sys.path.insert(0, ROOT)
 from workloads import configs as C, generators as G  # noqa: E402
 
 METRIC = "scanned tokens/s (SAE Top-k encode + postings) at 128K ctx"
-# Measured DRAM traffic of one query-SAE encode launch at the benchmark's size (see profiles/); set to None when
-# the encode kernel changes until the counters are taken again.
-ENCODE_QUERY_DRAM_BYTES = 1.41e9
+# Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, ncu) of one grouped encode launch of the benchmark
+# step (see profiles/); None when the encode kernel has changed since the counters were taken.
+ENCODE_DRAM_BYTES = {}          # (workload, timer name) -> bytes per launch
 UNIT = "tokens/s"
 
 
@@ -196,7 +196,7 @@ def run_ours(args, rank, world, local_rank):
     slots = [SaeSlot("key", key_saes, cfg.key.k, chunk)]
     if cfg.query:
         slots.append(SaeSlot("query", [S.Sae(*inp.sae("query", l)) for l in range(nl)], cfg.query.k, chunk))
-    pipe = ScanPipeline(slots)
+    pipe = ScanPipeline(slots, grouped=args.group)
     e2e_steps = max(2, min(args.steps, 8))
     total_steps = 2 * args.steps + args.warmup + e2e_steps + 4
     pipe.reserve_index((total_steps + 2) * chunk)
@@ -377,11 +377,31 @@ def run_ours(args, rank, world, local_rank):
 
     if rank != 0:
         return None
-    # dominant kernel: the encode with the most FLOPs (the query SAE where there is one)
-    dom = slots[-1]
-    shp = cfg.query if cfg.query else cfg.key
-    enc_avg_ms = kernel_ms["encode_" + dom.name]
-    flops = 2.0 * chunk * shp.d_in * shp.d_sae
+    # dominant kernel: the encode launch kind that carries the most FLOPs of a step (a grouped launch over layers and SAE
+    # streams, a grouped launch over one stream's layers, or single launches)
+    shapes = {s.name: (cfg.key if s.name == "key" else cfg.query) for s in slots}
+    best = None
+    for name in kernel_ms:
+        if not name.startswith("encode"):
+            continue
+        per_step = n_timed[name] / args.steps
+        if name == "encode_group":
+            fl_step = sum(nl * 2.0 * chunk * sh.d_in * sh.d_sae for sh in shapes.values())
+            desc = f"grouped launch over the {nl} layers of {' + '.join(shapes)} SAEs"
+        elif name.startswith("encode_group_"):
+            sh = shapes[name[len("encode_group_"):]]
+            fl_step = nl * 2.0 * chunk * sh.d_in * sh.d_sae
+            desc = f"grouped launch over the {nl} layers' {name[len('encode_group_'):]} SAEs {sh.d_in}->{sh.d_sae}, k={sh.k}"
+        else:
+            sh = shapes[name[len("encode_"):]]
+            fl_step = nl * 2.0 * chunk * sh.d_in * sh.d_sae
+            desc = f"{name[len('encode_'):]} SAE {sh.d_in}->{sh.d_sae}, k={sh.k}, one launch per layer"
+        if best is None or fl_step > best[0]:
+            best = (fl_step, name, per_step, desc)
+    fl_step, enc_name, per_step, desc = best
+    flops = fl_step / per_step
+    enc_avg_ms = kernel_ms[enc_name]
+    enc_desc = f"encode_tc_kernel, {desc} (T={chunk}; {per_step:g} launch(es) per step; duration includes the Top-k merge kernel)"
     tflops = flops / (enc_avg_ms * 1e-3) / 1e12
     peak, peak_source = pick_tensor_peak(peaks, ms * 1e-3)
     post_bytes = sum(nl * (chunk * s.k * 8 + (s.d_sae + 1) * 4) for s in slots)
@@ -395,13 +415,13 @@ def run_ours(args, rank, world, local_rank):
                 "steps": e2e_steps, "note": "every step's activations are copied from pinned host memory (double-buffered on a copy stream, overlapping the previous step's kernels) and the step's result is read back, all inside the timed region; postings also travel device->host (index append) in both numbers"},
         "gpu_launches": gpu_launches,
         "clocks": clocks,
-        "roofline": {"bound": "tensor", "kernel": f"encode_tc_kernel ({dom.name} SAE {shp.d_in}->{shp.d_sae}, k={shp.k}, T={chunk}; duration includes the Top-k merge kernel)",
+        "roofline": {"bound": "tensor", "kernel": enc_desc,
                      "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak, "peak_source": peak_source,
                      "frac_of_measured_burst": tflops / peaks["bf16_tflops"], "frac_of_measured_sustained": tflops / peaks["bf16_tflops_sustained"],
-                     "frac_of_nominal_2250": tflops / 2250.0, "launch_ms": enc_avg_ms, "launches_timed": n_timed["encode_" + dom.name],
+                     "frac_of_nominal_2250": tflops / 2250.0, "launch_ms": enc_avg_ms, "launches_timed": n_timed[enc_name], "flop_per_launch": flops,
                      # dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of this kernel (ncu, one pass);
                      # null when the kernel has changed since the counters were taken or the workload has no capture
-                     "traffic": ENCODE_QUERY_DRAM_BYTES if args.workload == "cfg3" else None, "traffic_unit": "bytes per launch"},
+                     "traffic": ENCODE_DRAM_BYTES.get((args.workload, enc_name)), "traffic_unit": "bytes per launch"},
         "roofline_postings": {"bound": "hbm", "kernel": "postings_partition_kernel + postings_bucket_kernel (all chunk-layers of a step in one batch)",
                               "achieved": post_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": post_gbs / peaks["hbm_gbs"],
                               "frac_of_nominal_8000": post_gbs / 8000.0, "peak_source": f"{peaks['source']} copy bandwidth",
@@ -771,6 +791,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference", "stub"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--group", default="auto", help="how a chunk's encodes are launched: all | slot | none | <stream name> | auto")
     ap.add_argument("--cpu-sample-tokens", type=int, default=2048, help="context tokens the CPU oracle is timed on for cpu_baseline")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.case:

@@ -46,6 +46,7 @@ typedef enum { S3_BF16 = 0, S3_F32 = 1 } s3_dtype;
 
 #define S3_MAX_K 128           /* largest Top-k per token                                           */
 #define S3_MAX_POSTINGS_ITEMS 32
+#define S3_MAX_ENCODE_ITEMS 8    /* encoder calls one grouped launch can serve                        */
 #define S3_MAX_SCORE_LAYERS 16
 #define S3_WS_HEADER_BYTES 64
 
@@ -104,6 +105,32 @@ s3_status s3_sae_preact(const s3_sae* sae, const void* d_x, int64_t ldx, int T, 
  * and the largest number of thread blocks a launch may use (0 = all SMs). Results do not depend on
  * either. */
 s3_status s3_sae_set_schedule(s3_sae* sae, int n_slices, int max_ctas);
+
+/* ------------------------------------------------------------------------------------------------
+ * Grouped SAE encode + Top-k            (paper Alg. 1 Phase 1: inside each chunk the scan loops over the
+ *                                        target layers, `for l in TargetLayers: feats <- E_l.encode(K_l)`;
+ *                                        Sec. 3.3 / 3.4: one SAE per target layer)
+ *
+ * Up to S3_MAX_ENCODE_ITEMS independent encoder calls (the layers' key SAEs of one chunk, key and query SAEs
+ * together, ...) as ONE persistent launch followed by one selection launch: the work units of all items are
+ * dealt out over the SMs by their modelled duration, so the SMs stay busy across items of unequal size and
+ * the launch ends evenly. Each item has its own encoder, input, T, k and outputs; the results are those of
+ * s3_sae_encode_topk item by item (bit-identical: the selection is exact, whatever the schedule).
+ * bf16 encoders only (S3_ERR_UNSUPPORTED otherwise); an item with T == 0 is skipped. `h_items` is a HOST
+ * array. Workspace: s3_sae_encode_grouped_workspace_bytes(h_items, n_items) (status block + every item's
+ * candidate lists).
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    const s3_sae* sae;
+    const void* d_x;     /* [T, d_in] with row pitch ldx */
+    int64_t ldx;
+    int32_t T, k;
+    int32_t* d_ids;      /* [T,k] */
+    float* d_vals;       /* [T,k] */
+} s3_encode_item;
+
+size_t s3_sae_encode_grouped_workspace_bytes(const s3_encode_item* h_items, int n_items);
+s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items, void* d_ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * SAE encode + ReLU + Top-k without any caller-provided scratch

@@ -17,6 +17,7 @@ S3_ERR_CAPACITY, S3_ERR_TIMEOUT, S3_ERR_STATE = -5, -6, -7
 S3_BF16, S3_F32 = 0, 1
 S3_SCORE_MINCOUNT, S3_SCORE_WEIGHTED = 0, 1
 S3_WS_HEADER_BYTES = 64
+S3_MAX_ENCODE_ITEMS = 8
 S3_STATIC_SCRATCH_BYTES = 16 << 20
 SCORE_LAUNCHES = 1            # kernels one span-scoring call enqueues
 
@@ -24,6 +25,7 @@ EXPORTS = [
     "s3_last_error", "s3_version", "s3_workspace_status",
     "s3_sae_prepared_bytes", "s3_sae_create", "s3_sae_destroy", "s3_sae_encode_workspace_bytes",
     "s3_sae_encode_topk", "s3_sae_set_schedule", "s3_sae_encode_topk_static",
+    "s3_sae_encode_grouped_workspace_bytes", "s3_sae_encode_topk_grouped",
     "s3_postings_workspace_bytes", "s3_postings_build", "s3_postings_build_batched",
     "s3_index_create", "s3_index_reserve", "s3_index_append", "s3_index_stream_wait", "s3_index_sync",
     "s3_index_stats", "s3_index_layer_postings", "s3_index_export_csr", "s3_index_destroy",
@@ -47,6 +49,11 @@ class PostingsItem(C.Structure):
     _fields_ = [("d_ids", C.c_void_p), ("d_vals", C.c_void_p), ("T", C.c_int32), ("k", C.c_int32),
                 ("d_sae", C.c_int32), ("reserved", C.c_int32), ("pos_base", C.c_int64),
                 ("d_row_ptr", C.c_void_p), ("d_pos", C.c_void_p), ("d_pval", C.c_void_p)]
+
+
+class EncodeItem(C.Structure):
+    _fields_ = [("sae", C.c_void_p), ("d_x", C.c_void_p), ("ldx", C.c_int64), ("T", C.c_int32), ("k", C.c_int32),
+                ("d_ids", C.c_void_p), ("d_vals", C.c_void_p)]
 
 
 class CsrView(C.Structure):
@@ -97,7 +104,7 @@ def lib():
         L.s3_last_error.restype = C.c_char_p
         for name in ("s3_sae_prepared_bytes", "s3_sae_encode_workspace_bytes", "s3_postings_workspace_bytes",
                      "s3_score_workspace_bytes", "s3_density_workspace_bytes", "s3_fuse_workspace_bytes",
-                     "s3_compact_workspace_bytes", "s3_sae_backward_workspace_bytes"):
+                     "s3_compact_workspace_bytes", "s3_sae_backward_workspace_bytes", "s3_sae_encode_grouped_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.s3_sae_prepared_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_sae_create.argtypes = [C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
@@ -109,6 +116,8 @@ def lib():
                                          C.c_void_p, C.c_size_t, C.c_void_p]
         L.s3_sae_encode_topk_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_void_p,
                                                 C.c_void_p, C.c_void_p, C.c_void_p]
+        L.s3_sae_encode_grouped_workspace_bytes.argtypes = [C.POINTER(EncodeItem), C.c_int]
+        L.s3_sae_encode_topk_grouped.argtypes = [C.POINTER(EncodeItem), C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
         L.s3_workspace_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
         L.s3_postings_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_postings_build.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_void_p,
@@ -239,6 +248,26 @@ def s3_sae_encode_topk(sae: Sae, x: torch.Tensor, k: int, ids: torch.Tensor, val
     assert tuple(ids.shape) == (T, k) and tuple(vals.shape) == (T, k)
     _check(lib().s3_sae_encode_topk(sae.handle, _ptr(x), x.stride(0) if T > 1 else max(x.stride(0), sae.d_in), T, k,
                                     _ptr(ids), _ptr(vals), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def make_encode_item(sae: Sae, x: torch.Tensor, k: int, ids: torch.Tensor, vals: torch.Tensor) -> EncodeItem:
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1 and x.shape[1] == sae.d_in
+    T = x.shape[0]
+    assert ids.dtype == torch.int32 and vals.dtype == torch.float32 and ids.is_contiguous() and vals.is_contiguous()
+    assert tuple(ids.shape) == (T, k) and tuple(vals.shape) == (T, k)
+    return EncodeItem(sae.handle, x.data_ptr(), x.stride(0) if T > 1 else max(x.stride(0), sae.d_in), T, k, ids.data_ptr(),
+                      vals.data_ptr())
+
+
+def s3_sae_encode_grouped_workspace_bytes(items: list[EncodeItem]) -> int:
+    arr = (EncodeItem * max(len(items), 1))(*items)
+    return int(lib().s3_sae_encode_grouped_workspace_bytes(arr, len(items)))
+
+
+def s3_sae_encode_topk_grouped(items: list[EncodeItem], ws: torch.Tensor, stream=None):
+    """Several encoder calls (make_encode_item) as one persistent launch plus one selection launch."""
+    arr = (EncodeItem * max(len(items), 1))(*items)
+    _check(lib().s3_sae_encode_topk_grouped(arr, len(items), _ptr(ws), ws.numel(), _stream(stream)))
 
 
 def s3_sae_encode_topk_static(sae: Sae, x: torch.Tensor, k: int, ids: torch.Tensor, vals: torch.Tensor,

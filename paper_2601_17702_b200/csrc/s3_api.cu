@@ -227,6 +227,60 @@ s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, in
     return S3_OK;
 }
 
+static s3_status check_encode_item(const s3_encode_item& it, int idx)
+{
+    S3_REQUIRE(it.sae != nullptr, S3_ERR_INVALID_ARG, "item %d: sae is null", idx);
+    S3_REQUIRE(it.sae->dtype == S3_BF16, S3_ERR_UNSUPPORTED, "item %d: the grouped launch takes bf16 encoders only", idx);
+    S3_REQUIRE(it.T >= 0, S3_ERR_INVALID_ARG, "item %d: T = %d is negative", idx, it.T);
+    S3_REQUIRE(it.k >= 1 && it.k <= it.sae->d_sae, S3_ERR_INVALID_ARG, "item %d: k = %d out of range [1, d_sae = %d]", idx, it.k,
+               it.sae->d_sae);
+    S3_REQUIRE(it.k <= S3_MAX_K, S3_ERR_UNSUPPORTED, "item %d: k = %d exceeds the supported maximum %d", idx, it.k, S3_MAX_K);
+    if (it.T == 0) return S3_OK;
+    S3_REQUIRE(it.d_x && it.d_ids && it.d_vals, S3_ERR_INVALID_ARG, "item %d: null device pointer", idx);
+    S3_REQUIRE(aligned16(it.d_x) && (reinterpret_cast<uintptr_t>(it.d_ids) & 3) == 0 && (reinterpret_cast<uintptr_t>(it.d_vals) & 3) == 0,
+               S3_ERR_INVALID_ARG, "item %d: misaligned device pointer", idx);
+    S3_REQUIRE(it.ldx >= it.sae->d_in && it.ldx % 8 == 0, S3_ERR_INVALID_ARG, "item %d: ldx = %lld must be a multiple of 8 and >= d_in",
+               idx, (long long)it.ldx);
+    return S3_OK;
+}
+
+size_t s3_sae_encode_grouped_workspace_bytes(const s3_encode_item* h_items, int n_items)
+{
+    if (!h_items || n_items < 0) return 0;
+    size_t n = 256;
+    for (int i = 0; i < n_items; ++i) {
+        const s3_encode_item& it = h_items[i];
+        if (!it.sae || it.sae->dtype != S3_BF16 || it.T <= 0 || it.k < 1) continue;
+        n += encode_tc_workspace_bytes(it.T, pick_slices(it.sae, it.T), it.k);
+    }
+    return n;
+}
+
+s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items, void* d_ws, size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(n_items >= 0, S3_ERR_INVALID_ARG, "n_items is negative");
+    if (n_items == 0) return S3_OK;
+    S3_REQUIRE(h_items != nullptr, S3_ERR_INVALID_ARG, "h_items is null");
+    S3_REQUIRE(n_items <= S3_MAX_ENCODE_ITEMS, S3_ERR_UNSUPPORTED, "n_items = %d exceeds %d", n_items, S3_MAX_ENCODE_ITEMS);
+    S3_REQUIRE(d_ws != nullptr && aligned16(d_ws), S3_ERR_INVALID_ARG, "d_ws is null or misaligned");
+    EncodeTcItem items[S3_MAX_ENCODE_ITEMS];
+    int n = 0, max_ctas = 0;
+    for (int i = 0; i < n_items; ++i) {
+        const s3_status st = check_encode_item(h_items[i], i);
+        if (st != S3_OK) return st;
+        const s3_encode_item& it = h_items[i];
+        if (it.T == 0) continue;
+        items[n++] = EncodeTcItem{&it.sae->tc, it.d_x, it.ldx, it.T, it.sae->d_in, it.sae->d_sae, it.k, pick_slices(it.sae, it.T),
+                                  it.d_ids, it.d_vals};
+        if (it.sae->max_ctas > 0 && (max_ctas == 0 || it.sae->max_ctas < max_ctas)) max_ctas = it.sae->max_ctas;
+    }
+    if (n == 0) return S3_OK;
+    const size_t need = s3_sae_encode_grouped_workspace_bytes(h_items, n_items);
+    S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
+    return launch_encode_tc_group(items, n, max_ctas, static_cast<unsigned char*>(d_ws) + 256, static_cast<uint32_t*>(d_ws),
+                                  static_cast<cudaStream_t>(stream));
+}
+
 s3_status s3_sae_preact(const s3_sae* sae, const void* d_x, int64_t ldx, int T, void* d_out, int64_t ld_out, s3_dtype out_dtype,
                         void* d_ws, size_t ws_bytes, void* stream)
 {

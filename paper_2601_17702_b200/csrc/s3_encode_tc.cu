@@ -32,6 +32,7 @@
 // and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <string.h>
 
 #include "s3_kernels.cuh"
 #include "s3_topk.cuh"
@@ -189,19 +190,60 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
                                 (static_cast<uint32_t>(PAIR_M >> 4) << 24);
 
-struct EncodeTcParams {
-    int T, d_in, d_sae, k;
-    int n_mtiles, n_col_tiles, n_slices, n_units, n_stages;
+constexpr int MAX_GROUP = S3_MAX_ENCODE_ITEMS;   // encoders one launch can serve
+constexpr int MAX_SCHED = 1024;                  // work units a launch can deal out by table
+constexpr int MAX_PAIRS = 96;                    // CTA pairs the table has room for
+
+// One encoder call of a grouped launch.
+struct ItemParams {
+    int T, d_in, k, kblocks;
+    int n_mtiles, n_col_tiles, n_slices;
+    int unit_start;            // first work unit of this item in the launch's flattened unit list
     uint32_t cap;              // candidate-list slots per (token, slice)
     const float* b_eff;
     uint64_t* cand;            // [T][n_slices][cap]
     uint32_t* counts;          // [T][n_slices]
     uint32_t* hint;            // [T] float bits of the best published bound
-    void* dense_out;           // dense mode: the pre-activations [T, ld_out], fp32 or bf16
-    long long ld_out;
-    int out_bf16;
-    uint32_t* status;
 };
+
+struct EncodeTcParams {
+    int n_items, n_units, n_stages;
+    int use_sched;             // 1: pair p runs units sched[pair_start[p] .. pair_start[p+1]); 0: units p, p + n_pairs, ...
+    uint32_t* status;
+    void* dense_out;           // dense mode (one item): the pre-activations [T, ld_out], fp32 or bf16
+    long long ld_out;
+    int out_bf16, d_sae;
+    ItemParams item[MAX_GROUP];
+    uint16_t pair_start[MAX_PAIRS + 1];
+    uint16_t sched[MAX_SCHED];
+};
+
+struct TensorMaps {
+    CUtensorMap x[MAX_GROUP];
+    CUtensorMap w[MAX_GROUP];
+};
+
+// The units of one CTA pair, in the order every role of both CTAs walks them.
+struct UnitWalk {
+    int i, end, step;
+};
+__device__ __forceinline__ UnitWalk unit_walk(const EncodeTcParams& p, int pair, int n_pairs)
+{
+    UnitWalk w;
+    if (p.use_sched) { w.i = p.pair_start[pair]; w.end = p.pair_start[pair + 1]; w.step = 1; }
+    else { w.i = pair; w.end = p.n_units; w.step = n_pairs; }
+    return w;
+}
+// Unit -> (item, column slice, row tile).
+__device__ __forceinline__ void unit_decode(const EncodeTcParams& p, const UnitWalk& w, int& item, int& slice, int& mt)
+{
+    const int u = p.use_sched ? static_cast<int>(p.sched[w.i]) : w.i;
+    item = p.n_items - 1;
+    while (item > 0 && p.item[item].unit_start > u) --item;
+    const int local = u - p.item[item].unit_start;
+    slice = local / p.item[item].n_mtiles;
+    mt = local - slice * p.item[item].n_mtiles;
+}
 
 // Shared-memory carve-up (all offsets from a 1024-byte aligned base).
 struct SmemLayout {
@@ -326,8 +368,7 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
 // the kernel is the same pipeline.
 template <bool DENSE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
-encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                 const EncodeTcParams p)
+encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant__ EncodeTcParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -344,7 +385,6 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int kblocks = (p.d_in + BK - 1) / BK;
     const uint32_t cta_rank = cluster_cta_rank();          // 0 = first CTA of the pair: issues the MMAs, owns the
     const bool first_cta = cta_rank == 0;                  // barriers that both CTAs signal (full, acc_empty)
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
@@ -373,15 +413,22 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
+            for (int j = 0; j < p.n_items; ++j) {
+                asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.x[j])) : "memory");
+                asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.w[j])) : "memory");
+            }
             uint32_t stage = 0, phase = 0;
             uint64_t issued = 0;
             bool ok = true;
-            for (int u = pair; u < p.n_units && ok; u += n_pairs) {
-                const int slice = u / p.n_mtiles, mt = u - slice * p.n_mtiles;
-                const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
-                const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
+            for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
+                int item, slice, mt;
+                unit_decode(p, uw, item, slice, mt);
+                const ItemParams& ip = p.item[item];
+                const CUtensorMap* map_x = &maps.x[item];
+                const CUtensorMap* map_w = &maps.w[item];
+                const int kblocks = ip.kblocks;
+                const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
+                const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
                 const int row0 = mt * PAIR_M + static_cast<int>(cta_rank) * BM;        // this CTA's tokens
                 for (int nt = tile_lo; nt < tile_hi && ok; ++nt) {
                     const int col0 = nt * BN + static_cast<int>(cta_rank) * (BN / 2);  // this CTA's half of the features
@@ -394,8 +441,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         }
                         if (first_cta) mbar_expect_tx(&full_bar[stage], 2 * STAGE_BYTES);
                         const uint32_t full_addr = map_to_cta(smem_u32(&full_bar[stage]), 0);
-                        tma_load_2d(smem_a + stage * A_STAGE_BYTES, &map_x, kb * BK, row0, full_addr);
-                        tma_load_2d(smem_b + stage * B_STAGE_BYTES, &map_w, kb * BK, col0, full_addr);
+                        tma_load_2d(smem_a + stage * A_STAGE_BYTES, map_x, kb * BK, row0, full_addr);
+                        tma_load_2d(smem_b + stage * B_STAGE_BYTES, map_w, kb * BK, col0, full_addr);
                         ++issued;
                         if (++stage == static_cast<uint32_t>(p.n_stages)) { stage = 0; phase ^= 1u; }
                     }
@@ -417,10 +464,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             uint32_t stage = 0, phase = 0;
             uint32_t tile_count = 0;
             bool ok = true;
-            for (int u = pair; u < p.n_units && ok; u += n_pairs) {
-                const int slice = u / p.n_mtiles;
-                const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
-                const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
+            for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
+                int item, slice, mt;
+                unit_decode(p, uw, item, slice, mt);
+                const ItemParams& ip = p.item[item];
+                const int kblocks = ip.kblocks;
+                const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
+                const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
                 for (int nt = tile_lo; nt < tile_hi && ok; ++nt, ++tile_count) {
                     const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
                     if (!mbar_wait(&acc_empty[ab], acc_phase ^ 1u, abort_flag)) {
@@ -462,19 +512,23 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         bool ok = true;
         // the accumulator is handed back on the first CTA's barrier
         const uint32_t acc_empty_addr[2] = {map_to_cta(smem_u32(&acc_empty[0]), 0), map_to_cta(smem_u32(&acc_empty[1]), 0)};
-        for (int u = pair; u < p.n_units && ok; u += n_pairs) {
-            const int slice = u / p.n_mtiles, mt = u - slice * p.n_mtiles;
-            const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * p.n_col_tiles / p.n_slices);
-            const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * p.n_col_tiles / p.n_slices);
+        for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
+            int item, slice, mt;
+            unit_decode(p, uw, item, slice, mt);
+            const ItemParams& ip = p.item[item];
+            const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
+            const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
             const int t = mt * PAIR_M + static_cast<int>(cta_rank) * BM + e;
-            const bool live = t < p.T;
-            uint64_t* glist = DENSE ? nullptr : p.cand + (static_cast<size_t>(live ? t : 0) * p.n_slices + slice) * p.cap;
+            const bool live = t < ip.T;
+            const int k = ip.k;
+            const uint32_t cap = ip.cap;
+            uint64_t* glist = DENSE ? nullptr : ip.cand + (static_cast<size_t>(live ? t : 0) * ip.n_slices + slice) * cap;
             if (!DENSE) {
 #pragma unroll 1
                 for (int sl = 0; sl < NB; ++sl) my_hist[sl * EPI_THREADS] = 0;
             }
             // start from the best bound another slice of these rows has published so far, if any
-            const uint32_t hint_in = (live && !DENSE) ? *reinterpret_cast<volatile const uint32_t*>(p.hint + t) : 0u;
+            const uint32_t hint_in = (live && !DENSE) ? *reinterpret_cast<volatile const uint32_t*>(ip.hint + t) : 0u;
             RowSel r;
             r.tau_floor = live ? __uint_as_float(hint_in) : INFINITY;    // rows past T select nothing
             r.tau = r.tau_floor;
@@ -492,7 +546,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (!__all_sync(0xffffffffu, arrived)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ab * BN + (static_cast<uint32_t>(quarter * 32) << 16);
-                const float4* bias4 = reinterpret_cast<const float4*>(p.b_eff + static_cast<size_t>(nt) * BN);
+                const float4* bias4 = reinterpret_cast<const float4*>(ip.b_eff + static_cast<size_t>(nt) * BN);
                 if (!DENSE && nt == tile_lo && __any_sync(0xffffffffu, live && r.tau == 0.0f)) {
                     // Cold start: without a bound every second value of the unit's first tile would go through the pending
                     // lists. A first pass over that tile only counts, per row, how many of its values exceed each of
@@ -530,7 +584,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         float bound = 0.0f;
 #pragma unroll
                         for (int lv = COLD_LEVELS - 1; lv >= 0; --lv)
-                            if (seen[lv] >= p.k && level[lv] > bound) bound = level[lv];       // levels descend with lv ascending
+                            if (seen[lv] >= k && level[lv] > bound) bound = level[lv];       // levels descend with lv ascending
                         r.tau_floor = r.tau = bound;
                     }
                 }
@@ -595,14 +649,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             slot[o3 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[3])) << 32) | (nc - 3u);
                             cnt += o3 + keep[3];
                         }
-                        if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) fold_pending(my_pend, my_hist, glist, r, cnt, p.k, p.cap);
+                        if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) fold_pending(my_pend, my_hist, glist, r, cnt, k, cap);
                     }
                 }
                 tc_fence_before();
                 mbar_arrive_cluster(acc_empty_addr[ab]);
             }
             if (ok && !DENSE) {
-                if (__any_sync(0xffffffffu, cnt > 0)) fold_pending(my_pend, my_hist, glist, r, cnt, p.k, p.cap);
+                if (__any_sync(0xffffffffu, cnt > 0)) fold_pending(my_pend, my_hist, glist, r, cnt, k, cap);
                 if (live) {
                     // The bound to publish: at least k values of this slice exceed it. An exact k-th value
                     // only bounds from below after stepping to the next float down.
@@ -622,8 +676,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         for (int q = 0; q < 16; ++q)
                             if (__uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > cut) glist[w++] = key[q];
                     }
-                    p.counts[static_cast<size_t>(t) * p.n_slices + slice] = w;
-                    if (out > hint_in) atomicMax(p.hint + t, out);
+                    ip.counts[static_cast<size_t>(t) * ip.n_slices + slice] = w;
+                    if (out > hint_in) atomicMax(ip.hint + t, out);
                 }
             }
         }
@@ -762,43 +816,81 @@ int encode_tc_min_slices(int d_sae) { return (encode_tc_col_tiles(d_sae) + 254) 
 size_t encode_tc_workspace_bytes(int T, int n_slices, int k)
 {
     const size_t t = static_cast<size_t>(T), s = static_cast<size_t>(n_slices);
-    return round_up(t * 4, 256) + round_up(t * s * 4, 256) + t * s * encode_tc_list_cap(k) * sizeof(uint64_t);
+    return round_up(t * 4, 256) + round_up(t * s * 4, 256) + round_up(t * s * encode_tc_list_cap(k) * sizeof(uint64_t), 256);
 }
 
 namespace {
 
-// Common launch of the two epilogue modes. Selection: d_scratch / d_ids / d_vals set, d_dense null. Dense: the reverse.
-s3_status launch_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k, int n_slices,
-                    int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals, void* d_dense, int64_t ld_out,
-                    bool out_bf16, cudaStream_t stream)
+// Modelled duration of one work unit, in tensor-pipe cycles: per 256-column tile the MMAs of its k-blocks or, for
+// narrow inputs, the Top-k filter of its 256 columns, whichever is longer.
+double unit_cost(int kblocks, int tiles, int k)
+{
+    const double mma = 600.0 * kblocks, filter = 12000.0 + 100.0 * k;
+    return tiles * (mma > filter ? mma : filter);
+}
+
+// Common launch of the two epilogue modes. Selection: items with d_ids / d_vals, scratch carved from d_scratch.
+// Dense: one item, d_dense set.
+s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* d_scratch, uint32_t* d_status, void* d_dense,
+                    int64_t ld_out, bool out_bf16, cudaStream_t stream)
 {
     const bool dense = d_dense != nullptr;
-    alignas(64) CUtensorMap map_x;
-    s3_status rc = make_map(&map_x, d_x, static_cast<uint64_t>(T), static_cast<uint64_t>(d_in), static_cast<uint64_t>(ldx), BM);
-    if (rc != S3_OK) return rc;
-
+    S3_REQUIRE(n_items >= 1 && n_items <= MAX_GROUP, S3_ERR_UNSUPPORTED, "%d encoders in one launch, at most %d", n_items, MAX_GROUP);
+    alignas(64) TensorMaps maps;
     EncodeTcParams p;
-    p.T = T; p.d_in = d_in; p.d_sae = d_sae; p.k = k;
-    p.n_mtiles = encode_tc_row_tiles(T);
-    p.n_col_tiles = encode_tc_col_tiles(d_sae);
-    S3_REQUIRE(n_slices >= encode_tc_min_slices(d_sae), S3_ERR_INVALID_ARG, "d_sae = %d needs at least %d column slices", d_sae,
-               encode_tc_min_slices(d_sae));
-    p.n_slices = n_slices;
-    p.n_units = p.n_mtiles * n_slices;
-    p.cap = encode_tc_list_cap(k);
-    p.b_eff = st->d_b_eff;
+    memset(&p, 0, sizeof(p));
+    p.n_items = n_items;
     p.status = d_status;
     p.dense_out = d_dense; p.ld_out = ld_out; p.out_bf16 = out_bf16 ? 1 : 0;
-    p.hint = nullptr; p.counts = nullptr; p.cand = nullptr;
-    if (!dense) {
-        unsigned char* base = static_cast<unsigned char*>(d_scratch);
-        p.hint = reinterpret_cast<uint32_t*>(base);
-        p.counts = reinterpret_cast<uint32_t*>(base + round_up(static_cast<size_t>(T) * 4, 256));
-        p.cand = reinterpret_cast<uint64_t*>(base + round_up(static_cast<size_t>(T) * 4, 256) +
-                                             round_up(static_cast<size_t>(T) * n_slices * 4, 256));
-        // no bound is known for any row yet
-        S3_CUDA_TRY(cudaMemsetAsync(p.hint, 0, static_cast<size_t>(T) * 4, stream));
+    p.d_sae = items[0].d_sae;
+
+    // items in descending order of their units' modelled duration, so that the short units fill the end of the launch
+    int order[MAX_GROUP];
+    double cost[MAX_GROUP];
+    for (int j = 0; j < n_items; ++j) {
+        order[j] = j;
+        const int nct = encode_tc_col_tiles(items[j].d_sae);
+        cost[j] = unit_cost((items[j].d_in + BK - 1) / BK, (nct + items[j].n_slices - 1) / items[j].n_slices, items[j].k);
     }
+    for (int a = 1; a < n_items; ++a)
+        for (int b = a; b > 0 && cost[order[b]] > cost[order[b - 1]]; --b) { const int t = order[b]; order[b] = order[b - 1]; order[b - 1] = t; }
+
+    unsigned char* base = static_cast<unsigned char*>(d_scratch);
+    size_t hint_bytes = 0;
+    for (int j = 0; j < n_items; ++j) hint_bytes += round_up(static_cast<size_t>(items[j].T) * 4, 256);
+    size_t hint_off = 0, off = hint_bytes;
+    int n_units = 0;
+    for (int q = 0; q < n_items; ++q) {
+        const EncodeTcItem& it = items[order[q]];
+        ItemParams& ip = p.item[q];
+        s3_status rc = make_map(&maps.x[q], it.d_x, static_cast<uint64_t>(it.T), static_cast<uint64_t>(it.d_in),
+                                static_cast<uint64_t>(it.ldx), BM);
+        if (rc != S3_OK) return rc;
+        memcpy(&maps.w[q], it.st->map_w, sizeof(CUtensorMap));
+        ip.T = it.T; ip.d_in = it.d_in; ip.k = it.k;
+        ip.kblocks = (it.d_in + BK - 1) / BK;
+        ip.n_mtiles = encode_tc_row_tiles(it.T);
+        ip.n_col_tiles = encode_tc_col_tiles(it.d_sae);
+        S3_REQUIRE(it.n_slices >= encode_tc_min_slices(it.d_sae), S3_ERR_INVALID_ARG, "d_sae = %d needs at least %d column slices",
+                   it.d_sae, encode_tc_min_slices(it.d_sae));
+        ip.n_slices = it.n_slices;
+        ip.unit_start = n_units;
+        n_units += ip.n_mtiles * it.n_slices;
+        ip.cap = encode_tc_list_cap(it.k);
+        ip.b_eff = it.st->d_b_eff;
+        if (!dense) {
+            const size_t t = static_cast<size_t>(it.T), sl = static_cast<size_t>(it.n_slices);
+            ip.hint = reinterpret_cast<uint32_t*>(base + hint_off);
+            hint_off += round_up(t * 4, 256);
+            ip.counts = reinterpret_cast<uint32_t*>(base + off);
+            off += round_up(t * sl * 4, 256);
+            ip.cand = reinterpret_cast<uint64_t*>(base + off);
+            off += round_up(t * sl * ip.cap * sizeof(uint64_t), 256);
+        }
+    }
+    p.n_units = n_units;
+    // no bound is known for any row yet
+    if (!dense) S3_CUDA_TRY(cudaMemsetAsync(base, 0, hint_bytes, stream));
 
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
@@ -810,7 +902,6 @@ s3_status launch_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T
                "shared memory too small for the encode pipeline");
     p.n_stages = n_stages;
     const size_t smem = smem_layout(n_stages).total + 1024;
-    const CUtensorMap& map_w = *reinterpret_cast<const CUtensorMap*>(st->map_w);
     static bool attr_set[64] = {};
     if (dev < 64 && !attr_set[dev]) {
         S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
@@ -819,33 +910,82 @@ s3_status launch_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T
     }
     int n_pairs = encode_tc_max_pairs();
     if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
-    if (p.n_units < n_pairs) n_pairs = p.n_units;
+    if (n_units < n_pairs) n_pairs = n_units;
+
+    // Units dealt out by modelled duration: in the flattened order (item, slice, row tile) each unit goes to the pair
+    // with the least work so far. Pairs therefore still walk the same slice of the same encoder at about the same time
+    // (its W_enc^T tiles are shared in L2), and a launch over unequal encoders ends evenly. Equal units come out
+    // round-robin, which is what the walk without a table does.
+    p.use_sched = 0;
+    if (n_items > 1 && n_units <= MAX_SCHED && n_pairs <= MAX_PAIRS) {
+        static thread_local uint16_t unit_pair[MAX_SCHED];
+        double load[MAX_PAIRS];
+        int count[MAX_PAIRS];
+        for (int q = 0; q < n_pairs; ++q) { load[q] = 0.0; count[q] = 0; }
+        int u = 0;
+        for (int q = 0; q < n_items; ++q) {
+            const int units = p.item[q].n_mtiles * p.item[q].n_slices;
+            const double c = cost[order[q]];
+            for (int i = 0; i < units; ++i, ++u) {
+                int best = 0;
+                for (int r = 1; r < n_pairs; ++r)
+                    if (load[r] < load[best]) best = r;
+                load[best] += c;
+                unit_pair[u] = static_cast<uint16_t>(best);
+                ++count[best];
+            }
+        }
+        int run = 0;
+        for (int q = 0; q < n_pairs; ++q) { p.pair_start[q] = static_cast<uint16_t>(run); run += count[q]; }
+        p.pair_start[n_pairs] = static_cast<uint16_t>(run);
+        int fill[MAX_PAIRS];
+        for (int q = 0; q < n_pairs; ++q) fill[q] = p.pair_start[q];
+        for (int i = 0; i < n_units; ++i) p.sched[fill[unit_pair[i]]++] = static_cast<uint16_t>(i);
+        p.use_sched = 1;
+    }
+
     if (dense) {
-        encode_tc_kernel<true><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(map_x, map_w, p);
+        encode_tc_kernel<true><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
         S3_CUDA_TRY(cudaGetLastError());
         return S3_OK;
     }
-    encode_tc_kernel<false><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(map_x, map_w, p);
+    encode_tc_kernel<false><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
     S3_CUDA_TRY(cudaGetLastError());
-    launch_candidate_merge(p.cand, p.counts, p.hint, T, n_slices, p.cap, k, d_ids, d_vals, stream);
+    MergeGroup mg;
+    mg.n_items = n_items;
+    int rows = 0;
+    for (int q = 0; q < n_items; ++q) {
+        const EncodeTcItem& it = items[order[q]];
+        const ItemParams& ip = p.item[q];
+        mg.item[q] = MergeItem{ip.cand, ip.counts, ip.hint, it.d_ids, it.d_vals, it.T, it.n_slices, it.k, ip.cap, rows};
+        rows += (it.T + kMergeRowsPerBlock - 1) / kMergeRowsPerBlock * kMergeRowsPerBlock;
+    }
+    launch_candidate_merge_group(mg, rows, stream);
     S3_CUDA_TRY(cudaGetLastError());
     return S3_OK;
 }
 
 }  // namespace
 
+s3_status launch_encode_tc_group(const EncodeTcItem* items, int n_items, int max_ctas, void* d_scratch, uint32_t* d_status,
+                                 cudaStream_t stream)
+{
+    return launch_tc(items, n_items, max_ctas, d_scratch, d_status, nullptr, 0, false, stream);
+}
+
 s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
                            int n_slices, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals,
                            cudaStream_t stream)
 {
-    return launch_tc(st, d_x, ldx, T, d_in, d_sae, k, n_slices, max_ctas, d_scratch, d_status, d_ids, d_vals, nullptr, 0, false, stream);
+    const EncodeTcItem it = {st, d_x, ldx, T, d_in, d_sae, k, n_slices, d_ids, d_vals};
+    return launch_tc(&it, 1, max_ctas, d_scratch, d_status, nullptr, 0, false, stream);
 }
 
 s3_status launch_preact_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int n_slices,
                            int max_ctas, uint32_t* d_status, void* d_out, int64_t ld_out, bool out_bf16, cudaStream_t stream)
 {
-    return launch_tc(st, d_x, ldx, T, d_in, d_sae, 1, n_slices, max_ctas, nullptr, d_status, nullptr, nullptr, d_out, ld_out, out_bf16,
-                     stream);
+    const EncodeTcItem it = {st, d_x, ldx, T, d_in, d_sae, 1, n_slices, nullptr, nullptr};
+    return launch_tc(&it, 1, max_ctas, nullptr, d_status, d_out, ld_out, out_bf16, stream);
 }
 
 }  // namespace s3

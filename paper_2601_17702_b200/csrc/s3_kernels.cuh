@@ -25,6 +25,19 @@ s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx
                            int n_slices, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals,
                            cudaStream_t stream);
 
+// Several encoder calls in one persistent launch (each with its own encoder, input, k and outputs); scratch as the sum of
+// encode_tc_workspace_bytes over the items.
+struct EncodeTcItem {
+    const EncodeTcState* st;
+    const void* d_x;
+    int64_t ldx;
+    int T, d_in, d_sae, k, n_slices;
+    int32_t* d_ids;
+    float* d_vals;
+};
+s3_status launch_encode_tc_group(const EncodeTcItem* items, int n_items, int max_ctas, void* d_scratch, uint32_t* d_status,
+                                 cudaStream_t stream);
+
 // The same GEMM with a dense epilogue: pre-activations [T, ld_out] as fp32 or bf16.
 s3_status launch_preact_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int n_slices,
                            int max_ctas, uint32_t* d_status, void* d_out, int64_t ld_out, bool out_bf16, cudaStream_t stream);

@@ -45,6 +45,25 @@ void launch_topk_merge(const uint64_t* d_part, int T, int n_slices, int k, int32
 
 // Candidate lists of the tensor-core encode: cand[(t * n_slices + slice) * cap + i], i < counts[t * n_slices + slice],
 // unordered keys; hint[t] = float bits of a bound that at least k values of row t exceed.
+// The same for the candidate lists of several encoder calls in one launch; row_start = first row of the item in the
+// launch's flattened row range (a multiple of kMergeRowsPerBlock).
+constexpr int kMergeRowsPerBlock = 4;
+struct MergeItem {
+    const uint64_t* cand;
+    const uint32_t* counts;
+    const uint32_t* hint;
+    int32_t* ids;
+    float* vals;
+    int T, n_slices, k;
+    uint32_t cap;
+    int row_start;
+};
+struct MergeGroup {
+    MergeItem item[S3_MAX_ENCODE_ITEMS];
+    int n_items;
+};
+void launch_candidate_merge_group(const MergeGroup& g, int total_rows, cudaStream_t stream);
+
 void launch_candidate_merge(const uint64_t* d_cand, const uint32_t* d_counts, const uint32_t* d_hint, int T, int n_slices,
                             uint32_t cap, int k, int32_t* d_ids, float* d_vals, cudaStream_t stream);
 

@@ -7,7 +7,7 @@ namespace s3 {
 
 namespace {
 
-constexpr int kMergeWarps = 4;
+constexpr int kMergeWarps = kMergeRowsPerBlock;
 
 // One warp per token: bitonic sort (descending) of the token's n_slices*k keys, padded with zeros to
 // a power of two, in the warp's private shared-memory segment.
@@ -50,16 +50,25 @@ topk_merge_kernel(const uint64_t* __restrict__ part, int T, int n, int npad, int
 constexpr int kCandBuf = 1024;   // survivor slots per warp
 
 __global__ void __launch_bounds__(kMergeWarps * 32)
-candidate_merge_kernel(const uint64_t* __restrict__ cand, const uint32_t* __restrict__ counts,
-                       const uint32_t* __restrict__ hint, int T, int n_slices, uint32_t cap, int k,
-                       int32_t* __restrict__ ids, float* __restrict__ vals)
+candidate_merge_kernel(const __grid_constant__ MergeGroup g)
 {
     __shared__ uint64_t cand_buf[kMergeWarps][kCandBuf];
     __shared__ uint32_t cand_hist[kMergeWarps][64];
     __shared__ uint32_t cand_start[kMergeWarps][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t = blockIdx.x * kMergeWarps + warp;
-    if (t >= T) return;
+    const int row = blockIdx.x * kMergeWarps + warp;
+    int item = g.n_items - 1;
+    while (item > 0 && g.item[item].row_start > row) --item;
+    const MergeItem& mi = g.item[item];
+    const int t = row - mi.row_start;
+    if (t >= mi.T) return;
+    const uint64_t* __restrict__ cand = mi.cand;
+    const uint32_t* __restrict__ counts = mi.counts;
+    const uint32_t* __restrict__ hint = mi.hint;
+    int32_t* __restrict__ ids = mi.ids;
+    float* __restrict__ vals = mi.vals;
+    const int n_slices = mi.n_slices, k = mi.k;
+    const uint32_t cap = mi.cap;
     uint64_t* buf = cand_buf[warp];
     const float tau = __uint_as_float(hint[t]);
     uint32_t n = 0;            // survivors so far (warp-uniform)
@@ -214,12 +223,20 @@ void launch_topk_merge(const uint64_t* d_part, int T, int n_slices, int k, int32
     topk_merge_kernel<<<grid, kMergeWarps * 32, smem, stream>>>(d_part, T, n, npad, k, d_ids, d_vals);
 }
 
+void launch_candidate_merge_group(const MergeGroup& g, int total_rows, cudaStream_t stream)
+{
+    if (total_rows <= 0) return;
+    candidate_merge_kernel<<<total_rows / kMergeWarps, kMergeWarps * 32, 0, stream>>>(g);
+}
+
 void launch_candidate_merge(const uint64_t* d_cand, const uint32_t* d_counts, const uint32_t* d_hint, int T, int n_slices,
                             uint32_t cap, int k, int32_t* d_ids, float* d_vals, cudaStream_t stream)
 {
     if (T <= 0) return;
-    const int grid = (T + kMergeWarps - 1) / kMergeWarps;
-    candidate_merge_kernel<<<grid, kMergeWarps * 32, 0, stream>>>(d_cand, d_counts, d_hint, T, n_slices, cap, k, d_ids, d_vals);
+    MergeGroup g;
+    g.n_items = 1;
+    g.item[0] = MergeItem{d_cand, d_counts, d_hint, d_ids, d_vals, T, n_slices, k, cap, 0};
+    launch_candidate_merge_group(g, (T + kMergeWarps - 1) / kMergeWarps * kMergeWarps, stream);
 }
 
 }  // namespace s3

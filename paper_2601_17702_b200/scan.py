@@ -11,6 +11,13 @@ import torch
 from . import binding as B
 
 
+# "auto" grouping: the layers of an SAE stream share one launch when the encoder's input is this narrow (the launch is
+# then bound by the Top-k filter, and a grouped launch keeps every SM busy to its end). Wider encoders are bound by the
+# operand feed and the power cap; there a launch whose CTA pairs all walk ONE encoder's weights in step is faster
+# (measured on the 4096 -> 32768 query encoders: four layers in one launch take 14 % longer than four launches).
+AUTO_GROUP_MAX_D_IN = 1024
+
+
 class SaeSlot:
     """One SAE stream of the scan (e.g. 'key' or 'query'): per-layer encoders plus the chunk-sized
     device buffers its outputs go through."""
@@ -30,9 +37,20 @@ class SaeSlot:
 
 
 class ScanPipeline:
-    def __init__(self, slots: list[SaeSlot]):
+    def __init__(self, slots: list[SaeSlot], grouped: bool | str = "auto"):
+        """grouped: how the encodes of a chunk are launched (bf16 encoders; fp32 ones always go one by one).
+        True / "all": the layers of all SAE streams in grouped launches (one persistent kernel per up to
+        S3_MAX_ENCODE_ITEMS encoders); "slot": one grouped launch per SAE stream; a stream's name (e.g. "key"): only
+        that stream's layers are grouped; False / "none": one launch pair per encoder; "auto" (default): per stream,
+        grouped when the encoder input is at most AUTO_GROUP_MAX_D_IN wide."""
         self.slots = slots
         self.n_layers = len(slots[0].saes)
+        mode = {True: "all", False: "none"}.get(grouped, grouped)
+        self.auto = mode == "auto"
+        if not all(sae.dtype == B.S3_BF16 for s in slots for sae in s.saes):
+            mode = "none"
+        self.group_mode = mode
+        self.ws_enc = None         # workspace of the grouped encode, sized at the first chunk
         n_post = sum(B.s3_postings_workspace_bytes(s.chunk, s.k, s.d_sae) for s in slots) * self.n_layers
         self.ws_post = B.new_workspace(n_post, slots[0].ids[0].device)
         self.launches = 0          # kernels of this library enqueued so far
@@ -59,17 +77,35 @@ class ScanPipeline:
         """x_by_slot[name][layer] is the [T, d_in] projection of this chunk for that SAE stream. append=False leaves
         out the hand-over to the host index (to time the device work without the copies)."""
         items = []
+        enc_items = []
         T = None
         for s in self.slots:
             xs = x_by_slot[s.name]
             for l in range(self.n_layers):
                 x = xs[l]
                 T = x.shape[0]
-                with self._timed("encode_" + s.name):
-                    B.s3_sae_encode_topk(s.saes[l], x, s.k, s.ids[l][:T], s.vals[l][:T], s.ws)
-                self.launches += 2
+                if self.group_mode in ("all", "slot", s.name) or (self.auto and s.saes[l].d_in <= AUTO_GROUP_MAX_D_IN):
+                    enc_items.append((s.name, B.make_encode_item(s.saes[l], x, s.k, s.ids[l][:T], s.vals[l][:T])))
+                else:
+                    with self._timed("encode_" + s.name):
+                        B.s3_sae_encode_topk(s.saes[l], x, s.k, s.ids[l][:T], s.vals[l][:T], s.ws)
+                    self.launches += 2
                 items.append(B.make_postings_item(s.ids[l][:T], s.d_sae, pos_base, s.row_ptr[l], s.pos[l],
                                                   s.vals[l][:T] if s.pval else None, s.pval[l] if s.pval else None))
+        groups = []
+        for name, item in enc_items:
+            new_group = not groups or len(groups[-1][1]) == B.S3_MAX_ENCODE_ITEMS or (self.group_mode != "all" and groups[-1][0] != name)
+            if new_group:
+                groups.append((name, []))
+            groups[-1][1].append(item)
+        need = max((B.s3_sae_encode_grouped_workspace_bytes(g) for _, g in groups), default=0)
+        if groups and (self.ws_enc is None or self.ws_enc.numel() < need):
+            assert self.ws_enc is None, "the grouped-encode workspace is sized by the first (full) chunk"
+            self.ws_enc = B.new_workspace(need, self.slots[0].ids[0].device)
+        for name, group in groups:
+            with self._timed("encode_group" if self.group_mode == "all" else "encode_group_" + name):
+                B.s3_sae_encode_topk_grouped(group, self.ws_enc)
+            self.launches += 2         # persistent encode over all items, selection over all items
         # the previous chunk's device->host copies read row_ptr/pos: order the overwrite after them
         for s in self.slots:
             s.index.stream_wait()
@@ -88,6 +124,8 @@ class ScanPipeline:
             s.index.sync()
             code = B.s3_workspace_status(s.ws)
             assert code == 0
+        if self.ws_enc is not None:
+            assert B.s3_workspace_status(self.ws_enc) == 0
         assert B.s3_workspace_status(self.ws_post) == 0
 
     def close(self):

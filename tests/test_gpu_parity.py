@@ -532,3 +532,44 @@ def test_cfg1_scan_and_retrieval_end_to_end():
     pre = O.preact(x.numpy(), W.numpy(), b_enc.numpy(), b_dec.numpy())
     check_topk_against_preact(pre, ids_h, vals.cpu().numpy(), k, TOL_F32)
     ix.close()
+
+
+# ------------------------------------------------------------------------------------ grouped encode
+
+def test_grouped_encode_equals_the_single_calls_bit_for_bit():
+    """Several encoders of unequal shape, input length and k in one grouped launch (Alg. 1 Phase 1: the layers'
+    SAEs of one chunk): every item's ids and values are those of its own s3_sae_encode_topk call, and those match
+    the oracle. An empty item is skipped."""
+    d = dev()
+    shapes = [(700, 256, 4096, 32), (300, 1024, 8192, 64), (513, 128, 2048, 8), (0, 64, 512, 4), (1000, 512, 16384, 16),
+              (260, 64, 1024, 128), (90, 192, 1000, 16)]
+    saes, xs, xs_d, outs, items = [], [], [], [], []
+    for i, (T, d_in, d_sae, k) in enumerate(shapes):
+        W, b_enc, b_dec = G.sae_weights(300 + i, 0, d_in, d_sae, torch.bfloat16)
+        x = G.activations(400 + i, 0, 0, max(T, 1), d_in, torch.bfloat16)[:T]
+        sae = S.Sae(W.to(d), b_enc.to(d), b_dec.to(d))
+        ids = torch.full((T, k), -5, dtype=torch.int32, device=d)
+        vals = torch.full((T, k), -5.0, dtype=torch.float32, device=d)
+        saes.append((sae, W, b_enc, b_dec))
+        xs.append(x)
+        outs.append((ids, vals))
+        xs_d.append(x.to(d))
+        items.append(S.make_encode_item(sae, xs_d[-1], k, ids, vals))
+    ws = S.new_workspace(S.s3_sae_encode_grouped_workspace_bytes(items))
+    S.s3_sae_encode_topk_grouped(items, ws)
+    assert S.s3_workspace_status(ws) == 0
+    for (T, d_in, d_sae, k), (sae, W, b_enc, b_dec), x, (ids, vals) in zip(shapes, saes, xs, outs):
+        if T == 0:
+            continue
+        ids1, vals1 = gpu_encode(W, b_enc, b_dec, x, k)
+        np.testing.assert_array_equal(ids.cpu().numpy(), ids1)
+        np.testing.assert_array_equal(vals.cpu().numpy(), vals1)
+        pre = O.preact(x.float().numpy(), W.float().numpy(), b_enc.numpy(), b_dec.numpy())
+        check_topk_against_preact(pre, ids.cpu().numpy(), vals.cpu().numpy(), k, TOL_BF16)
+    # a second launch over the leftovers of the first gives the same bits
+    for ids, vals in outs:
+        ids.fill_(-9)
+    S.s3_sae_encode_topk_grouped(items, ws)
+    for (T, d_in, d_sae, k), (sae, W, b_enc, b_dec), x, (ids, vals) in zip(shapes, saes, xs, outs):
+        if T:
+            np.testing.assert_array_equal(ids.cpu().numpy(), gpu_encode(W, b_enc, b_dec, x, k)[0])
