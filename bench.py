@@ -545,7 +545,7 @@ def run_case(args):
         # retrieval scoring alone: a random index of L tokens (k ids per token out of D features) as one
         # merged CSR, Q queries of nq tokens with kq ids each; bytes = gathered postings + lexical scores + outputs
         r = C.CFG4
-        nQ = args.queries or nQ
+        nQ = args.queries or r.Q
         L = args.tokens or r.scan.L
         k, D = (r.scan.key.k, r.scan.key.d_sae) if not args.tokens else (16, 8192)
         stride = r.stride if not args.tokens else 64
@@ -575,7 +575,8 @@ def run_case(args):
         gathered = 0
         for q in range(nQ):
             gathered += int(lens[torch.unique(q_ids[0, q].flatten().long())].sum().item())
-        run = lambda i: S.s3_coactivation_score_topspans(csr, D, L, q_ids, q_vals, r.width, stride, r.s, r.alpha, r.beta, ws,
+        sws = S.new_workspace(S.s3_score_workspace_bytes(nQ, r.nq, r.kq, 1, ns, r.s), dev)
+        run = lambda i: S.s3_coactivation_score_topspans(csr, D, L, q_ids, q_vals, r.width, stride, r.s, r.alpha, r.beta, sws,
                                                          bm25, top_idx=top_idx, top_score=top_score)
         if args.compact:
             # the same index in block-delta form: build timed once, then the scorer decodes blocks in its gather
@@ -589,7 +590,7 @@ def run_case(args):
             ref_idx, ref_score = run(0)
             ref_idx, ref_score = ref_idx.clone(), ref_score.clone()
             run = lambda i: S.s3_coactivation_score_topspans_compact([comp], D, L, q_ids, q_vals, r.width, stride, r.s, r.alpha,
-                                                                     r.beta, ws, bm25, top_idx=top_idx, top_score=top_score)
+                                                                     r.beta, sws, bm25, top_idx=top_idx, top_score=top_score)
             run(0)
             torch.cuda.synchronize()
             out.update(compact_bytes=comp.nbytes(), compact_build_ms=e0.elapsed_time(e1),

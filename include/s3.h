@@ -255,7 +255,11 @@ s3_status s3_index_destroy(s3_index* index);
  *   mode S3_SCORE_MINCOUNT : base[q,j] = sum_l sum_f min(cQ_l(f), cS_l(f,j))          (integer, exact)
  *   mode S3_SCORE_WEIGHTED : base[q,j] = sum_l sum_f aQ_l(f) * IDF_l(f) * cS_l(f,j)   (Eq. 6 summed over
  *        the span; IDF(f) = 1/(ln(1+freq(f))+1), freq = the feature's posting-list length in layer l;
- *        features with freq > stop_freq are skipped when stop_freq > 0; accumulated in fp64)
+ *        features with freq > stop_freq are skipped when stop_freq > 0). The weights aQ*IDF (fp64) are
+ *        rounded to a fixed-point grid of at least 40 bits below the query's largest weight and summed as
+ *        integers, so the result does not depend on the order of the additions: it is identical from run
+ *        to run, and within 1e-5 (relative) of the fp64 sum whenever a span's weights lie within a factor
+ *        2^20 of the query's largest.
  * with cS_l(f,j) = number of postings of f inside span j.
  * Fusion: score = fl32(fl32(alpha*base) + fl32(beta*bm25[q,j])) (bm25 nullable: score = fl32(alpha*base)).
  * Output: the s best spans per query by (score descending, span index ascending); padded with
@@ -266,7 +270,12 @@ s3_status s3_index_destroy(s3_index* index);
  * Limits: n_layers <= S3_MAX_SCORE_LAYERS; nq*k <= 4096; n_spans <= 16384; s <= 64;
  *         width, stride >= 1. Per query the kernel keeps 4 (min-count) or 8 (weighted) bytes per span and
  *         about 28 bytes per query entry in shared memory; a combination beyond the SM's capacity
- *         (only weighted mode near both maxima) returns S3_ERR_UNSUPPORTED.
+ *         (only weighted mode near both maxima) returns S3_ERR_UNSUPPORTED. n_spans == 0 (L < width) writes
+ *         index -1 / score 0 for every query and reads no posting.
+ * Workspace: the status block is enough (then one thread block works on each query). With
+ *         s3_score_workspace_bytes(Q, ...) bytes a batch of few queries is cut over several blocks per query
+ *         (a single query runs on up to 148 of them); the blocks add their partial sums in the workspace,
+ *         which the call clears first. Results are the same either way.
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
     const uint64_t* d_row_ptr;

@@ -351,8 +351,8 @@ s3_status s3_postings_build(const int32_t* d_ids, const float* d_vals, int T, in
 // ---------------------------------------------------------------------------------------------- scoring
 size_t s3_score_workspace_bytes(int Q, int nq, int k, int n_layers, int n_spans, int s)
 {
-    (void)Q; (void)nq; (void)k; (void)n_layers; (void)n_spans; (void)s;
-    return S3_WS_HEADER_BYTES;
+    (void)nq; (void)k; (void)n_layers; (void)s;
+    return 256 + score_workspace_bytes(Q, n_spans);
 }
 
 }  // extern "C"
@@ -401,7 +401,7 @@ s3_status s3_coactivation_score_topspans(const s3_csr_view* h_layers, int n_laye
     for (int l = 0; l < n_layers; ++l)
         S3_REQUIRE(h_layers[l].d_row_ptr && (h_layers[l].d_pos || n_spans == 0), S3_ERR_INVALID_ARG, "layer %d: null CSR pointer", l);
     return launch_score(h_layers, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, (int)n_spans, p, d_bm25, ld_bm25, d_top_idx,
-                        d_top_score, d_all_scores, static_cast<cudaStream_t>(stream));
+                        d_top_score, d_all_scores, d_ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 s3_status s3_coactivation_score_topspans_compact(const s3_compact_view* h_layers, int n_layers, int d_sae, int64_t L,
@@ -419,7 +419,7 @@ s3_status s3_coactivation_score_topspans_compact(const s3_compact_view* h_layers
                        h_layers[l].d_payload,
                    S3_ERR_INVALID_ARG, "layer %d: null pointer in the compact view", l);
     return launch_score_compact(h_layers, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, (int)n_spans, p, d_bm25, ld_bm25,
-                                d_top_idx, d_top_score, d_all_scores, static_cast<cudaStream_t>(stream));
+                                d_top_idx, d_top_score, d_all_scores, d_ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 // ---------------------------------------------------------------------------------------------- compact index

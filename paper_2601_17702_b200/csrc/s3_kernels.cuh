@@ -52,15 +52,16 @@ s3_status launch_encode_simt(const float* d_x, int64_t ldx, const float* d_W, co
 size_t postings_workspace_bytes(int T, int k, int d_sae);   // table bytes of one item (multiple of 256)
 s3_status launch_postings(const s3_postings_item* h_items, int n_items, void* d_ws, size_t ws_bytes, cudaStream_t stream);
 
+size_t score_workspace_bytes(int Q, int n_spans);   // after the 256-byte head of the workspace: tickets + shared difference arrays
 s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
                        const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
                        const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
-                       float* d_all_scores, cudaStream_t stream);
+                       float* d_all_scores, void* d_ws, size_t ws_bytes, cudaStream_t stream);
 
 s3_status launch_score_compact(const s3_compact_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
                                const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
                                const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
-                               float* d_all_scores, cudaStream_t stream);
+                               float* d_all_scores, void* d_ws, size_t ws_bytes, cudaStream_t stream);
 void compact_bound(uint64_t n_postings, int d_sae, uint64_t* max_blocks, uint64_t* max_words);
 size_t compact_workspace_bytes(uint64_t n_postings, int d_sae);
 s3_status launch_compact_build(const uint64_t* d_row_ptr, const int32_t* d_pos, int d_sae, int64_t stop_freq,

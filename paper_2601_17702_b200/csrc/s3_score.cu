@@ -1,14 +1,20 @@
 // Query-time span scoring (Sec. 3.5, Eq. 5-6; appendix IDF definition) fused with score fusion and
-// top-s selection. One thread block per query:
+// top-s selection. A query is handled by one thread block or, when there are fewer queries than the GPU
+// has room for, by several blocks that each take a share of its posting lists:
 //   a. aggregate the query tokens' Top-k into unique features with cQ (token count) and aQ (summed
 //      activation): block bitonic sort of (id, entry) keys, then run detection;
-//   b. fetch the unique features' list bounds in one parallel sweep, cut all lists into 32-posting
-//      pieces and deal the pieces out evenly over the warps (a long list is simply many pieces, so
-//      skewed list lengths do not unbalance the block). Every posting works out by itself which
-//      spans it still adds to (see posting_range), for any width/stride. Min-count mode records the
-//      range as +1/-1 in a difference array that one prefix sum turns into min(cQ, cS) totals;
-//      weighted mode adds aQ*IDF to each span of the range in fp64;
-//   c. fuse with the lexical score vector and pick the s best spans (score desc, index asc).
+//   b. fetch the unique features' list bounds in one parallel sweep and cut all lists into 32-posting
+//      pieces (a long list is simply many pieces, so skewed list lengths do not unbalance anything). The
+//      block tabulates one 16-byte descriptor per piece of its share (where the piece starts, how many
+//      postings it has, cQ, the feature) and its warps walk the pieces, one broadcast descriptor load per
+//      piece. Every posting works out by itself which spans it still adds to (see posting_range), for any
+//      width/stride, and records the range as +w / -w in a difference array in shared memory that one
+//      prefix sum turns into per-span totals: w = 1 in min-count mode (totals are min(cQ, cS) sums), and in
+//      weighted mode w = aQ*IDF as a fixed-point integer whose unit is chosen per query from the largest
+//      weight, so that the sums are exact integers and do not depend on the order of the additions;
+//   c. fuse with the lexical score vector and pick the s best spans (score desc, index asc). With several
+//      blocks per query each adds its difference array to the query's array in the workspace; the block
+//      that arrives last (a ticket counter, nobody waits) finishes the query.
 #include "s3_kernels.cuh"
 #include "s3_query.cuh"
 
@@ -20,6 +26,18 @@ struct CompactLayers {
     s3_compact_view v[S3_MAX_SCORE_LAYERS];
 };
 constexpr int CBATCH = 8;        // compact index: blocks of 32 postings a warp decodes side by side
+constexpr int WINP = 1024;       // pieces whose descriptors are tabulated at a time
+constexpr int MAX_SPLIT = 148;   // blocks per query at most
+
+// One 32-posting piece of a posting list.
+struct PieceDesc {
+    unsigned long long start;    // raw CSR: index of the piece's first posting in pos; compact: its block index
+    uint32_t first_i;            // list index of the piece's first posting
+    uint32_t meta;               // postings in the piece (6 bits) | cQ << 6 (13 bits) | unique-feature index << 19
+};
+__device__ __forceinline__ uint32_t piece_count(uint32_t meta) { return meta & 63u; }
+__device__ __forceinline__ uint32_t piece_cq(uint32_t meta) { return (meta >> 6) & 0x1FFFu; }
+__device__ __forceinline__ uint32_t piece_owner(uint32_t meta) { return meta >> 19; }
 
 struct ScoreArgs {
     const int32_t* q_ids;
@@ -34,7 +52,30 @@ struct ScoreArgs {
     int64_t stop_freq;
     int stride_shift;   // log2(stride) when the stride is a power of two, else -1
     unsigned long long stride_magic;   // ceil(2^64 / stride) (stride >= 2)
+    int n_split;                       // blocks per query
+    unsigned long long* acc_g;         // [Q][n_spans + 2] sum of the blocks' difference arrays (n_split > 1), zeroed by the launcher
+    uint32_t* tickets;                 // [Q] blocks of the query that have added theirs, zeroed by the launcher
 };
+
+// Shared-memory carve-up, identical on host and device.
+struct ScoreLayout {
+    uint32_t acc_off, ulo_off, keys_off, ufeat_off, ustart_off, uaq_off, uw_off, table_off, total;
+};
+__host__ __device__ inline ScoreLayout score_layout(int nk, int npad, int n_spans, bool weighted)
+{
+    ScoreLayout L;
+    uint32_t o = 0;
+    L.acc_off = o;    o += (static_cast<uint32_t>(n_spans) + 2) * (weighted ? 8u : 4u);  o = (o + 15u) & ~15u;
+    L.ulo_off = o;    o += static_cast<uint32_t>(nk) * 8u;
+    L.uw_off = o;     o += weighted ? static_cast<uint32_t>(nk) * 8u : 0u;
+    L.table_off = o;  o += WINP * 16u;
+    L.keys_off = o;   o += static_cast<uint32_t>(npad) * 4u;
+    L.ufeat_off = o;  o += (static_cast<uint32_t>(nk) + 1u) * 4u;                      // cstart[u] replaces ufeat[u]
+    L.ustart_off = o; o += (static_cast<uint32_t>(nk) + 1u) * 4u;
+    L.uaq_off = o;    o += weighted ? static_cast<uint32_t>(nk) * 4u : 0u;
+    L.total = o + 16u;
+    return L;
+}
 
 __device__ __forceinline__ uint32_t orderable(float v)
 {
@@ -114,55 +155,132 @@ __device__ __noinline__ int block_positions_now(const s3_compact_view& v, uint32
     return block_positions(h, lane, lo, hi);
 }
 
-template <bool POW2, bool COMPACT>
+// Adds w to the difference array at j_lo and takes it away again after j_hi.
+template <bool WEIGHTED>
+__device__ __forceinline__ void add_range(int* acc_i, unsigned long long* acc_w, int j_lo, int j_hi, unsigned long long w)
+{
+    if (j_lo > j_hi) return;
+    if (WEIGHTED) {
+        atomicAdd(&acc_w[j_lo], w);
+        atomicAdd(&acc_w[j_hi + 1], 0ull - w);
+    } else {
+        atomicAdd(&acc_i[j_lo], 1);
+        atomicAdd(&acc_i[j_hi + 1], -1);
+    }
+}
+
+__device__ __forceinline__ double block_max_double(double v, double* red /*[SW]*/)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    double m = red[0];
+    for (int w = 1; w < SW; ++w) m = fmax(m, red[w]);
+    return m;
+}
+
+template <bool POW2, bool COMPACT, bool WEIGHTED>
 __global__ void __launch_bounds__(ST)
 score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__ CompactLayers clayers,
              const __grid_constant__ ScoreArgs a)
 {
     extern __shared__ __align__(16) unsigned char score_smem_raw[];
-    const bool weighted = a.mode == S3_SCORE_WEIGHTED;
-    const ScoreSmem SL = score_smem(a.nk, a.npad, a.n_spans, weighted);
-    int* acc_i = reinterpret_cast<int*>(score_smem_raw + SL.acc_off);          // min-count: difference array [n_spans+1]
-    double* acc_d = reinterpret_cast<double*>(score_smem_raw + SL.acc_off);    // weighted: fp64 per span
-    uint32_t* sel = reinterpret_cast<uint32_t*>(score_smem_raw + SL.acc_off);  // phase c: orderable fused scores
+    const ScoreLayout SL = score_layout(a.nk, a.npad, a.n_spans, WEIGHTED);
+    int* acc_i = reinterpret_cast<int*>(score_smem_raw + SL.acc_off);                              // min-count: difference array [n_spans+2]
+    unsigned long long* acc_w = reinterpret_cast<unsigned long long*>(score_smem_raw + SL.acc_off);  // weighted: fixed-point, same shape
+    uint32_t* sel = reinterpret_cast<uint32_t*>(score_smem_raw + SL.acc_off);                       // phase c: orderable fused scores
     unsigned long long* ulo = reinterpret_cast<unsigned long long*>(score_smem_raw + SL.ulo_off);
+    long long* uw = reinterpret_cast<long long*>(score_smem_raw + SL.uw_off);                       // weighted: fixed-point aQ*IDF
+    PieceDesc* table = reinterpret_cast<PieceDesc*>(score_smem_raw + SL.table_off);
     uint32_t* keys = reinterpret_cast<uint32_t*>(score_smem_raw + SL.keys_off);
     uint32_t* ulen = keys;                                                      // keys are dead once aQ is summed
     int32_t* ufeat = reinterpret_cast<int32_t*>(score_smem_raw + SL.ufeat_off);
     int32_t* ustart = reinterpret_cast<int32_t*>(score_smem_raw + SL.ustart_off);
     float* uaq = reinterpret_cast<float*>(score_smem_raw + SL.uaq_off);
-    uint16_t* owner = reinterpret_cast<uint16_t*>(score_smem_raw + SL.owner_off);
-    uint32_t* cstart = reinterpret_cast<uint32_t*>(score_smem_raw + SL.cstart_off);   // same storage as ufeat: a thread
-                                                                                        // reads ufeat[u], then writes cstart[u]
+    uint32_t* cstart = reinterpret_cast<uint32_t*>(score_smem_raw + SL.ufeat_off);   // same storage as ufeat: a thread
+                                                                                       // reads ufeat[u], then writes cstart[u]
     __shared__ uint32_t ws[SW + 1];
     __shared__ unsigned long long red[SW];
     __shared__ int n_unique_s;
+    __shared__ uint32_t ticket_s;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int q = blockIdx.x;
+    const int q = blockIdx.x / a.n_split, part = blockIdx.x - q * a.n_split;
 
-    if (weighted) { for (int j = tid; j < a.n_spans + 1; j += ST) acc_d[j] = 0.0; }
+    if (WEIGHTED) { for (int j = tid; j < a.n_spans + 2; j += ST) acc_w[j] = 0ull; }
     else          { for (int j = tid; j < a.n_spans + 2; j += ST) acc_i[j] = 0; }
     __syncthreads();
+
+    // Weighted mode: the unit of the fixed-point weights. A first pass over the layers finds the query's largest
+    // weight and its number of postings; unit = 2^(exponent of the largest weight + 1 - bits) with bits chosen so
+    // that the sum of all contributions stays below 2^62.
+    int wexp = 0;                 // weights are stored as llrint(ldexp(w, wexp))
+    if (WEIGHTED) {
+        double wmax = 0.0;
+        unsigned long long n_post = 0;
+        for (int l = 0; l < a.n_layers; ++l) {
+            const int32_t* qi = a.q_ids + ((size_t)l * a.Q + q) * a.nk;
+            const float* qv = a.q_vals + ((size_t)l * a.Q + q) * a.nk;
+            const int U = aggregate_query(qi, qv, a.nk, a.npad, a.d_sae, true, keys, ufeat, ustart, uaq, ws, &n_unique_s);
+            const uint32_t pieces = cut_lists(layers.v[l].d_row_ptr, U, a.stop_freq, ufeat, ulo, ulen, cstart, ws,
+                                              COMPACT ? clayers.v[l].d_blk_ptr : nullptr);
+            n_post += static_cast<unsigned long long>(pieces) * PIECE;
+            double m = 0.0;
+            for (int u = tid; u < U; u += ST)
+                if (ulen[u]) m = fmax(m, static_cast<double>(uaq[u]) * (1.0 / (log(1.0 + static_cast<double>(ulen[u])) + 1.0)));
+            wmax = fmax(wmax, block_max_double(m, reinterpret_cast<double*>(red)));
+            __syncthreads();
+        }
+        int bits = 61;
+        while (bits > 20 && (n_post >> (61 - bits)) != 0ull) --bits;          // n_post < 2^(61 - bits + 1)
+        wexp = wmax > 0.0 ? bits - 1 - ilogb(wmax) : 0;
+    }
 
     for (int l = 0; l < a.n_layers; ++l) {
         const int32_t* qi = a.q_ids + ((size_t)l * a.Q + q) * a.nk;
         const float* qv = a.q_vals + ((size_t)l * a.Q + q) * a.nk;
-        const int U = aggregate_query(qi, qv, a.nk, a.npad, a.d_sae, weighted, keys, ufeat, ustart, uaq, ws, &n_unique_s);
+        const int U = aggregate_query(qi, qv, a.nk, a.npad, a.d_sae, WEIGHTED, keys, ufeat, ustart, uaq, ws, &n_unique_s);
         // b. list bounds of every unique feature (independent loads), then the pieces' prefix sum
         const int32_t* __restrict__ pos = layers.v[l].d_pos;
-        const uint32_t piece_total = cut_lists(layers.v[l].d_row_ptr, U, weighted ? a.stop_freq : 0, ufeat, ulo, ulen, cstart, ws,
+        const uint32_t piece_total = cut_lists(layers.v[l].d_row_ptr, U, WEIGHTED ? a.stop_freq : 0, ufeat, ulo, ulen, cstart, ws,
                                                COMPACT ? clayers.v[l].d_blk_ptr : nullptr);
+        if (WEIGHTED) {
+            for (int u = tid; u < U; u += ST) {
+                const double w = static_cast<double>(uaq[u]) * (1.0 / (log(1.0 + static_cast<double>(ulen[u])) + 1.0));
+                uw[u] = ulen[u] ? __double2ll_rn(ldexp(w, wexp)) : 0ll;
+            }
+            __syncthreads();
+        }
+        // this block's share of the layer's pieces
+        const uint32_t share0 = static_cast<uint32_t>(static_cast<uint64_t>(piece_total) * part / a.n_split);
+        const uint32_t share1 = static_cast<uint32_t>(static_cast<uint64_t>(piece_total) * (part + 1) / a.n_split);
 
-        // The pieces are walked a window at a time; inside a window every warp takes an equal share. BATCH
-        // pieces per round: first all their loads are issued, then their updates, so that a warp has BATCH
-        // independent memory round trips in flight instead of one.
-        for (uint32_t win0 = 0; win0 < piece_total; win0 += WIN) {
-            const uint32_t win1 = piece_total - win0 < WIN ? piece_total : win0 + WIN;
-            tabulate_owners(cstart, U, win0, win1, owner);
+        // The share is walked a window at a time; inside a window every warp takes an equal run of consecutive
+        // pieces. BATCH pieces per round: first all their loads are issued, then their updates, so that a warp has
+        // BATCH independent memory round trips in flight instead of one.
+        for (uint32_t win0 = share0; win0 < share1; win0 += WINP) {
+            const uint32_t win1 = share1 - win0 < WINP ? share1 : win0 + WINP;
+            // descriptors: owner by binary search in the pieces' prefix (last u with cstart[u] <= c; pieces of
+            // empty lists share a start), one piece per thread and step
+            for (uint32_t c = win0 + tid; c < win1; c += ST) {
+                int lo = 0, hi = U;
+                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (cstart[mid] <= c) lo = mid; else hi = mid; }
+                const uint32_t j = c - cstart[lo];
+                const uint32_t left = ulen[lo] - PIECE * j;
+                PieceDesc d;
+                d.start = ulo[lo] + (COMPACT ? j : PIECE * j);
+                d.first_i = PIECE * j;
+                d.meta = (left < PIECE ? left : PIECE) | (static_cast<uint32_t>(ustart[lo + 1] - ustart[lo]) << 6) |
+                         (static_cast<uint32_t>(lo) << 19);
+                table[c - win0] = d;
+            }
+            __syncthreads();
             const uint32_t n_win = win1 - win0;
-            const uint32_t c_begin = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * warp / SW);
-            const uint32_t c_end = win0 + static_cast<uint32_t>(static_cast<uint64_t>(n_win) * (warp + 1) / SW);
+            const uint32_t c_begin = static_cast<uint32_t>(static_cast<uint64_t>(n_win) * warp / SW);
+            const uint32_t c_end = static_cast<uint32_t>(static_cast<uint64_t>(n_win) * (warp + 1) / SW);
             if constexpr (COMPACT) {
                 // A piece is one block of the compact index. The headers of the next CBATCH blocks are fetched while
                 // the payload words of the current ones are in flight, so a batch waits for one memory round trip.
@@ -170,16 +288,14 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
                 // targets lie in at most two blocks, x = floor((32 j - cQ)/32) and x + 1. Block j itself is at hand; an
                 // earlier block j - d is piece b - d of this warp (its pieces are consecutive) and is taken from the
                 // batch or from the last two blocks of the previous batch; only when it lies further back (the start
-                // of the warp's share, cQ > 64) is it decoded on the spot.
+                // of the warp's run, cQ > 64) is it decoded on the spot.
                 const s3_compact_view& cv = clayers.v[l];
                 auto fetch_head = [&](uint32_t c) {
                     PieceHead h;
                     h.first = 0; h.desc = 0; h.cnt = 0;
                     if (c < c_end) {
-                        const int u = owner[c - win0];
-                        const uint32_t j = c - cstart[u];
-                        const uint32_t left = ulen[u] - 32u * j;
-                        h = block_head(cv, static_cast<uint32_t>(ulo[u]) + j, left < 32u ? left : 32u);
+                        const PieceDesc d = table[c];
+                        h = block_head(cv, static_cast<uint32_t>(d.start), piece_count(d.meta));
                     }
                     return h;
                 };
@@ -206,24 +322,24 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
                         if (hc[b].cnt == 0) continue;                      // uniform over the warp
                         const int p = block_positions(hc[b], lane, lo[b], hi[b]);
                         hist[b + 2] = p;
-                        const int u = owner[c0 + b - win0];
+                        const PieceDesc d = table[c0 + b];
                         int p_prev = -1;
-                        if (!weighted) {
-                            const int j = static_cast<int>(c0 + b - cstart[u]);
-                            const int cq = ustart[u + 1] - ustart[u];
+                        if (!WEIGHTED) {
+                            const int j = static_cast<int>(d.first_i >> 5);
+                            const int cq = static_cast<int>(piece_cq(d.meta));
                             const int x = (32 * j - cq) >> 5;              // floor, may be negative
                             int pr[3] = {p, -1, -1};
 #pragma unroll
                             for (int r = 1; r <= 2; ++r) {
                                 const int xb = x + r - 1;
                                 if (xb >= 0 && xb < j) {
-                                    const int d = j - xb;
-                                    if (d <= b + avail) {
+                                    const int dd = j - xb;
+                                    if (dd <= b + avail) {
 #pragma unroll
                                         for (int e = 1; e <= b + 2; ++e)
-                                            if (d == e) pr[r] = hist[b + 2 - e];
+                                            if (dd == e) pr[r] = hist[b + 2 - e];
                                     } else {
-                                        pr[r] = block_positions_now(cv, static_cast<uint32_t>(ulo[u]) + xb, lane);
+                                        pr[r] = block_positions_now(cv, static_cast<uint32_t>(d.start) - dd, lane);
                                     }
                                 }
                             }
@@ -240,33 +356,27 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
                         if (p < 0) continue;
                         int j_lo, j_hi;
                         posting_range<POW2>(a, p, p_prev, j_lo, j_hi);
-                        if (weighted) {
-                            const double w = static_cast<double>(uaq[u]) * (1.0 / (log(1.0 + static_cast<double>(ulen[u])) + 1.0));
-                            for (int jj = j_lo; jj <= j_hi; ++jj) atomicAdd(&acc_d[jj], w);
-                        } else if (j_lo <= j_hi) {
-                            atomicAdd(&acc_i[j_lo], 1);
-                            atomicAdd(&acc_i[j_hi + 1], -1);
-                        }
+                        add_range<WEIGHTED>(acc_i, acc_w, j_lo, j_hi, WEIGHTED ? static_cast<unsigned long long>(uw[piece_owner(d.meta)]) : 1ull);
                     }
                     carry2 = hist[CBATCH]; carry1 = hist[CBATCH + 1];
                 }
             } else
             for (uint32_t c0 = c_begin; c0 < c_end; c0 += BATCH) {
-                int p[BATCH], p_prev[BATCH], ub[BATCH];
+                int p[BATCH], p_prev[BATCH];
+                uint32_t own[BATCH];
 #pragma unroll
                 for (int b = 0; b < BATCH; ++b) {
-                    const uint32_t c = c0 + b;
-                    p[b] = -1; p_prev[b] = -1; ub[b] = 0;
-                    if (c < c_end) {
-                        const int u = owner[c - win0];
-                        ub[b] = u;
-                        const int32_t* __restrict__ list = pos + ulo[u];
-                        const uint32_t i = (c - cstart[u]) * PIECE + lane;
-                        if (i < ulen[u]) {
-                            p[b] = __ldg(list + i);
-                            if (!weighted) {
-                                const uint32_t cq = static_cast<uint32_t>(ustart[u + 1] - ustart[u]);
-                                if (i >= cq) p_prev[b] = __ldg(list + i - cq);
+                    p[b] = -1; p_prev[b] = -1; own[b] = 0;
+                    if (c0 + b < c_end) {
+                        const uint4 raw = *reinterpret_cast<const uint4*>(&table[c0 + b]);       // one broadcast load per piece
+                        const unsigned long long start = (static_cast<unsigned long long>(raw.y) << 32) | raw.x;
+                        own[b] = piece_owner(raw.w);
+                        if (static_cast<uint32_t>(lane) < piece_count(raw.w)) {
+                            const int32_t* __restrict__ src = pos + start + lane;
+                            p[b] = __ldg(src);
+                            if (!WEIGHTED) {
+                                const uint32_t cq = piece_cq(raw.w);
+                                if (raw.z + lane >= cq) p_prev[b] = __ldg(src - cq);
                             }
                         }
                     }
@@ -276,22 +386,55 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
                     if (p[b] < 0) continue;
                     int j_lo, j_hi;
                     posting_range<POW2>(a, p[b], p_prev[b], j_lo, j_hi);
-                    if (weighted) {
-                        const double w = static_cast<double>(uaq[ub[b]]) *
-                                         (1.0 / (log(1.0 + static_cast<double>(ulen[ub[b]])) + 1.0));
-                        for (int j = j_lo; j <= j_hi; ++j) atomicAdd(&acc_d[j], w);
-                    } else if (j_lo <= j_hi) {
-                        atomicAdd(&acc_i[j_lo], 1);
-                        atomicAdd(&acc_i[j_hi + 1], -1);
-                    }
+                    add_range<WEIGHTED>(acc_i, acc_w, j_lo, j_hi, WEIGHTED ? static_cast<unsigned long long>(uw[own[b]]) : 1ull);
                 }
             }
             __syncthreads();
         }
     }
 
-    // min-count mode: difference array -> per-span totals (inclusive prefix sum, in place)
-    if (!weighted) {
+    // Several blocks per query: add this block's difference array to the query's in the workspace; the block that
+    // takes the last ticket reads the sum back and finishes the query.
+    if (a.n_split > 1) {
+        unsigned long long* g = a.acc_g + static_cast<size_t>(q) * (a.n_spans + 2);
+        for (int j = tid; j < a.n_spans + 2; j += ST) {
+            if (WEIGHTED) { if (acc_w[j]) atomicAdd(&g[j], acc_w[j]); }
+            else if (acc_i[j]) atomicAdd(reinterpret_cast<int*>(&g[j]), acc_i[j]);
+        }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) ticket_s = atomicAdd(&a.tickets[q], 1u);
+        __syncthreads();
+        if (ticket_s != static_cast<uint32_t>(a.n_split - 1)) return;
+        __threadfence();
+        for (int j = tid; j < a.n_spans + 2; j += ST) {
+            const unsigned long long v = __ldcg(&g[j]);
+            if (WEIGHTED) acc_w[j] = v; else acc_i[j] = static_cast<int>(static_cast<uint32_t>(v));
+        }
+        __syncthreads();
+    }
+
+    // difference array -> per-span totals (inclusive prefix sum, in place)
+    if (WEIGHTED) {
+        unsigned long long carry = 0;
+        for (int j0 = 0; j0 < a.n_spans; j0 += ST) {
+            const int j = j0 + tid;
+            unsigned long long inc = j < a.n_spans ? acc_w[j] : 0ull;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += n;
+            }
+            __syncthreads();
+            if (lane == 31) red[warp] = inc;
+            __syncthreads();
+            unsigned long long before = carry;
+            for (int w = 0; w < warp; ++w) before += red[w];
+            if (j < a.n_spans) acc_w[j] = before + inc;
+            for (int w = 0; w < SW; ++w) carry += red[w];
+        }
+        __syncthreads();
+    } else {
         uint32_t carry = 0;
         for (int j0 = 0; j0 < a.n_spans; j0 += ST) {
             const int j = j0 + tid;
@@ -311,7 +454,8 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
         const int j = j0 + tid;
         float v = 0.0f;
         if (j < a.n_spans) {
-            const float base = weighted ? __double2float_rn(acc_d[j]) : __int2float_rn(acc_i[j]);
+            const float base = WEIGHTED ? __double2float_rn(ldexp(static_cast<double>(static_cast<long long>(acc_w[j])), -wexp))
+                                        : __int2float_rn(acc_i[j]);
             v = __fmul_rn(a.alpha, base);
             if (a.bm25) v = __fadd_rn(v, __fmul_rn(a.beta, a.bm25[(size_t)q * a.ld_bm25 + j]));
             if (a.all_scores) a.all_scores[(size_t)q * a.n_spans + j] = v;
@@ -351,25 +495,54 @@ score_kernel(const __grid_constant__ ScoreLayers layers, const __grid_constant__
     }
 }
 
+// No span fits into the context: every query gets s times "no span".
+__global__ void score_empty_kernel(int32_t* top_idx, float* top_score, size_t n)
+{
+    const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < n) { top_idx[i] = -1; top_score[i] = 0.0f; }
+}
+
+template <bool POW2, bool COMPACT, bool WEIGHTED>
+s3_status launch_variant(const ScoreLayers& layers, const CompactLayers& cl, const ScoreArgs& a, size_t smem, int max_smem, int dev,
+                         cudaStream_t stream)
+{
+    static bool attr_set[64] = {};
+    if (dev >= 64 || !attr_set[dev]) {
+        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<POW2, COMPACT, WEIGHTED>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+        if (dev < 64) attr_set[dev] = true;
+    }
+    score_kernel<POW2, COMPACT, WEIGHTED><<<a.Q * a.n_split, ST, smem, stream>>>(layers, cl, a);
+    S3_CUDA_TRY(cudaGetLastError());
+    return S3_OK;
+}
+
 }  // namespace
+
+size_t score_workspace_bytes(int Q, int n_spans)
+{
+    if (Q <= 0 || n_spans <= 0) return 0;
+    return round_up(static_cast<size_t>(Q) * 4, 256) + static_cast<size_t>(Q) * (n_spans + 2) * 8;
+}
 
 namespace {
 
 s3_status launch_score_impl(const ScoreLayers& layers, const CompactLayers* clayers, int n_layers, int d_sae, const int32_t* d_q_ids,
                             const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
                             const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
-                            float* d_all_scores, cudaStream_t stream)
+                            float* d_all_scores, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
+    if (n_spans == 0) {
+        const size_t n = static_cast<size_t>(Q) * p->s;
+        score_empty_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(d_top_idx, d_top_score, n);
+        S3_CUDA_TRY(cudaGetLastError());
+        return S3_OK;
+    }
     static int max_smem_dev[64] = {};
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
     int max_smem = dev < 64 ? max_smem_dev[dev] : 0;
     if (max_smem == 0) {
         S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
-        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
-        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
-        S3_CUDA_TRY(cudaFuncSetAttribute(score_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
         if (dev < 64) max_smem_dev[dev] = max_smem;
     }
     ScoreArgs a;
@@ -382,19 +555,31 @@ s3_status launch_score_impl(const ScoreLayers& layers, const CompactLayers* clay
     a.alpha = p->alpha; a.beta = p->beta; a.stop_freq = p->stop_freq;
     a.stride_shift = (p->stride & (p->stride - 1)) == 0 ? __builtin_ctz(static_cast<unsigned>(p->stride)) : -1;
     a.stride_magic = p->stride >= 2 ? ~0ull / static_cast<unsigned long long>(p->stride) + 1ull : 0ull;
-    const size_t smem = score_smem(a.nk, npad, n_spans, p->mode == S3_SCORE_WEIGHTED).total;
+    const bool weighted = p->mode == S3_SCORE_WEIGHTED;
+    const size_t smem = score_layout(a.nk, npad, n_spans, weighted).total;
     S3_REQUIRE(smem + 2048 <= static_cast<size_t>(max_smem), S3_ERR_UNSUPPORTED,
                "n_spans = %d with nq*k = %d needs %zu bytes of shared memory per query, %d available", n_spans, a.nk, smem,
                max_smem - 2048);
-    if (clayers) {
-        if (a.stride_shift >= 0) score_kernel<true, true><<<Q, ST, smem, stream>>>(layers, *clayers, a);
-        else score_kernel<false, true><<<Q, ST, smem, stream>>>(layers, *clayers, a);
-    } else {
-        CompactLayers none = {};
-        if (a.stride_shift >= 0) score_kernel<true, false><<<Q, ST, smem, stream>>>(layers, none, a);
-        else score_kernel<false, false><<<Q, ST, smem, stream>>>(layers, none, a);
+    // Few queries: cut each over several blocks (about two blocks per SM in all) when the workspace has room for the
+    // queries' shared difference arrays; otherwise one block per query.
+    a.n_split = 1;
+    a.acc_g = nullptr; a.tickets = nullptr;
+    const int want = 2 * device_sm_count() / Q;
+    if (want > 1 && ws_bytes >= 256 + score_workspace_bytes(Q, n_spans)) {
+        a.n_split = want > MAX_SPLIT ? MAX_SPLIT : want;
+        a.tickets = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(d_ws) + 256);
+        a.acc_g = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(d_ws) + 256 + round_up(static_cast<size_t>(Q) * 4, 256));
+        // the shared sums and tickets start from zero (a small range: this path is taken for few queries only)
+        S3_CUDA_TRY(cudaMemsetAsync(a.tickets, 0, score_workspace_bytes(Q, n_spans), stream));
     }
-    S3_CUDA_TRY(cudaGetLastError());
+    CompactLayers none = {};
+    const CompactLayers& cl = clayers ? *clayers : none;
+    const bool pow2 = a.stride_shift >= 0, compact = clayers != nullptr;
+#define S3_SCORE_CASE(P, C, W) \
+    if (pow2 == P && compact == C && weighted == W) return launch_variant<P, C, W>(layers, cl, a, smem, max_smem, dev, stream);
+    S3_SCORE_CASE(true, false, false) S3_SCORE_CASE(false, false, false) S3_SCORE_CASE(true, true, false) S3_SCORE_CASE(false, true, false)
+    S3_SCORE_CASE(true, false, true) S3_SCORE_CASE(false, false, true) S3_SCORE_CASE(true, true, true) S3_SCORE_CASE(false, true, true)
+#undef S3_SCORE_CASE
     return S3_OK;
 }
 
@@ -403,18 +588,18 @@ s3_status launch_score_impl(const ScoreLayers& layers, const CompactLayers* clay
 s3_status launch_score(const s3_csr_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
                        const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
                        const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
-                       float* d_all_scores, cudaStream_t stream)
+                       float* d_all_scores, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
     ScoreLayers layers = {};
     for (int l = 0; l < n_layers; ++l) layers.v[l] = h_layers[l];
     return launch_score_impl(layers, nullptr, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, n_spans, p, d_bm25, ld_bm25,
-                             d_top_idx, d_top_score, d_all_scores, stream);
+                             d_top_idx, d_top_score, d_all_scores, d_ws, ws_bytes, stream);
 }
 
 s3_status launch_score_compact(const s3_compact_view* h_layers, int n_layers, int d_sae, const int32_t* d_q_ids,
                                const float* d_q_vals, int Q, int nq, int k, int n_spans, const s3_score_params* p,
                                const float* d_bm25, int64_t ld_bm25, int32_t* d_top_idx, float* d_top_score,
-                               float* d_all_scores, cudaStream_t stream)
+                               float* d_all_scores, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
     ScoreLayers layers = {};
     CompactLayers cl = {};
@@ -424,7 +609,7 @@ s3_status launch_score_compact(const s3_compact_view* h_layers, int n_layers, in
         layers.v[l].d_pos = nullptr;
     }
     return launch_score_impl(layers, &cl, n_layers, d_sae, d_q_ids, d_q_vals, Q, nq, k, n_spans, p, d_bm25, ld_bm25,
-                             d_top_idx, d_top_score, d_all_scores, stream);
+                             d_top_idx, d_top_score, d_all_scores, d_ws, ws_bytes, stream);
 }
 
 }  // namespace s3

@@ -134,7 +134,9 @@ def gpu_score_compact(ctx, q, qv, d_sae, width, stride, s, alpha, beta, bm25, mo
     ns = C.n_spans(L, width, stride)
     Q = q.shape[1]
     alls = torch.zeros((Q, max(ns, 1)), dtype=torch.float32, device=d)
-    ws = S.new_workspace(64)
+    # odd list totals: the full workspace, so that each query is cut over many thread blocks; even ones: one block per query
+    split = int(layers[0].row_ptr[-1]) % 2 == 1
+    ws = S.new_workspace(S.s3_score_workspace_bytes(Q, q.shape[2], q.shape[3], n_layers, ns, s) if split else 64)
     bm = None if bm25 is None else torch.as_tensor(bm25).to(d).contiguous()
     ti, ts = S.s3_coactivation_score_topspans_compact(layers, d_sae, L, torch.as_tensor(q).to(d).contiguous(),
                                                       torch.as_tensor(qv).to(d).contiguous(), width, stride, s, alpha, beta,

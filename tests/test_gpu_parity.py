@@ -415,7 +415,8 @@ def test_index_append_export_matches_oracle_merge():
 
 # ------------------------------------------------------------------------------------ scoring
 
-def gpu_score(ctx_ids, q_ids, q_vals, d_sae, width, stride, s, alpha, beta, bm25=None, mode=0, stop_freq=0):
+def gpu_score(ctx_ids, q_ids, q_vals, d_sae, width, stride, s, alpha, beta, bm25=None, mode=0, stop_freq=0, split=False):
+    """split: give the call the full workspace, so that the few queries of these tests are cut over many blocks each."""
     d = dev()
     n_layers, L, k = ctx_ids.shape
     layers = []
@@ -426,7 +427,8 @@ def gpu_score(ctx_ids, q_ids, q_vals, d_sae, width, stride, s, alpha, beta, bm25
     ns = C.n_spans(L, width, stride)
     Q = q_ids.shape[1]
     alls = torch.zeros((Q, max(ns, 1)), dtype=torch.float32, device=d)
-    ws = S.new_workspace(64)
+    ws = S.new_workspace(S.s3_score_workspace_bytes(Q, q_ids.shape[2], q_ids.shape[3], n_layers, ns, s) if split else 64)
+    ws[64:] = 0xA5                              # whatever an earlier call left there must not matter
     bm = None if bm25 is None else torch.as_tensor(bm25).to(d).contiguous()
     ti, ts = S.s3_coactivation_score_topspans(layers, d_sae, L, torch.as_tensor(q_ids).to(d).contiguous(),
                                               torch.as_tensor(q_vals).to(d).contiguous(), width, stride, s, alpha, beta,
@@ -458,10 +460,11 @@ def test_score_mincount_exact(L, k, d_sae, n_layers, Q, nq, kq, width, stride, s
         if ns == 0:
             b = None
         oi, os_, oall = O.fuse_select(co, b, alpha, beta, s)
-        ti, ts, alls = gpu_score(ctx, q, qv, d_sae, width, stride, s, alpha, beta, b)
-        np.testing.assert_array_equal(alls, oall)
-        np.testing.assert_array_equal(ti, oi)
-        np.testing.assert_array_equal(ts, os_)
+        for split in (False, True):
+            ti, ts, alls = gpu_score(ctx, q, qv, d_sae, width, stride, s, alpha, beta, b, split=split)
+            np.testing.assert_array_equal(alls, oall)
+            np.testing.assert_array_equal(ti, oi)
+            np.testing.assert_array_equal(ts, os_)
 
 
 def test_score_weighted_mode():
@@ -477,6 +480,26 @@ def test_score_weighted_mode():
         for qi in range(Q):                       # the selected spans are the best ones of the GPU's own scores
             order = sorted(range(alls.shape[1]), key=lambda j: (-float(alls[qi, j]), j))[:s]
             assert ti[qi].tolist() == order
+        # the weights are summed as fixed-point integers: the same bits from run to run and however the query is
+        # cut over thread blocks
+        for split in (False, True, True):
+            ti2, ts2, alls2 = gpu_score(ctx, q, qv, d_sae, width, stride, s, 1.0, 0.0, None, 1, stop, split=split)
+            np.testing.assert_array_equal(alls2, alls)
+            np.testing.assert_array_equal(ti2, ti)
+            np.testing.assert_array_equal(ts2, ts)
+
+
+def test_score_weighted_wide_weight_range():
+    """Activations spread over five decades: spans that hold a large weight agree with the fp64 sum to 1e-5; the fixed-point
+    grid lies 2^-40 below the query's largest weight."""
+    L, k, d_sae, Q, nq, kq, width, stride, s = 3000, 8, 256, 2, 6, 8, 64, 16, 8
+    ctx = _rand_ids(L, k, d_sae, 250)[None]
+    q = _rand_ids(Q * nq, kq, d_sae, 251).reshape(1, Q, nq, kq)
+    qv = (10.0 ** np.random.default_rng(29).uniform(-3, 2, q.shape)).astype(np.float32)
+    w = O.score_spans(ctx, q, qv, d_sae, width, stride, 1, 0)
+    _, _, oall = O.fuse_select(w, None, 1.0, 0.0, s)
+    _, _, alls = gpu_score(ctx, q, qv, d_sae, width, stride, s, 1.0, 0.0, None, 1, 0)
+    np.testing.assert_allclose(alls, oall, rtol=1e-5, atol=0)
 
 
 def test_hand_example_on_gpu(golden_dir):
