@@ -338,8 +338,8 @@ s3_status s3_position_density_topcenters(const s3_csr_view* h_layers, int n_laye
 
 /* ------------------------------------------------------------------------------------------------
  * Head aggregation + Top-k       (paper Sec. 3.3: the SAE reads one head's projection, x in R^d_head, with one
- *                                 feature-ID space for all of them; Sec. 3.4: k is "the Top-k sparsity per token
- *                                 after head aggregation". The rule itself is not given; this is the reading.)
+ *                                 feature-ID space for all of them; Sec. 3.4 defines k as the per-token sparsity
+ *                                 once the heads are aggregated. The rule itself is not given; this is the reading.)
  *
  * d_ids / d_vals [T, H, k] hold, per token, the Top-k codes of its H heads (e.g. s3_sae_encode_topk on the
  * [T*H, d_head] view of the projections). Per token: a(f) = sum of f's activations over the heads whose code

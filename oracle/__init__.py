@@ -279,8 +279,8 @@ def prune_stop_features(row_ptr, pos, stop_freq: int):
 
 # ---------------------------------------------------------------------------------------------- head aggregation
 def head_aggregate(ids, vals, k_out: int):
-    """Sec. 3.3 / 3.4: the SAE reads one head's projection (x in R^d_head) and the index keeps "the Top-k sparsity per
-    token after head aggregation"; the aggregation rule is not given. Reading: all heads share one feature-ID space;
+    """Sec. 3.3 / 3.4: the SAE reads one head's projection (x in R^d_head), while Sec. 3.4 counts k features per token
+    once the heads have been aggregated; the aggregation rule is not given. Reading: all heads share one feature-ID space;
     a token's activation of feature f is the sum over the heads whose Top-k holds f (fp32, heads in ascending order,
     which is the precision the selection is made in), and the token keeps the k_out largest sums > 0, ordered by
     (sum descending, id ascending), padded with id -1 / value 0.

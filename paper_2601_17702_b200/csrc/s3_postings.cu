@@ -36,7 +36,7 @@ constexpr int RUN_PAIRS = NT * PER;      // pairs per run at most
 constexpr int B_MAX = 4 * NT;            // buckets per item at most (four per thread in the scan)
 constexpr int FB_MAX = 12;               // at most 4096 features per bucket
 constexpr int CAP = 8192;                // entries sorted at once in shared memory
-constexpr int TBL_BITS = 13;             // (feature, window) counters of one sort
+constexpr int TBL_BITS = 12;             // (feature, window) counters of one sort
 constexpr int TBL = 1 << TBL_BITS;
 constexpr int MAX_RUNS = 4 * NT;         // runs whose segment table fits in shared memory
 constexpr int BM_WORDS = 2 * CAP;        // bitmap words of the single-list path (e_stage + sorted)
@@ -123,23 +123,30 @@ postings_partition_kernel(const __grid_constant__ PostingsPlan pl)
     for (int b = tid; b < B; b += NT) hist[b] = 0;
     __syncthreads();
 
-    uint32_t e[PER], ba[PER];                  // entry; bucket << 16 | arrival rank inside the bucket
+    // all loads first, so that the run's sixteen memory round trips per thread overlap
+    int32_t fid[PER];
 #pragma unroll
     for (int j = 0; j < PER; ++j) {
         const uint32_t p = tid + j * NT;
+        fid[j] = p < n_pairs ? __ldcs(src + p) : -1;
+    }
+    uint32_t e[PER], ba[PER];                  // entry; bucket << 16 | arrival rank inside the bucket
+    bool bad = false;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        const uint32_t p = tid + j * NT;
+        const int32_t f = fid[j];
         ba[j] = 0xFFFFFFFFu;
         e[j] = 0;
-        if (p < n_pairs) {
-            const int32_t f = __ldcs(src + p);
-            if (f >= d_sae) dev_set_error(pl.status, DEV_BAD_FEATURE_ID);
-            else if (f >= 0) {
-                const uint32_t b = (uint32_t)f >> fbits;
-                const uint32_t t = (uint32_t)t_lo + (k == 1 ? p : __umulhi(p, magic));
-                e[j] = (((uint32_t)f & fmask) << tbits) | t;
-                ba[j] = (b << 16) | atomicAdd(&hist[b], 1u);
-            }
+        if (f >= d_sae) bad = true;
+        else if (f >= 0) {
+            const uint32_t b = (uint32_t)f >> fbits;
+            const uint32_t t = (uint32_t)t_lo + (k == 1 ? p : __umulhi(p, magic));
+            e[j] = (((uint32_t)f & fmask) << tbits) | t;
+            ba[j] = (b << 16) | atomicAdd(&hist[b], 1u);
         }
     }
+    if (bad) dev_set_error(pl.status, DEV_BAD_FEATURE_ID);
     __syncthreads();
 
     // exclusive scan of the bucket counts, four per thread; the directory row goes out on the way
@@ -261,14 +268,16 @@ __device__ void sort_range(const BucketCtx& c, uint32_t f_lo, uint32_t f_hi, uin
     __syncthreads();
     const uint32_t n = FILTER ? c.counters[0] : n_known;
 
-    // exclusive scan of the counters in (feature, window) order: eight words (16 counters) per thread
+    // exclusive scan of the counters in (feature, window) order: TBL / 2 / NT words (two counters each) per thread
     {
-        uint4* t4 = reinterpret_cast<uint4*>(c.tbl) + 2 * tid;
-        uint4 v0 = t4[0], v1 = t4[1];
-        uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        constexpr int WPT = TBL / 2 / NT;
+        static_assert(WPT == 4, "one uint4 of counters per thread");
+        uint4* t4 = reinterpret_cast<uint4*>(c.tbl) + tid;
+        const uint4 v0 = t4[0];
+        uint32_t w[WPT] = {v0.x, v0.y, v0.z, v0.w};
         uint32_t run = 0;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < WPT; ++q) {
             const uint32_t lo = w[q] & 0xFFFFu, hi = w[q] >> 16;
             w[q] = run | ((run + lo) << 16);
             run += lo + hi;
@@ -276,9 +285,8 @@ __device__ void sort_range(const BucketCtx& c, uint32_t f_lo, uint32_t f_hi, uin
         uint32_t total;
         const uint32_t base = block_scan_excl(run, c.warp_sums, &total) * 0x00010001u;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) w[q] += base;
+        for (int q = 0; q < WPT; ++q) w[q] += base;
         t4[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        t4[1] = make_uint4(w[4], w[5], w[6], w[7]);
     }
     __syncthreads();
 
@@ -427,6 +435,47 @@ postings_bucket_kernel(const __grid_constant__ PostingsPlan pl)
     // the bucket's segment in every run: first output offset = sum of the starts, size = sum of the lengths
     uint32_t bucket_base = 0, n_total = 0;
     const bool table_fits = c.n_runs <= MAX_RUNS;
+    if (c.n_runs <= 128) {
+        // the usual chunk: one warp, four runs per lane, shuffles only
+        if (tid < 32) {
+            uint32_t s4[4], l4[4], sum_s = 0, sum_l = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int r = 4 * tid + q;
+                s4[q] = l4[q] = 0;
+                if (r < c.n_runs) {
+                    const uint16_t* d = c.dir + (size_t)r * (c.B + 1) + c.b;
+                    s4[q] = __ldg(d);
+                    l4[q] = __ldg(d + 1) - s4[q];
+                }
+                sum_s += s4[q];
+                sum_l += l4[q];
+            }
+            uint32_t inc = sum_l;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
+                if (tid >= o) inc += u;
+                sum_s += __shfl_xor_sync(0xffffffffu, sum_s, o);
+            }
+            uint32_t off = inc - sum_l;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int r = 4 * tid + q;
+                if (r < c.n_runs) {
+                    c.seg[r] = (uint16_t)s4[q];
+                    c.seg[MAX_RUNS + r] = (uint16_t)l4[q];
+                    c.seg[2 * MAX_RUNS + r] = (uint16_t)off;
+                }
+                off += l4[q];
+            }
+            if (tid == 31) { counters[0] = sum_s; counters[1] = inc; }
+        }
+        __syncthreads();
+        bucket_base = counters[0];
+        n_total = counters[1];
+        __syncthreads();
+    } else
     for (int r0 = 0; r0 < c.n_runs; r0 += MAX_RUNS) {
         uint32_t s4[4], l4[4], sum_s = 0, sum_l = 0;
 #pragma unroll
