@@ -8,7 +8,7 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 x bf16 -> fp32) into
 //               one of two 128x256 accumulators in tensor memory, tcgen05.commit frees the stage /
 //               publishes the accumulator;
-//   warps 2-5   epilogue: thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
+//   warps 2-5   epilogue (one group of four warps; see EPI_GROUPS): thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
 //               biased and compared with the row's bound tau, a value that at least k pre-activations
 //               of the row are known to exceed. Survivors go, branch-free, to a short pending list in
 //               shared memory. When some lane's list is nearly full the warp folds its lists: each
@@ -46,8 +46,15 @@ constexpr int PAIR_M = 2 * BM;                      // tokens per tile over the 
 constexpr int A_STAGE_BYTES = BM * BK * 2;         // 16 KB: this CTA's 128 tokens
 constexpr int B_STAGE_BYTES = (BN / 2) * BK * 2;   // 16 KB: this CTA's half of the tile's 256 features
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;   // per CTA; a stage is complete after twice that
-constexpr int NUM_THREADS = 192;
-constexpr int EPI_THREADS = 128;
+// Epilogue warp groups: each takes 256 / EPI_GROUPS columns of every tile, with its own bound, histogram and candidate
+// list per row. Two groups were measured and are not used: every list needs its own k survivors, so the work of folding
+// survivors, which is what bounds the narrow encoders, stays the same per thread (key SAE 0.326 ms instead of 0.313).
+#ifndef S3_EPI_GROUPS
+#define S3_EPI_GROUPS 1
+#endif
+constexpr int EPI_GROUPS = S3_EPI_GROUPS;
+constexpr int EPI_THREADS = 128 * EPI_GROUPS;
+constexpr int NUM_THREADS = 64 + EPI_THREADS;
 constexpr int TMEM_COLS = 512;
 constexpr int BATCH = 32;                    // columns per tcgen05.ld
 constexpr int STEP = 8;                      // columns filtered between two checks of the pending lists
@@ -505,9 +512,12 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
     } else {
         // ---------------- epilogue: bias + ReLU + candidate selection ----------------
         const int quarter = warp & 3;               // TMEM lanes this warp may read
+        const int grp = (warp - 2) >> 2;            // which share of a tile's columns this warp filters
         const int e = quarter * 32 + lane;          // row inside the 128-token block
-        uint64_t* my_pend = pend + e;
-        uint16_t* my_hist = hist + e;
+        uint64_t* my_pend = pend + grp * 128 + e;
+        uint16_t* my_hist = hist + grp * 128 + e;
+        constexpr int CB_PER_GROUP = BN / BATCH / EPI_GROUPS;
+        const int cb_lo = grp * CB_PER_GROUP, cb_hi = cb_lo + CB_PER_GROUP;
         uint32_t tile_count = 0;
         bool ok = true;
         // the accumulator is handed back on the first CTA's barrier
@@ -522,7 +532,9 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             const bool live = t < ip.T;
             const int k = ip.k;
             const uint32_t cap = ip.cap;
-            uint64_t* glist = DENSE ? nullptr : ip.cand + (static_cast<size_t>(live ? t : 0) * ip.n_slices + slice) * cap;
+            // each group keeps its own candidate list, bound and histogram for its columns of the row
+            const size_t list_idx = (static_cast<size_t>(live ? t : 0) * ip.n_slices + slice) * EPI_GROUPS + grp;
+            uint64_t* glist = DENSE ? nullptr : ip.cand + list_idx * cap;
             if (!DENSE) {
 #pragma unroll 1
                 for (int sl = 0; sl < NB; ++sl) my_hist[sl * EPI_THREADS] = 0;
@@ -556,7 +568,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                     float level[COLD_LEVELS];
                     int seen[COLD_LEVELS];
 #pragma unroll 1
-                    for (int cb = 0; cb < BN / BATCH; ++cb) {
+                    for (int cb = cb_lo; cb < cb_hi; ++cb) {
                         uint32_t acc[32];
                         tc_ld32(taddr + cb * BATCH, acc);
                         float bias[BATCH];
@@ -566,7 +578,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                             bias[4 * j4 + 0] = b4.x; bias[4 * j4 + 1] = b4.y; bias[4 * j4 + 2] = b4.z; bias[4 * j4 + 3] = b4.w;
                         }
                         tc_wait_ld();
-                        if (cb == 0) {
+                        if (cb == cb_lo) {
                             float top = 0.0f;
 #pragma unroll
                             for (int q = 0; q < BATCH; ++q) top = fmaxf(top, __uint_as_float(acc[q]) + bias[q]);
@@ -589,7 +601,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                     }
                 }
 #pragma unroll 1
-                for (int cb = 0; cb < BN / BATCH; ++cb) {
+                for (int cb = cb_lo; cb < cb_hi; ++cb) {
                     uint32_t acc[32];
                     tc_ld32(taddr + cb * BATCH, acc);
                     float bias[BATCH];
@@ -676,7 +688,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                         for (int q = 0; q < 16; ++q)
                             if (__uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > cut) glist[w++] = key[q];
                     }
-                    ip.counts[static_cast<size_t>(t) * ip.n_slices + slice] = w;
+                    ip.counts[list_idx] = w;
                     if (out > hint_in) atomicMax(ip.hint + t, out);
                 }
             }
@@ -808,14 +820,15 @@ int encode_tc_max_pairs()
     return n;
 }
 
-uint32_t encode_tc_list_cap(int k) { return static_cast<uint32_t>(k < 4 ? 64 : 16 * k); }
+// Slots of one candidate list (one per row, slice and epilogue group); a list that fills up is pruned in place.
+uint32_t encode_tc_list_cap(int k) { return static_cast<uint32_t>((k < 4 ? 64 : 16 * k) / EPI_GROUPS); }
 
 // Column tiles per slice may not exceed 255: a row's histogram counters are 16 bits wide.
 int encode_tc_min_slices(int d_sae) { return (encode_tc_col_tiles(d_sae) + 254) / 255; }
 
 size_t encode_tc_workspace_bytes(int T, int n_slices, int k)
 {
-    const size_t t = static_cast<size_t>(T), s = static_cast<size_t>(n_slices);
+    const size_t t = static_cast<size_t>(T), s = static_cast<size_t>(n_slices) * EPI_GROUPS;    // candidate lists per row
     return round_up(t * 4, 256) + round_up(t * s * 4, 256) + round_up(t * s * encode_tc_list_cap(k) * sizeof(uint64_t), 256);
 }
 
@@ -879,7 +892,7 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
         ip.cap = encode_tc_list_cap(it.k);
         ip.b_eff = it.st->d_b_eff;
         if (!dense) {
-            const size_t t = static_cast<size_t>(it.T), sl = static_cast<size_t>(it.n_slices);
+            const size_t t = static_cast<size_t>(it.T), sl = static_cast<size_t>(it.n_slices) * EPI_GROUPS;
             ip.hint = reinterpret_cast<uint32_t*>(base + hint_off);
             hint_off += round_up(t * 4, 256);
             ip.counts = reinterpret_cast<uint32_t*>(base + off);
@@ -957,7 +970,7 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     for (int q = 0; q < n_items; ++q) {
         const EncodeTcItem& it = items[order[q]];
         const ItemParams& ip = p.item[q];
-        mg.item[q] = MergeItem{ip.cand, ip.counts, ip.hint, it.d_ids, it.d_vals, it.T, it.n_slices, it.k, ip.cap, rows};
+        mg.item[q] = MergeItem{ip.cand, ip.counts, ip.hint, it.d_ids, it.d_vals, it.T, it.n_slices * EPI_GROUPS, it.k, ip.cap, rows};
         rows += (it.T + kMergeRowsPerBlock - 1) / kMergeRowsPerBlock * kMergeRowsPerBlock;
     }
     launch_candidate_merge_group(mg, rows, stream);
