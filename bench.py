@@ -36,7 +36,7 @@ from workloads import configs as C, generators as G  # noqa: E402
 METRIC = "scanned tokens/s (SAE Top-k encode + postings) at 128K ctx"
 # Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, ncu) of one grouped encode launch of the benchmark
 # step (see profiles/); None when the encode kernel has changed since the counters were taken.
-ENCODE_DRAM_BYTES = {}          # (workload, timer name) -> bytes per launch
+ENCODE_DRAM_BYTES = {("cfg3", "encode_query"): 1.14e9}    # (workload, timer name) -> bytes per launch
 UNIT = "tokens/s"
 
 
@@ -132,7 +132,7 @@ class ClockSampler:
                 "samples": len(sel), "reasons": sorted(reasons), "source": self.source}
 
 
-WORKLOADS = {"cfg3": (C.CFG3, C.CFG4), "cfg5": (C.CFG5, None), "cfg2": (C.CFG2, None)}
+WORKLOADS = {"cfg3": (C.CFG3, C.CFG4), "cfg5": (C.CFG5, None), "cfg2": (C.CFG2, None), "cfg1": (C.CFG1, None)}
 
 
 def workload_config(cfg, rcfg, L_idx, ns):
@@ -404,18 +404,26 @@ def run_ours(args, rank, world, local_rank):
     enc_desc = f"encode_tc_kernel, {desc} (T={chunk}; {per_step:g} launch(es) per step; duration includes the Top-k merge kernel)"
     tflops = flops / (enc_avg_ms * 1e-3) / 1e12
     peak, peak_source = pick_tensor_peak(peaks, ms * 1e-3)
+    bound = "tensor"
+    if cfg.dtype == torch.float32:
+        # fp32 inputs run on the FFMA kernel: 128 FMA lanes per SM and clock, at the clock sampled during the run
+        sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+        mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        bound, peak = "alu", sm_count * 128 * 2 * mhz * 1e6 / 1e12
+        peak_source = f"{sm_count} SMs x 128 fp32 FMA lanes x 2 FLOP x {mhz:.0f} MHz (sampled)"
+        enc_desc = enc_desc.replace("encode_tc_kernel", "encode_simt_kernel")
     post_bytes = sum(nl * (chunk * s.k * 8 + (s.d_sae + 1) * 4) for s in slots)
     post_gbs = post_bytes / (kernel_ms["postings"] * 1e-3) / 1e9
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+        "dtype": "f32" if cfg.dtype == torch.float32 else "bf16", "data": "synthetic",
         "config": workload_config(cfg, rcfg, L_idx, ns),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "note": "every step's activations are copied from pinned host memory (double-buffered on a copy stream, overlapping the previous step's kernels) and the step's result is read back, all inside the timed region; postings also travel device->host (index append) in both numbers"},
         "gpu_launches": gpu_launches,
         "clocks": clocks,
-        "roofline": {"bound": "tensor", "kernel": enc_desc,
+        "roofline": {"bound": bound, "kernel": enc_desc,
                      "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak, "peak_source": peak_source,
                      "frac_of_measured_burst": tflops / peaks["bf16_tflops"], "frac_of_measured_sustained": tflops / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": tflops / 2250.0, "launch_ms": enc_avg_ms, "launches_timed": n_timed[enc_name], "flop_per_launch": flops,
@@ -777,7 +785,7 @@ def run_stub(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads | train | project (--k = output width)")
-    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS), help="cfg3 = the 128K-token 4-layer key+query scan the metric is quoted on (default); cfg5 = the 1M-token 8-layer Zipf scan; cfg2 = the 32K-token one-layer scan")
+    ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS), help="cfg3 = the 128K-token 4-layer key+query scan the metric is quoted on (default); cfg5 = the 1M-token 8-layer Zipf scan; cfg2 = the 32K-token one-layer scan; cfg1 = the tiny fp32 scan")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)
     ap.add_argument("--max-ctas", type=int, default=0)

@@ -267,6 +267,8 @@ __device__ void sort_range(const BucketCtx& c, uint32_t f_lo, uint32_t f_hi, uin
     }
     __syncthreads();
     const uint32_t n = FILTER ? c.counters[0] : n_known;
+    __syncthreads();
+    if (tid == 0) c.counters[0] = 0;            // from here on: the number of large groups
 
     // exclusive scan of the counters in (feature, window) order: TBL / 2 / NT words (two counters each) per thread
     {
@@ -303,11 +305,16 @@ __device__ void sort_range(const BucketCtx& c, uint32_t f_lo, uint32_t f_hi, uin
     }
     __syncthreads();
 
-    // groups of two or more entries: insertion sort by token (a repeated token breaks the input contract)
+    // groups of two or more entries (a repeated token breaks the input contract). Up to eight entries: insertion sort
+    // by the group's thread. Larger groups (a feature present in many tokens of one window) go to a second list that
+    // the warps take one group at a time: every entry counts the group's smaller tokens, which is its rank.
     const uint32_t n_conf = c.counters[1];
+    uint16_t* big = c.a_stage;                  // ranks are dead after phase B
+    uint32_t* tmp = c.e_stage;                  // so are the staged entries
     for (uint32_t ci = tid; ci < n_conf; ci += NT) {
         const uint32_t g = conf[ci];
         const uint32_t s = tbl16[g], e_ = g + 1 < (uint32_t)TBL ? tbl16[g + 1] : n;
+        if (e_ - s > 8u) { big[atomicAdd(&c.counters[0], 1u)] = (uint16_t)g; continue; }
         for (uint32_t x = s + 1; x < e_; ++x) {
             const uint32_t v = c.sorted[x];
             const uint32_t vi = vals ? c.sorted_idx[x] : 0u;
@@ -320,6 +327,28 @@ __device__ void sort_range(const BucketCtx& c, uint32_t f_lo, uint32_t f_hi, uin
             }
             c.sorted[y] = v;
             if (vals) c.sorted_idx[y] = vi;
+        }
+    }
+    __syncthreads();
+    const uint32_t n_big = c.counters[0];
+    for (uint32_t bi = warp; bi < n_big; bi += NW) {
+        const uint32_t g = big[bi];
+        const uint32_t s = tbl16[g], e_ = g + 1 < (uint32_t)TBL ? tbl16[g + 1] : n, cnt = e_ - s;
+        for (uint32_t i = lane; i < cnt; i += 32) {
+            const uint32_t v = c.sorted[s + i];
+            uint32_t rank = 0;
+            for (uint32_t j = 0; j < cnt; ++j) {
+                const uint32_t u = c.sorted[s + j];
+                rank += (u < v || (u == v && j < i)) ? 1u : 0u;
+                if (u == v && j != i) dev_set_error(c.status, DEV_DUPLICATE_ID);
+            }
+            tmp[s + rank] = v;
+            if (vals) c.idx_stage[s + rank] = c.sorted_idx[s + i];
+        }
+        __syncwarp();
+        for (uint32_t i = lane; i < cnt; i += 32) {
+            c.sorted[s + i] = tmp[s + i];
+            if (vals) c.sorted_idx[s + i] = c.idx_stage[s + i];
         }
     }
     __syncthreads();

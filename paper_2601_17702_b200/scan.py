@@ -46,9 +46,9 @@ class ScanPipeline:
         self.slots = slots
         self.n_layers = len(slots[0].saes)
         mode = {True: "all", False: "none"}.get(grouped, grouped)
-        self.auto = mode == "auto"
         if not all(sae.dtype == B.S3_BF16 for s in slots for sae in s.saes):
             mode = "none"
+        self.auto = mode == "auto"
         self.group_mode = mode
         self.ws_enc = None         # workspace of the grouped encode, sized at the first chunk
         n_post = sum(B.s3_postings_workspace_bytes(s.chunk, s.k, s.d_sae) for s in slots) * self.n_layers
