@@ -623,6 +623,30 @@ def run_case(args):
             if not args.no_union:
                 S.s3_head_aggregate_topk(ids.view(T, H, k), vals.view(T, H, k), D, k)
         out.update(T=T, H=H, d_head=d_head, d_sae=D, k=k, flop=2.0 * T * H * d_head * D)
+    elif args.case == "project_encode":
+        # the key projection of a Llama-3.1-8B layer (d_model 4096 -> 8 KV heads of 128) and the per-head SAE (128 -> 16384) of one
+        # chunk: fused (the projected tile stays on the SM) or, with --no-union, as the chain projection -> bf16 K -> encode
+        d_model, H, D, k = 4096, 8, cfg.key.d_sae, args.k or cfg.key.k
+        T = args.tokens or cfg.chunk
+        g = torch.Generator(device=dev).manual_seed(1)
+        Wp = (torch.randn((d_model, H * 128), device=dev, generator=g) / d_model ** 0.5).to(torch.bfloat16)
+        proj = S.Sae(Wp, torch.zeros(H * 128, device=dev), torch.zeros(d_model, device=dev))
+        W = (torch.randn((128, D), device=dev, generator=g) / 128 ** 0.5).to(torch.bfloat16)
+        sae = S.Sae(W, torch.zeros(D, device=dev), torch.zeros(128, device=dev))
+        hs = [torch.randn((T, d_model), device=dev, generator=g).to(torch.bfloat16) for _ in range(2)]
+        ids = torch.empty((T, H, k), dtype=torch.int32, device=dev)
+        vals = torch.empty((T, H, k), dtype=torch.float32, device=dev)
+        xbuf = torch.empty((T, H * 128), dtype=torch.bfloat16, device=dev)
+        pws = S.new_workspace(64, dev)
+        ws = S.new_workspace(max(S.s3_sae_project_encode_workspace_bytes(sae, T, H, k), sae.encode_workspace_bytes(T * H, k)), dev)
+
+        def run(i):
+            if args.no_union:
+                S.s3_sae_preact(proj, hs[i % 2], torch.bfloat16, xbuf, pws)
+                S.s3_sae_encode_topk(sae, xbuf.view(T * H, 128), k, ids.view(T * H, k), vals.view(T * H, k), ws)
+            else:
+                S.s3_sae_project_encode_topk(proj, sae, hs[i % 2], H, k, ids, vals, ws)
+        out.update(T=T, d_model=d_model, H=H, d_sae=D, k=k, fused=not args.no_union, flop=2.0 * T * d_model * H * 128 + 2.0 * T * H * 128 * D)
     elif args.case == "project":
         # the upstream projections of a Llama-3.1-8B layer on one chunk (d_model 4096 -> keys 1024, queries 4096) through the
         # dense-epilogue form of the encode GEMM, bf16 in and out
@@ -784,7 +808,7 @@ def run_stub(args, rank, world):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads | train | project (--k = output width)")
+    ap.add_argument("--case", default=None, help="run one kernel alone: encode_key | encode_query | encode_retrieval | postings | score | density | decode | heads | train | project (--k = output width) | project_encode (--no-union: unfused chain)")
     ap.add_argument("--workload", default="cfg3", choices=sorted(WORKLOADS), help="cfg3 = the 128K-token 4-layer key+query scan the metric is quoted on (default); cfg5 = the 1M-token 8-layer Zipf scan; cfg2 = the 32K-token one-layer scan; cfg1 = the tiny fp32 scan")
     ap.add_argument("--tokens", type=int, default=0)
     ap.add_argument("--slices", type=int, default=0)

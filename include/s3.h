@@ -133,6 +133,27 @@ size_t s3_sae_encode_grouped_workspace_bytes(const s3_encode_item* h_items, int 
 s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items, void* d_ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * Upstream projection fused with the per-head encode
+ *            (paper appendix on chunk-independent prefill: the keys of a chunk are K = W_K h; Sec. 3.3: the SAE
+ *             reads one head's projection, x in R^d_head, with one encoder and one feature-ID space for all heads)
+ *
+ * `proj` is a bf16 handle (s3_sae_create) over W_proj [d_model, n_heads * 128] with bias b_enc and b_dec = 0, i.e.
+ * x = h W_proj + b; `sae` is the bf16 encoder of one head (d_in = 128). For every token t and head j:
+ *     x[t,j,:] = bf16(h[t,:] W_proj[:, 128 j : 128 (j+1)] + b)         (fp32 accumulation, round to nearest even)
+ *     ids / vals [t,j,:] = the Top-k code of x[t,j,:] as s3_sae_encode_topk defines it.
+ * A CTA pair computes the head's 256 x 128 tile of x, keeps it in shared memory as the encode GEMM's token operand and
+ * runs the encoder's column tiles on it, so x reaches neither HBM nor L2. The result equals, bit for bit,
+ * s3_sae_preact (bf16 output) followed by s3_sae_encode_topk on the [T * n_heads, 128] view, and feeds
+ * s3_head_aggregate_topk. h is [T, d_model] bf16 with row pitch ldh (multiple of 8).
+ * Limits: d_head = 128 exactly; k <= S3_MAX_K; d_sae <= 65280. Workspace:
+ * s3_sae_project_encode_workspace_bytes(sae, T, n_heads, k).
+ * ---------------------------------------------------------------------------------------------- */
+size_t s3_sae_project_encode_workspace_bytes(const s3_sae* sae, int T_max, int n_heads, int k);
+s3_status s3_sae_project_encode_topk(const s3_sae* proj, const s3_sae* sae, const void* d_h, int64_t ldh, int T, int n_heads,
+                                     int k, int32_t* d_ids /*[T,n_heads,k]*/, float* d_vals /*[T,n_heads,k]*/,
+                                     void* d_ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * SAE encode + ReLU + Top-k without any caller-provided scratch
  *
  * (The paper has no counterpart of this call: it exists for the way some programs have to use this

@@ -26,6 +26,7 @@ EXPORTS = [
     "s3_sae_prepared_bytes", "s3_sae_create", "s3_sae_destroy", "s3_sae_encode_workspace_bytes",
     "s3_sae_encode_topk", "s3_sae_set_schedule", "s3_sae_encode_topk_static",
     "s3_sae_encode_grouped_workspace_bytes", "s3_sae_encode_topk_grouped",
+    "s3_sae_project_encode_workspace_bytes", "s3_sae_project_encode_topk",
     "s3_postings_workspace_bytes", "s3_postings_build", "s3_postings_build_batched",
     "s3_index_create", "s3_index_reserve", "s3_index_append", "s3_index_stream_wait", "s3_index_sync",
     "s3_index_stats", "s3_index_layer_postings", "s3_index_export_csr", "s3_index_destroy",
@@ -104,7 +105,8 @@ def lib():
         L.s3_last_error.restype = C.c_char_p
         for name in ("s3_sae_prepared_bytes", "s3_sae_encode_workspace_bytes", "s3_postings_workspace_bytes",
                      "s3_score_workspace_bytes", "s3_density_workspace_bytes", "s3_fuse_workspace_bytes",
-                     "s3_compact_workspace_bytes", "s3_sae_backward_workspace_bytes", "s3_sae_encode_grouped_workspace_bytes"):
+                     "s3_compact_workspace_bytes", "s3_sae_backward_workspace_bytes", "s3_sae_encode_grouped_workspace_bytes",
+                     "s3_sae_project_encode_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.s3_sae_prepared_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_sae_create.argtypes = [C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
@@ -118,6 +120,9 @@ def lib():
                                                 C.c_void_p, C.c_void_p, C.c_void_p]
         L.s3_sae_encode_grouped_workspace_bytes.argtypes = [C.POINTER(EncodeItem), C.c_int]
         L.s3_sae_encode_topk_grouped.argtypes = [C.POINTER(EncodeItem), C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_sae_project_encode_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int]
+        L.s3_sae_project_encode_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                                 C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.s3_workspace_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
         L.s3_postings_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         L.s3_postings_build.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_void_p,
@@ -268,6 +273,22 @@ def s3_sae_encode_topk_grouped(items: list[EncodeItem], ws: torch.Tensor, stream
     """Several encoder calls (make_encode_item) as one persistent launch plus one selection launch."""
     arr = (EncodeItem * max(len(items), 1))(*items)
     _check(lib().s3_sae_encode_topk_grouped(arr, len(items), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def s3_sae_project_encode_workspace_bytes(sae: Sae, T_max: int, n_heads: int, k: int) -> int:
+    return int(lib().s3_sae_project_encode_workspace_bytes(sae.handle, T_max, n_heads, k))
+
+
+def s3_sae_project_encode_topk(proj: Sae, sae: Sae, h: torch.Tensor, n_heads: int, k: int, ids: torch.Tensor, vals: torch.Tensor,
+                               ws: torch.Tensor, stream=None):
+    """h [T, d_model] bf16 -> per (token, head) Top-k codes ids / vals [T, n_heads, k] of x = h W_proj + b read head by head
+    through the 128-wide encoder `sae`; `proj` is a Sae handle over W_proj [d_model, n_heads * 128] (b_dec = 0)."""
+    assert h.is_cuda and h.dim() == 2 and h.stride(1) == 1 and h.shape[1] == proj.d_in
+    T = h.shape[0]
+    assert ids.dtype == torch.int32 and vals.dtype == torch.float32 and ids.is_contiguous() and vals.is_contiguous()
+    assert tuple(ids.shape) == (T, n_heads, k) and tuple(vals.shape) == (T, n_heads, k)
+    _check(lib().s3_sae_project_encode_topk(proj.handle, sae.handle, _ptr(h), h.stride(0) if T > 1 else max(h.stride(0), proj.d_in),
+                                            T, n_heads, k, _ptr(ids), _ptr(vals), _ptr(ws), ws.numel(), _stream(stream)))
 
 
 def s3_sae_encode_topk_static(sae: Sae, x: torch.Tensor, k: int, ids: torch.Tensor, vals: torch.Tensor,

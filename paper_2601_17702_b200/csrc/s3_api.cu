@@ -281,6 +281,35 @@ s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items,
                                   static_cast<cudaStream_t>(stream));
 }
 
+size_t s3_sae_project_encode_workspace_bytes(const s3_sae* sae, int T_max, int n_heads, int k)
+{
+    if (!sae || T_max < 0 || n_heads < 1 || k < 1 || sae->dtype != S3_BF16) return 0;
+    return 256 + encode_proj_tc_workspace_bytes(T_max, n_heads, k);
+}
+
+s3_status s3_sae_project_encode_topk(const s3_sae* proj, const s3_sae* sae, const void* d_h, int64_t ldh, int T, int n_heads, int k,
+                                     int32_t* d_ids, float* d_vals, void* d_ws, size_t ws_bytes, void* stream)
+{
+    S3_REQUIRE(proj != nullptr && sae != nullptr, S3_ERR_INVALID_ARG, "null handle");
+    S3_REQUIRE(proj->dtype == S3_BF16 && sae->dtype == S3_BF16, S3_ERR_UNSUPPORTED, "bf16 projection and encoder only");
+    S3_REQUIRE(sae->d_in == 128, S3_ERR_UNSUPPORTED, "the per-head encoder must read d_head = 128 values, not %d", sae->d_in);
+    S3_REQUIRE(n_heads >= 1 && proj->d_sae == n_heads * 128, S3_ERR_INVALID_ARG, "the projection yields %d columns, %d heads of 128 expected",
+               proj->d_sae, n_heads);
+    S3_REQUIRE(T >= 0, S3_ERR_INVALID_ARG, "T = %d is negative", T);
+    S3_REQUIRE(k >= 1 && k <= sae->d_sae, S3_ERR_INVALID_ARG, "k = %d out of range [1, d_sae = %d]", k, sae->d_sae);
+    S3_REQUIRE(k <= S3_MAX_K, S3_ERR_UNSUPPORTED, "k = %d exceeds the supported maximum %d", k, S3_MAX_K);
+    S3_REQUIRE(static_cast<int64_t>(T) * n_heads <= INT32_MAX, S3_ERR_UNSUPPORTED, "T * n_heads exceeds 2^31");
+    if (T == 0) return S3_OK;
+    S3_REQUIRE(d_h && d_ids && d_vals && d_ws, S3_ERR_INVALID_ARG, "null device pointer");
+    S3_REQUIRE(aligned16(d_h) && aligned16(d_ws), S3_ERR_INVALID_ARG, "misaligned device pointer");
+    S3_REQUIRE(ldh >= proj->d_in && ldh % 8 == 0, S3_ERR_INVALID_ARG, "ldh = %lld must be a multiple of 8 and >= d_model", (long long)ldh);
+    const size_t need = s3_sae_project_encode_workspace_bytes(sae, T, n_heads, k);
+    S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
+    return launch_encode_proj_tc(&proj->tc, &sae->tc, d_h, ldh, T, proj->d_in, n_heads, sae->d_sae, k, sae->max_ctas,
+                                 static_cast<unsigned char*>(d_ws) + 256, static_cast<uint32_t*>(d_ws), d_ids, d_vals,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 s3_status s3_sae_preact(const s3_sae* sae, const void* d_x, int64_t ldx, int T, void* d_out, int64_t ld_out, s3_dtype out_dtype,
                         void* d_ws, size_t ws_bytes, void* stream)
 {

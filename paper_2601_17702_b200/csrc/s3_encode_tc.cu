@@ -131,6 +131,30 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
+// The same with a cluster-scope release: what the arriving thread wrote to its own shared memory (made visible to the
+// asynchronous proxy with fence.proxy.async first) is ordered before the other CTA's waiter.
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Bounded wait with a cluster-scope acquire (the barrier is signalled by threads of both CTAs).
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag)
+{
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if ((it & 1023u) == 1023u && *abort_flag) return false;
+    }
+    return false;
+}
+
 // Tile load of one CTA of the pair into its own shared memory; the bytes are counted on the mbarrier at
 // cluster address `bar_addr` (the first CTA's), which the .cta_group::2 form allows to lie in the peer CTA.
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_addr)
@@ -197,6 +221,12 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
                                 (static_cast<uint32_t>(PAIR_M >> 4) << 24);
 
+// The same with N = 128: the upstream projection of one head (d_head = 128 output columns).
+constexpr int PROJ_N = 128;
+constexpr uint32_t kInstrDescN128 = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(PROJ_N >> 3) << 17) |
+                                    (static_cast<uint32_t>(PAIR_M >> 4) << 24);
+constexpr int M_SELECT = 0, M_DENSE = 1, M_PROJ = 2;   // epilogue modes of the kernel
+
 constexpr int MAX_GROUP = S3_MAX_ENCODE_ITEMS;   // encoders one launch can serve
 constexpr int MAX_SCHED = 1024;                  // work units a launch can deal out by table
 constexpr int MAX_PAIRS = 96;                    // CTA pairs the table has room for
@@ -220,6 +250,10 @@ struct EncodeTcParams {
     void* dense_out;           // dense mode (one item): the pre-activations [T, ld_out], fp32 or bf16
     long long ld_out;
     int out_bf16, d_sae;
+    // projection mode (one item): the encoder's input is one head of x = h W_proj + b, computed by the same CTA pair just
+    // before the head's tiles. Units are (row tile, head); outputs are indexed by row = token * heads + head.
+    int proj_heads, proj_kblocks;      // heads (0 = no projection), k-blocks of the projection's inner dimension
+    const float* proj_bias;            // [heads * 128]
     ItemParams item[MAX_GROUP];
     uint16_t pair_start[MAX_PAIRS + 1];
     uint16_t sched[MAX_SCHED];
@@ -228,6 +262,7 @@ struct EncodeTcParams {
 struct TensorMaps {
     CUtensorMap x[MAX_GROUP];
     CUtensorMap w[MAX_GROUP];
+    CUtensorMap wk;                    // projection mode: W_proj^T [heads * 128, d_model], box of 64 rows
 };
 
 // The units of one CTA pair, in the order every role of both CTAs walks them.
@@ -245,6 +280,12 @@ __device__ __forceinline__ UnitWalk unit_walk(const EncodeTcParams& p, int pair,
 __device__ __forceinline__ void unit_decode(const EncodeTcParams& p, const UnitWalk& w, int& item, int& slice, int& mt)
 {
     const int u = p.use_sched ? static_cast<int>(p.sched[w.i]) : w.i;
+    if (p.proj_heads > 0) {            // (row tile, head), heads of a row tile next to each other: they share the tile of h
+        item = 0;
+        mt = u / p.proj_heads;
+        slice = u - mt * p.proj_heads;
+        return;
+    }
     item = p.n_items - 1;
     while (item > 0 && p.item[item].unit_start > u) --item;
     const int local = u - p.item[item].unit_start;
@@ -254,17 +295,19 @@ __device__ __forceinline__ void unit_decode(const EncodeTcParams& p, const UnitW
 
 // Shared-memory carve-up (all offsets from a 1024-byte aligned base).
 struct SmemLayout {
-    uint32_t a_off, b_off, pend_off, hist_off, bar_off, total;
+    uint32_t a_off, b_off, x_off, pend_off, hist_off, bar_off, total;
 };
-__host__ __device__ inline SmemLayout smem_layout(int n_stages)
+constexpr int X_TILE_BYTES = 2 * A_STAGE_BYTES;    // projection mode: this CTA's 128 tokens x 128 projected columns, two k-blocks
+__host__ __device__ inline SmemLayout smem_layout(int n_stages, bool proj = false)
 {
     SmemLayout L;
     L.a_off = 0;
     L.b_off = L.a_off + n_stages * A_STAGE_BYTES;
-    L.pend_off = L.b_off + n_stages * B_STAGE_BYTES;
+    L.x_off = L.b_off + n_stages * B_STAGE_BYTES;
+    L.pend_off = L.x_off + (proj ? X_TILE_BYTES : 0);
     L.hist_off = L.pend_off + PEND_CAP * EPI_THREADS * 8;
     L.bar_off = L.hist_off + NB * EPI_THREADS * 2;
-    L.total = L.bar_off + (2 * n_stages + 4) * 8 + 16;
+    L.total = L.bar_off + (2 * n_stages + 5) * 8 + 16;
     return L;
 }
 
@@ -373,22 +416,25 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
 
 // DENSE: the epilogue writes the pre-activations themselves (row-major, fp32 or bf16) instead of selecting; the rest of
 // the kernel is the same pipeline.
-template <bool DENSE>
+template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant__ EncodeTcParams p)
 {
+    constexpr bool DENSE = MODE == M_DENSE, PROJ = MODE == M_PROJ;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const SmemLayout L = smem_layout(p.n_stages);
+    const SmemLayout L = smem_layout(p.n_stages, PROJ);
     unsigned char* smem_a = smem + L.a_off;
     unsigned char* smem_b = smem + L.b_off;
+    unsigned char* smem_x = smem + L.x_off;                // projection mode: the head's projected tile, the encode's A operand
     uint64_t* pend = reinterpret_cast<uint64_t*>(smem + L.pend_off);
     uint16_t* hist = reinterpret_cast<uint16_t*>(smem + L.hist_off);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L.bar_off);
     uint64_t* empty_bar = full_bar + p.n_stages;
     uint64_t* acc_full = empty_bar + p.n_stages;
     uint64_t* acc_empty = acc_full + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* x_ready = acc_empty + 2;                     // projection mode: both CTAs' projected tiles are in shared memory
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(x_ready + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -402,6 +448,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
         // acc_empty: every epilogue thread of both CTAs, on the first CTA's barrier
         for (int s = 0; s < p.n_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 2 * EPI_THREADS); }
+        mbar_init(x_ready, 2 * EPI_THREADS);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -434,9 +481,27 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                 const CUtensorMap* map_x = &maps.x[item];
                 const CUtensorMap* map_w = &maps.w[item];
                 const int kblocks = ip.kblocks;
-                const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
-                const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
+                const int tile_lo = PROJ ? 0 : static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
+                const int tile_hi = PROJ ? ip.n_col_tiles : static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
                 const int row0 = mt * PAIR_M + static_cast<int>(cta_rank) * BM;        // this CTA's tokens
+                if constexpr (PROJ) {
+                    // the head's projection first: 128 tokens of h and this CTA's 64 of the head's 128 rows of W_proj^T per k-block
+                    const int wrow0 = slice * PROJ_N + static_cast<int>(cta_rank) * (PROJ_N / 2);
+                    for (int kb = 0; kb < p.proj_kblocks; ++kb) {
+                        if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag)) {
+                            dev_set_error(p.status, DEV_TIMEOUT_SMEM_EMPTY);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        if (first_cta) mbar_expect_tx(&full_bar[stage], 2 * (A_STAGE_BYTES + B_STAGE_BYTES / 2));
+                        const uint32_t full_addr = map_to_cta(smem_u32(&full_bar[stage]), 0);
+                        tma_load_2d(smem_a + stage * A_STAGE_BYTES, map_x, kb * BK, row0, full_addr);
+                        tma_load_2d(smem_b + stage * B_STAGE_BYTES, &maps.wk, kb * BK, wrow0, full_addr);
+                        ++issued;
+                        if (++stage == static_cast<uint32_t>(p.n_stages)) { stage = 0; phase ^= 1u; }
+                    }
+                }
                 for (int nt = tile_lo; nt < tile_hi && ok; ++nt) {
                     const int col0 = nt * BN + static_cast<int>(cta_rank) * (BN / 2);  // this CTA's half of the features
                     for (int kb = 0; kb < kblocks; ++kb) {
@@ -446,9 +511,9 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                             ok = false;
                             break;
                         }
-                        if (first_cta) mbar_expect_tx(&full_bar[stage], 2 * STAGE_BYTES);
+                        if (first_cta) mbar_expect_tx(&full_bar[stage], PROJ ? 2 * B_STAGE_BYTES : 2 * STAGE_BYTES);
                         const uint32_t full_addr = map_to_cta(smem_u32(&full_bar[stage]), 0);
-                        tma_load_2d(smem_a + stage * A_STAGE_BYTES, map_x, kb * BK, row0, full_addr);
+                        if (!PROJ) tma_load_2d(smem_a + stage * A_STAGE_BYTES, map_x, kb * BK, row0, full_addr);
                         tma_load_2d(smem_b + stage * B_STAGE_BYTES, map_w, kb * BK, col0, full_addr);
                         ++issued;
                         if (++stage == static_cast<uint32_t>(p.n_stages)) { stage = 0; phase ^= 1u; }
@@ -469,15 +534,58 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
         // ---------------- MMA issuer (first CTA of the pair only) ----------------
         if (lane == 0 && first_cta) {
             uint32_t stage = 0, phase = 0;
-            uint32_t tile_count = 0;
+            uint32_t tile_count = 0, unit_count = 0;
             bool ok = true;
             for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
                 int item, slice, mt;
                 unit_decode(p, uw, item, slice, mt);
                 const ItemParams& ip = p.item[item];
                 const int kblocks = ip.kblocks;
-                const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
-                const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
+                const int tile_lo = PROJ ? 0 : static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
+                const int tile_hi = PROJ ? ip.n_col_tiles : static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
+                if constexpr (PROJ) {
+                    // The projection takes its turn in the accumulator rotation like a tile (128 columns of it). Its MMAs
+                    // are issued after the previous head's, so when its accumulator completes the shared-memory tile of the
+                    // previous head is no longer read and the epilogue may overwrite it.
+                    const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+                    if (!mbar_wait(&acc_empty[ab], acc_phase ^ 1u, abort_flag)) {
+                        dev_set_error(p.status, DEV_TIMEOUT_ACC_EMPTY);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + ab * BN;
+                    for (int kb = 0; kb < p.proj_kblocks; ++kb) {
+                        if (!mbar_wait(&full_bar[stage], phase, abort_flag)) {
+                            dev_set_error(p.status, DEV_TIMEOUT_TMA_FULL);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint64_t da = make_smem_desc(smem_u32(smem_a + stage * A_STAGE_BYTES));
+                        const uint64_t db = make_smem_desc(smem_u32(smem_b + stage * B_STAGE_BYTES));
+#pragma unroll
+                        for (int kk = 0; kk < BK / UMMA_K; ++kk)
+                            tc_mma_bf16(d_tmem, da + static_cast<uint64_t>(kk * 2), db + static_cast<uint64_t>(kk * 2), kInstrDescN128,
+                                        (kb | kk) != 0 ? 1u : 0u);
+                        tc_commit_pair(&empty_bar[stage]);
+                        if (++stage == static_cast<uint32_t>(p.n_stages)) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    tc_commit_pair(&acc_full[ab]);
+                    ++tile_count;
+                    // the projected tile (bf16, swizzled like a TMA tile) of both CTAs must be in shared memory
+                    if (!mbar_wait_cluster(x_ready, unit_count & 1u, abort_flag)) {
+                        dev_set_error(p.status, DEV_TIMEOUT_ACC_FULL);
+                        *abort_flag = 1;
+                        ok = false;
+                        break;
+                    }
+                    ++unit_count;
+                    tc_fence_after();
+                }
                 for (int nt = tile_lo; nt < tile_hi && ok; ++nt, ++tile_count) {
                     const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
                     if (!mbar_wait(&acc_empty[ab], acc_phase ^ 1u, abort_flag)) {
@@ -496,7 +604,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                             break;
                         }
                         tc_fence_after();
-                        const uint64_t da = make_smem_desc(smem_u32(smem_a + stage * A_STAGE_BYTES));
+                        const uint64_t da = make_smem_desc(PROJ ? smem_u32(smem_x + kb * A_STAGE_BYTES) : smem_u32(smem_a + stage * A_STAGE_BYTES));
                         const uint64_t db = make_smem_desc(smem_u32(smem_b + stage * B_STAGE_BYTES));
 #pragma unroll
                         for (int kk = 0; kk < BK / UMMA_K; ++kk)
@@ -526,26 +634,72 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             int item, slice, mt;
             unit_decode(p, uw, item, slice, mt);
             const ItemParams& ip = p.item[item];
-            const int tile_lo = static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
-            const int tile_hi = static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
+            const int tile_lo = PROJ ? 0 : static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
+            const int tile_hi = PROJ ? ip.n_col_tiles : static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
             const int t = mt * PAIR_M + static_cast<int>(cta_rank) * BM + e;
             const bool live = t < ip.T;
             const int k = ip.k;
             const uint32_t cap = ip.cap;
+            // projection mode: the unit's "slice" is the head; a (token, head) pair is one output row with one list
+            const size_t orow = PROJ ? static_cast<size_t>(live ? t : 0) * p.proj_heads + slice : static_cast<size_t>(live ? t : 0);
             // each group keeps its own candidate list, bound and histogram for its columns of the row
-            const size_t list_idx = (static_cast<size_t>(live ? t : 0) * ip.n_slices + slice) * EPI_GROUPS + grp;
+            const size_t list_idx = PROJ ? orow * EPI_GROUPS + grp : (orow * ip.n_slices + slice) * EPI_GROUPS + grp;
             uint64_t* glist = DENSE ? nullptr : ip.cand + list_idx * cap;
             if (!DENSE) {
 #pragma unroll 1
                 for (int sl = 0; sl < NB; ++sl) my_hist[sl * EPI_THREADS] = 0;
             }
             // start from the best bound another slice of these rows has published so far, if any
-            const uint32_t hint_in = (live && !DENSE) ? *reinterpret_cast<volatile const uint32_t*>(ip.hint + t) : 0u;
+            const uint32_t hint_in = (live && !DENSE) ? *reinterpret_cast<volatile const uint32_t*>(ip.hint + orow) : 0u;
             RowSel r;
             r.tau_floor = live ? __uint_as_float(hint_in) : INFINITY;    // rows past T select nothing
             r.tau = r.tau_floor;
             r.hbase = -1; r.istar = 0; r.above = 0; r.gcnt = 0; r.floor_exact = false;
             int cnt = 0;                            // entries in this row's pending list
+            if constexpr (PROJ) {
+                // The head's projection: accumulator -> + bias -> bf16 (round to nearest even, as the dense epilogue stores
+                // it) -> this CTA's shared-memory tile in the layout of a 128-byte-swizzled TMA tile (two k-blocks of 128 rows x
+                // 64 columns; the 16-byte chunk c of row r sits at chunk c ^ (r & 7)), where the encode's MMAs read it as A.
+                const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+                const bool arrived = mbar_wait(&acc_full[ab], acc_phase, abort_flag);
+                if (!arrived) {
+                    dev_set_error(p.status, DEV_TIMEOUT_ACC_FULL);
+                    *abort_flag = 1;
+                }
+                if (!__all_sync(0xffffffffu, arrived)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ab * BN + (static_cast<uint32_t>(quarter * 32) << 16);
+                constexpr int PB = PROJ_N / BATCH / EPI_GROUPS;           // batches of 32 columns per group
+                unsigned char* xrow = smem_x + (e >> 3) * 1024 + (e & 7) * 128;
+#pragma unroll 1
+                for (int cb = grp * PB; cb < (grp + 1) * PB; ++cb) {
+                    uint32_t acc[32];
+                    tc_ld32(taddr + cb * BATCH, acc);
+                    const float4* pb4 = reinterpret_cast<const float4*>(p.proj_bias + slice * PROJ_N + cb * BATCH);
+                    float bias[BATCH];
+#pragma unroll
+                    for (int j4 = 0; j4 < BATCH / 4; ++j4) {
+                        const float4 b4 = __ldg(pb4 + j4);
+                        bias[4 * j4 + 0] = b4.x; bias[4 * j4 + 1] = b4.y; bias[4 * j4 + 2] = b4.z; bias[4 * j4 + 3] = b4.w;
+                    }
+                    tc_wait_ld();
+#pragma unroll
+                    for (int g8 = 0; g8 < BATCH / 8; ++g8) {
+                        __nv_bfloat162 h2[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            h2[q] = __floats2bfloat162_rn(__uint_as_float(acc[g8 * 8 + 2 * q]) + bias[g8 * 8 + 2 * q],
+                                                          __uint_as_float(acc[g8 * 8 + 2 * q + 1]) + bias[g8 * 8 + 2 * q + 1]);
+                        const int chunk = (cb & 1) * 4 + g8;              // 16-byte chunk inside the row's 128 bytes of this k-block
+                        *reinterpret_cast<uint4*>(xrow + (cb >> 1) * A_STAGE_BYTES + ((chunk ^ (e & 7)) << 4)) = *reinterpret_cast<const uint4*>(h2);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy stores -> visible to the MMA's reads
+                tc_fence_before();
+                mbar_arrive_cluster(acc_empty_addr[ab]);
+                mbar_arrive_cluster_release(map_to_cta(smem_u32(x_ready), 0));
+                ++tile_count;
+            }
             for (int nt = tile_lo; nt < tile_hi && ok; ++nt, ++tile_count) {
                 const uint32_t ab = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
                 const bool arrived = mbar_wait(&acc_full[ab], acc_phase, abort_flag);
@@ -689,7 +843,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                             if (__uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > cut) glist[w++] = key[q];
                     }
                     ip.counts[list_idx] = w;
-                    if (out > hint_in) atomicMax(ip.hint + t, out);
+                    if (out > hint_in) atomicMax(ip.hint + orow, out);
                 }
             }
         }
@@ -917,8 +1071,8 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     const size_t smem = smem_layout(n_stages).total + 1024;
     static bool attr_set[64] = {};
     if (dev < 64 && !attr_set[dev]) {
-        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
-        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_SELECT>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_DENSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set[dev] = true;
     }
     int n_pairs = encode_tc_max_pairs();
@@ -958,11 +1112,11 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     }
 
     if (dense) {
-        encode_tc_kernel<true><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
+        encode_tc_kernel<M_DENSE><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
         S3_CUDA_TRY(cudaGetLastError());
         return S3_OK;
     }
-    encode_tc_kernel<false><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
+    encode_tc_kernel<M_SELECT><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
     S3_CUDA_TRY(cudaGetLastError());
     MergeGroup mg;
     mg.n_items = n_items;
@@ -1000,5 +1154,75 @@ s3_status launch_preact_tc(const EncodeTcState* st, const void* d_x, int64_t ldx
     const EncodeTcItem it = {st, d_x, ldx, T, d_in, d_sae, 1, n_slices, nullptr, nullptr};
     return launch_tc(&it, 1, max_ctas, nullptr, d_status, d_out, ld_out, out_bf16, stream);
 }
+
+size_t encode_proj_tc_workspace_bytes(int T, int n_heads, int k)
+{
+    return encode_tc_workspace_bytes(T * n_heads, 1, k);
+}
+
+// Projection of one head + encode of that head in the same CTA pair: h [T, d_model] -> x = h W_proj + b (bf16, kept in shared
+// memory) -> Top-k of the d_head = 128 wide encoder, per (token, head).
+s3_status launch_encode_proj_tc(const EncodeTcState* proj, const EncodeTcState* st, const void* d_h, int64_t ldh, int T, int d_model,
+                                int n_heads, int d_sae, int k, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids,
+                                float* d_vals, cudaStream_t stream)
+{
+    alignas(64) TensorMaps maps;
+    EncodeTcParams p;
+    memset(&p, 0, sizeof(p));
+    memset(&maps, 0, sizeof(maps));
+    s3_status rc = make_map(&maps.x[0], d_h, static_cast<uint64_t>(T), static_cast<uint64_t>(d_model), static_cast<uint64_t>(ldh), BM);
+    if (rc != S3_OK) return rc;
+    rc = make_map(&maps.wk, proj->d_wt, static_cast<uint64_t>(n_heads) * PROJ_N, static_cast<uint64_t>(d_model),
+                  static_cast<uint64_t>(d_model), PROJ_N / 2);
+    if (rc != S3_OK) return rc;
+    memcpy(&maps.w[0], st->map_w, sizeof(CUtensorMap));
+    p.n_items = 1;
+    p.status = d_status;
+    p.d_sae = d_sae;
+    p.proj_heads = n_heads;
+    p.proj_kblocks = (d_model + BK - 1) / BK;
+    p.proj_bias = proj->d_b_eff;
+    ItemParams& ip = p.item[0];
+    ip.T = T; ip.d_in = PROJ_N; ip.k = k; ip.kblocks = PROJ_N / BK;
+    ip.n_mtiles = encode_tc_row_tiles(T);
+    ip.n_col_tiles = encode_tc_col_tiles(d_sae);
+    S3_REQUIRE(encode_tc_min_slices(d_sae) == 1, S3_ERR_UNSUPPORTED, "d_sae = %d is too wide for one column slice per head", d_sae);
+    ip.n_slices = 1;
+    ip.unit_start = 0;
+    ip.cap = encode_tc_list_cap(k);
+    ip.b_eff = st->d_b_eff;
+    const size_t rows = static_cast<size_t>(T) * n_heads, lists = EPI_GROUPS;
+    unsigned char* base = static_cast<unsigned char*>(d_scratch);
+    ip.hint = reinterpret_cast<uint32_t*>(base);
+    ip.counts = reinterpret_cast<uint32_t*>(base + round_up(rows * 4, 256));
+    ip.cand = reinterpret_cast<uint64_t*>(base + round_up(rows * 4, 256) + round_up(rows * lists * 4, 256));
+    p.n_units = ip.n_mtiles * n_heads;
+    S3_CUDA_TRY(cudaMemsetAsync(ip.hint, 0, rows * 4, stream));
+
+    int dev = 0;
+    S3_CUDA_TRY(cudaGetDevice(&dev));
+    int max_smem = 0;
+    S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    int n_stages = 6;
+    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, true).total) + 1024 > max_smem) --n_stages;
+    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, true).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
+               "shared memory too small for the encode pipeline");
+    p.n_stages = n_stages;
+    const size_t smem = smem_layout(n_stages, true).total + 1024;
+    static bool attr_set[64] = {};
+    if (dev < 64 && !attr_set[dev]) {
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        attr_set[dev] = true;
+    }
+    int n_pairs = encode_tc_max_pairs();
+    if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
+    if (p.n_units < n_pairs) n_pairs = p.n_units;
+    encode_tc_kernel<M_PROJ><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
+    S3_CUDA_TRY(cudaGetLastError());
+    launch_candidate_merge(ip.cand, ip.counts, ip.hint, static_cast<int>(rows), static_cast<int>(lists), ip.cap, k, d_ids, d_vals, stream);
+    S3_CUDA_TRY(cudaGetLastError());
+    return S3_OK;
+}
+
 
 }  // namespace s3

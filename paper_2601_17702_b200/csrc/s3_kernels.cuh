@@ -38,6 +38,13 @@ struct EncodeTcItem {
 s3_status launch_encode_tc_group(const EncodeTcItem* items, int n_items, int max_ctas, void* d_scratch, uint32_t* d_status,
                                  cudaStream_t stream);
 
+// Projection of a head and its encode in one launch (the projected tile never leaves the SM): proj maps d_model -> n_heads * 128,
+// st is the 128-wide encoder shared by the heads; ids / vals [T, n_heads, k].
+size_t encode_proj_tc_workspace_bytes(int T, int n_heads, int k);
+s3_status launch_encode_proj_tc(const EncodeTcState* proj, const EncodeTcState* st, const void* d_h, int64_t ldh, int T, int d_model,
+                                int n_heads, int d_sae, int k, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids,
+                                float* d_vals, cudaStream_t stream);
+
 // The same GEMM with a dense epilogue: pre-activations [T, ld_out] as fp32 or bf16.
 s3_status launch_preact_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int n_slices,
                            int max_ctas, uint32_t* d_status, void* d_out, int64_t ld_out, bool out_bf16, cudaStream_t stream);
