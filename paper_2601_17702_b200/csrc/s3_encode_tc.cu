@@ -8,7 +8,7 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 x bf16 -> fp32) into
 //               one of two 128x256 accumulators in tensor memory, tcgen05.commit frees the stage /
 //               publishes the accumulator;
-//   warps 2-5   epilogue (one group of four warps; see EPI_GROUPS): thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
+//   warps 2-5   epilogue (four warps per group, one or two groups: see MAX_EPI_GROUPS): thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
 //               biased and compared with the row's bound tau, a value that at least k pre-activations
 //               of the row are known to exceed. Survivors go, branch-free, to a short pending list in
 //               shared memory. When some lane's list is nearly full the warp folds its lists: each
@@ -46,15 +46,14 @@ constexpr int PAIR_M = 2 * BM;                      // tokens per tile over the 
 constexpr int A_STAGE_BYTES = BM * BK * 2;         // 16 KB: this CTA's 128 tokens
 constexpr int B_STAGE_BYTES = (BN / 2) * BK * 2;   // 16 KB: this CTA's half of the tile's 256 features
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;   // per CTA; a stage is complete after twice that
-// Epilogue warp groups: each takes 256 / EPI_GROUPS columns of every tile, with its own bound, histogram and candidate
-// list per row. Two groups were measured and are not used: every list needs its own k survivors, so the work of folding
-// survivors, which is what bounds the narrow encoders, stays the same per thread (key SAE 0.326 ms instead of 0.313).
-#ifndef S3_EPI_GROUPS
-#define S3_EPI_GROUPS 1
-#endif
-constexpr int EPI_GROUPS = S3_EPI_GROUPS;
-constexpr int EPI_THREADS = 128 * EPI_GROUPS;
-constexpr int NUM_THREADS = 64 + EPI_THREADS;
+// Epilogue warp groups (template parameter GROUPS of the kernel): each group of four warps takes 256 / GROUPS columns of
+// every tile, with its own bound, histogram and candidate list per row. One group serves encoders whose tiles take the
+// tensor pipe or the operand feed longer than the filter (d_in >= 1024); two groups serve narrow encoders, where the filter
+// of a single warp per scheduler is the bottleneck and a second warp hides its latencies (d_in 128, k 32: 1.73 -> 1.48 ms;
+// d_in 512, k 16: 1.89 -> 1.71 ms; d_in 1024: 0.646 -> 0.657 ms, hence one group there). The gain is limited because every
+// list needs its own k survivors, so the work of folding survivors does not shrink with the columns per thread.
+constexpr int MAX_EPI_GROUPS = 2;
+constexpr int kTwoGroupsMaxDin = 512;         // encoders at most this wide run with two epilogue groups
 constexpr int TMEM_COLS = 512;
 constexpr int BATCH = 32;                    // columns per tcgen05.ld
 constexpr int STEP = 8;                      // columns filtered between two checks of the pending lists
@@ -298,8 +297,9 @@ struct SmemLayout {
     uint32_t a_off, b_off, x_off, pend_off, hist_off, bar_off, total;
 };
 constexpr int X_TILE_BYTES = 2 * A_STAGE_BYTES;    // projection mode: this CTA's 128 tokens x 128 projected columns, two k-blocks
-__host__ __device__ inline SmemLayout smem_layout(int n_stages, bool proj = false)
+__host__ __device__ inline SmemLayout smem_layout(int n_stages, bool proj, int groups)
 {
+    const int EPI_THREADS = 128 * groups;
     SmemLayout L;
     L.a_off = 0;
     L.b_off = L.a_off + n_stages * A_STAGE_BYTES;
@@ -326,6 +326,7 @@ struct RowSel {
 // if the list stays nearly full it keeps only its k largest keys and restarts the histogram from there.
 // New entries always come from later columns than the list's, so after the exact cut a value equal to
 // the k-th key's can no longer win (ties go to the lower id) and the strict comparison stays exact.
+template <int EPI_THREADS>
 __device__ __noinline__ void prune_list(uint64_t* glist, uint16_t* my_hist, RowSel& r, int k, uint32_t cap)
 {
     uint32_t w = 0;
@@ -360,11 +361,12 @@ __device__ __noinline__ void prune_list(uint64_t* glist, uint16_t* my_hist, RowS
 
 // Folds the warp's pending lists (cnt entries per lane) into candidate lists and histograms, then
 // raises each row's bound as far as the histogram allows. Called by all 32 lanes.
+template <int EPI_THREADS>
 __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_hist, uint64_t* glist, RowSel& r, int& cnt,
                                              int k, uint32_t cap)
 {
     if (__any_sync(0xffffffffu, r.gcnt + cnt > cap)) {
-        if (r.gcnt + cnt > cap) prune_list(glist, my_hist, r, k, cap);
+        if (r.gcnt + cnt > cap) prune_list<EPI_THREADS>(glist, my_hist, r, k, cap);
     }
     if (r.hbase < 0 && cnt > 0) {
         uint32_t ref = __float_as_uint(r.tau);
@@ -416,14 +418,15 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
 
 // DENSE: the epilogue writes the pre-activations themselves (row-major, fp32 or bf16) instead of selecting; the rest of
 // the kernel is the same pipeline.
-template <int MODE>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+template <int MODE, int GROUPS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(64 + 128 * GROUPS, 1)
 encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant__ EncodeTcParams p)
 {
     constexpr bool DENSE = MODE == M_DENSE, PROJ = MODE == M_PROJ;
+    constexpr int EPI_GROUPS = GROUPS, EPI_THREADS = 128 * GROUPS;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const SmemLayout L = smem_layout(p.n_stages, PROJ);
+    const SmemLayout L = smem_layout(p.n_stages, PROJ, GROUPS);
     unsigned char* smem_a = smem + L.a_off;
     unsigned char* smem_b = smem + L.b_off;
     unsigned char* smem_x = smem + L.x_off;                // projection mode: the head's projected tile, the encode's A operand
@@ -815,14 +818,14 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                             slot[o3 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[3])) << 32) | (nc - 3u);
                             cnt += o3 + keep[3];
                         }
-                        if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) fold_pending(my_pend, my_hist, glist, r, cnt, k, cap);
+                        if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) fold_pending<EPI_THREADS>(my_pend, my_hist, glist, r, cnt, k, cap);
                     }
                 }
                 tc_fence_before();
                 mbar_arrive_cluster(acc_empty_addr[ab]);
             }
             if (ok && !DENSE) {
-                if (__any_sync(0xffffffffu, cnt > 0)) fold_pending(my_pend, my_hist, glist, r, cnt, k, cap);
+                if (__any_sync(0xffffffffu, cnt > 0)) fold_pending<EPI_THREADS>(my_pend, my_hist, glist, r, cnt, k, cap);
                 if (live) {
                     // The bound to publish: at least k values of this slice exceed it. An exact k-th value
                     // only bounds from below after stepping to the next float down.
@@ -975,15 +978,16 @@ int encode_tc_max_pairs()
 }
 
 // Slots of one candidate list (one per row, slice and epilogue group); a list that fills up is pruned in place.
-uint32_t encode_tc_list_cap(int k) { return static_cast<uint32_t>((k < 4 ? 64 : 16 * k) / EPI_GROUPS); }
+uint32_t encode_tc_list_cap(int k, int groups) { return static_cast<uint32_t>((k < 4 ? 64 : 16 * k) / groups); }
 
 // Column tiles per slice may not exceed 255: a row's histogram counters are 16 bits wide.
 int encode_tc_min_slices(int d_sae) { return (encode_tc_col_tiles(d_sae) + 254) / 255; }
 
 size_t encode_tc_workspace_bytes(int T, int n_slices, int k)
 {
-    const size_t t = static_cast<size_t>(T), s = static_cast<size_t>(n_slices) * EPI_GROUPS;    // candidate lists per row
-    return round_up(t * 4, 256) + round_up(t * s * 4, 256) + round_up(t * s * encode_tc_list_cap(k) * sizeof(uint64_t), 256);
+    // sized for either number of epilogue groups: two lists of half the slots take the room of one list
+    const size_t t = static_cast<size_t>(T), s = static_cast<size_t>(n_slices) * MAX_EPI_GROUPS;    // candidate lists per row
+    return round_up(t * 4, 256) + round_up(t * s * 4, 256) + round_up(t * s * encode_tc_list_cap(k, MAX_EPI_GROUPS) * sizeof(uint64_t), 256);
 }
 
 namespace {
@@ -1010,6 +1014,9 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     p.status = d_status;
     p.dense_out = d_dense; p.ld_out = ld_out; p.out_bf16 = out_bf16 ? 1 : 0;
     p.d_sae = items[0].d_sae;
+    int max_d_in = 0;
+    for (int j = 0; j < n_items; ++j) max_d_in = items[j].d_in > max_d_in ? items[j].d_in : max_d_in;
+    const int groups = (!dense && max_d_in <= kTwoGroupsMaxDin) ? 2 : 1;
 
     // items in descending order of their units' modelled duration, so that the short units fill the end of the launch
     int order[MAX_GROUP];
@@ -1043,10 +1050,10 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
         ip.n_slices = it.n_slices;
         ip.unit_start = n_units;
         n_units += ip.n_mtiles * it.n_slices;
-        ip.cap = encode_tc_list_cap(it.k);
+        ip.cap = encode_tc_list_cap(it.k, groups);
         ip.b_eff = it.st->d_b_eff;
         if (!dense) {
-            const size_t t = static_cast<size_t>(it.T), sl = static_cast<size_t>(it.n_slices) * EPI_GROUPS;
+            const size_t t = static_cast<size_t>(it.T), sl = static_cast<size_t>(it.n_slices) * groups;
             ip.hint = reinterpret_cast<uint32_t*>(base + hint_off);
             hint_off += round_up(t * 4, 256);
             ip.counts = reinterpret_cast<uint32_t*>(base + off);
@@ -1064,15 +1071,16 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     int max_smem = 0;
     S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     int n_stages = 6;
-    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages).total) + 1024 > max_smem) --n_stages;
-    S3_REQUIRE(static_cast<int>(smem_layout(n_stages).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
+    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, false, groups).total) + 1024 > max_smem) --n_stages;
+    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, false, groups).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
                "shared memory too small for the encode pipeline");
     p.n_stages = n_stages;
-    const size_t smem = smem_layout(n_stages).total + 1024;
+    const size_t smem = smem_layout(n_stages, false, groups).total + 1024;
     static bool attr_set[64] = {};
     if (dev < 64 && !attr_set[dev]) {
-        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_SELECT>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
-        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_DENSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_SELECT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_SELECT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_DENSE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set[dev] = true;
     }
     int n_pairs = encode_tc_max_pairs();
@@ -1112,11 +1120,12 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     }
 
     if (dense) {
-        encode_tc_kernel<M_DENSE><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
+        encode_tc_kernel<M_DENSE, 1><<<2 * n_pairs, 64 + 128, smem, stream>>>(maps, p);
         S3_CUDA_TRY(cudaGetLastError());
         return S3_OK;
     }
-    encode_tc_kernel<M_SELECT><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
+    if (groups == 2) encode_tc_kernel<M_SELECT, 2><<<2 * n_pairs, 64 + 256, smem, stream>>>(maps, p);
+    else encode_tc_kernel<M_SELECT, 1><<<2 * n_pairs, 64 + 128, smem, stream>>>(maps, p);
     S3_CUDA_TRY(cudaGetLastError());
     MergeGroup mg;
     mg.n_items = n_items;
@@ -1124,7 +1133,7 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     for (int q = 0; q < n_items; ++q) {
         const EncodeTcItem& it = items[order[q]];
         const ItemParams& ip = p.item[q];
-        mg.item[q] = MergeItem{ip.cand, ip.counts, ip.hint, it.d_ids, it.d_vals, it.T, it.n_slices * EPI_GROUPS, it.k, ip.cap, rows};
+        mg.item[q] = MergeItem{ip.cand, ip.counts, ip.hint, it.d_ids, it.d_vals, it.T, it.n_slices * groups, it.k, ip.cap, rows};
         rows += (it.T + kMergeRowsPerBlock - 1) / kMergeRowsPerBlock * kMergeRowsPerBlock;
     }
     launch_candidate_merge_group(mg, rows, stream);
@@ -1189,9 +1198,10 @@ s3_status launch_encode_proj_tc(const EncodeTcState* proj, const EncodeTcState* 
     S3_REQUIRE(encode_tc_min_slices(d_sae) == 1, S3_ERR_UNSUPPORTED, "d_sae = %d is too wide for one column slice per head", d_sae);
     ip.n_slices = 1;
     ip.unit_start = 0;
-    ip.cap = encode_tc_list_cap(k);
+    constexpr int groups = 2;                  // d_head = 128: the narrow-encoder configuration
+    ip.cap = encode_tc_list_cap(k, groups);
     ip.b_eff = st->d_b_eff;
-    const size_t rows = static_cast<size_t>(T) * n_heads, lists = EPI_GROUPS;
+    const size_t rows = static_cast<size_t>(T) * n_heads, lists = groups;
     unsigned char* base = static_cast<unsigned char*>(d_scratch);
     ip.hint = reinterpret_cast<uint32_t*>(base);
     ip.counts = reinterpret_cast<uint32_t*>(base + round_up(rows * 4, 256));
@@ -1204,20 +1214,20 @@ s3_status launch_encode_proj_tc(const EncodeTcState* proj, const EncodeTcState* 
     int max_smem = 0;
     S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     int n_stages = 6;
-    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, true).total) + 1024 > max_smem) --n_stages;
-    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, true).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
+    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, true, groups).total) + 1024 > max_smem) --n_stages;
+    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, true, groups).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
                "shared memory too small for the encode pipeline");
     p.n_stages = n_stages;
-    const size_t smem = smem_layout(n_stages, true).total + 1024;
+    const size_t smem = smem_layout(n_stages, true, groups).total + 1024;
     static bool attr_set[64] = {};
     if (dev < 64 && !attr_set[dev]) {
-        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+        S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_PROJ, groups>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set[dev] = true;
     }
     int n_pairs = encode_tc_max_pairs();
     if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
     if (p.n_units < n_pairs) n_pairs = p.n_units;
-    encode_tc_kernel<M_PROJ><<<2 * n_pairs, NUM_THREADS, smem, stream>>>(maps, p);
+    encode_tc_kernel<M_PROJ, groups><<<2 * n_pairs, 64 + 128 * groups, smem, stream>>>(maps, p);
     S3_CUDA_TRY(cudaGetLastError());
     launch_candidate_merge(ip.cand, ip.counts, ip.hint, static_cast<int>(rows), static_cast<int>(lists), ip.cap, k, d_ids, d_vals, stream);
     S3_CUDA_TRY(cudaGetLastError());
