@@ -59,6 +59,10 @@ constexpr int BATCH = 32;                    // columns per tcgen05.ld
 constexpr int STEP = 8;                      // columns filtered between two checks of the pending lists
 constexpr int PEND_CAP = 2 * STEP;           // pending-list slots per row
 constexpr int NB = 64;                       // histogram buckets per row
+#ifndef S3_FOLD_CHUNK
+#define S3_FOLD_CHUNK 4
+#endif
+constexpr int FOLD_CHUNK = S3_FOLD_CHUNK;    // pending entries a fold handles per step
 constexpr int kCompactMinTiles = 32;          // units of at least this many column tiles compact their candidate lists
 constexpr int COLD_LEVELS = 6;                // trial bounds of the cold-start pass, as fractions of the first batch's maximum
 __device__ constexpr float kColdFraction[COLD_LEVELS] = {0.80f, 0.65f, 0.52f, 0.40f, 0.30f, 0.20f};
@@ -382,18 +386,38 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
         }
     }
     const int nmax = __reduce_max_sync(0xffffffffu, cnt);
-    for (int i = 0; i < nmax; ++i) {
-        if (i < cnt) {
-            const uint64_t key = my_pend[i * EPI_THREADS];
-            const uint32_t vb = static_cast<uint32_t>(key >> 32);
-            if (__uint_as_float(vb) > r.tau) {
-                int idx = static_cast<int>(vb >> HSHIFT) - r.hbase;
-                idx = idx < 0 ? 0 : (idx > NB - 1 ? NB - 1 : idx);
-                my_hist[idx * EPI_THREADS] += 1;
+    // FOLD_CHUNK entries at a time: their loads first, then the list stores, then the histogram, so that the
+    // shared-memory round trips of a chunk overlap instead of forming one dependent chain per entry
+    for (int i0 = 0; i0 < nmax; i0 += FOLD_CHUNK) {
+        uint64_t key[FOLD_CHUNK];
+        int idx[FOLD_CHUNK];
+        bool ok[FOLD_CHUNK];
+#pragma unroll
+        for (int q = 0; q < FOLD_CHUNK; ++q) key[q] = (i0 + q < cnt) ? my_pend[(i0 + q) * EPI_THREADS] : 0ull;
+#pragma unroll
+        for (int q = 0; q < FOLD_CHUNK; ++q) {
+            const uint32_t vb = static_cast<uint32_t>(key[q] >> 32);
+            ok[q] = (i0 + q < cnt) && __uint_as_float(vb) > r.tau;
+            int ix = static_cast<int>(vb >> HSHIFT) - r.hbase;
+            idx[q] = ix < 0 ? 0 : (ix > NB - 1 ? NB - 1 : ix);
+        }
+#pragma unroll
+        for (int q = 0; q < FOLD_CHUNK; ++q)
+            if (ok[q]) glist[r.gcnt++] = key[q];
+        // one histogram update per run of equal buckets (survivors cluster in the buckets just above the bound)
+        int run_idx = -1, run_n = 0;
+#pragma unroll
+        for (int q = 0; q < FOLD_CHUNK; ++q) {
+            if (ok[q]) {
+                if (idx[q] == run_idx) ++run_n;
+                else {
+                    if (run_n) my_hist[run_idx * EPI_THREADS] += static_cast<uint16_t>(run_n);
+                    run_idx = idx[q]; run_n = 1;
+                }
                 r.above += 1;
-                glist[r.gcnt++] = key;
             }
         }
+        if (run_n) my_hist[run_idx * EPI_THREADS] += static_cast<uint16_t>(run_n);
     }
     cnt = 0;
     while (r.istar < NB - 1) {
