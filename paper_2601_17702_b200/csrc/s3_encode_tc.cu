@@ -836,10 +836,10 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                             const int o1 = keep[0], o2 = o1 + keep[1], o3 = o2 + keep[2];
                             uint64_t* slot = my_pend + cnt * EPI_THREADS;
                             const uint32_t nc = ncol0 - static_cast<uint32_t>(h * STEP + j);
-                            slot[0] = (static_cast<uint64_t>(__float_as_uint(v[0])) << 32) | nc;
-                            slot[o1 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[1])) << 32) | (nc - 1u);
-                            slot[o2 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[2])) << 32) | (nc - 2u);
-                            slot[o3 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[3])) << 32) | (nc - 3u);
+                            if (keep[0]) slot[0] = (static_cast<uint64_t>(__float_as_uint(v[0])) << 32) | nc;
+                            if (keep[1]) slot[o1 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[1])) << 32) | (nc - 1u);
+                            if (keep[2]) slot[o2 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[2])) << 32) | (nc - 2u);
+                            if (keep[3]) slot[o3 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[3])) << 32) | (nc - 3u);
                             cnt += o3 + keep[3];
                         }
                         if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) fold_pending<EPI_THREADS>(my_pend, my_hist, glist, r, cnt, k, cap);
