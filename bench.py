@@ -196,7 +196,7 @@ def run_ours(args, rank, world, local_rank):
     slots = [SaeSlot("key", key_saes, cfg.key.k, chunk)]
     if cfg.query:
         slots.append(SaeSlot("query", [S.Sae(*inp.sae("query", l)) for l in range(nl)], cfg.query.k, chunk))
-    pipe = ScanPipeline(slots, grouped=args.group)
+    pipe = ScanPipeline(slots, grouped=args.group, overlap=args.overlap)
     e2e_steps = max(2, min(args.steps, 8))
     total_steps = 2 * args.steps + args.warmup + e2e_steps + 4
     pipe.reserve_index((total_steps + 2) * chunk)
@@ -824,6 +824,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference", "stub"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--overlap", action="store_true", help="run the grouped launch of narrow encoders on a second stream beside the wide encoders' launches (on the SMs those leave free) instead of after them")
     ap.add_argument("--group", default="auto", help="how a chunk's encodes are launched: all | slot | none | <stream name> | auto")
     ap.add_argument("--cpu-sample-tokens", type=int, default=2048, help="context tokens the CPU oracle is timed on for cpu_baseline")
     args = ap.parse_args()

@@ -117,7 +117,8 @@ s3_status s3_sae_set_schedule(s3_sae* sae, int n_slices, int max_ctas);
  * the launch ends evenly. Each item has its own encoder, input, T, k and outputs; the results are those of
  * s3_sae_encode_topk item by item (bit-identical: the selection is exact, whatever the schedule).
  * bf16 encoders only (S3_ERR_UNSUPPORTED otherwise); an item with T == 0 is skipped. `h_items` is a HOST
- * array. Workspace: s3_sae_encode_grouped_workspace_bytes(h_items, n_items) (status block + every item's
+ * array. max_ctas > 0 limits the launch to that many thread blocks (an even number is used), for launches that
+ * share the GPU with another stream's kernel. Workspace: s3_sae_encode_grouped_workspace_bytes(h_items, n_items) (status block + every item's
  * candidate lists).
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
@@ -130,7 +131,11 @@ typedef struct {
 } s3_encode_item;
 
 size_t s3_sae_encode_grouped_workspace_bytes(const s3_encode_item* h_items, int n_items);
-s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items, void* d_ws, size_t ws_bytes, void* stream);
+s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items, int max_ctas /*0 = all SMs*/,
+                                     void* d_ws, size_t ws_bytes, void* stream);
+/* Thread blocks (one per SM) that s3_sae_encode_topk will occupy for T tokens: a launch over few work units leaves SMs
+ * free, on which a grouped launch limited with max_ctas can run at the same time from another stream. */
+int s3_sae_encode_ctas(const s3_sae* sae, int T);
 
 /* ------------------------------------------------------------------------------------------------
  * Upstream projection fused with the per-head encode

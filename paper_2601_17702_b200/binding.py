@@ -25,7 +25,7 @@ EXPORTS = [
     "s3_last_error", "s3_version", "s3_workspace_status",
     "s3_sae_prepared_bytes", "s3_sae_create", "s3_sae_destroy", "s3_sae_encode_workspace_bytes",
     "s3_sae_encode_topk", "s3_sae_set_schedule", "s3_sae_encode_topk_static",
-    "s3_sae_encode_grouped_workspace_bytes", "s3_sae_encode_topk_grouped",
+    "s3_sae_encode_grouped_workspace_bytes", "s3_sae_encode_topk_grouped", "s3_sae_encode_ctas",
     "s3_sae_project_encode_workspace_bytes", "s3_sae_project_encode_topk",
     "s3_postings_workspace_bytes", "s3_postings_build", "s3_postings_build_batched",
     "s3_index_create", "s3_index_reserve", "s3_index_append", "s3_index_stream_wait", "s3_index_sync",
@@ -119,7 +119,8 @@ def lib():
         L.s3_sae_encode_topk_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_void_p,
                                                 C.c_void_p, C.c_void_p, C.c_void_p]
         L.s3_sae_encode_grouped_workspace_bytes.argtypes = [C.POINTER(EncodeItem), C.c_int]
-        L.s3_sae_encode_topk_grouped.argtypes = [C.POINTER(EncodeItem), C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_sae_encode_topk_grouped.argtypes = [C.POINTER(EncodeItem), C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.s3_sae_encode_ctas.argtypes = [C.c_void_p, C.c_int]
         L.s3_sae_project_encode_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int]
         L.s3_sae_project_encode_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                                  C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -269,10 +270,16 @@ def s3_sae_encode_grouped_workspace_bytes(items: list[EncodeItem]) -> int:
     return int(lib().s3_sae_encode_grouped_workspace_bytes(arr, len(items)))
 
 
-def s3_sae_encode_topk_grouped(items: list[EncodeItem], ws: torch.Tensor, stream=None):
-    """Several encoder calls (make_encode_item) as one persistent launch plus one selection launch."""
+def s3_sae_encode_topk_grouped(items: list[EncodeItem], ws: torch.Tensor, max_ctas: int = 0, stream=None):
+    """Several encoder calls (make_encode_item) as one persistent launch plus one selection launch; max_ctas > 0
+    limits the launch to that many thread blocks."""
     arr = (EncodeItem * max(len(items), 1))(*items)
-    _check(lib().s3_sae_encode_topk_grouped(arr, len(items), _ptr(ws), ws.numel(), _stream(stream)))
+    _check(lib().s3_sae_encode_topk_grouped(arr, len(items), max_ctas, _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def s3_sae_encode_ctas(sae: Sae, T: int) -> int:
+    """Thread blocks an s3_sae_encode_topk launch over T tokens occupies."""
+    return int(lib().s3_sae_encode_ctas(sae.handle, T))
 
 
 def s3_sae_project_encode_workspace_bytes(sae: Sae, T_max: int, n_heads: int, k: int) -> int:

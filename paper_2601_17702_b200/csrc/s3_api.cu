@@ -256,15 +256,27 @@ size_t s3_sae_encode_grouped_workspace_bytes(const s3_encode_item* h_items, int 
     return n;
 }
 
-s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items, void* d_ws, size_t ws_bytes, void* stream)
+int s3_sae_encode_ctas(const s3_sae* sae, int T)
 {
+    if (!sae || T <= 0) return 0;
+    if (sae->dtype != S3_BF16) return device_sm_count();
+    const int units = row_tiles(sae, T) * pick_slices(sae, T);
+    int pairs = encode_tc_max_pairs();
+    if (sae->max_ctas > 0 && sae->max_ctas / 2 < pairs) pairs = sae->max_ctas / 2 > 0 ? sae->max_ctas / 2 : 1;
+    return 2 * (units < pairs ? units : pairs);
+}
+
+s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items, int max_ctas_arg, void* d_ws, size_t ws_bytes,
+                                     void* stream)
+{
+    S3_REQUIRE(max_ctas_arg >= 0, S3_ERR_INVALID_ARG, "max_ctas is negative");
     S3_REQUIRE(n_items >= 0, S3_ERR_INVALID_ARG, "n_items is negative");
     if (n_items == 0) return S3_OK;
     S3_REQUIRE(h_items != nullptr, S3_ERR_INVALID_ARG, "h_items is null");
     S3_REQUIRE(n_items <= S3_MAX_ENCODE_ITEMS, S3_ERR_UNSUPPORTED, "n_items = %d exceeds %d", n_items, S3_MAX_ENCODE_ITEMS);
     S3_REQUIRE(d_ws != nullptr && aligned16(d_ws), S3_ERR_INVALID_ARG, "d_ws is null or misaligned");
     EncodeTcItem items[S3_MAX_ENCODE_ITEMS];
-    int n = 0, max_ctas = 0;
+    int n = 0, max_ctas = max_ctas_arg;
     for (int i = 0; i < n_items; ++i) {
         const s3_status st = check_encode_item(h_items[i], i);
         if (st != S3_OK) return st;

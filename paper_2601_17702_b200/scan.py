@@ -37,14 +37,21 @@ class SaeSlot:
 
 
 class ScanPipeline:
-    def __init__(self, slots: list[SaeSlot], grouped: bool | str = "auto"):
+    def __init__(self, slots: list[SaeSlot], grouped: bool | str = "auto", overlap: bool = False):
         """grouped: how the encodes of a chunk are launched (bf16 encoders; fp32 ones always go one by one).
         True / "all": the layers of all SAE streams in grouped launches (one persistent kernel per up to
         S3_MAX_ENCODE_ITEMS encoders); "slot": one grouped launch per SAE stream; a stream's name (e.g. "key"): only
         that stream's layers are grouped; False / "none": one launch pair per encoder; "auto" (default): per stream,
-        grouped when the encoder input is at most AUTO_GROUP_MAX_D_IN wide."""
+        grouped when the encoder input is at most AUTO_GROUP_MAX_D_IN wide.
+        overlap: when a chunk has both wide encoders (launched one by one, each leaving some SMs without a work unit) and
+        a grouped launch of narrow ones, the grouped launch runs on a second stream, limited to the SMs the wide launches
+        leave free, so that it proceeds beside them instead of after them. Off by default: measured on the 128K-token
+        workload the four key encoders then take the whole window of the query launches on the 10 free CTA pairs (8.3 ms
+        instead of 1.3 ms alone) while each query launch runs 6 % slower beside them, and the step gets no shorter."""
         self.slots = slots
         self.n_layers = len(slots[0].saes)
+        self.overlap = overlap
+        self.side = None           # second stream of the overlapped grouped launch
         mode = {True: "all", False: "none"}.get(grouped, grouped)
         if not all(sae.dtype == B.S3_BF16 for s in slots for sae in s.saes):
             mode = "none"
@@ -78,6 +85,7 @@ class ScanPipeline:
         out the hand-over to the host index (to time the device work without the copies)."""
         items = []
         enc_items = []
+        singles = []
         T = None
         for s in self.slots:
             xs = x_by_slot[s.name]
@@ -87,9 +95,7 @@ class ScanPipeline:
                 if self.group_mode in ("all", "slot", s.name) or (self.auto and s.saes[l].d_in <= AUTO_GROUP_MAX_D_IN):
                     enc_items.append((s.name, B.make_encode_item(s.saes[l], x, s.k, s.ids[l][:T], s.vals[l][:T])))
                 else:
-                    with self._timed("encode_" + s.name):
-                        B.s3_sae_encode_topk(s.saes[l], x, s.k, s.ids[l][:T], s.vals[l][:T], s.ws)
-                    self.launches += 2
+                    singles.append((s, l, x))
                 items.append(B.make_postings_item(s.ids[l][:T], s.d_sae, pos_base, s.row_ptr[l], s.pos[l],
                                                   s.vals[l][:T] if s.pval else None, s.pval[l] if s.pval else None))
         groups = []
@@ -102,10 +108,28 @@ class ScanPipeline:
         if groups and (self.ws_enc is None or self.ws_enc.numel() < need):
             assert self.ws_enc is None, "the grouped-encode workspace is sized by the first (full) chunk"
             self.ws_enc = B.new_workspace(need, self.slots[0].ids[0].device)
-        for name, group in groups:
-            with self._timed("encode_group" if self.group_mode == "all" else "encode_group_" + name):
-                B.s3_sae_encode_topk_grouped(group, self.ws_enc)
-            self.launches += 2         # persistent encode over all items, selection over all items
+
+        # SMs the wide launches leave without a work unit: the grouped launch of the narrow encoders can have them
+        free_ctas = 0
+        if self.overlap and groups and singles:
+            n_sm = torch.cuda.get_device_properties(self.slots[0].ids[0].device).multi_processor_count
+            free_ctas = min(n_sm - B.s3_sae_encode_ctas(s.saes[l], x.shape[0]) for s, l, x in singles)
+        main = torch.cuda.current_stream()
+        if free_ctas >= 2:
+            if self.side is None:
+                self.side = torch.cuda.Stream(device=self.slots[0].ids[0].device)
+            self.side.wait_stream(main)          # the chunk's inputs, and the previous chunk's postings that read ids, are done
+        for s, l, x in singles:
+            with self._timed("encode_" + s.name):
+                B.s3_sae_encode_topk(s.saes[l], x, s.k, s.ids[l][:x.shape[0]], s.vals[l][:x.shape[0]], s.ws)
+            self.launches += 2
+        with torch.cuda.stream(self.side if free_ctas >= 2 else main):
+            for name, group in groups:
+                with self._timed("encode_group" if self.group_mode == "all" else "encode_group_" + name):
+                    B.s3_sae_encode_topk_grouped(group, self.ws_enc, free_ctas if free_ctas >= 2 else 0)
+                self.launches += 2         # persistent encode over all items, selection over all items
+        if free_ctas >= 2:
+            main.wait_stream(self.side)
         # the previous chunk's device->host copies read row_ptr/pos: order the overwrite after them
         for s in self.slots:
             s.index.stream_wait()

@@ -589,10 +589,10 @@ def test_grouped_encode_equals_the_single_calls_bit_for_bit():
         np.testing.assert_array_equal(vals.cpu().numpy(), vals1)
         pre = O.preact(x.float().numpy(), W.float().numpy(), b_enc.numpy(), b_dec.numpy())
         check_topk_against_preact(pre, ids.cpu().numpy(), vals.cpu().numpy(), k, TOL_BF16)
-    # a second launch over the leftovers of the first gives the same bits
+    # a second launch over the leftovers of the first, limited to a few thread blocks, gives the same bits
     for ids, vals in outs:
         ids.fill_(-9)
-    S.s3_sae_encode_topk_grouped(items, ws)
+    S.s3_sae_encode_topk_grouped(items, ws, max_ctas=20)
     for (T, d_in, d_sae, k), (sae, W, b_enc, b_dec), x, (ids, vals) in zip(shapes, saes, xs, outs):
         if T:
             np.testing.assert_array_equal(ids.cpu().numpy(), gpu_encode(W, b_enc, b_dec, x, k)[0])
