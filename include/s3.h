@@ -136,6 +136,17 @@ s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items,
 /* Thread blocks (one per SM) that s3_sae_encode_topk will occupy for T tokens: a launch over few work units leaves SMs
  * free, on which a grouped launch limited with max_ctas can run at the same time from another stream. */
 int s3_sae_encode_ctas(const s3_sae* sae, int T);
+/* The work units a launch over n_items bf16 encoder calls (HOST arrays T, d_in, d_sae, k) is cut into on n_pairs pairs of
+ * thread blocks; host arithmetic only, no device is touched. A unit is a run of 256-column tiles of one 256-token row
+ * tile of one item, and its survivors go to one of the row's candidate lists ("slot"). Encoders whose weights stay in L2
+ * are cut into one contiguous share of equal modelled duration per pair (pieces of at least three column tiles, a row
+ * tile spread over neighbouring pairs); wider encoders keep uniform column slices walked in step, so that the pairs read
+ * the same weight tiles at the same time. Writes six integers per unit to h_units (pair, item, row tile, first column
+ * tile, one past the last, slot), at most max_units units, and every item's slots per row to h_slots [n_items].
+ * Returns the number of units, -1 when the launch deals uniform slices round-robin without a unit table (only h_slots is
+ * written), -2 on invalid arguments. The selection result never depends on the schedule (Eq. 3 is exact). */
+int s3_encode_schedule_describe(const int32_t* T, const int32_t* d_in, const int32_t* d_sae, const int32_t* k, int n_items,
+                                int n_pairs, int32_t* h_units, int max_units, int32_t* h_slots);
 
 /* ------------------------------------------------------------------------------------------------
  * Upstream projection fused with the per-head encode

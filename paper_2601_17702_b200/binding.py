@@ -25,7 +25,7 @@ EXPORTS = [
     "s3_last_error", "s3_version", "s3_workspace_status",
     "s3_sae_prepared_bytes", "s3_sae_create", "s3_sae_destroy", "s3_sae_encode_workspace_bytes",
     "s3_sae_encode_topk", "s3_sae_set_schedule", "s3_sae_encode_topk_static",
-    "s3_sae_encode_grouped_workspace_bytes", "s3_sae_encode_topk_grouped", "s3_sae_encode_ctas",
+    "s3_sae_encode_grouped_workspace_bytes", "s3_sae_encode_topk_grouped", "s3_sae_encode_ctas", "s3_encode_schedule_describe",
     "s3_sae_project_encode_workspace_bytes", "s3_sae_project_encode_topk",
     "s3_postings_workspace_bytes", "s3_postings_build", "s3_postings_build_batched",
     "s3_index_create", "s3_index_reserve", "s3_index_append", "s3_index_stream_wait", "s3_index_sync",
@@ -121,6 +121,8 @@ def lib():
         L.s3_sae_encode_grouped_workspace_bytes.argtypes = [C.POINTER(EncodeItem), C.c_int]
         L.s3_sae_encode_topk_grouped.argtypes = [C.POINTER(EncodeItem), C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
         L.s3_sae_encode_ctas.argtypes = [C.c_void_p, C.c_int]
+        L.s3_encode_schedule_describe.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int,
+                                                  C.c_void_p]
         L.s3_sae_project_encode_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int]
         L.s3_sae_project_encode_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                                  C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -280,6 +282,23 @@ def s3_sae_encode_topk_grouped(items: list[EncodeItem], ws: torch.Tensor, max_ct
 def s3_sae_encode_ctas(sae: Sae, T: int) -> int:
     """Thread blocks an s3_sae_encode_topk launch over T tokens occupies."""
     return int(lib().s3_sae_encode_ctas(sae.handle, T))
+
+
+def s3_encode_schedule_describe(items, n_pairs: int, max_units: int = 4096):
+    """items: (T, d_in, d_sae, k) per encoder call. Returns (units int32 [n, 6] = pair, item, row tile, first column tile, one
+    past the last, slot; or None when the launch deals uniform slices without a table, slots per row of every item)."""
+    import numpy as np
+    a = np.ascontiguousarray(np.asarray(items, dtype=np.int32).reshape(-1, 4).T)
+    n = a.shape[1]
+    units = np.zeros((max_units, 6), dtype=np.int32)
+    slots = np.zeros(n, dtype=np.int32)
+    rc = int(lib().s3_encode_schedule_describe(a[0].ctypes.data, a[1].ctypes.data, a[2].ctypes.data, a[3].ctypes.data, n, n_pairs,
+                                               units.ctypes.data, max_units, slots.ctypes.data))
+    if rc == -2:
+        raise ValueError("invalid schedule query")
+    if rc > max_units:
+        raise ValueError(f"{rc} units, room for {max_units}")
+    return (units[:rc] if rc >= 0 else None), slots
 
 
 def s3_sae_project_encode_workspace_bytes(sae: Sae, T_max: int, n_heads: int, k: int) -> int:

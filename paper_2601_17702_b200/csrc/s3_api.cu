@@ -69,13 +69,13 @@ constexpr int kMaxSlices = 16;
 int col_tiles(const s3_sae* sae) { return sae->dtype == S3_BF16 ? encode_tc_col_tiles(sae->d_sae) : encode_simt_col_tiles(sae->d_sae); }
 int row_tiles(const s3_sae* sae, int T) { return sae->dtype == S3_BF16 ? encode_tc_row_tiles(T) : encode_simt_row_tiles(T); }
 
-// Number of column slices per row block. The kernel runs `units = row_tiles * slices` work units on
-// at most n_sm thread blocks; the modelled time is waves * tiles-per-slice plus a small charge per
-// slice for restarting the Top-k filter and for the merge.
+// Uniform column slices per row block: the caller's override (s3_sae_set_schedule), clamped to what the kernel takes; for
+// the fp32 kernel without an override, enough (row block, slice) thread blocks to cover the SMs. The bf16 launch
+// schedules itself when there is no override.
 int pick_slices(const s3_sae* sae, int T)
 {
     const int nct = col_tiles(sae);
-    int cap = nct < kMaxSlices ? nct : kMaxSlices;
+    const int cap = nct < kMaxSlices ? nct : kMaxSlices;
     const int lo = sae->dtype == S3_BF16 ? encode_tc_min_slices(sae->d_sae) : 1;
     if (sae->n_slices_override > 0) {
         const int s = sae->n_slices_override < cap ? sae->n_slices_override : cap;
@@ -84,24 +84,8 @@ int pick_slices(const s3_sae* sae, int T)
     const int nrt = row_tiles(sae, T);
     int n_sm = device_sm_count();
     if (sae->max_ctas > 0 && sae->max_ctas < n_sm) n_sm = sae->max_ctas;
-    if (sae->dtype == S3_BF16) {         // the tensor-core kernel runs one unit per CTA pair
-        n_sm = encode_tc_max_pairs();
-        if (sae->max_ctas > 0 && sae->max_ctas / 2 < n_sm) n_sm = sae->max_ctas / 2 > 0 ? sae->max_ctas / 2 : 1;
-    }
-    if (sae->dtype == S3_F32) {   // non-persistent kernel: enough blocks to cover the SMs
-        int s = (n_sm + nrt - 1) / nrt;
-        return s < 1 ? 1 : (s > cap ? cap : s);
-    }
-    int best = 1;
-    double best_cost = 1e30;
-    for (int s = lo; s <= cap; ++s) {
-        const int units = nrt * s;
-        const int waves = (units + n_sm - 1) / n_sm;
-        const int len = (nct + s - 1) / s;
-        const double cost = (double)waves * len + 0.25 * s * waves;
-        if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
-    }
-    return best;
+    const int s = (n_sm + nrt - 1) / nrt;
+    return s < lo ? lo : (s > cap ? cap : s);
 }
 
 }  // namespace
@@ -207,15 +191,18 @@ s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, in
                S3_ERR_INVALID_ARG, "misaligned device pointer");
     S3_REQUIRE(ldx >= sae->d_in, S3_ERR_INVALID_ARG, "ldx = %lld is smaller than d_in = %d", (long long)ldx, sae->d_in);
     if (sae->dtype == S3_BF16) S3_REQUIRE(ldx % 8 == 0, S3_ERR_INVALID_ARG, "ldx = %lld must be a multiple of 8 for bf16", (long long)ldx);
-    const int n_slices = pick_slices(sae, T);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint32_t* status = static_cast<uint32_t*>(d_ws);
     if (sae->dtype == S3_BF16) {
-        const size_t need = S3_WS_HEADER_BYTES + 192 + encode_tc_workspace_bytes(T, n_slices, k);
+        // column slices: the caller's override, else the launch's own schedule
+        const int forced = sae->n_slices_override > 0 ? pick_slices(sae, T) : 0;
+        const EncodeTcItem it = {&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, k, forced, d_ids, d_vals};
+        const size_t need = S3_WS_HEADER_BYTES + 192 + encode_tc_group_workspace_need(&it, 1, sae->max_ctas);
         S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
-        return launch_encode_tc(&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, k, n_slices, sae->max_ctas,
+        return launch_encode_tc(&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, k, forced, sae->max_ctas,
                                 static_cast<unsigned char*>(d_ws) + 256, status, d_ids, d_vals, st);
     }
+    const int n_slices = pick_slices(sae, T);
     const size_t need = S3_WS_HEADER_BYTES + (size_t)T * n_slices * k * sizeof(uint64_t);
     S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
     uint64_t* part = reinterpret_cast<uint64_t*>(static_cast<unsigned char*>(d_ws) + S3_WS_HEADER_BYTES);
@@ -251,7 +238,9 @@ size_t s3_sae_encode_grouped_workspace_bytes(const s3_encode_item* h_items, int 
     for (int i = 0; i < n_items; ++i) {
         const s3_encode_item& it = h_items[i];
         if (!it.sae || it.sae->dtype != S3_BF16 || it.T <= 0 || it.k < 1) continue;
-        n += encode_tc_workspace_bytes(it.T, pick_slices(it.sae, it.T), it.k);
+        // a caller's slice override counts as given; otherwise the bound that holds whatever schedule the launch picks
+        n += it.sae->n_slices_override > 0 ? encode_tc_workspace_bytes(it.T, pick_slices(it.sae, it.T), it.k)
+                                           : encode_tc_workspace_bound(it.T, it.k);
     }
     return n;
 }
@@ -260,10 +249,23 @@ int s3_sae_encode_ctas(const s3_sae* sae, int T)
 {
     if (!sae || T <= 0) return 0;
     if (sae->dtype != S3_BF16) return device_sm_count();
-    const int units = row_tiles(sae, T) * pick_slices(sae, T);
-    int pairs = encode_tc_max_pairs();
-    if (sae->max_ctas > 0 && sae->max_ctas / 2 < pairs) pairs = sae->max_ctas / 2 > 0 ? sae->max_ctas / 2 : 1;
-    return 2 * (units < pairs ? units : pairs);
+    const EncodeTcItem it = {&sae->tc, nullptr, 0, T, sae->d_in, sae->d_sae, 1, sae->n_slices_override > 0 ? pick_slices(sae, T) : 0,
+                             nullptr, nullptr};
+    return encode_tc_group_ctas(&it, 1, sae->max_ctas);
+}
+
+int s3_encode_schedule_describe(const int32_t* T, const int32_t* d_in, const int32_t* d_sae, const int32_t* k, int n_items,
+                                int n_pairs, int32_t* h_units, int max_units, int32_t* h_slots)
+{
+    if (!T || !d_in || !d_sae || !k || !h_slots || n_items < 1 || n_items > S3_MAX_ENCODE_ITEMS || n_pairs < 1 || max_units < 0 ||
+        (max_units > 0 && !h_units))
+        return -2;
+    EncodeTcItem items[S3_MAX_ENCODE_ITEMS];
+    for (int i = 0; i < n_items; ++i) {
+        if (T[i] < 1 || d_in[i] < 1 || d_sae[i] < 1 || k[i] < 1) return -2;
+        items[i] = EncodeTcItem{nullptr, nullptr, 0, T[i], d_in[i], d_sae[i], k[i], 0, nullptr, nullptr};
+    }
+    return encode_tc_describe_schedule(items, n_items, n_pairs, h_units, max_units, h_slots);
 }
 
 s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items, int max_ctas_arg, void* d_ws, size_t ws_bytes,
@@ -282,12 +284,12 @@ s3_status s3_sae_encode_topk_grouped(const s3_encode_item* h_items, int n_items,
         if (st != S3_OK) return st;
         const s3_encode_item& it = h_items[i];
         if (it.T == 0) continue;
-        items[n++] = EncodeTcItem{&it.sae->tc, it.d_x, it.ldx, it.T, it.sae->d_in, it.sae->d_sae, it.k, pick_slices(it.sae, it.T),
-                                  it.d_ids, it.d_vals};
+        items[n++] = EncodeTcItem{&it.sae->tc, it.d_x, it.ldx, it.T, it.sae->d_in, it.sae->d_sae, it.k,
+                                  it.sae->n_slices_override > 0 ? pick_slices(it.sae, it.T) : 0, it.d_ids, it.d_vals};
         if (it.sae->max_ctas > 0 && (max_ctas == 0 || it.sae->max_ctas < max_ctas)) max_ctas = it.sae->max_ctas;
     }
     if (n == 0) return S3_OK;
-    const size_t need = s3_sae_encode_grouped_workspace_bytes(h_items, n_items);
+    const size_t need = 256 + encode_tc_group_workspace_need(items, n, max_ctas);
     S3_REQUIRE(ws_bytes >= need, S3_ERR_CAPACITY, "workspace holds %zu bytes, %zu needed", ws_bytes, need);
     return launch_encode_tc_group(items, n, max_ctas, static_cast<unsigned char*>(d_ws) + 256, static_cast<uint32_t*>(d_ws),
                                   static_cast<cudaStream_t>(stream));
@@ -337,7 +339,7 @@ s3_status s3_sae_preact(const s3_sae* sae, const void* d_x, int64_t ldx, int T, 
     const int vec = out_dtype == S3_BF16 ? 8 : 4;
     S3_REQUIRE(ld_out >= sae->d_sae && ld_out % vec == 0, S3_ERR_INVALID_ARG, "ld_out = %lld must be a multiple of %d and >= d_sae",
                (long long)ld_out, vec);
-    return launch_preact_tc(&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, pick_slices(sae, T), sae->max_ctas,
+    return launch_preact_tc(&sae->tc, d_x, ldx, T, sae->d_in, sae->d_sae, sae->n_slices_override > 0 ? pick_slices(sae, T) : 0, sae->max_ctas,
                             static_cast<uint32_t*>(d_ws), d_out, ld_out, out_dtype == S3_BF16, static_cast<cudaStream_t>(stream));
 }
 

@@ -231,8 +231,15 @@ constexpr uint32_t kInstrDescN128 = (1u << 4) | (1u << 7) | (1u << 10) | (static
 constexpr int M_SELECT = 0, M_DENSE = 1, M_PROJ = 2;   // epilogue modes of the kernel
 
 constexpr int MAX_GROUP = S3_MAX_ENCODE_ITEMS;   // encoders one launch can serve
-constexpr int MAX_SCHED = 1024;                  // work units a launch can deal out by table
+constexpr int MAX_SCHED = 2048;                  // work units a launch can deal out by table
 constexpr int MAX_PAIRS = 96;                    // CTA pairs the table has room for
+
+// One work unit of a table-driven launch: column tiles [tile_lo, tile_hi) of row tile mt of an item; its survivors go
+// to candidate list `slot` of the rows.
+struct UnitDesc {
+    uint16_t mt, tile_lo, tile_hi;
+    uint8_t item, slot;
+};
 
 // One encoder call of a grouped launch.
 struct ItemParams {
@@ -248,7 +255,7 @@ struct ItemParams {
 
 struct EncodeTcParams {
     int n_items, n_units, n_stages;
-    int use_sched;             // 1: pair p runs units sched[pair_start[p] .. pair_start[p+1]); 0: units p, p + n_pairs, ...
+    int use_sched;             // 1: pair p runs units unit[pair_start[p] .. pair_start[p+1]); 0: units p, p + n_pairs, ...
     uint32_t* status;
     void* dense_out;           // dense mode (one item): the pre-activations [T, ld_out], fp32 or bf16
     long long ld_out;
@@ -259,7 +266,7 @@ struct EncodeTcParams {
     const float* proj_bias;            // [heads * 128]
     ItemParams item[MAX_GROUP];
     uint16_t pair_start[MAX_PAIRS + 1];
-    uint16_t sched[MAX_SCHED];
+    UnitDesc unit[MAX_SCHED];
 };
 
 struct TensorMaps {
@@ -279,26 +286,39 @@ __device__ __forceinline__ UnitWalk unit_walk(const EncodeTcParams& p, int pair,
     else { w.i = pair; w.end = p.n_units; w.step = n_pairs; }
     return w;
 }
-// Unit -> (item, column slice, row tile).
-__device__ __forceinline__ void unit_decode(const EncodeTcParams& p, const UnitWalk& w, int& item, int& slice, int& mt)
+// Unit -> item, candidate-list slot ("slice"), row tile and the column tiles [tile_lo, tile_hi) it covers.
+struct Unit {
+    int item, slice, mt, tile_lo, tile_hi;
+};
+__device__ __forceinline__ Unit unit_decode(const EncodeTcParams& p, const UnitWalk& w)
 {
-    const int u = p.use_sched ? static_cast<int>(p.sched[w.i]) : w.i;
-    if (p.proj_heads > 0) {            // (row tile, head), heads of a row tile next to each other: they share the tile of h
-        item = 0;
-        mt = u / p.proj_heads;
-        slice = u - mt * p.proj_heads;
-        return;
+    Unit u;
+    if (p.use_sched) {
+        const UnitDesc d = p.unit[w.i];
+        u.item = d.item; u.slice = d.slot; u.mt = d.mt; u.tile_lo = d.tile_lo; u.tile_hi = d.tile_hi;
+        return u;
     }
-    item = p.n_items - 1;
-    while (item > 0 && p.item[item].unit_start > u) --item;
-    const int local = u - p.item[item].unit_start;
-    slice = local / p.item[item].n_mtiles;
-    mt = local - slice * p.item[item].n_mtiles;
+    if (p.proj_heads > 0) {            // (row tile, head), heads of a row tile next to each other: they share the tile of h
+        u.item = 0;
+        u.mt = w.i / p.proj_heads;
+        u.slice = w.i - u.mt * p.proj_heads;
+        u.tile_lo = 0; u.tile_hi = p.item[0].n_col_tiles;
+        return u;
+    }
+    u.item = p.n_items - 1;
+    while (u.item > 0 && p.item[u.item].unit_start > w.i) --u.item;
+    const ItemParams& ip = p.item[u.item];
+    const int local = w.i - ip.unit_start;
+    u.slice = local / ip.n_mtiles;
+    u.mt = local - u.slice * ip.n_mtiles;
+    u.tile_lo = static_cast<int>(static_cast<int64_t>(u.slice) * ip.n_col_tiles / ip.n_slices);
+    u.tile_hi = static_cast<int>(static_cast<int64_t>(u.slice + 1) * ip.n_col_tiles / ip.n_slices);
+    return u;
 }
 
 // Shared-memory carve-up (all offsets from a 1024-byte aligned base).
 struct SmemLayout {
-    uint32_t a_off, b_off, x_off, pend_off, hist_off, bar_off, total;
+    uint32_t a_off, b_off, x_off, pend_off, hist_off, xtau_off, bar_off, total;
 };
 constexpr int X_TILE_BYTES = 2 * A_STAGE_BYTES;    // projection mode: this CTA's 128 tokens x 128 projected columns, two k-blocks
 __host__ __device__ inline SmemLayout smem_layout(int n_stages, bool proj, int groups)
@@ -310,7 +330,8 @@ __host__ __device__ inline SmemLayout smem_layout(int n_stages, bool proj, int g
     L.x_off = L.b_off + n_stages * B_STAGE_BYTES;
     L.pend_off = L.x_off + (proj ? X_TILE_BYTES : 0);
     L.hist_off = L.pend_off + PEND_CAP * EPI_THREADS * 8;
-    L.bar_off = L.hist_off + NB * EPI_THREADS * 2;
+    L.xtau_off = L.hist_off + NB * EPI_THREADS * 2;
+    L.bar_off = L.xtau_off + BM * 16;
     L.total = L.bar_off + (2 * n_stages + 5) * 8 + 16;
     return L;
 }
@@ -324,7 +345,18 @@ struct RowSel {
     uint32_t above;     // survivors counted in slots >= istar
     uint32_t gcnt;      // entries in the row's candidate list
     bool floor_exact;   // tau_floor is the value of the list's exact k-th key
+    float ext;          // best bound learnt from the row's other lists (other column pieces, the other epilogue group)
+    float cut;          // max(tau, ext): what a value must exceed to be kept
 };
+
+// The bound this list may announce: at least k of its values exceed it. An exact k-th value only bounds from below after
+// stepping to the next float down.
+__device__ __forceinline__ uint32_t announced_bound(const RowSel& r)
+{
+    uint32_t out = __float_as_uint(r.tau);
+    if (r.istar == 0 && r.floor_exact && out > 0u) out -= 1u;
+    return out;
+}
 
 // Rare path: the candidate list cannot take the pending entries. Drops what is not above the bound;
 // if the list stays nearly full it keeps only its k largest keys and restarts the histogram from there.
@@ -336,7 +368,7 @@ __device__ __noinline__ void prune_list(uint64_t* glist, uint16_t* my_hist, RowS
     uint32_t w = 0;
     for (uint32_t i = 0; i < r.gcnt; ++i) {
         const uint64_t key = glist[i];
-        if (__uint_as_float(static_cast<uint32_t>(key >> 32)) > r.tau) glist[w++] = key;
+        if (__uint_as_float(static_cast<uint32_t>(key >> 32)) > r.cut) glist[w++] = key;
     }
     r.gcnt = w;
     if (r.gcnt + PEND_CAP <= cap) return;
@@ -354,6 +386,7 @@ __device__ __noinline__ void prune_list(uint64_t* glist, uint16_t* my_hist, RowS
     r.gcnt = k;
     const uint32_t vb = static_cast<uint32_t>(glist[k - 1] >> 32);
     r.tau_floor = r.tau = __uint_as_float(vb);
+    r.cut = fmaxf(r.tau, r.ext);
     r.floor_exact = true;
 #pragma unroll 1
     for (int s = 0; s < NB; ++s) my_hist[s * EPI_THREADS] = 0;
@@ -370,10 +403,14 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
                                              int k, uint32_t cap)
 {
     if (__any_sync(0xffffffffu, r.gcnt + cnt > cap)) {
-        if (r.gcnt + cnt > cap) prune_list<EPI_THREADS>(glist, my_hist, r, k, cap);
+        if (r.gcnt + cnt > cap) {
+            RowSel t = r;            // the rare path works on a copy: the row's own state never has its address taken and stays in registers
+            prune_list<EPI_THREADS>(glist, my_hist, t, k, cap);
+            r = t;
+        }
     }
     if (r.hbase < 0 && cnt > 0) {
-        uint32_t ref = __float_as_uint(r.tau);
+        uint32_t ref = __float_as_uint(r.cut);
         if (ref == 0) {      // no bound yet: centre the window on the largest value seen so far
             for (int i = 0; i < cnt; ++i) {
                 const uint32_t vb = static_cast<uint32_t>(my_pend[i * EPI_THREADS] >> 32);
@@ -397,7 +434,7 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
 #pragma unroll
         for (int q = 0; q < FOLD_CHUNK; ++q) {
             const uint32_t vb = static_cast<uint32_t>(key[q] >> 32);
-            ok[q] = (i0 + q < cnt) && __uint_as_float(vb) > r.tau;
+            ok[q] = (i0 + q < cnt) && __uint_as_float(vb) > r.cut;
             int ix = static_cast<int>(vb >> HSHIFT) - r.hbase;
             idx[q] = ix < 0 ? 0 : (ix > NB - 1 ? NB - 1 : ix);
         }
@@ -438,6 +475,7 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
     }
     // "value >= edge" is "value > the float just below the edge"
     r.tau = r.istar > 0 ? __uint_as_float((static_cast<uint32_t>(r.hbase + r.istar) << HSHIFT) - 1u) : r.tau_floor;
+    r.cut = fmaxf(r.tau, r.ext);
 }
 
 // DENSE: the epilogue writes the pre-activations themselves (row-major, fp32 or bf16) instead of selecting; the rest of
@@ -456,6 +494,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
     unsigned char* smem_x = smem + L.x_off;                // projection mode: the head's projected tile, the encode's A operand
     uint64_t* pend = reinterpret_cast<uint64_t*>(smem + L.pend_off);
     uint16_t* hist = reinterpret_cast<uint16_t*>(smem + L.hist_off);
+    uint32_t* xtau32 = reinterpret_cast<uint32_t*>(smem + L.xtau_off);   // [unit number mod 4][row]: best bound of the row's lists
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L.bar_off);
     uint64_t* empty_bar = full_bar + p.n_stages;
     uint64_t* acc_full = empty_bar + p.n_stages;
@@ -475,6 +514,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
         // acc_empty: every epilogue thread of both CTAs, on the first CTA's barrier
         for (int s = 0; s < p.n_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 2 * EPI_THREADS); }
+        for (int i = 0; i < 4 * BM; ++i) xtau32[i] = 0u;
         mbar_init(x_ready, 2 * EPI_THREADS);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -502,14 +542,12 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             uint64_t issued = 0;
             bool ok = true;
             for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
-                int item, slice, mt;
-                unit_decode(p, uw, item, slice, mt);
+                const Unit un = unit_decode(p, uw);
+                const int item = un.item, slice = un.slice, mt = un.mt, tile_lo = un.tile_lo, tile_hi = un.tile_hi;
                 const ItemParams& ip = p.item[item];
                 const CUtensorMap* map_x = &maps.x[item];
                 const CUtensorMap* map_w = &maps.w[item];
                 const int kblocks = ip.kblocks;
-                const int tile_lo = PROJ ? 0 : static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
-                const int tile_hi = PROJ ? ip.n_col_tiles : static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
                 const int row0 = mt * PAIR_M + static_cast<int>(cta_rank) * BM;        // this CTA's tokens
                 if constexpr (PROJ) {
                     // the head's projection first: 128 tokens of h and this CTA's 64 of the head's 128 rows of W_proj^T per k-block
@@ -564,12 +602,9 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             uint32_t tile_count = 0, unit_count = 0;
             bool ok = true;
             for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
-                int item, slice, mt;
-                unit_decode(p, uw, item, slice, mt);
-                const ItemParams& ip = p.item[item];
-                const int kblocks = ip.kblocks;
-                const int tile_lo = PROJ ? 0 : static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
-                const int tile_hi = PROJ ? ip.n_col_tiles : static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
+                const Unit un = unit_decode(p, uw);
+                const int tile_lo = un.tile_lo, tile_hi = un.tile_hi;
+                const int kblocks = p.item[un.item].kblocks;
                 if constexpr (PROJ) {
                     // The projection takes its turn in the accumulator rotation like a tile (128 columns of it). Its MMAs
                     // are issued after the previous head's, so when its accumulator completes the shared-memory tile of the
@@ -653,16 +688,14 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
         uint16_t* my_hist = hist + grp * 128 + e;
         constexpr int CB_PER_GROUP = BN / BATCH / EPI_GROUPS;
         const int cb_lo = grp * CB_PER_GROUP, cb_hi = cb_lo + CB_PER_GROUP;
-        uint32_t tile_count = 0;
+        uint32_t tile_count = 0, unit_seq = 0;
         bool ok = true;
         // the accumulator is handed back on the first CTA's barrier
         const uint32_t acc_empty_addr[2] = {map_to_cta(smem_u32(&acc_empty[0]), 0), map_to_cta(smem_u32(&acc_empty[1]), 0)};
         for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
-            int item, slice, mt;
-            unit_decode(p, uw, item, slice, mt);
-            const ItemParams& ip = p.item[item];
-            const int tile_lo = PROJ ? 0 : static_cast<int>(static_cast<int64_t>(slice) * ip.n_col_tiles / ip.n_slices);
-            const int tile_hi = PROJ ? ip.n_col_tiles : static_cast<int>(static_cast<int64_t>(slice + 1) * ip.n_col_tiles / ip.n_slices);
+            const Unit un = unit_decode(p, uw);
+            const int slice = un.slice, mt = un.mt, tile_lo = un.tile_lo, tile_hi = un.tile_hi;
+            const ItemParams& ip = p.item[un.item];
             const int t = mt * PAIR_M + static_cast<int>(cta_rank) * BM + e;
             const bool live = t < ip.T;
             const int k = ip.k;
@@ -682,7 +715,19 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             r.tau_floor = live ? __uint_as_float(hint_in) : INFINITY;    // rows past T select nothing
             r.tau = r.tau_floor;
             r.hbase = -1; r.istar = 0; r.above = 0; r.gcnt = 0; r.floor_exact = false;
+            r.ext = r.cut = r.tau;
             int cnt = 0;                            // entries in this row's pending list
+            // Bounds are shared while the unit runs: a bound that k values of one list exceed holds for the whole row, so every
+            // other list of the row (the other epilogue group's, other column pieces' on other SMs) may drop what does not
+            // beat it. Without this each list gathers its own k survivors and the folding work grows with the number of lists.
+            ++unit_seq;
+            // The groups exchange bounds through xtau32[unit number mod 4][row]. A group cannot start a tile before every
+            // group has finished the tile two before it (the accumulator it needs is handed back by all of them), so the
+            // groups are never more than two units apart: the slot of unit n + 2, cleared here by each group, is not in
+            // use by anyone (unit n - 2 is over for all), and both groups have cleared it before either reaches unit n + 2.
+            if (EPI_GROUPS > 1) xtau32[((unit_seq + 2u) & 3u) * BM + e] = 0u;
+            const bool share_row = !DENSE && !PROJ && live && ip.n_slices > 1;     // other units hold pieces of these rows
+            uint32_t announced = hint_in;
             if constexpr (PROJ) {
                 // The head's projection: accumulator -> + bias -> bf16 (round to nearest even, as the dense epilogue stores
                 // it) -> this CTA's shared-memory tile in the layout of a 128-byte-swizzled TMA tile (two k-blocks of 128 rows x
@@ -781,6 +826,8 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                         r.tau_floor = r.tau = bound;
                     }
                 }
+                // the row's published bound as of now; used from the tile's second batch on, so the load's latency is covered
+                const uint32_t row_bound = share_row ? *reinterpret_cast<volatile const uint32_t*>(ip.hint + orow) : 0u;
 #pragma unroll 1
                 for (int cb = cb_lo; cb < cb_hi; ++cb) {
                     uint32_t acc[32];
@@ -790,6 +837,11 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                     for (int j4 = 0; j4 < BATCH / 4; ++j4) {
                         const float4 b4 = __ldg(bias4 + cb * (BATCH / 4) + j4);
                         bias[4 * j4 + 0] = b4.x; bias[4 * j4 + 1] = b4.y; bias[4 * j4 + 2] = b4.z; bias[4 * j4 + 3] = b4.w;
+                    }
+                    if constexpr (!DENSE) {
+                        if (EPI_GROUPS > 1) r.ext = fmaxf(r.ext, __uint_as_float(xtau32[(unit_seq & 3u) * BM + e]));
+                        if (cb == cb_lo + 1) r.ext = fmaxf(r.ext, __uint_as_float(row_bound));
+                        r.cut = fmaxf(r.cut, r.ext);
                     }
                     tc_wait_ld();
                     if constexpr (DENSE) {
@@ -831,7 +883,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 v[q] = __uint_as_float(acc[h * STEP + j + q]) + bias[h * STEP + j + q];
-                                keep[q] = (v[q] > r.tau) ? 1 : 0;
+                                keep[q] = (v[q] > r.cut) ? 1 : 0;
                             }
                             const int o1 = keep[0], o2 = o1 + keep[1], o3 = o2 + keep[2];
                             uint64_t* slot = my_pend + cnt * EPI_THREADS;
@@ -842,7 +894,15 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                             if (keep[3]) slot[o3 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[3])) << 32) | (nc - 3u);
                             cnt += o3 + keep[3];
                         }
-                        if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) fold_pending<EPI_THREADS>(my_pend, my_hist, glist, r, cnt, k, cap);
+                        if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) {
+                            fold_pending<EPI_THREADS>(my_pend, my_hist, glist, r, cnt, k, cap);
+                            const uint32_t now = announced_bound(r);       // tell the row's other lists when the bound has risen
+                            if (now > announced) {
+                                announced = now;
+                                if (EPI_GROUPS > 1) atomicMax(&xtau32[(unit_seq & 3u) * BM + e], now);
+                                if (share_row) atomicMax(ip.hint + orow, now);
+                            }
+                        }
                     }
                 }
                 tc_fence_before();
@@ -851,10 +911,9 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             if (ok && !DENSE) {
                 if (__any_sync(0xffffffffu, cnt > 0)) fold_pending<EPI_THREADS>(my_pend, my_hist, glist, r, cnt, k, cap);
                 if (live) {
-                    // The bound to publish: at least k values of this slice exceed it. An exact k-th value
-                    // only bounds from below after stepping to the next float down.
-                    uint32_t out = __float_as_uint(r.tau);
-                    if (r.istar == 0 && r.floor_exact && out > 0u) out -= 1u;
+                    // what the merge may cut the row's lists at: this list's own bound or a better one learnt meanwhile
+                    uint32_t out = announced_bound(r);
+                    if (__float_as_uint(r.ext) > out) out = __float_as_uint(r.ext);
                     // The list was filled under bounds that rose along the slice (about k (1 + ln(columns / k))
                     // entries); only what beats the final bound can still matter, so the list is compacted once
                     // here and the merge reads a fraction of it. The pass is a tail of dependent round trips after the
@@ -1007,21 +1066,282 @@ uint32_t encode_tc_list_cap(int k, int groups) { return static_cast<uint32_t>((k
 // Column tiles per slice may not exceed 255: a row's histogram counters are 16 bits wide.
 int encode_tc_min_slices(int d_sae) { return (encode_tc_col_tiles(d_sae) + 254) / 255; }
 
-size_t encode_tc_workspace_bytes(int T, int n_slices, int k)
+// Scratch of one item whose rows hold `lists` (row, slot) candidate lists in all: the rows' bounds, the lists' lengths and
+// the lists. Sized for either number of epilogue groups: two lists of half the slots take the room of one list.
+static size_t lists_bytes(int T, size_t lists, int k)
 {
-    // sized for either number of epilogue groups: two lists of half the slots take the room of one list
-    const size_t t = static_cast<size_t>(T), s = static_cast<size_t>(n_slices) * MAX_EPI_GROUPS;    // candidate lists per row
-    return round_up(t * 4, 256) + round_up(t * s * 4, 256) + round_up(t * s * encode_tc_list_cap(k, MAX_EPI_GROUPS) * sizeof(uint64_t), 256);
+    const size_t s = lists * MAX_EPI_GROUPS;
+    return round_up(static_cast<size_t>(T) * 4, 256) + round_up(s * 4, 256) +
+           round_up(s * encode_tc_list_cap(k, MAX_EPI_GROUPS) * sizeof(uint64_t), 256);
+}
+
+size_t encode_tc_workspace_bytes(int T, int n_slices, int k) { return lists_bytes(T, static_cast<size_t>(T) * n_slices, k); }
+
+// Slots per row any automatic schedule stays within: a row tile is cut where a pair's share ends, so it holds about
+// pairs / row tiles pieces plus the ends; uniform slices are held to the same number.
+static int slot_bound(int T, int n_pairs)
+{
+    const int n = encode_tc_row_tiles(T);
+    const int b = 4 + (n_pairs + n - 1) / n;
+    return b < 16 ? b : 16;
+}
+
+// Scratch that holds any automatic schedule of T tokens, and of fewer: T * slot_bound(T) <= 5 T + 256 pairs, which grows
+// with T, so a workspace sized for a full chunk also serves the shorter last one.
+size_t encode_tc_workspace_bound(int T, int k)
+{
+    const size_t t = static_cast<size_t>(T);
+    size_t lists = 5 * t + 256 * static_cast<size_t>(encode_tc_max_pairs());
+    if (lists > 16 * t) lists = 16 * t;
+    return lists_bytes(T, lists, k);
 }
 
 namespace {
 
-// Modelled duration of one work unit, in tensor-pipe cycles: per 256-column tile the MMAs of its k-blocks or, for
-// narrow inputs, the Top-k filter of its 256 columns, whichever is longer.
-double unit_cost(int kblocks, int tiles, int k)
+// ---- work units of a launch -----------------------------------------------------------------------------
+// Modelled durations in SM cycles. A 256-column tile takes the MMAs of its k-blocks or the Top-k filter of its columns,
+// whichever is longer; a unit also pays for its cold start (one extra pass over its first tile) and its last fold.
+struct CostModel {
+    double tile, unit;
+};
+CostModel cost_model(int kblocks, int k, int groups, bool dense)
 {
-    const double mma = 600.0 * kblocks, filter = 12000.0 + 100.0 * k;
-    return tiles * (mma > filter ? mma : filter);
+    const double mma = 600.0 * kblocks;
+    const double filter = dense ? 6000.0 : (12000.0 + 100.0 * k) / (groups == 2 ? 1.5 : 1.0);
+    CostModel c;
+    c.tile = mma > filter ? mma : filter;
+    c.unit = dense ? 2000.0 : 16000.0 + 100.0 * k;
+    return c;
+}
+
+constexpr int kMaxSlots = 16;                       // candidate lists per row and epilogue group at most
+constexpr int kMinPiece = 3;                        // a row is not cut into pieces shorter than this many column tiles
+constexpr size_t kRoundBytes = size_t(48) << 20;    // encoder weights that pairs may walk at the same time (they should stay in L2)
+
+struct Schedule {
+    int order[MAX_GROUP];             // launch position -> caller's item
+    int slots[MAX_GROUP];             // candidate lists per row of the item at each launch position
+    int n_pairs, n_units, groups;
+    bool table;                       // units come from unit[] / pair_start[]; otherwise uniform slices dealt round-robin
+    UnitDesc unit[MAX_SCHED];
+    uint16_t pair_start[MAX_PAIRS + 1];
+};
+
+// Uniform column slices of one encoder: the count that minimises waves * tiles-per-slice plus a charge per slice.
+int uniform_slices(int T, int nct, int d_sae, int n_pairs)
+{
+    const int n_mtiles = encode_tc_row_tiles(T);
+    const int lo = encode_tc_min_slices(d_sae);
+    int cap = nct < kMaxSlots ? nct : kMaxSlots;
+    if (slot_bound(T, n_pairs) < cap) cap = slot_bound(T, n_pairs);
+    if (cap < lo) cap = lo;
+    int best = lo;
+    double best_cost = 1e30;
+    for (int sl = lo; sl <= cap; ++sl) {
+        const int units = n_mtiles * sl;
+        const int waves = (units + n_pairs - 1) / n_pairs;
+        const int len = (nct + sl - 1) / sl;
+        const double cost = static_cast<double>(waves) * len + 0.25 * sl * waves;
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = sl; }
+    }
+    return best;
+}
+
+// Balanced plan. The items (in launch order) are taken in rounds whose encoder weights fit in L2 together; the tiles of a
+// round, in the order (item, row tile, column tile), are cut into one contiguous range per CTA pair of equal modelled
+// duration, and a range is cut into units at the row-tile boundaries. A row tile therefore ends up in a few pieces held by
+// neighbouring pairs, each piece with its own candidate list. Fails (false) when an encoder is too wide for a round, a
+// row would need more than kMaxSlots pieces, or the units do not fit the table.
+bool plan_balanced(const EncodeTcItem* items, const int* order, int n_items, int n_pairs, int groups, bool dense, Schedule& sc)
+{
+    static thread_local UnitDesc gen[MAX_SCHED];
+    static thread_local uint16_t gen_pair[MAX_SCHED];
+    int n = 0;
+    int q0 = 0;
+    while (q0 < n_items) {
+        size_t bytes = 0;
+        int q1 = q0;
+        while (q1 < n_items) {
+            const EncodeTcItem& it = items[order[q1]];
+            const size_t w = static_cast<size_t>(it.d_sae) * it.d_in * 2;
+            if (w > kRoundBytes) return false;
+            if (q1 > q0 && bytes + w > kRoundBytes) break;
+            bytes += w;
+            ++q1;
+        }
+        double rem = 0.0;
+        for (int q = q0; q < q1; ++q) {
+            const EncodeTcItem& it = items[order[q]];
+            const CostModel c = cost_model((it.d_in + BK - 1) / BK, it.k, groups, dense);
+            rem += static_cast<double>(encode_tc_row_tiles(it.T)) * (encode_tc_col_tiles(it.d_sae) * c.tile + c.unit);
+        }
+        // a pair's share: what is left, plus the start-up of the piece that every later cut adds, over the pairs left
+        auto share = [&](int pr, double unit) { return (rem + unit * (n_pairs - pr - 1)) / (n_pairs - pr); };
+        int pr = 0;
+        double acc = 0.0;
+        double target = share(0, cost_model((items[order[q0]].d_in + BK - 1) / BK, items[order[q0]].k, groups, dense).unit);
+        for (int q = q0; q < q1; ++q) {
+            const EncodeTcItem& it = items[order[q]];
+            const CostModel c = cost_model((it.d_in + BK - 1) / BK, it.k, groups, dense);
+            const int n_mtiles = encode_tc_row_tiles(it.T), nct = encode_tc_col_tiles(it.d_sae);
+            if (n_mtiles > 65535 || nct > 65535) return false;
+            const int max_pieces = slot_bound(it.T, n_pairs);
+            int slots = 1;
+            for (int mt = 0; mt < n_mtiles; ++mt) {
+                int lo = 0, pieces = 0;
+                while (lo < nct) {
+                    const int left = nct - lo;
+                    int take;
+                    if (pr == n_pairs - 1) take = left;
+                    else {
+                        const int fit = static_cast<int>((target - acc - c.unit) / c.tile + 0.5);
+                        if (fit >= left) take = left;
+                        else if (left - fit < kMinPiece && left - kMinPiece >= kMinPiece) take = left - kMinPiece;   // leave a whole piece
+                        else if (left - fit < kMinPiece) take = left;
+                        else if (fit < kMinPiece) {
+                            if (acc > 0.0) {              // this pair is full: the row goes on with the next one
+                                ++pr; acc = 0.0; target = share(pr, c.unit);
+                                continue;
+                            }
+                            take = left < kMinPiece ? left : kMinPiece;
+                        } else take = fit;
+                    }
+                    if (take > 255) take = 255;           // a row's histogram counters are 16 bits wide
+                    if (n >= MAX_SCHED || pieces >= max_pieces) return false;
+                    gen[n].mt = static_cast<uint16_t>(mt);
+                    gen[n].tile_lo = static_cast<uint16_t>(lo);
+                    gen[n].tile_hi = static_cast<uint16_t>(lo + take);
+                    gen[n].item = static_cast<uint8_t>(q);
+                    gen[n].slot = static_cast<uint8_t>(pieces);
+                    gen_pair[n] = static_cast<uint16_t>(pr);
+                    ++n;
+                    acc += c.unit + take * c.tile;
+                    rem -= take * c.tile + (pieces == 0 ? c.unit : 0.0);
+                    ++pieces;
+                    lo += take;
+                    if (pr < n_pairs - 1 && acc >= target - 0.5 * c.tile) { ++pr; acc = 0.0; target = share(pr, c.unit); }
+                }
+                slots = pieces > slots ? pieces : slots;
+            }
+            sc.slots[q] = slots;
+        }
+        q0 = q1;
+    }
+    // bucket by pair, keeping the order of generation (rounds in launch order)
+    int count[MAX_PAIRS] = {};
+    for (int i = 0; i < n; ++i) ++count[gen_pair[i]];
+    int run = 0, used = 0;
+    for (int q = 0; q < n_pairs; ++q) {
+        sc.pair_start[q] = static_cast<uint16_t>(run);
+        run += count[q];
+        if (count[q]) used = q + 1;
+    }
+    for (int q = n_pairs; q <= MAX_PAIRS; ++q) sc.pair_start[q] = static_cast<uint16_t>(run);
+    int fill[MAX_PAIRS];
+    for (int q = 0; q < n_pairs; ++q) fill[q] = sc.pair_start[q];
+    for (int i = 0; i < n; ++i) sc.unit[fill[gen_pair[i]]++] = gen[i];
+    sc.n_units = n;
+    sc.n_pairs = used;
+    sc.table = true;
+    return true;
+}
+
+// Uniform slices, whole (row tile, slice) units; with several items and room in the table the units are dealt out by
+// modelled duration (each to the pair with the least work so far), otherwise round-robin without a table.
+void plan_uniform(const EncodeTcItem* items, const int* order, int n_items, int n_pairs, int groups, bool dense, Schedule& sc)
+{
+    int n_units = 0;
+    for (int q = 0; q < n_items; ++q) {
+        const EncodeTcItem& it = items[order[q]];
+        const int n_mtiles = encode_tc_row_tiles(it.T), nct = encode_tc_col_tiles(it.d_sae);
+        sc.slots[q] = it.n_slices > 0 ? it.n_slices : uniform_slices(it.T, nct, it.d_sae, n_pairs);
+        n_units += n_mtiles * sc.slots[q];
+    }
+    sc.n_units = n_units;
+    sc.n_pairs = n_units < n_pairs ? n_units : n_pairs;
+    sc.table = false;
+    if (n_items < 2 || n_units > MAX_SCHED) return;
+    static thread_local uint16_t unit_pair[MAX_SCHED];
+    static thread_local UnitDesc gen[MAX_SCHED];
+    double load[MAX_PAIRS];
+    int count[MAX_PAIRS];
+    for (int q = 0; q < sc.n_pairs; ++q) { load[q] = 0.0; count[q] = 0; }
+    int u = 0;
+    for (int q = 0; q < n_items; ++q) {
+        const EncodeTcItem& it = items[order[q]];
+        const int n_mtiles = encode_tc_row_tiles(it.T), nct = encode_tc_col_tiles(it.d_sae);
+        if (n_mtiles > 65535 || nct > 65535) return;
+        const CostModel c = cost_model((it.d_in + BK - 1) / BK, it.k, groups, dense);
+        for (int sl = 0; sl < sc.slots[q]; ++sl) {
+            const int lo = static_cast<int>(static_cast<int64_t>(sl) * nct / sc.slots[q]);
+            const int hi = static_cast<int>(static_cast<int64_t>(sl + 1) * nct / sc.slots[q]);
+            for (int mt = 0; mt < n_mtiles; ++mt, ++u) {
+                int best = 0;
+                for (int r = 1; r < sc.n_pairs; ++r)
+                    if (load[r] < load[best]) best = r;
+                load[best] += c.unit + (hi - lo) * c.tile;
+                unit_pair[u] = static_cast<uint16_t>(best);
+                ++count[best];
+                gen[u].mt = static_cast<uint16_t>(mt);
+                gen[u].tile_lo = static_cast<uint16_t>(lo);
+                gen[u].tile_hi = static_cast<uint16_t>(hi);
+                gen[u].item = static_cast<uint8_t>(q);
+                gen[u].slot = static_cast<uint8_t>(sl);
+            }
+        }
+    }
+    int run = 0;
+    for (int q = 0; q < sc.n_pairs; ++q) { sc.pair_start[q] = static_cast<uint16_t>(run); run += count[q]; }
+    for (int q = sc.n_pairs; q <= MAX_PAIRS; ++q) sc.pair_start[q] = static_cast<uint16_t>(run);
+    int fill[MAX_PAIRS];
+    for (int q = 0; q < sc.n_pairs; ++q) fill[q] = sc.pair_start[q];
+    for (int i = 0; i < n_units; ++i) sc.unit[fill[unit_pair[i]]++] = gen[i];
+    sc.table = true;
+}
+
+// The schedule of a launch: launch order of the items (descending modelled tile duration, so that the short tiles fill
+// the end), epilogue groups, CTA pairs and the units. Items that leave n_slices at 0 get the balanced plan when it
+// applies; an item with n_slices > 0 forces uniform slices for the whole launch.
+void build_schedule(const EncodeTcItem* items, int n_items, int max_ctas, bool dense, Schedule& sc, int device_pairs = 0)
+{
+    int max_d_in = 0;
+    bool forced = false;
+    for (int j = 0; j < n_items; ++j) {
+        max_d_in = items[j].d_in > max_d_in ? items[j].d_in : max_d_in;
+        forced = forced || items[j].n_slices > 0;
+    }
+    sc.groups = (!dense && max_d_in <= kTwoGroupsMaxDin) ? 2 : 1;
+    double cost[MAX_GROUP];
+    for (int j = 0; j < n_items; ++j) {
+        sc.order[j] = j;
+        cost[j] = cost_model((items[j].d_in + BK - 1) / BK, items[j].k, sc.groups, dense).tile;
+    }
+    for (int a = 1; a < n_items; ++a)
+        for (int b = a; b > 0 && cost[sc.order[b]] > cost[sc.order[b - 1]]; --b) {
+            const int t = sc.order[b]; sc.order[b] = sc.order[b - 1]; sc.order[b - 1] = t;
+        }
+    int n_pairs = device_pairs > 0 ? device_pairs : encode_tc_max_pairs();
+    if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
+    if (n_pairs > MAX_PAIRS) n_pairs = MAX_PAIRS;
+    // Cutting row tiles at the pairs' shares costs extra pieces (each gathers its own survivors at first), so it is not
+    // done where whole row tiles already fill the pairs' waves evenly. (Eight 512-wide layers of 16384 tokens, 512 row
+    // tiles in 7 waves of 74: whole rows 1.49 ms, cut 1.54 ms; one 1024-wide layer of 8192 tokens, 32 row tiles: two
+    // uniform slices 0.298 ms, cut 0.284 ms; 256 row tiles of a 128-wide encoder, k = 128: 2.54 ms against 2.36 ms.)
+    bool even_without_cuts = false;
+    if (!forced) {
+        int units = 0;
+        for (int j = 0; j < n_items; ++j) units += encode_tc_row_tiles(items[j].T) * encode_tc_min_slices(items[j].d_sae);
+        const int waves = (units + n_pairs - 1) / n_pairs;
+        even_without_cuts = static_cast<double>(units) >= 0.93 * waves * n_pairs;
+    }
+    if (forced || even_without_cuts || !plan_balanced(items, sc.order, n_items, n_pairs, sc.groups, dense, sc))
+        plan_uniform(items, sc.order, n_items, n_pairs, sc.groups, dense, sc);
+}
+
+Schedule& schedule_buffer()
+{
+    static thread_local Schedule sc;
+    return sc;
 }
 
 // Common launch of the two epilogue modes. Selection: items with d_ids / d_vals, scratch carved from d_scratch.
@@ -1032,32 +1352,30 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     const bool dense = d_dense != nullptr;
     S3_REQUIRE(n_items >= 1 && n_items <= MAX_GROUP, S3_ERR_UNSUPPORTED, "%d encoders in one launch, at most %d", n_items, MAX_GROUP);
     alignas(64) TensorMaps maps;
-    EncodeTcParams p;
+    static thread_local EncodeTcParams p;
     memset(&p, 0, sizeof(p));
     p.n_items = n_items;
     p.status = d_status;
     p.dense_out = d_dense; p.ld_out = ld_out; p.out_bf16 = out_bf16 ? 1 : 0;
     p.d_sae = items[0].d_sae;
-    int max_d_in = 0;
-    for (int j = 0; j < n_items; ++j) max_d_in = items[j].d_in > max_d_in ? items[j].d_in : max_d_in;
-    const int groups = (!dense && max_d_in <= kTwoGroupsMaxDin) ? 2 : 1;
+    for (int j = 0; j < n_items; ++j)
+        S3_REQUIRE(items[j].n_slices == 0 || items[j].n_slices >= encode_tc_min_slices(items[j].d_sae), S3_ERR_INVALID_ARG,
+                   "d_sae = %d needs at least %d column slices", items[j].d_sae, encode_tc_min_slices(items[j].d_sae));
+    Schedule& sc = schedule_buffer();
+    build_schedule(items, n_items, max_ctas, dense, sc);
+    const int groups = sc.groups;
+    const int* order = sc.order;
 
-    // items in descending order of their units' modelled duration, so that the short units fill the end of the launch
-    int order[MAX_GROUP];
-    double cost[MAX_GROUP];
-    for (int j = 0; j < n_items; ++j) {
-        order[j] = j;
-        const int nct = encode_tc_col_tiles(items[j].d_sae);
-        cost[j] = unit_cost((items[j].d_in + BK - 1) / BK, (nct + items[j].n_slices - 1) / items[j].n_slices, items[j].k);
-    }
-    for (int a = 1; a < n_items; ++a)
-        for (int b = a; b > 0 && cost[order[b]] > cost[order[b - 1]]; --b) { const int t = order[b]; order[b] = order[b - 1]; order[b - 1] = t; }
-
+    // scratch: every item's bounds, then every item's list lengths (one memset clears both: a row tile cut into fewer
+    // pieces than the item's slot count leaves the other slots empty), then the lists
     unsigned char* base = static_cast<unsigned char*>(d_scratch);
-    size_t hint_bytes = 0;
-    for (int j = 0; j < n_items; ++j) hint_bytes += round_up(static_cast<size_t>(items[j].T) * 4, 256);
-    size_t hint_off = 0, off = hint_bytes;
-    int n_units = 0;
+    size_t hint_bytes = 0, count_bytes = 0;
+    for (int q = 0; q < n_items; ++q) {
+        const EncodeTcItem& it = items[order[q]];
+        hint_bytes += round_up(static_cast<size_t>(it.T) * 4, 256);
+        count_bytes += round_up(static_cast<size_t>(it.T) * sc.slots[q] * groups * 4, 256);
+    }
+    size_t hint_off = 0, count_off = hint_bytes, off = hint_bytes + count_bytes;
     for (int q = 0; q < n_items; ++q) {
         const EncodeTcItem& it = items[order[q]];
         ItemParams& ip = p.item[q];
@@ -1069,26 +1387,28 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
         ip.kblocks = (it.d_in + BK - 1) / BK;
         ip.n_mtiles = encode_tc_row_tiles(it.T);
         ip.n_col_tiles = encode_tc_col_tiles(it.d_sae);
-        S3_REQUIRE(it.n_slices >= encode_tc_min_slices(it.d_sae), S3_ERR_INVALID_ARG, "d_sae = %d needs at least %d column slices",
-                   it.d_sae, encode_tc_min_slices(it.d_sae));
-        ip.n_slices = it.n_slices;
-        ip.unit_start = n_units;
-        n_units += ip.n_mtiles * it.n_slices;
+        ip.n_slices = sc.slots[q];
+        ip.unit_start = q == 0 ? 0 : p.item[q - 1].unit_start + p.item[q - 1].n_mtiles * p.item[q - 1].n_slices;
         ip.cap = encode_tc_list_cap(it.k, groups);
         ip.b_eff = it.st->d_b_eff;
         if (!dense) {
-            const size_t t = static_cast<size_t>(it.T), sl = static_cast<size_t>(it.n_slices) * groups;
+            const size_t t = static_cast<size_t>(it.T), sl = static_cast<size_t>(ip.n_slices) * groups;
             ip.hint = reinterpret_cast<uint32_t*>(base + hint_off);
             hint_off += round_up(t * 4, 256);
-            ip.counts = reinterpret_cast<uint32_t*>(base + off);
-            off += round_up(t * sl * 4, 256);
+            ip.counts = reinterpret_cast<uint32_t*>(base + count_off);
+            count_off += round_up(t * sl * 4, 256);
             ip.cand = reinterpret_cast<uint64_t*>(base + off);
             off += round_up(t * sl * ip.cap * sizeof(uint64_t), 256);
         }
     }
-    p.n_units = n_units;
-    // no bound is known for any row yet
-    if (!dense) S3_CUDA_TRY(cudaMemsetAsync(base, 0, hint_bytes, stream));
+    p.n_units = sc.n_units;
+    p.use_sched = sc.table ? 1 : 0;
+    if (sc.table) {
+        memcpy(p.pair_start, sc.pair_start, sizeof(p.pair_start));
+        memcpy(p.unit, sc.unit, sizeof(UnitDesc) * static_cast<size_t>(sc.n_units));
+    }
+    // no bound is known for any row yet, and no list holds anything
+    if (!dense) S3_CUDA_TRY(cudaMemsetAsync(base, 0, hint_bytes + (sc.table ? count_bytes : 0), stream));
 
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
@@ -1107,41 +1427,7 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
         S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_DENSE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set[dev] = true;
     }
-    int n_pairs = encode_tc_max_pairs();
-    if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
-    if (n_units < n_pairs) n_pairs = n_units;
-
-    // Units dealt out by modelled duration: in the flattened order (item, slice, row tile) each unit goes to the pair
-    // with the least work so far. Pairs therefore still walk the same slice of the same encoder at about the same time
-    // (its W_enc^T tiles are shared in L2), and a launch over unequal encoders ends evenly. Equal units come out
-    // round-robin, which is what the walk without a table does.
-    p.use_sched = 0;
-    if (n_items > 1 && n_units <= MAX_SCHED && n_pairs <= MAX_PAIRS) {
-        static thread_local uint16_t unit_pair[MAX_SCHED];
-        double load[MAX_PAIRS];
-        int count[MAX_PAIRS];
-        for (int q = 0; q < n_pairs; ++q) { load[q] = 0.0; count[q] = 0; }
-        int u = 0;
-        for (int q = 0; q < n_items; ++q) {
-            const int units = p.item[q].n_mtiles * p.item[q].n_slices;
-            const double c = cost[order[q]];
-            for (int i = 0; i < units; ++i, ++u) {
-                int best = 0;
-                for (int r = 1; r < n_pairs; ++r)
-                    if (load[r] < load[best]) best = r;
-                load[best] += c;
-                unit_pair[u] = static_cast<uint16_t>(best);
-                ++count[best];
-            }
-        }
-        int run = 0;
-        for (int q = 0; q < n_pairs; ++q) { p.pair_start[q] = static_cast<uint16_t>(run); run += count[q]; }
-        p.pair_start[n_pairs] = static_cast<uint16_t>(run);
-        int fill[MAX_PAIRS];
-        for (int q = 0; q < n_pairs; ++q) fill[q] = p.pair_start[q];
-        for (int i = 0; i < n_units; ++i) p.sched[fill[unit_pair[i]]++] = static_cast<uint16_t>(i);
-        p.use_sched = 1;
-    }
+    const int n_pairs = sc.n_pairs;
 
     if (dense) {
         encode_tc_kernel<M_DENSE, 1><<<2 * n_pairs, 64 + 128, smem, stream>>>(maps, p);
@@ -1157,7 +1443,7 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     for (int q = 0; q < n_items; ++q) {
         const EncodeTcItem& it = items[order[q]];
         const ItemParams& ip = p.item[q];
-        mg.item[q] = MergeItem{ip.cand, ip.counts, ip.hint, it.d_ids, it.d_vals, it.T, it.n_slices * groups, it.k, ip.cap, rows};
+        mg.item[q] = MergeItem{ip.cand, ip.counts, ip.hint, it.d_ids, it.d_vals, it.T, ip.n_slices * groups, it.k, ip.cap, rows};
         rows += (it.T + kMergeRowsPerBlock - 1) / kMergeRowsPerBlock * kMergeRowsPerBlock;
     }
     launch_candidate_merge_group(mg, rows, stream);
@@ -1166,6 +1452,44 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
 }
 
 }  // namespace
+
+size_t encode_tc_group_workspace_need(const EncodeTcItem* items, int n_items, int max_ctas)
+{
+    if (n_items < 1 || n_items > MAX_GROUP) return 0;
+    Schedule& sc = schedule_buffer();
+    build_schedule(items, n_items, max_ctas, false, sc);
+    size_t n = 0;
+    for (int q = 0; q < n_items; ++q) n += encode_tc_workspace_bytes(items[sc.order[q]].T, sc.slots[q], items[sc.order[q]].k);
+    return n;
+}
+
+// The units of the launch over these items on n_pairs CTA pairs, six integers each: pair, item (caller's index), row
+// tile, first column tile, one past the last column tile, candidate-list slot. Returns the unit count (also when it
+// exceeds max_units; only max_units are written), or -1 when the launch deals uniform slices round-robin without a table.
+int encode_tc_describe_schedule(const EncodeTcItem* items, int n_items, int n_pairs, int32_t* out, int max_units, int32_t* slots_out)
+{
+    if (n_items < 1 || n_items > MAX_GROUP || n_pairs < 1) return -2;
+    Schedule& sc = schedule_buffer();
+    build_schedule(items, n_items, 2 * n_pairs, false, sc, n_pairs);
+    for (int q = 0; q < n_items; ++q) slots_out[sc.order[q]] = sc.slots[q];
+    if (!sc.table) return -1;
+    for (int pr = 0; pr < sc.n_pairs; ++pr)
+        for (int i = sc.pair_start[pr]; i < sc.pair_start[pr + 1]; ++i) {
+            if (i >= max_units) continue;
+            const UnitDesc& u = sc.unit[i];
+            int32_t* o = out + static_cast<size_t>(i) * 6;
+            o[0] = pr; o[1] = sc.order[u.item]; o[2] = u.mt; o[3] = u.tile_lo; o[4] = u.tile_hi; o[5] = u.slot;
+        }
+    return sc.n_units;
+}
+
+int encode_tc_group_ctas(const EncodeTcItem* items, int n_items, int max_ctas)
+{
+    if (n_items < 1 || n_items > MAX_GROUP) return 0;
+    Schedule& sc = schedule_buffer();
+    build_schedule(items, n_items, max_ctas, false, sc);
+    return 2 * sc.n_pairs;
+}
 
 s3_status launch_encode_tc_group(const EncodeTcItem* items, int n_items, int max_ctas, void* d_scratch, uint32_t* d_status,
                                  cudaStream_t stream)

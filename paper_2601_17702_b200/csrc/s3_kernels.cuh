@@ -20,6 +20,7 @@ int encode_tc_row_tiles(int T);
 int encode_tc_min_slices(int d_sae);
 int encode_tc_max_pairs();         // CTA pairs (work units in flight) of the bf16 encode on this device
 size_t encode_tc_workspace_bytes(int T, int n_slices, int k);     // scratch after the status block
+size_t encode_tc_workspace_bound(int T, int k);    // holds any automatic schedule of T tokens or fewer
 // Encode kernel + candidate merge: writes ids / vals [T,k].
 s3_status launch_encode_tc(const EncodeTcState* st, const void* d_x, int64_t ldx, int T, int d_in, int d_sae, int k,
                            int n_slices, int max_ctas, void* d_scratch, uint32_t* d_status, int32_t* d_ids, float* d_vals,
@@ -31,10 +32,14 @@ struct EncodeTcItem {
     const EncodeTcState* st;
     const void* d_x;
     int64_t ldx;
-    int T, d_in, d_sae, k, n_slices;
+    int T, d_in, d_sae, k, n_slices;      // n_slices: uniform column slices per row tile; 0 = scheduled by the launch
     int32_t* d_ids;
     float* d_vals;
 };
+// Exact scratch bytes and thread blocks of the launch these items would get (only T, d_in, d_sae, k, n_slices are read).
+size_t encode_tc_group_workspace_need(const EncodeTcItem* items, int n_items, int max_ctas);
+int encode_tc_group_ctas(const EncodeTcItem* items, int n_items, int max_ctas);
+int encode_tc_describe_schedule(const EncodeTcItem* items, int n_items, int n_pairs, int32_t* out, int max_units, int32_t* slots_out);
 s3_status launch_encode_tc_group(const EncodeTcItem* items, int n_items, int max_ctas, void* d_scratch, uint32_t* d_status,
                                  cudaStream_t stream);
 
