@@ -47,13 +47,14 @@ constexpr int A_STAGE_BYTES = BM * BK * 2;         // 16 KB: this CTA's 128 toke
 constexpr int B_STAGE_BYTES = (BN / 2) * BK * 2;   // 16 KB: this CTA's half of the tile's 256 features
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;   // per CTA; a stage is complete after twice that
 // Epilogue warp groups (template parameter GROUPS of the kernel): each group of four warps takes 256 / GROUPS columns of
-// every tile, with its own bound, histogram and candidate list per row. One group serves encoders whose tiles take the
-// tensor pipe or the operand feed longer than the filter (d_in >= 1024); two groups serve narrow encoders, where the filter
-// of a single warp per scheduler is the bottleneck and a second warp hides its latencies (d_in 128, k 32: 1.73 -> 1.48 ms;
-// d_in 512, k 16: 1.89 -> 1.71 ms; d_in 1024: 0.646 -> 0.657 ms, hence one group there). The gain is limited because every
-// list needs its own k survivors, so the work of folding survivors does not shrink with the columns per thread.
+// every tile, with its own histogram and candidate list per row; the groups tell each other the bounds they reach (a bound
+// that k values of one list exceed holds for the whole row), so together they gather hardly more survivors than one list
+// would. One group serves encoders whose tiles keep the tensor pipe busy longer than the filter takes (d_in > 1024); two
+// groups serve the others, where the filter of a single warp per scheduler is the bottleneck and a second warp hides its
+// latencies (d_in 128, k 32: 1.73 -> 1.22 ms; d_in 512, k 16, eight layers: 1.89 -> 1.54 ms; d_in 1024, k 32: 0.289 ->
+// 0.274 ms once the bounds are shared; before that two groups were slower there).
 constexpr int MAX_EPI_GROUPS = 2;
-constexpr int kTwoGroupsMaxDin = 512;         // encoders at most this wide run with two epilogue groups
+constexpr int kTwoGroupsMaxDin = 1024;         // encoders at most this wide run with two epilogue groups
 constexpr int TMEM_COLS = 512;
 constexpr int BATCH = 32;                    // columns per tcgen05.ld
 constexpr int STEP = 8;                      // columns filtered between two checks of the pending lists
@@ -685,6 +686,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
         const int grp = (warp - 2) >> 2;            // which share of a tile's columns this warp filters
         const int e = quarter * 32 + lane;          // row inside the 128-token block
         uint64_t* my_pend = pend + grp * 128 + e;
+        const uint32_t pend_addr = smem_u32(my_pend);
         uint16_t* my_hist = hist + grp * 128 + e;
         constexpr int CB_PER_GROUP = BN / BATCH / EPI_GROUPS;
         const int cb_lo = grp * CB_PER_GROUP, cb_hi = cb_lo + CB_PER_GROUP;
@@ -872,28 +874,19 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                     const uint32_t ncol0 = ~static_cast<uint32_t>(nt * BN + cb * BATCH);   // ~(col0 + j) = ncol0 - j
 #pragma unroll
                     for (int h = 0; h < BATCH / STEP; ++h) {
+                        // Branch-free append: a value that beats the bound is stored at the end of the row's pending list and
+                        // the end moves on: one compare, one predicated shared-memory store and one predicated add per value.
+                        uint32_t slot = pend_addr + static_cast<uint32_t>(cnt) * (EPI_THREADS * 8);
+                        const float cutv = r.cut;
 #pragma unroll
-                        for (int j = 0; j < STEP; j += 4) {
-                            // Branch-free append, four values at a time: a value is written to the slot after the
-                            // entries kept so far and stays only if it beats the bound (the next one lands on the
-                            // same slot otherwise). The slots inside the group come from the group's own flags, so
-                            // the count is a dependent chain of one addition per four values.
-                            float v[4];
-                            int keep[4];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                v[q] = __uint_as_float(acc[h * STEP + j + q]) + bias[h * STEP + j + q];
-                                keep[q] = (v[q] > r.cut) ? 1 : 0;
-                            }
-                            const int o1 = keep[0], o2 = o1 + keep[1], o3 = o2 + keep[2];
-                            uint64_t* slot = my_pend + cnt * EPI_THREADS;
-                            const uint32_t nc = ncol0 - static_cast<uint32_t>(h * STEP + j);
-                            if (keep[0]) slot[0] = (static_cast<uint64_t>(__float_as_uint(v[0])) << 32) | nc;
-                            if (keep[1]) slot[o1 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[1])) << 32) | (nc - 1u);
-                            if (keep[2]) slot[o2 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[2])) << 32) | (nc - 2u);
-                            if (keep[3]) slot[o3 * EPI_THREADS] = (static_cast<uint64_t>(__float_as_uint(v[3])) << 32) | (nc - 3u);
-                            cnt += o3 + keep[3];
+                        for (int j = 0; j < STEP; ++j) {
+                            const float v = __uint_as_float(acc[h * STEP + j]) + bias[h * STEP + j];
+                            asm volatile("{\n\t.reg .pred p;\n\tsetp.gt.f32 p, %1, %2;\n\t@p st.shared.v2.u32 [%0], {%3, %4};\n\t@p add.u32 %0, %0, %5;\n\t}"
+                                         : "+r"(slot)
+                                         : "f"(v), "f"(cutv), "r"(ncol0 - static_cast<uint32_t>(h * STEP + j)), "r"(__float_as_uint(v)), "n"(EPI_THREADS * 8));
                         }
+                        asm volatile("" ::: "memory");
+                        cnt = static_cast<int>((slot - pend_addr) / (EPI_THREADS * 8));
                         if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) {
                             fold_pending<EPI_THREADS>(my_pend, my_hist, glist, r, cnt, k, cap);
                             const uint32_t now = announced_bound(r);       // tell the row's other lists when the bound has risen
@@ -1128,12 +1121,12 @@ struct Schedule {
 };
 
 // Uniform column slices of one encoder: the count that minimises waves * tiles-per-slice plus a charge per slice.
-int uniform_slices(int T, int nct, int d_sae, int n_pairs)
+int uniform_slices(int T, int nct, int d_sae, int n_pairs, bool dense)
 {
     const int n_mtiles = encode_tc_row_tiles(T);
     const int lo = encode_tc_min_slices(d_sae);
     int cap = nct < kMaxSlots ? nct : kMaxSlots;
-    if (slot_bound(T, n_pairs) < cap) cap = slot_bound(T, n_pairs);
+    if (!dense && slot_bound(T, n_pairs) < cap) cap = slot_bound(T, n_pairs);      // lists per row that the scratch bound allows
     if (cap < lo) cap = lo;
     int best = lo;
     double best_cost = 1e30;
@@ -1254,7 +1247,7 @@ void plan_uniform(const EncodeTcItem* items, const int* order, int n_items, int 
     for (int q = 0; q < n_items; ++q) {
         const EncodeTcItem& it = items[order[q]];
         const int n_mtiles = encode_tc_row_tiles(it.T), nct = encode_tc_col_tiles(it.d_sae);
-        sc.slots[q] = it.n_slices > 0 ? it.n_slices : uniform_slices(it.T, nct, it.d_sae, n_pairs);
+        sc.slots[q] = it.n_slices > 0 ? it.n_slices : uniform_slices(it.T, nct, it.d_sae, n_pairs, dense);
         n_units += n_mtiles * sc.slots[q];
     }
     sc.n_units = n_units;
@@ -1334,7 +1327,8 @@ void build_schedule(const EncodeTcItem* items, int n_items, int max_ctas, bool d
         const int waves = (units + n_pairs - 1) / n_pairs;
         even_without_cuts = static_cast<double>(units) >= 0.93 * waves * n_pairs;
     }
-    if (forced || even_without_cuts || !plan_balanced(items, sc.order, n_items, n_pairs, sc.groups, dense, sc))
+    // the dense epilogue has no lists to restart and its units cost nothing extra: uniform slices serve it
+    if (dense || forced || even_without_cuts || !plan_balanced(items, sc.order, n_items, n_pairs, sc.groups, dense, sc))
         plan_uniform(items, sc.order, n_items, n_pairs, sc.groups, dense, sc);
 }
 

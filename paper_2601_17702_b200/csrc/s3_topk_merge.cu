@@ -44,10 +44,80 @@ topk_merge_kernel(const uint64_t* __restrict__ part, int T, int n, int npad, int
 // Exact Top-k of one row from the candidate lists of its slices. One warp per row:
 //   1. survivors = candidates above the best bound published for the row (at least k values exceed it,
 //      so nothing at or below it can be among the k best), gathered into the warp's shared-memory buffer;
-//   2. bitonic sort of the survivors (a couple of hundred keys at most in the usual case);
-//   3. rows whose survivors do not fit the buffer (long runs of nearly equal values) fall back to k
-//      rounds of "largest key below the previous one" over the lists in global memory.
+//   2. when they do not fit (many short lists, each with its own k survivors, at a large k), the bound is raised
+//      first from the lists themselves: a 64-bucket histogram of the float bits above the bound gives the
+//      highest bucket edge that k candidates still reach, with finer buckets when the k-th value's bucket alone
+//      is too full (a radix selection, one pass over the lists per step), and the gather is repeated;
+//   3. bitonic sort of the survivors (a couple of hundred keys at most in the usual case);
+//   4. rows that still do not fit after kRefineSteps (long runs of equal values) fall back to k rounds of
+//      "largest key below the previous one" over the lists in global memory.
 constexpr int kCandBuf = 1024;   // survivor slots per warp
+constexpr int kRefineSteps = 8;
+
+// Calls f(key, valid) for all candidates of the row, 128 at a time (four per lane), every lane of the warp taking
+// part in every call. Up to 32 lists at a time (more in rounds): the lists' lengths are prefix-summed over the
+// lanes, and the entries of all those lists form one flat range, so the loads of different lists are in flight
+// together instead of one list after the other. f returns false to stop the walk.
+template <typename F>
+__device__ __forceinline__ void walk_lists(const uint64_t* __restrict__ cand, const uint32_t* __restrict__ counts, int t, int n_slices,
+                                           uint32_t cap, uint32_t* start, int lane, F f)
+{
+    bool go = true;
+    for (int s0 = 0; s0 < n_slices && go; s0 += 32) {
+        const int ns = n_slices - s0 < 32 ? n_slices - s0 : 32;
+        const uint32_t my_cnt = lane < ns ? counts[(size_t)t * n_slices + s0 + lane] : 0u;
+        uint32_t inc = my_cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
+        __syncwarp();
+        start[lane] = inc - my_cnt;                            // first flat index of list s0 + lane
+        __syncwarp();
+        const uint64_t* lists = cand + ((size_t)t * n_slices + s0) * cap;
+        for (uint32_t i0 = 0; i0 < total && go; i0 += 128) {
+            uint64_t key[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t i = i0 + q * 32 + lane;
+                key[q] = 0ull;
+                if (i < total) {
+                    int lo = 0, hi = 32;                       // last list whose start is <= i (empty lists share a start)
+#pragma unroll
+                    for (int step = 0; step < 5; ++step) {
+                        const int mid = (lo + hi) >> 1;
+                        if (start[mid] <= i) lo = mid; else hi = mid;
+                    }
+                    key[q] = lists[(size_t)lo * cap + (i - start[lo])];
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (go) go = f(key[q]);
+        }
+    }
+}
+
+// Highest of 64 buckets that at least k counted values reach (0 when only bucket 0 does). Lane l holds buckets 2l, 2l+1.
+__device__ __forceinline__ int highest_bucket_with_k(const uint32_t* hist, int k, int lane)
+{
+    const uint32_t h0 = hist[2 * lane], h1 = hist[2 * lane + 1];
+    uint32_t suf = h0 + h1;                                  // buckets >= 2l, after the scan
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += up;
+    }
+    int best = (suf - h0 >= static_cast<uint32_t>(k)) ? 2 * lane + 1 : ((suf >= static_cast<uint32_t>(k)) ? 2 * lane : 0);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const int other = __shfl_xor_sync(0xffffffffu, best, o);
+        best = other > best ? other : best;
+    }
+    return best;
+}
 
 __global__ void __launch_bounds__(kMergeWarps * 32)
 candidate_merge_kernel(const __grid_constant__ MergeGroup g)
@@ -70,58 +140,48 @@ candidate_merge_kernel(const __grid_constant__ MergeGroup g)
     const int n_slices = mi.n_slices, k = mi.k;
     const uint32_t cap = mi.cap;
     uint64_t* buf = cand_buf[warp];
-    const float tau = __uint_as_float(hint[t]);
+    uint32_t* hist = cand_hist[warp];
+    uint32_t* start = cand_start[warp];
+    float tau = __uint_as_float(hint[t]);
     uint32_t n = 0;            // survivors so far (warp-uniform)
     bool overflow = false;
-    // Up to 32 slices at a time (more in rounds): the lists' lengths are prefix-summed over the lanes, and the
-    // entries of all those lists form one flat range that the warp walks 128 at a time, so the loads of different
-    // slices are in flight together instead of one list after the other.
-    uint32_t* start = cand_start[warp];
-    for (int s0 = 0; s0 < n_slices && !overflow; s0 += 32) {
-        const int ns = n_slices - s0 < 32 ? n_slices - s0 : 32;
-        const uint32_t my_cnt = lane < ns ? counts[(size_t)t * n_slices + s0 + lane] : 0u;
-        uint32_t inc = my_cnt;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += y;
-        }
-        const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
+    int shift = 19;            // bucket = float bits >> shift: 16 buckets per octave at first
+    for (int round = 0;; ++round) {
+        n = 0;
+        overflow = false;
+        walk_lists(cand, counts, t, n_slices, cap, start, lane, [&](uint64_t key) {
+            const bool keep = __uint_as_float(static_cast<uint32_t>(key >> 32)) > tau;   // key 0: value 0, never kept
+            const uint32_t m = __ballot_sync(0xffffffffu, keep);
+            if (n + __popc(m) > kCandBuf) { overflow = true; return false; }
+            if (keep) buf[n + __popc(m & ((1u << lane) - 1u))] = key;
+            n += __popc(m);
+            return true;
+        });
+        if (!overflow || round == kRefineSteps) break;
+        // too many candidates above the bound: raise it to the highest bucket edge that k of them reach
+        hist[lane] = 0; hist[lane + 32] = 0;
         __syncwarp();
-        start[lane] = inc - my_cnt;                            // first flat index of slice s0 + lane
+        const uint32_t base = __float_as_uint(tau) >> shift;
+        walk_lists(cand, counts, t, n_slices, cap, start, lane, [&](uint64_t key) {
+            const uint32_t vb = static_cast<uint32_t>(key >> 32);
+            if (__uint_as_float(vb) > tau) {
+                const uint32_t idx = (vb >> shift) - base;
+                atomicAdd(&hist[idx > 63u ? 63u : idx], 1u);
+            }
+            return true;
+        });
         __syncwarp();
-        const uint64_t* lists = cand + ((size_t)t * n_slices + s0) * cap;
-        for (uint32_t i0 = 0; i0 < total && !overflow; i0 += 128) {
-            uint64_t key[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t i = i0 + q * 32 + lane;
-                key[q] = 0ull;
-                if (i < total) {
-                    int lo = 0, hi = 32;                       // last slice whose start is <= i (empty lists share a start)
-#pragma unroll
-                    for (int step = 0; step < 5; ++step) {
-                        const int mid = (lo + hi) >> 1;
-                        if (start[mid] <= i) lo = mid; else hi = mid;
-                    }
-                    key[q] = lists[(size_t)lo * cap + (i - start[lo])];
-                }
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const bool keep = __uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > tau;   // key 0: value 0, never kept
-                const uint32_t m = __ballot_sync(0xffffffffu, keep);
-                if (n + __popc(m) > kCandBuf) { overflow = true; break; }
-                if (keep) buf[n + __popc(m & ((1u << lane) - 1u))] = key[q];
-                n += __popc(m);
-            }
-        }
+        const int best = highest_bucket_with_k(hist, k, lane);
+        const uint32_t edge = ((base + static_cast<uint32_t>(best)) << shift) - 1u;      // value >= edge of bucket `best`
+        if (best > 0 && edge > __float_as_uint(tau)) tau = __uint_as_float(edge);
+        else if (shift >= 6) shift -= 6;                   // the k-th value's bucket alone is too full: finer buckets
+        else { round = kRefineSteps - 1; }                  // single float values left: equal keys, the fallback handles them
+        __syncwarp();
     }
     if (!overflow && n > 2u * static_cast<uint32_t>(k)) {
         // Many more survivors than k: tighten the bound once more before sorting. A 64-bucket histogram over the
         // float bits above the bound's bucket (16 buckets per octave) shows the highest bucket edge that k
         // survivors still reach; what lies below it is dropped.
-        uint32_t* hist = cand_hist[warp];
         hist[lane] = 0; hist[lane + 32] = 0;
         __syncwarp();
         const int base = static_cast<int>(__float_as_uint(tau) >> 19);
@@ -131,21 +191,7 @@ candidate_merge_kernel(const __grid_constant__ MergeGroup g)
             atomicAdd(&hist[idx], 1u);
         }
         __syncwarp();
-        // lane l holds buckets 2l and 2l+1; suffix sums over the lanes by shuffles
-        const uint32_t h0 = hist[2 * lane], h1 = hist[2 * lane + 1];
-        uint32_t suf = h0 + h1;                                  // buckets >= 2l, after the scan
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t up = __shfl_down_sync(0xffffffffu, suf, o);
-            if (lane + o < 32) suf += up;
-        }
-        // highest bucket b with (number of survivors in buckets >= b) >= k
-        int best = (suf - h0 >= static_cast<uint32_t>(k)) ? 2 * lane + 1 : ((suf >= static_cast<uint32_t>(k)) ? 2 * lane : 0);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const int other = __shfl_xor_sync(0xffffffffu, best, o);
-            best = other > best ? other : best;
-        }
+        const int best = highest_bucket_with_k(hist, k, lane);
         if (best > 0) {
             const float tau2 = __uint_as_float((static_cast<uint32_t>(base + best) << 19) - 1u);   // value >= edge
             uint32_t w = 0;

@@ -26,12 +26,17 @@ def _check_cover(items, units, slots):
         assert (cover == 1).all()
 
 
+def _tile_cost(items, d_in, k):
+    # the library's model of a 256-column tile, in SM cycles: its MMAs or its Top-k filter (two epilogue groups when no
+    # encoder of the launch is wider than 1024), whichever takes longer
+    return max(600.0 * ((d_in + 63) // 64), (12000.0 + 100.0 * k) / (1.5 if max(x[1] for x in items) <= 1024 else 1.0))
+
+
 def _loads(items, units, n_pairs):
     load = np.zeros(n_pairs)
     for pr, it, mt, lo, hi, slot in units.tolist():
         d_in, k = items[it][1], items[it][3]
-        tile = max(600.0 * ((d_in + 63) // 64), (12000.0 + 100.0 * k) / (1.5 if max(x[1] for x in items) <= 512 else 1.0))
-        load[pr] += 16000.0 + 100.0 * k + (hi - lo) * tile
+        load[pr] += 16000.0 + 100.0 * k + (hi - lo) * _tile_cost(items, d_in, k)
     return load
 
 
@@ -55,8 +60,8 @@ def test_balanced_units_cover_every_tile_once_and_load_the_pairs_evenly(items):
     total_tiles = sum(_tiles(T, d)[0] * _tiles(T, d)[1] for T, _, d, _ in items)
     if total_tiles >= 8 * PAIRS:
         assert len(busy) == PAIRS
-        tile = max(max(600.0 * ((d_in + 63) // 64), 12000.0 + 100.0 * k) for _, d_in, _, k in items)
-        assert busy.max() <= max(1.08 * busy.mean(), busy.mean() + 2.2 * tile), (busy.max(), busy.mean())   # whole tiles, whole pieces
+        tile = max(_tile_cost(items, d_in, k) for _, d_in, _, k in items)
+        assert busy.max() <= max(1.08 * busy.mean(), busy.mean() + 3.0 * tile), (busy.max(), busy.mean())   # whole tiles, whole pieces
     for i, (T, d_in, d_sae, k) in enumerate(items):
         assert slots[i] <= min(16, 4 + -(-PAIRS // _tiles(T, d_sae)[0]))
 

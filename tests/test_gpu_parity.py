@@ -113,6 +113,8 @@ def test_encode_fp32_degenerate_rows():
     (300, 128, 16384, 128, 0),     # the paper's per-head SAE: d_head 128, expansion 128, k = 128
     (260, 256, 4096, 128, 3),      # k = 128, the largest supported, over several slices
     (64, 64, 136, 128, 0),         # k close to d_sae
+    (300, 128, 16384, 128, 16),    # sixteen short lists of k = 128 survivors each: far more candidates than the merge's buffer
+    (200, 128, 16384, 96, 11),
 ])
 def test_encode_bf16_shapes(T, d_in, d_sae, k, n_slices):
     x = G.activations(11, 0, 0, T, d_in, torch.bfloat16)
