@@ -1103,7 +1103,7 @@ CostModel cost_model(int kblocks, int k, int groups, bool dense)
     const double filter = dense ? 6000.0 : (12000.0 + 100.0 * k) / (groups == 2 ? 1.5 : 1.0);
     CostModel c;
     c.tile = mma > filter ? mma : filter;
-    c.unit = dense ? 2000.0 : 16000.0 + 100.0 * k;
+    c.unit = dense ? 2000.0 : 5000.0 + 100.0 * k;       // measured closer to 16000 + 100 k, but shares cut with the smaller charge end more evenly
     return c;
 }
 

@@ -36,7 +36,7 @@ def _loads(items, units, n_pairs):
     load = np.zeros(n_pairs)
     for pr, it, mt, lo, hi, slot in units.tolist():
         d_in, k = items[it][1], items[it][3]
-        load[pr] += 16000.0 + 100.0 * k + (hi - lo) * _tile_cost(items, d_in, k)
+        load[pr] += 5000.0 + 100.0 * k + (hi - lo) * _tile_cost(items, d_in, k)
     return load
 
 
