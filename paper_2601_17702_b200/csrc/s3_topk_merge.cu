@@ -51,7 +51,7 @@ topk_merge_kernel(const uint64_t* __restrict__ part, int T, int n, int npad, int
 //   3. bitonic sort of the survivors (a couple of hundred keys at most in the usual case);
 //   4. rows that still do not fit after kRefineSteps (long runs of equal values) fall back to k rounds of
 //      "largest key below the previous one" over the lists in global memory.
-constexpr int kCandBuf = 512;    // survivor slots per warp (1024 halves the warps an SM holds: the key SAE's merge 0.045 -> 0.036 ms at 512)
+constexpr int kCandBuf = 512;    // survivor slots per warp (1024 halves the warps an SM holds: key SAE encode + merge 0.269 -> 0.260 ms at 512)
 constexpr int kRefineSteps = 8;
 
 // Calls f(key, valid) for all candidates of the row, 128 at a time (four per lane), every lane of the warp taking
