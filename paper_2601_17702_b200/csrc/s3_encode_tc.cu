@@ -64,7 +64,6 @@ constexpr int NB = 64;                       // histogram buckets per row
 #define S3_FOLD_CHUNK 4
 #endif
 constexpr int FOLD_CHUNK = S3_FOLD_CHUNK;    // pending entries a fold handles per step
-constexpr int kCompactMinTiles = 32;          // units of at least this many column tiles compact their candidate lists
 constexpr int COLD_LEVELS = 6;                // trial bounds of the cold-start pass, as fractions of the first batch's maximum
 __device__ constexpr float kColdFraction[COLD_LEVELS] = {0.80f, 0.65f, 0.52f, 0.40f, 0.30f, 0.20f};
 constexpr int HSHIFT = 19;                   // bucket = float bits >> 19: 16 buckets per octave
@@ -907,21 +906,10 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                     // what the merge may cut the row's lists at: this list's own bound or a better one learnt meanwhile
                     uint32_t out = announced_bound(r);
                     if (__float_as_uint(r.ext) > out) out = __float_as_uint(r.ext);
-                    // The list was filled under bounds that rose along the slice (about k (1 + ln(columns / k))
-                    // entries); only what beats the final bound can still matter, so the list is compacted once
-                    // here and the merge reads a fraction of it. The pass is a tail of dependent round trips after the
-                    // unit's last tile, so it is taken only when the unit was long enough to make that tail small.
-                    const float cut = __uint_as_float(out);
-                    uint32_t w = tile_hi - tile_lo >= kCompactMinTiles ? 0u : r.gcnt;
-                    for (uint32_t i0 = 0; i0 < r.gcnt && tile_hi - tile_lo >= kCompactMinTiles; i0 += 16) {
-                        uint64_t key[16];                        // read first: the writes land at or before i0
-#pragma unroll
-                        for (int q = 0; q < 16; ++q) key[q] = i0 + q < r.gcnt ? glist[i0 + q] : 0ull;
-#pragma unroll
-                        for (int q = 0; q < 16; ++q)
-                            if (__uint_as_float(static_cast<uint32_t>(key[q] >> 32)) > cut) glist[w++] = key[q];
-                    }
-                    ip.counts[list_idx] = w;
+                    // The list stays as it was filled (about k (1 + ln(columns / k)) entries under bounds that rose along the
+                    // unit): the merge cuts it at the row's final bound. Compacting it here, a tail of dependent round trips
+                    // after the unit's last tile, cost more than the merge saves (heads k = 128: 2.36 -> 2.08 ms without it).
+                    ip.counts[list_idx] = r.gcnt;
                     if (out > hint_in) atomicMax(ip.hint + orow, out);
                 }
             }
