@@ -1280,6 +1280,69 @@ void plan_uniform(const EncodeTcItem* items, const int* order, int n_items, int 
     sc.table = true;
 }
 
+// Banded walk of one encoder whose weights do not stay in L2: bands of R row tiles, each band swept by its S column
+// slices at the same time (one unit per pair), band after band. The hot set is then a band's token tiles (R x 2 MB at
+// d_in 4096, re-read for every column tile) plus the windows of W_enc^T that the slices stream; with all row tiles in
+// one band the token tiles alone fill the L2 and W_enc^T is read about four times (query SAE, T 8192: 1.03-1.27 GB of
+// DRAM traffic with 32 row tiles x 2 slices, 0.76-0.80 GB with two bands of 16 x 4, the same 1.57 ms; 12 x 6 and 8 x 8
+// are 4 and 11 % slower: more lists per row). Four slices, more when there are too few row tiles to fill the pairs.
+bool plan_banded(const EncodeTcItem& it, int n_pairs, Schedule& sc)
+{
+    static thread_local UnitDesc gen[MAX_SCHED];
+    static thread_local uint16_t gen_pair[MAX_SCHED];
+    const int n_mtiles = encode_tc_row_tiles(it.T), nct = encode_tc_col_tiles(it.d_sae);
+    // (S, R): the modelled time is bands x tiles per slice (+ a quarter tile per slice and band, as for uniform slices);
+    // among the choices within 3 % of the best, the fewest slices whose band of token tiles stays under 40 MB, else the best.
+    const int s_lo = encode_tc_min_slices(it.d_sae);
+    int s_hi = slot_bound(it.T, n_pairs) < nct ? slot_bound(it.T, n_pairs) : nct;
+    s_hi = s_hi > kMaxSlots ? kMaxSlots : s_hi;
+    if (s_hi < s_lo) return false;
+    const int r_hot = static_cast<int>((size_t(40) << 20) / (static_cast<size_t>(PAIR_M) * it.d_in * 2));
+    auto band_rows = [&](int S) {
+        int R = n_pairs / S;
+        R = R < 1 ? 1 : (R > n_mtiles ? n_mtiles : R);
+        const int bands = (n_mtiles + R - 1) / R;
+        return (n_mtiles + bands - 1) / bands;                  // bands of equal height
+    };
+    auto modelled = [&](int S) {
+        const int R = band_rows(S), bands = (n_mtiles + R - 1) / R;
+        return bands * ((nct + S - 1) / S) + 0.25 * S * bands;
+    };
+    double best = 1e30;
+    for (int c = s_lo; c <= s_hi; ++c) best = modelled(c) < best ? modelled(c) : best;
+    int S = 0;
+    for (int c = s_lo; c <= s_hi && S == 0; ++c)
+        if (modelled(c) <= 1.03 * best && band_rows(c) <= r_hot) S = c;
+    for (int c = s_lo; c <= s_hi && S == 0; ++c)
+        if (modelled(c) <= best + 1e-9) S = c;
+    const int R = band_rows(S);
+    if (S > kMaxSlots || n_mtiles > 65535 || n_mtiles * S > MAX_SCHED || (nct + S - 1) / S > 255) return false;
+    int n = 0;
+    for (int b0 = 0; b0 < n_mtiles; b0 += R) {
+        const int rows = n_mtiles - b0 < R ? n_mtiles - b0 : R;
+        int i = 0;
+        for (int sl = 0; sl < S; ++sl)
+            for (int r = 0; r < rows; ++r, ++i, ++n) {
+                gen[n].mt = static_cast<uint16_t>(b0 + r);
+                gen[n].tile_lo = static_cast<uint16_t>(static_cast<int64_t>(sl) * nct / S);
+                gen[n].tile_hi = static_cast<uint16_t>(static_cast<int64_t>(sl + 1) * nct / S);
+                gen[n].item = 0;
+                gen[n].slot = static_cast<uint8_t>(sl);
+                gen_pair[n] = static_cast<uint16_t>(i % n_pairs);
+            }
+    }
+    int count[MAX_PAIRS] = {};
+    for (int i = 0; i < n; ++i) ++count[gen_pair[i]];
+    int run = 0, used = 0;
+    for (int q = 0; q < n_pairs; ++q) { sc.pair_start[q] = static_cast<uint16_t>(run); run += count[q]; if (count[q]) used = q + 1; }
+    for (int q = n_pairs; q <= MAX_PAIRS; ++q) sc.pair_start[q] = static_cast<uint16_t>(run);
+    int fill[MAX_PAIRS];
+    for (int q = 0; q < n_pairs; ++q) fill[q] = sc.pair_start[q];
+    for (int i = 0; i < n; ++i) sc.unit[fill[gen_pair[i]]++] = gen[i];
+    sc.n_units = n; sc.n_pairs = used; sc.table = true; sc.slots[0] = S;
+    return true;
+}
+
 // The schedule of a launch: launch order of the items (descending modelled tile duration, so that the short tiles fill
 // the end), epilogue groups, CTA pairs and the units. Items that leave n_slices at 0 get the balanced plan when it
 // applies; an item with n_slices > 0 forces uniform slices for the whole launch.
@@ -1316,6 +1379,9 @@ void build_schedule(const EncodeTcItem* items, int n_items, int max_ctas, bool d
         even_without_cuts = static_cast<double>(units) >= 0.93 * waves * n_pairs;
     }
     // the dense epilogue has no lists to restart and its units cost nothing extra: uniform slices serve it
+    if (!dense && !forced && n_items == 1 && static_cast<size_t>(items[0].d_sae) * items[0].d_in * 2 > kRoundBytes &&
+        plan_banded(items[0], n_pairs, sc))
+        return;
     if (dense || forced || even_without_cuts || !plan_balanced(items, sc.order, n_items, n_pairs, sc.groups, dense, sc))
         plan_uniform(items, sc.order, n_items, n_pairs, sc.groups, dense, sc);
 }

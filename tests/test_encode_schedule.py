@@ -66,14 +66,31 @@ def test_balanced_units_cover_every_tile_once_and_load_the_pairs_evenly(items):
         assert slots[i] <= min(16, 4 + -(-PAIRS // _tiles(T, d_sae)[0]))
 
 
-def test_wide_encoder_keeps_uniform_slices_walked_in_step():
-    # 4096 -> 32768: 268 MB of weights, far more than L2; its pairs must read the same weight tiles at the same time
-    units, slots = B.s3_encode_schedule_describe([(8192, 4096, 32768, 64)], PAIRS)
-    assert units is None and 1 <= slots[0] <= 16
-    # two wide items: still uniform slices, dealt out by table
-    units, slots = B.s3_encode_schedule_describe([(8192, 4096, 32768, 64), (4096, 4096, 32768, 64)], PAIRS)
+def test_wide_encoder_walks_bands_of_row_tiles_with_its_slices_in_step():
+    # 4096 -> 32768: 268 MB of weights, far more than L2. Its row tiles are not cut at shares; bands of row tiles are swept
+    # by uniform column slices, one unit per pair, so the pairs of a slice read the same weight tiles at the same time
+    # and a band's token tiles (16 x 2 MB) stay in L2.
+    item = (8192, 4096, 32768, 64)
+    units, slots = B.s3_encode_schedule_describe([item], PAIRS)
+    assert units is not None and slots[0] == 4 and len(units) == 128
+    _check_cover([item], units, slots)
+    assert set((lo, hi) for _, _, _, lo, hi, _ in units.tolist()) == {(0, 32), (32, 64), (64, 96), (96, 128)}
+    for pr in range(64):
+        mine = units[units[:, 0] == pr]
+        assert len(mine) == 2 and mine[0, 2] < 16 <= mine[1, 2]                 # first a unit of band 0, then one of band 1
+        assert (mine[0, 3], mine[0, 4]) == (mine[1, 3], mine[1, 4])             # the same slice in both bands
+    assert units[:, 0].max() == 63
+    # 37 row tiles: two slices over all of them keep every pair busy (74 units of 64 tiles); bands of four slices would take 96
+    units, slots = B.s3_encode_schedule_describe([(9472, 4096, 32768, 64)], PAIRS)
+    assert slots[0] == 2 and len(units) == 74 and np.bincount(units[:, 0]).max() == 1
+    # few row tiles: more slices, one band
+    units, slots = B.s3_encode_schedule_describe([(2048, 4096, 32768, 64)], PAIRS)
+    assert slots[0] == 9 and len(units) == 72
+    # two wide items in one launch: uniform slices, dealt out by table
+    both = [(8192, 4096, 32768, 64), (4096, 4096, 32768, 64)]
+    units, slots = B.s3_encode_schedule_describe(both, PAIRS)
     assert units is not None
-    _check_cover([(8192, 4096, 32768, 64), (4096, 4096, 32768, 64)], units, slots)
+    _check_cover(both, units, slots)
     for i in (0, 1):
         mine = units[units[:, 1] == i]
         assert len(set((lo, hi) for _, _, _, lo, hi, _ in mine.tolist())) == slots[i]      # the same slices in every row tile
