@@ -289,6 +289,7 @@ __device__ __forceinline__ UnitWalk unit_walk(const EncodeTcParams& p, int pair,
 // Unit -> item, candidate-list slot ("slice"), row tile and the column tiles [tile_lo, tile_hi) it covers.
 struct Unit {
     int item, slice, mt, tile_lo, tile_hi;
+    int head;              // projection mode: the head whose projection the unit computes first (0 otherwise)
 };
 __device__ __forceinline__ Unit unit_decode(const EncodeTcParams& p, const UnitWalk& w)
 {
@@ -296,12 +297,19 @@ __device__ __forceinline__ Unit unit_decode(const EncodeTcParams& p, const UnitW
     if (p.use_sched) {
         const UnitDesc d = p.unit[w.i];
         u.item = d.item; u.slice = d.slot; u.mt = d.mt; u.tile_lo = d.tile_lo; u.tile_hi = d.tile_hi;
+        u.head = 0;
+        if (p.proj_heads > 0) {        // the table's row index runs over (row tile, head)
+            u.mt = d.mt / p.proj_heads;
+            u.head = d.mt - u.mt * p.proj_heads;
+        }
         return u;
     }
+    u.head = 0;
     if (p.proj_heads > 0) {            // (row tile, head), heads of a row tile next to each other: they share the tile of h
         u.item = 0;
         u.mt = w.i / p.proj_heads;
-        u.slice = w.i - u.mt * p.proj_heads;
+        u.head = w.i - u.mt * p.proj_heads;
+        u.slice = 0;
         u.tile_lo = 0; u.tile_hi = p.item[0].n_col_tiles;
         return u;
     }
@@ -543,7 +551,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             bool ok = true;
             for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
                 const Unit un = unit_decode(p, uw);
-                const int item = un.item, slice = un.slice, mt = un.mt, tile_lo = un.tile_lo, tile_hi = un.tile_hi;
+                const int item = un.item, mt = un.mt, tile_lo = un.tile_lo, tile_hi = un.tile_hi;
                 const ItemParams& ip = p.item[item];
                 const CUtensorMap* map_x = &maps.x[item];
                 const CUtensorMap* map_w = &maps.w[item];
@@ -551,7 +559,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                 const int row0 = mt * PAIR_M + static_cast<int>(cta_rank) * BM;        // this CTA's tokens
                 if constexpr (PROJ) {
                     // the head's projection first: 128 tokens of h and this CTA's 64 of the head's 128 rows of W_proj^T per k-block
-                    const int wrow0 = slice * PROJ_N + static_cast<int>(cta_rank) * (PROJ_N / 2);
+                    const int wrow0 = un.head * PROJ_N + static_cast<int>(cta_rank) * (PROJ_N / 2);
                     for (int kb = 0; kb < p.proj_kblocks; ++kb) {
                         if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag)) {
                             dev_set_error(p.status, DEV_TIMEOUT_SMEM_EMPTY);
@@ -701,10 +709,10 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             const bool live = t < ip.T;
             const int k = ip.k;
             const uint32_t cap = ip.cap;
-            // projection mode: the unit's "slice" is the head; a (token, head) pair is one output row with one list
-            const size_t orow = PROJ ? static_cast<size_t>(live ? t : 0) * p.proj_heads + slice : static_cast<size_t>(live ? t : 0);
+            // projection mode: a (token, head) pair is one output row
+            const size_t orow = PROJ ? static_cast<size_t>(live ? t : 0) * p.proj_heads + un.head : static_cast<size_t>(live ? t : 0);
             // each group keeps its own candidate list, bound and histogram for its columns of the row
-            const size_t list_idx = PROJ ? orow * EPI_GROUPS + grp : (orow * ip.n_slices + slice) * EPI_GROUPS + grp;
+            const size_t list_idx = (orow * ip.n_slices + slice) * EPI_GROUPS + grp;
             uint64_t* glist = DENSE ? nullptr : ip.cand + list_idx * cap;
             if (!DENSE) {
 #pragma unroll 1
@@ -727,7 +735,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             // groups are never more than two units apart: the slot of unit n + 2, cleared here by each group, is not in
             // use by anyone (unit n - 2 is over for all), and both groups have cleared it before either reaches unit n + 2.
             if (EPI_GROUPS > 1) xtau32[((unit_seq + 2u) & 3u) * BM + e] = 0u;
-            const bool share_row = !DENSE && !PROJ && live && ip.n_slices > 1;     // other units hold pieces of these rows
+            const bool share_row = !DENSE && live && ip.n_slices > 1;     // other units hold pieces of these rows
             uint32_t announced = hint_in;
             if constexpr (PROJ) {
                 // The head's projection: accumulator -> + bias -> bf16 (round to nearest even, as the dense epilogue stores
@@ -748,7 +756,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                 for (int cb = grp * PB; cb < (grp + 1) * PB; ++cb) {
                     uint32_t acc[32];
                     tc_ld32(taddr + cb * BATCH, acc);
-                    const float4* pb4 = reinterpret_cast<const float4*>(p.proj_bias + slice * PROJ_N + cb * BATCH);
+                    const float4* pb4 = reinterpret_cast<const float4*>(p.proj_bias + un.head * PROJ_N + cb * BATCH);
                     float bias[BATCH];
 #pragma unroll
                     for (int j4 = 0; j4 < BATCH / 4; ++j4) {
@@ -1133,7 +1141,8 @@ int uniform_slices(int T, int nct, int d_sae, int n_pairs, bool dense)
 // duration, and a range is cut into units at the row-tile boundaries. A row tile therefore ends up in a few pieces held by
 // neighbouring pairs, each piece with its own candidate list. Fails (false) when an encoder is too wide for a round, a
 // row would need more than kMaxSlots pieces, or the units do not fit the table.
-bool plan_balanced(const EncodeTcItem* items, const int* order, int n_items, int n_pairs, int groups, bool dense, Schedule& sc)
+bool plan_balanced(const EncodeTcItem* items, const int* order, int n_items, int n_pairs, int groups, bool dense, Schedule& sc,
+                   double extra_unit_cost = 0.0)
 {
     static thread_local UnitDesc gen[MAX_SCHED];
     static thread_local uint16_t gen_pair[MAX_SCHED];
@@ -1153,17 +1162,19 @@ bool plan_balanced(const EncodeTcItem* items, const int* order, int n_items, int
         double rem = 0.0;
         for (int q = q0; q < q1; ++q) {
             const EncodeTcItem& it = items[order[q]];
-            const CostModel c = cost_model((it.d_in + BK - 1) / BK, it.k, groups, dense);
+            CostModel c = cost_model((it.d_in + BK - 1) / BK, it.k, groups, dense);
+            c.unit += extra_unit_cost;
             rem += static_cast<double>(encode_tc_row_tiles(it.T)) * (encode_tc_col_tiles(it.d_sae) * c.tile + c.unit);
         }
         // a pair's share: what is left, plus the start-up of the piece that every later cut adds, over the pairs left
         auto share = [&](int pr, double unit) { return (rem + unit * (n_pairs - pr - 1)) / (n_pairs - pr); };
         int pr = 0;
         double acc = 0.0;
-        double target = share(0, cost_model((items[order[q0]].d_in + BK - 1) / BK, items[order[q0]].k, groups, dense).unit);
+        double target = share(0, cost_model((items[order[q0]].d_in + BK - 1) / BK, items[order[q0]].k, groups, dense).unit + extra_unit_cost);
         for (int q = q0; q < q1; ++q) {
             const EncodeTcItem& it = items[order[q]];
-            const CostModel c = cost_model((it.d_in + BK - 1) / BK, it.k, groups, dense);
+            CostModel c = cost_model((it.d_in + BK - 1) / BK, it.k, groups, dense);
+            c.unit += extra_unit_cost;
             const int n_mtiles = encode_tc_row_tiles(it.T), nct = encode_tc_col_tiles(it.d_sae);
             if (n_mtiles > 65535 || nct > 65535) return false;
             const int max_pieces = slot_bound(it.T, n_pairs);
@@ -1560,9 +1571,12 @@ s3_status launch_preact_tc(const EncodeTcState* st, const void* d_x, int64_t ldx
     return launch_tc(&it, 1, max_ctas, nullptr, d_status, d_out, ld_out, out_bf16, stream);
 }
 
+// The (row tile, head) pairs of a projection launch as the row tiles of one 128-wide encoder, for the schedule.
+static int proj_schedule_rows(int T, int n_heads) { return encode_tc_row_tiles(T) * n_heads * PAIR_M; }
+
 size_t encode_proj_tc_workspace_bytes(int T, int n_heads, int k)
 {
-    return encode_tc_workspace_bytes(T * n_heads, 1, k);
+    return encode_tc_workspace_bound(proj_schedule_rows(T, n_heads), k);      // holds whatever pieces the launch cuts
 }
 
 // Projection of one head + encode of that head in the same CTA pair: h [T, d_model] -> x = h W_proj + b (bf16, kept in shared
@@ -1572,7 +1586,7 @@ s3_status launch_encode_proj_tc(const EncodeTcState* proj, const EncodeTcState* 
                                 float* d_vals, cudaStream_t stream)
 {
     alignas(64) TensorMaps maps;
-    EncodeTcParams p;
+    static thread_local EncodeTcParams p;
     memset(&p, 0, sizeof(p));
     memset(&maps, 0, sizeof(maps));
     s3_status rc = make_map(&maps.x[0], d_h, static_cast<uint64_t>(T), static_cast<uint64_t>(d_model), static_cast<uint64_t>(ldh), BM);
@@ -1592,18 +1606,41 @@ s3_status launch_encode_proj_tc(const EncodeTcState* proj, const EncodeTcState* 
     ip.n_mtiles = encode_tc_row_tiles(T);
     ip.n_col_tiles = encode_tc_col_tiles(d_sae);
     S3_REQUIRE(encode_tc_min_slices(d_sae) == 1, S3_ERR_UNSUPPORTED, "d_sae = %d is too wide for one column slice per head", d_sae);
-    ip.n_slices = 1;
     ip.unit_start = 0;
     constexpr int groups = 2;                  // d_head = 128: the narrow-encoder configuration
     ip.cap = encode_tc_list_cap(k, groups);
     ip.b_eff = st->d_b_eff;
-    const size_t rows = static_cast<size_t>(T) * n_heads, lists = groups;
+    int n_pairs = encode_tc_max_pairs();
+    if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
+    if (n_pairs > MAX_PAIRS) n_pairs = MAX_PAIRS;
+    // Units: whole (row tile, head) pairs when they fill the pairs' waves evenly; otherwise the column tiles of all
+    // (row tile, head) pairs are cut at the pairs' shares like a narrow encoder's row tiles, every piece computing its
+    // head's projection again first (64 k-blocks into half an accumulator: about two column tiles' worth of time).
+    ip.n_slices = 1;
+    p.n_units = ip.n_mtiles * n_heads;
+    {
+        const int waves = (p.n_units + n_pairs - 1) / n_pairs;
+        const bool even = static_cast<double>(p.n_units) >= 0.93 * waves * n_pairs;
+        const EncodeTcItem fake = {st, nullptr, 0, proj_schedule_rows(T, n_heads), PROJ_N, d_sae, k, 0, nullptr, nullptr};
+        const int order0 = 0;
+        Schedule& sc = schedule_buffer();
+        const double proj_cost = 300.0 * p.proj_kblocks + 3000.0;
+        if (!even && ip.n_mtiles * n_heads <= 65535 && plan_balanced(&fake, &order0, 1, n_pairs, groups, false, sc, proj_cost)) {
+            ip.n_slices = sc.slots[0];
+            p.n_units = sc.n_units;
+            p.use_sched = 1;
+            memcpy(p.pair_start, sc.pair_start, sizeof(p.pair_start));
+            memcpy(p.unit, sc.unit, sizeof(UnitDesc) * static_cast<size_t>(sc.n_units));
+            n_pairs = sc.n_pairs;
+        } else if (p.n_units < n_pairs) n_pairs = p.n_units;
+    }
+    const size_t rows = static_cast<size_t>(T) * n_heads, lists = static_cast<size_t>(ip.n_slices) * groups;
     unsigned char* base = static_cast<unsigned char*>(d_scratch);
     ip.hint = reinterpret_cast<uint32_t*>(base);
     ip.counts = reinterpret_cast<uint32_t*>(base + round_up(rows * 4, 256));
     ip.cand = reinterpret_cast<uint64_t*>(base + round_up(rows * 4, 256) + round_up(rows * lists * 4, 256));
-    p.n_units = ip.n_mtiles * n_heads;
-    S3_CUDA_TRY(cudaMemsetAsync(ip.hint, 0, rows * 4, stream));
+    // bounds, and the lengths of the lists (a row cut into fewer pieces than the slot count leaves the other slots empty)
+    S3_CUDA_TRY(cudaMemsetAsync(base, 0, round_up(rows * 4, 256) + (p.use_sched ? rows * lists * 4 : 0), stream));
 
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
@@ -1620,9 +1657,6 @@ s3_status launch_encode_proj_tc(const EncodeTcState* proj, const EncodeTcState* 
         S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_PROJ, groups>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
         attr_set[dev] = true;
     }
-    int n_pairs = encode_tc_max_pairs();
-    if (max_ctas > 0 && max_ctas / 2 < n_pairs) n_pairs = max_ctas / 2 > 0 ? max_ctas / 2 : 1;
-    if (p.n_units < n_pairs) n_pairs = p.n_units;
     encode_tc_kernel<M_PROJ, groups><<<2 * n_pairs, 64 + 128 * groups, smem, stream>>>(maps, p);
     S3_CUDA_TRY(cudaGetLastError());
     launch_candidate_merge(ip.cand, ip.counts, ip.hint, static_cast<int>(rows), static_cast<int>(lists), ip.cap, k, d_ids, d_vals, stream);
