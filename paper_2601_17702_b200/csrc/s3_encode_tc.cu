@@ -2,34 +2,43 @@
 //
 //   pre[t,f] = sum_i x[t,i] * W_enc[i,f] + b_eff[f],   b_eff = b_enc - W_enc^T b_dec   (folded once)
 //
-// Persistent, warp-specialised kernel, one CTA per SM:
-//   warp 0      TMA producer: streams 128x64 tiles of x and 256x64 tiles of W_enc^T (K-major, 128-byte
-//               swizzle) into a ring of shared-memory stages, completion on mbarriers;
-//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 x bf16 -> fp32) into
-//               one of two 128x256 accumulators in tensor memory, tcgen05.commit frees the stage /
-//               publishes the accumulator;
-//   warps 2-5   epilogue (four warps per group, one or two groups: see MAX_EPI_GROUPS): thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
-//               biased and compared with the row's bound tau, a value that at least k pre-activations
-//               of the row are known to exceed. Survivors go, branch-free, to a short pending list in
-//               shared memory. When some lane's list is nearly full the warp folds its lists: each
-//               survivor is appended to the row's candidate list in global memory and counted in a
-//               small per-row histogram over the float's exponent and top mantissa bits; as soon as k
-//               survivors lie in buckets above the bound's bucket, tau moves up to the next bucket edge.
-//               tau therefore tracks the row's running k-th largest value to within one bucket (about
-//               4 %) at a few instructions per survivor, and no ordered structure is kept on the SM.
-// A work unit is (128-token block, slice of 256-column tiles). A finished unit publishes its final
-// bound per row; units of the same rows that start later begin with it (any published bound is valid:
-// k values above it exist). The candidate lists of all slices, a few hundred keys per row, are
-// reduced to the exact Top-k by the merge kernel (s3_topk_merge.cu), which first drops everything not
-// above the best published bound. Only candidates leave the SM (as 64-bit keys); the pre-activation
-// matrix is never written to memory.
+// Persistent, warp-specialised kernel; the two CTAs of a cluster (one per SM) work as a pair on 256-token x
+// 256-feature tiles:
+//   warp 0      TMA producer: per k-block each CTA streams its 128 tokens of x and its half of the tile's 256
+//               rows of W_enc^T (K-major, 128-byte swizzle) into a ring of shared-memory stages; all copies of
+//               a stage are counted on the first CTA's mbarrier;
+//   warp 1      MMA issuer (first CTA only): one thread issues tcgen05.mma.cta_group::2 (M=256 over the pair,
+//               N=256, K=16, bf16 x bf16 -> fp32) into one of two 256-column accumulators in each CTA's tensor
+//               memory; tcgen05.commit, multicast to both CTAs, frees the stage / publishes the accumulator;
+//   warps 2..   epilogue, four warps per group, one or two groups (template parameter GROUPS; two groups split a
+//               tile's columns): thread = token row (TMEM lane). Each 32-column batch is read with tcgen05.ld,
+//               biased and compared with the row's bound, a value that at least k pre-activations of the row are
+//               known to exceed. Survivors go, branch-free, to a short pending list in shared memory. When some
+//               lane's list is nearly full the warp folds its lists: each survivor is appended to the row's
+//               candidate list in global memory and counted in a small per-row histogram over the float's
+//               exponent and top mantissa bits; as soon as k survivors lie in buckets above the bound's bucket,
+//               the bound moves up to the next bucket edge. It therefore tracks the row's running k-th largest
+//               value to within one bucket (about 4 %) at a few instructions per survivor, and no ordered
+//               structure is kept on the SM.
+// A work unit is a run of column tiles of one 256-token row tile of one encoder call (up to 8 calls per launch).
+// The host cuts the launch into units (build_schedule): shares of equal modelled duration per CTA pair for
+// encoders whose weights stay in L2, bands of row tiles swept by uniform column slices in step for wider ones,
+// whole (row tile, slice) units otherwise; the units travel in the launch parameters. Every unit keeps its own
+// candidate list per row and epilogue group. Bounds are shared: a bound that k values of one list exceed holds for
+// the whole row, so a list announces its bound whenever it rises (to the other group through shared memory, to
+// the row's other pieces through a per-row word in global memory) and every list drops what does not beat the
+// best bound it has seen. The lists, a few hundred keys per row, are reduced to the exact Top-k by the merge
+// kernel (s3_topk_merge.cu), which first drops everything not above the row's best bound. Only candidates leave
+// the SM (as 64-bit keys); the pre-activation matrix is never written to memory.
 //
-// A candidate list that would overflow is first compacted against the current bound and, if that
-// does not free enough room (many nearly equal values), cut down to its exact k largest keys.
+// A candidate list that would overflow is first compacted against the current bound and, if that does not free
+// enough room (many nearly equal values), cut down to its exact k largest keys.
 //
-// Every mbarrier wait is bounded; a wait that runs out records which one in the workspace status
-// word, raises a CTA-wide abort flag, and the CTA drains its own TMA copies, frees its tensor memory
-// and exits.
+// The same pipeline serves two more epilogues: DENSE writes the pre-activations themselves (the upstream
+// projections), PROJ computes a head's projection into shared memory first and encodes from there.
+//
+// Every mbarrier wait is bounded; a wait that runs out records which one in the workspace status word, raises a
+// CTA-wide abort flag, and the CTA drains its own TMA copies, frees its tensor memory and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <string.h>
