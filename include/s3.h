@@ -101,9 +101,9 @@ s3_status s3_sae_encode_topk(const s3_sae* sae, const void* d_x, int64_t ldx, in
  * d_out 16-byte aligned. Workspace: the 64-byte status block only. */
 s3_status s3_sae_preact(const s3_sae* sae, const void* d_x, int64_t ldx, int T, void* d_out, int64_t ld_out,
                         s3_dtype out_dtype, void* d_ws, size_t ws_bytes, void* stream);
-/* Tuning knob: number of column slices each row block of the encode is split into (0 = automatic)
- * and the largest number of thread blocks a launch may use (0 = all SMs). Results do not depend on
- * either. */
+/* Tuning knob: number of uniform column slices each row block of the encode is split into (0 = the launch cuts its own
+ * work units, see s3_encode_schedule_describe) and the largest number of thread blocks a launch may use (0 = all SMs).
+ * Results do not depend on either. */
 s3_status s3_sae_set_schedule(s3_sae* sae, int n_slices, int max_ctas);
 
 /* ------------------------------------------------------------------------------------------------
@@ -113,13 +113,13 @@ s3_status s3_sae_set_schedule(s3_sae* sae, int n_slices, int max_ctas);
  *
  * Up to S3_MAX_ENCODE_ITEMS independent encoder calls (the layers' key SAEs of one chunk, key and query SAEs
  * together, ...) as ONE persistent launch followed by one selection launch: the work units of all items are
- * dealt out over the SMs by their modelled duration, so the SMs stay busy across items of unequal size and
+ * cut and dealt out over the SMs by their modelled duration, so the SMs stay busy across items of unequal size and
  * the launch ends evenly. Each item has its own encoder, input, T, k and outputs; the results are those of
  * s3_sae_encode_topk item by item (bit-identical: the selection is exact, whatever the schedule).
  * bf16 encoders only (S3_ERR_UNSUPPORTED otherwise); an item with T == 0 is skipped. `h_items` is a HOST
  * array. max_ctas > 0 limits the launch to that many thread blocks (an even number is used), for launches that
- * share the GPU with another stream's kernel. Workspace: s3_sae_encode_grouped_workspace_bytes(h_items, n_items) (status block + every item's
- * candidate lists).
+ * share the GPU with another stream's kernel. Workspace: s3_sae_encode_grouped_workspace_bytes(h_items, n_items) (status block + room for every item's
+ * candidate lists under any schedule; it grows with T, so the size for a full chunk also serves a shorter last one).
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
     const s3_sae* sae;
@@ -140,8 +140,8 @@ int s3_sae_encode_ctas(const s3_sae* sae, int T);
  * thread blocks; host arithmetic only, no device is touched. A unit is a run of 256-column tiles of one 256-token row
  * tile of one item, and its survivors go to one of the row's candidate lists ("slot"). Encoders whose weights stay in L2
  * are cut into one contiguous share of equal modelled duration per pair (pieces of at least three column tiles, a row
- * tile spread over neighbouring pairs); wider encoders keep uniform column slices walked in step, so that the pairs read
- * the same weight tiles at the same time. Writes six integers per unit to h_units (pair, item, row tile, first column
+ * tile spread over neighbouring pairs); wider encoders walk bands of row tiles with uniform column slices in step, so that the pairs of a
+ * slice read the same weight tiles at the same time and a band's token tiles stay in L2. Writes six integers per unit to h_units (pair, item, row tile, first column
  * tile, one past the last, slot), at most max_units units, and every item's slots per row to h_slots [n_items].
  * Returns the number of units, -1 when the launch deals uniform slices round-robin without a unit table (only h_slots is
  * written), -2 on invalid arguments. The selection result never depends on the schedule (Eq. 3 is exact). */
