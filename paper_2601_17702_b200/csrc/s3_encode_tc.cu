@@ -67,7 +67,11 @@ constexpr int kTwoGroupsMaxDin = 1024;         // encoders at most this wide run
 constexpr int TMEM_COLS = 512;
 constexpr int BATCH = 32;                    // columns per tcgen05.ld
 constexpr int STEP = 8;                      // columns filtered between two checks of the pending lists
-constexpr int PEND_CAP = 2 * STEP;           // pending-list slots per row
+// Pending-list slots per row, chosen per launch: more slots mean fewer, fuller folds (k = 128 on 128-wide encoders: 2.10
+// -> 1.94 ms with 24) but, with two epilogue groups, one pipeline stage less (16 KB per group at 16 slots, 24 KB at 24),
+// which costs the eight 512-wide k = 16 layers 2.6 %. Launches with k >= 32 take 24, the others 16.
+constexpr int PEND_CAP_MIN = 2 * STEP, PEND_CAP_MAX = 3 * STEP;
+__host__ __device__ inline int pend_cap_for(int max_k) { return max_k >= 32 ? PEND_CAP_MAX : PEND_CAP_MIN; }
 constexpr int NB = 64;                       // histogram buckets per row
 #ifndef S3_FOLD_CHUNK
 #define S3_FOLD_CHUNK 4
@@ -264,6 +268,7 @@ struct ItemParams {
 
 struct EncodeTcParams {
     int n_items, n_units, n_stages;
+    int pend_cap;              // pending-list slots per row (shared memory)
     int use_sched;             // 1: pair p runs units unit[pair_start[p] .. pair_start[p+1]); 0: units p, p + n_pairs, ...
     uint32_t* status;
     void* dense_out;           // dense mode (one item): the pre-activations [T, ld_out], fp32 or bf16
@@ -338,7 +343,7 @@ struct SmemLayout {
     uint32_t a_off, b_off, x_off, pend_off, hist_off, xtau_off, bar_off, total;
 };
 constexpr int X_TILE_BYTES = 2 * A_STAGE_BYTES;    // projection mode: this CTA's 128 tokens x 128 projected columns, two k-blocks
-__host__ __device__ inline SmemLayout smem_layout(int n_stages, bool proj, int groups)
+__host__ __device__ inline SmemLayout smem_layout(int n_stages, bool proj, int groups, int pend_cap)
 {
     const int EPI_THREADS = 128 * groups;
     SmemLayout L;
@@ -346,7 +351,7 @@ __host__ __device__ inline SmemLayout smem_layout(int n_stages, bool proj, int g
     L.b_off = L.a_off + n_stages * A_STAGE_BYTES;
     L.x_off = L.b_off + n_stages * B_STAGE_BYTES;
     L.pend_off = L.x_off + (proj ? X_TILE_BYTES : 0);
-    L.hist_off = L.pend_off + PEND_CAP * EPI_THREADS * 8;
+    L.hist_off = L.pend_off + pend_cap * EPI_THREADS * 8;
     L.xtau_off = L.hist_off + NB * EPI_THREADS * 2;
     L.bar_off = L.xtau_off + BM * 16;
     L.total = L.bar_off + (2 * n_stages + 5) * 8 + 16;
@@ -388,7 +393,7 @@ __device__ __noinline__ void prune_list(uint64_t* glist, uint16_t* my_hist, RowS
         if (__uint_as_float(static_cast<uint32_t>(key >> 32)) > r.cut) glist[w++] = key;
     }
     r.gcnt = w;
-    if (r.gcnt + PEND_CAP <= cap) return;
+    if (r.gcnt + PEND_CAP_MAX <= cap) return;
     for (int a = 0; a < k; ++a) {
         uint32_t best = a;
         uint64_t kb = glist[a];
@@ -505,7 +510,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
     constexpr int EPI_GROUPS = GROUPS, EPI_THREADS = 128 * GROUPS;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const SmemLayout L = smem_layout(p.n_stages, PROJ, GROUPS);
+    const SmemLayout L = smem_layout(p.n_stages, PROJ, GROUPS, p.pend_cap);
     unsigned char* smem_a = smem + L.a_off;
     unsigned char* smem_b = smem + L.b_off;
     unsigned char* smem_x = smem + L.x_off;                // projection mode: the head's projected tile, the encode's A operand
@@ -708,6 +713,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
         const int cb_lo = grp * CB_PER_GROUP, cb_hi = cb_lo + CB_PER_GROUP;
         uint32_t tile_count = 0, unit_seq = 0;
         bool ok = true;
+        const int fold_at = p.pend_cap - STEP;      // a lane with more pending entries than this may not take another STEP values
         // the accumulator is handed back on the first CTA's barrier
         const uint32_t acc_empty_addr[2] = {map_to_cta(smem_u32(&acc_empty[0]), 0), map_to_cta(smem_u32(&acc_empty[1]), 0)};
         for (UnitWalk uw = unit_walk(p, pair, n_pairs); uw.i < uw.end && ok; uw.i += uw.step) {
@@ -903,7 +909,7 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
                         }
                         asm volatile("" ::: "memory");
                         cnt = static_cast<int>((slot - pend_addr) / (EPI_THREADS * 8));
-                        if (__any_sync(0xffffffffu, cnt > PEND_CAP - STEP)) {
+                        if (__any_sync(0xffffffffu, cnt > fold_at)) {
                             fold_pending<EPI_THREADS>(my_pend, my_hist, glist, r, cnt, k, cap);
                             const uint32_t now = announced_bound(r);       // tell the row's other lists when the bound has risen
                             if (now > announced) {
@@ -1478,16 +1484,21 @@ s3_status launch_tc(const EncodeTcItem* items, int n_items, int max_ctas, void* 
     // no bound is known for any row yet, and no list holds anything
     if (!dense) S3_CUDA_TRY(cudaMemsetAsync(base, 0, hint_bytes + (sc.table ? count_bytes : 0), stream));
 
+    {
+        int max_k = 0;
+        for (int j = 0; j < n_items; ++j) max_k = items[j].k > max_k ? items[j].k : max_k;
+        p.pend_cap = pend_cap_for(max_k);
+    }
     int dev = 0;
     S3_CUDA_TRY(cudaGetDevice(&dev));
     int max_smem = 0;
     S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     int n_stages = 6;
-    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, false, groups).total) + 1024 > max_smem) --n_stages;
-    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, false, groups).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
+    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, false, groups, p.pend_cap).total) + 1024 > max_smem) --n_stages;
+    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, false, groups, p.pend_cap).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
                "shared memory too small for the encode pipeline");
     p.n_stages = n_stages;
-    const size_t smem = smem_layout(n_stages, false, groups).total + 1024;
+    const size_t smem = smem_layout(n_stages, false, groups, p.pend_cap).total + 1024;
     static bool attr_set[64] = {};
     if (dev < 64 && !attr_set[dev]) {
         S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_SELECT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
@@ -1655,12 +1666,13 @@ s3_status launch_encode_proj_tc(const EncodeTcState* proj, const EncodeTcState* 
     S3_CUDA_TRY(cudaGetDevice(&dev));
     int max_smem = 0;
     S3_CUDA_TRY(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    p.pend_cap = pend_cap_for(k);
     int n_stages = 6;
-    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, true, groups).total) + 1024 > max_smem) --n_stages;
-    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, true, groups).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
+    while (n_stages > 2 && static_cast<int>(smem_layout(n_stages, true, groups, p.pend_cap).total) + 1024 > max_smem) --n_stages;
+    S3_REQUIRE(static_cast<int>(smem_layout(n_stages, true, groups, p.pend_cap).total) + 1024 <= max_smem, S3_ERR_UNSUPPORTED,
                "shared memory too small for the encode pipeline");
     p.n_stages = n_stages;
-    const size_t smem = smem_layout(n_stages, true, groups).total + 1024;
+    const size_t smem = smem_layout(n_stages, true, groups, p.pend_cap).total + 1024;
     static bool attr_set[64] = {};
     if (dev < 64 && !attr_set[dev]) {
         S3_CUDA_TRY(cudaFuncSetAttribute(encode_tc_kernel<M_PROJ, groups>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
