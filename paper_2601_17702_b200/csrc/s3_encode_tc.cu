@@ -77,8 +77,8 @@ constexpr int NB = 64;                       // histogram buckets per row
 #define S3_FOLD_CHUNK 4
 #endif
 constexpr int FOLD_CHUNK = S3_FOLD_CHUNK;    // pending entries a fold handles per step
-constexpr int COLD_LEVELS = 6;                // trial bounds of the cold-start pass, as fractions of the first batch's maximum
-__device__ constexpr float kColdFraction[COLD_LEVELS] = {0.80f, 0.65f, 0.52f, 0.40f, 0.30f, 0.20f};
+constexpr int COLD_LEVELS = 3;                // trial bounds of the cold-start pass, as fractions of the first batch's maximum
+__device__ constexpr float kColdFraction[COLD_LEVELS] = {0.60f, 0.40f, 0.20f};      // six or eight levels cost more than they save (about 1 %)
 constexpr int HSHIFT = 19;                   // bucket = float bits >> 19: 16 buckets per octave
 constexpr uint32_t WAIT_LIMIT = 1u << 26;    // try_wait polls before a wait is declared dead (~1 s)
 
@@ -421,7 +421,8 @@ __device__ __noinline__ void prune_list(uint64_t* glist, uint16_t* my_hist, RowS
 // Folds the warp's pending lists (cnt entries per lane) into candidate lists and histograms, then
 // raises each row's bound as far as the histogram allows. Called by all 32 lanes.
 template <int EPI_THREADS>
-__device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_hist, uint64_t* glist, RowSel& r, int& cnt,
+__device__ __forceinline__ void fold_pending(uint64_t* __restrict__ my_pend, uint16_t* __restrict__ my_hist, uint64_t* __restrict__ glist,
+                                             RowSel& r, int& cnt,
                                              int k, uint32_t cap)
 {
     if (__any_sync(0xffffffffu, r.gcnt + cnt > cap)) {
@@ -445,14 +446,22 @@ __device__ __forceinline__ void fold_pending(uint64_t* my_pend, uint16_t* my_his
         }
     }
     const int nmax = __reduce_max_sync(0xffffffffu, cnt);
-    // FOLD_CHUNK entries at a time: their loads first, then the list stores, then the histogram, so that the
-    // shared-memory round trips of a chunk overlap instead of forming one dependent chain per entry
+    // FOLD_CHUNK entries at a time: their loads first (those of the next chunk are issued before this chunk is worked on),
+    // then the list stores, then the histogram, so that the shared-memory round trips overlap instead of forming one
+    // dependent chain per entry
+    uint64_t nxt[FOLD_CHUNK];
+#pragma unroll
+    for (int q = 0; q < FOLD_CHUNK; ++q) nxt[q] = (q < cnt) ? my_pend[q * EPI_THREADS] : 0ull;
     for (int i0 = 0; i0 < nmax; i0 += FOLD_CHUNK) {
         uint64_t key[FOLD_CHUNK];
         int idx[FOLD_CHUNK];
         bool ok[FOLD_CHUNK];
 #pragma unroll
-        for (int q = 0; q < FOLD_CHUNK; ++q) key[q] = (i0 + q < cnt) ? my_pend[(i0 + q) * EPI_THREADS] : 0ull;
+        for (int q = 0; q < FOLD_CHUNK; ++q) key[q] = nxt[q];
+        if (i0 + FOLD_CHUNK < nmax) {
+#pragma unroll
+            for (int q = 0; q < FOLD_CHUNK; ++q) nxt[q] = (i0 + FOLD_CHUNK + q < cnt) ? my_pend[(i0 + FOLD_CHUNK + q) * EPI_THREADS] : 0ull;
+        }
 #pragma unroll
         for (int q = 0; q < FOLD_CHUNK; ++q) {
             const uint32_t vb = static_cast<uint32_t>(key[q] >> 32);
