@@ -28,22 +28,26 @@ def _sample_rows(T, n=48):
                                      np.arange(255, 258), np.arange(127, 130)]))
 
 
-@pytest.mark.parametrize("which,layer,chunk_idx", [("key", 0, 0), ("key", 3, 15), ("query", 2, 7)])
-def test_cfg3_full_chunk_encode_sampled_rows(which, layer, chunk_idx):
+# one chunk per call as the scan does it (the query SAE's launch walks two bands of 16 row tiles with four column slices
+# each; the key SAE's row tiles are cut at the thread-block pairs' shares), and two chunks of the query SAE in one call
+# (four bands)
+@pytest.mark.parametrize("which,layer,chunk_idx,n_chunks", [("key", 0, 0, 1), ("key", 3, 15, 1), ("query", 2, 7, 1), ("query", 0, 2, 2)])
+def test_cfg3_full_chunk_encode_sampled_rows(which, layer, chunk_idx, n_chunks):
     cfg = C.CFG3
     shp = cfg.key if which == "key" else cfg.query
     inp = C.ScanInputs(cfg)
     W, b_enc, b_dec = inp.sae(which, layer)
-    x = inp.x(which, layer, chunk_idx * cfg.chunk, cfg.chunk)
+    T = n_chunks * cfg.chunk
+    x = inp.x(which, layer, chunk_idx * cfg.chunk, T)
     d = _dev()
     sae = S.Sae(W.to(d), b_enc.to(d), b_dec.to(d))
-    ws = S.new_workspace(sae.encode_workspace_bytes(cfg.chunk, shp.k))
-    ids = torch.full((cfg.chunk, shp.k), -7, dtype=torch.int32, device=d)
-    vals = torch.full((cfg.chunk, shp.k), -7.0, dtype=torch.float32, device=d)
+    ws = S.new_workspace(sae.encode_workspace_bytes(T, shp.k))
+    ids = torch.full((T, shp.k), -7, dtype=torch.int32, device=d)
+    vals = torch.full((T, shp.k), -7.0, dtype=torch.float32, device=d)
     S.s3_sae_encode_topk(sae, x.to(d), shp.k, ids, vals, ws)
     assert S.s3_workspace_status(ws) == 0
     ids, vals = ids.cpu().numpy(), vals.cpu().numpy()
-    rows = _sample_rows(cfg.chunk)
+    rows = _sample_rows(T)
     pre = O.preact(x[rows].float().numpy(), W.float().numpy(), b_enc.numpy(), b_dec.numpy())
     stats = {}
     check_topk_against_preact(pre, ids[rows], vals[rows], shp.k, TOL_BF16, stats)
