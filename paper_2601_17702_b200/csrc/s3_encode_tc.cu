@@ -42,6 +42,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <string.h>
+#include <vector>
 
 #include "s3_kernels.cuh"
 #include "s3_topk.cuh"
@@ -1315,56 +1316,62 @@ void plan_uniform(const EncodeTcItem* items, const int* order, int n_items, int 
     sc.table = true;
 }
 
-// Banded walk of one encoder whose weights do not stay in L2: bands of R row tiles, each band swept by its S column
-// slices at the same time (one unit per pair), band after band. The hot set is then a band's token tiles (R x 2 MB at
-// d_in 4096, re-read for every column tile) plus the windows of W_enc^T that the slices stream; with all row tiles in
-// one band the token tiles alone fill the L2 and W_enc^T is read about four times (query SAE, T 8192: 1.03-1.27 GB of
-// DRAM traffic with 32 row tiles x 2 slices, 0.76-0.80 GB with two bands of 16 x 4, the same 1.57 ms; 12 x 6 and 8 x 8
-// are 4 and 11 % slower: more lists per row). Four slices, more when there are too few row tiles to fill the pairs.
+// Banded walk of one encoder whose weights do not stay in L2: bands of row tiles, each band swept by its column
+// slices at the same time (one unit per pair), band after band. The hot set is then a band's token tiles (2 MB per row
+// tile at d_in 4096, re-read for every column tile) plus the windows of W_enc^T that the slices stream; with all row
+// tiles in one band the token tiles alone fill the L2 and W_enc^T is read about four times (query SAE, T 8192: 1.03-1.27
+// GB of DRAM traffic with 32 row tiles x 2 slices). A band holds as many row tiles as there are pairs per slice, and
+// each band picks its own slice count so that the pairs' total stays short: 32 row tiles on 74 pairs go as 18 x 4 slices
+// (32 column tiles each) + 14 x 5 (26 each), 58 tiles on the busiest pair instead of the 64 of 16 x 4 + 16 x 4 (1.58 ->
+// 1.53 ms, 0.89 GB; bands of 12 x 6 and 8 x 8 alone are 4 and 11 % slower: more lists per row).
 bool plan_banded(const EncodeTcItem& it, int n_pairs, Schedule& sc)
 {
     static thread_local UnitDesc gen[MAX_SCHED];
     static thread_local uint16_t gen_pair[MAX_SCHED];
     const int n_mtiles = encode_tc_row_tiles(it.T), nct = encode_tc_col_tiles(it.d_sae);
-    // (S, R): the modelled time is bands x tiles per slice (+ a quarter tile per slice and band, as for uniform slices);
-    // among the choices within 3 % of the best, the fewest slices whose band of token tiles stays under 40 MB, else the best.
+    // modelled time of a band: its tiles per slice, a quarter tile per slice, 6 % more when its token tiles exceed 40 MB
     const int s_lo = encode_tc_min_slices(it.d_sae);
     int s_hi = slot_bound(it.T, n_pairs) < nct ? slot_bound(it.T, n_pairs) : nct;
     s_hi = s_hi > kMaxSlots ? kMaxSlots : s_hi;
     if (s_hi < s_lo) return false;
     const int r_hot = static_cast<int>((size_t(40) << 20) / (static_cast<size_t>(PAIR_M) * it.d_in * 2));
-    auto band_rows = [&](int S) {
-        int R = n_pairs / S;
-        R = R < 1 ? 1 : (R > n_mtiles ? n_mtiles : R);
-        const int bands = (n_mtiles + R - 1) / R;
-        return (n_mtiles + bands - 1) / bands;                  // bands of equal height
-    };
-    auto modelled = [&](int S) {
-        const int R = band_rows(S), bands = (n_mtiles + R - 1) / R;
-        return bands * ((nct + S - 1) / S) + 0.25 * S * bands;
-    };
-    double best = 1e30;
-    for (int c = s_lo; c <= s_hi; ++c) best = modelled(c) < best ? modelled(c) : best;
-    int S = 0;
-    for (int c = s_lo; c <= s_hi && S == 0; ++c)
-        if (modelled(c) <= 1.03 * best && band_rows(c) <= r_hot) S = c;
-    for (int c = s_lo; c <= s_hi && S == 0; ++c)
-        if (modelled(c) <= best + 1e-9) S = c;
-    const int R = band_rows(S);
-    if (S > kMaxSlots || n_mtiles > 65535 || n_mtiles * S > MAX_SCHED || (nct + S - 1) / S > 255) return false;
-    int n = 0;
-    for (int b0 = 0; b0 < n_mtiles; b0 += R) {
-        const int rows = n_mtiles - b0 < R ? n_mtiles - b0 : R;
-        int i = 0;
-        for (int sl = 0; sl < S; ++sl)
-            for (int r = 0; r < rows; ++r, ++i, ++n) {
+    // bands may differ in their slice count: cost[n] = least modelled time of the last n row tiles, band by band
+    static thread_local std::vector<double> cost;
+    static thread_local std::vector<uint8_t> pick;
+    cost.assign(n_mtiles + 1, 0.0);
+    pick.assign(n_mtiles + 1, 0);
+    for (int left = 1; left <= n_mtiles; ++left) {
+        double best = 1e30;
+        int arg = s_lo;
+        for (int c = s_lo; c <= s_hi; ++c) {
+            int R = n_pairs / c;
+            R = R < 1 ? 1 : (R > left ? left : R);
+            const int len = (nct + c - 1) / c;
+            const double t = len + 0.25 * c + (R > r_hot ? 0.06 * len : 0.0) + cost[left - R];
+            if (t < best - 1e-9) { best = t; arg = c; }
+        }
+        cost[left] = best;
+        pick[left] = static_cast<uint8_t>(arg);
+    }
+    int n = 0, S = 0, offset = 0;
+    if (n_mtiles > 65535) return false;
+    for (int b0 = 0; b0 < n_mtiles;) {
+        const int left = n_mtiles - b0, c = pick[left];
+        int rows = n_pairs / c;
+        rows = rows < 1 ? 1 : (rows > left ? left : rows);
+        if ((nct + c - 1) / c > 255 || n + rows * c > MAX_SCHED) return false;
+        S = c > S ? c : S;
+        for (int sl = 0; sl < c; ++sl)
+            for (int r = 0; r < rows; ++r, ++n) {
                 gen[n].mt = static_cast<uint16_t>(b0 + r);
-                gen[n].tile_lo = static_cast<uint16_t>(static_cast<int64_t>(sl) * nct / S);
-                gen[n].tile_hi = static_cast<uint16_t>(static_cast<int64_t>(sl + 1) * nct / S);
+                gen[n].tile_lo = static_cast<uint16_t>(static_cast<int64_t>(sl) * nct / c);
+                gen[n].tile_hi = static_cast<uint16_t>(static_cast<int64_t>(sl + 1) * nct / c);
                 gen[n].item = 0;
                 gen[n].slot = static_cast<uint8_t>(sl);
-                gen_pair[n] = static_cast<uint16_t>(i % n_pairs);
+                gen_pair[n] = static_cast<uint16_t>((offset + sl * rows + r) % n_pairs);
             }
+        offset = (offset + rows * c) % n_pairs;
+        b0 += rows;
     }
     int count[MAX_PAIRS] = {};
     for (int i = 0; i < n; ++i) ++count[gen_pair[i]];

@@ -69,17 +69,20 @@ def test_balanced_units_cover_every_tile_once_and_load_the_pairs_evenly(items):
 def test_wide_encoder_walks_bands_of_row_tiles_with_its_slices_in_step():
     # 4096 -> 32768: 268 MB of weights, far more than L2. Its row tiles are not cut at shares; bands of row tiles are swept
     # by uniform column slices, one unit per pair, so the pairs of a slice read the same weight tiles at the same time
-    # and a band's token tiles (16 x 2 MB) stay in L2.
+    # and a band's token tiles (18 x 2 MB) stay in L2. Each band has its own slice count.
     item = (8192, 4096, 32768, 64)
     units, slots = B.s3_encode_schedule_describe([item], PAIRS)
-    assert units is not None and slots[0] == 4 and len(units) == 128
+    assert units is not None and slots[0] == 5 and len(units) == 18 * 4 + 14 * 5
     _check_cover([item], units, slots)
-    assert set((lo, hi) for _, _, _, lo, hi, _ in units.tolist()) == {(0, 32), (32, 64), (64, 96), (96, 128)}
-    for pr in range(64):
+    first, second = units[units[:, 2] < 18], units[units[:, 2] >= 18]
+    assert set((lo, hi) for _, _, _, lo, hi, _ in first.tolist()) == {(0, 32), (32, 64), (64, 96), (96, 128)}      # 18 row tiles x 4 slices
+    assert len(set((lo, hi) for _, _, _, lo, hi, _ in second.tolist())) == 5 and (second[:, 4] - second[:, 3]).max() == 26
+    assert len(np.unique(first[:, 0])) == 72 and len(np.unique(second[:, 0])) == 70            # one unit per pair and band
+    tiles = np.bincount(units[:, 0], weights=units[:, 4] - units[:, 3], minlength=PAIRS)
+    assert tiles.max() == 58 and (tiles > 0).all()                                             # 64 with two bands of 16 x 4
+    for pr in range(PAIRS):
         mine = units[units[:, 0] == pr]
-        assert len(mine) == 2 and mine[0, 2] < 16 <= mine[1, 2]                 # first a unit of band 0, then one of band 1
-        assert (mine[0, 3], mine[0, 4]) == (mine[1, 3], mine[1, 4])             # the same slice in both bands
-    assert units[:, 0].max() == 63
+        assert len(mine) <= 2 and (np.diff(mine[:, 2]) > 0).all()                              # band 0's unit first
     # 37 row tiles: two slices over all of them keep every pair busy (74 units of 64 tiles); bands of four slices would take 96
     units, slots = B.s3_encode_schedule_describe([(9472, 4096, 32768, 64)], PAIRS)
     assert slots[0] == 2 and len(units) == 74 and np.bincount(units[:, 0]).max() == 1
