@@ -755,10 +755,14 @@ encode_tc_kernel(const __grid_constant__ TensorMaps maps, const __grid_constant_
             // other list of the row (the other epilogue group's, other column pieces' on other SMs) may drop what does not
             // beat it. Without this each list gathers its own k survivors and the folding work grows with the number of lists.
             ++unit_seq;
-            // The groups exchange bounds through xtau32[unit number mod 4][row]. A group cannot start a tile before every
-            // group has finished the tile two before it (the accumulator it needs is handed back by all of them), so the
-            // groups are never more than two units apart: the slot of unit n + 2, cleared here by each group, is not in
-            // use by anyone (unit n - 2 is over for all), and both groups have cleared it before either reaches unit n + 2.
+            // The groups exchange bounds through xtau32[unit number mod 4][row]; unit n + 2 shares its slot with unit n - 2
+            // and each group clears it here, at the start of its unit n. A group announces only before it hands a tile's
+            // accumulator back, and no group can start a tile before every group has handed back the tile two before it.
+            // So (a) whichever group clears last has itself finished announcing for unit n - 2, and the other finished
+            // before its own, earlier clear: after the last clear the slot is zero and nobody writes to it for unit n - 2
+            // any more (the leading group's clear may still fall among the lagging group's announcements; that only loses
+            // a bound); (b) a group can reach unit n + 2 only after the other has finished the first tile of unit n, i.e.
+            // after both clears, so nothing read or announced for unit n + 2 meets an older unit's value.
             if (EPI_GROUPS > 1) xtau32[((unit_seq + 2u) & 3u) * BM + e] = 0u;
             const bool share_row = !DENSE && live && ip.n_slices > 1;     // other units hold pieces of these rows
             uint32_t announced = hint_in;
