@@ -35,7 +35,8 @@ def test_hand_example():
     (33, 3, 5, 40, 7),            # entry count not a power of two, heavy overlap between heads
     (10, 1, 16, 100, 16),         # one head: identity
     (7, 4, 8, 64, 40),            # more outputs wanted than unique features
-    (300, 8, 128, 16384, 128),    # the paper's k = 128 per head: 1024 entries per token, the largest one warp takes
+    (300, 8, 128, 16384, 128),    # the paper's k = 128 per head: 1024 entries per token
+    (300, 4, 128, 16384, 128),    # 512 entries per token, the largest one warp takes
 ])
 def test_parity(T, H, k, D, k_out):
     rng = np.random.default_rng(T + H)
